@@ -1,0 +1,175 @@
+/*
+ * snapstream.h -- C ABI of the SnapStream hot path for NVIDIA B200 (sm_100a).
+ *
+ * SnapStream (arXiv 2511.03092) compresses a prompt's KV cache once, at prefill, into a
+ * fixed number of slots  [ sinks | recent-token ring | SnapKV top-K ]  (Section 3.1) and then
+ * decodes over that fixed-size cache, writing each new token's K/V into the ring at the index
+ * of Eq. 3 (Section 3.3).  This library implements exactly that path:
+ *
+ *   snap_cache_layout   slot arithmetic of Section 3.1
+ *   snap_compress       Section 3.2: Eq. 4 scores -> Eq. 1 window sum -> Eq. 2 pool + top-K ->
+ *                       ring construction (Section 3.2.1) and gather into the cache
+ *   snap_append_kv      Eq. 3 scatter of one new token per sequence
+ *   snap_decode_attn    Section 3.3: (optional Eq. 3 scatter, then) attention of one query token
+ *                       per sequence over the valid cache slots
+ *
+ * Conventions
+ *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are plain
+ *     host memory.  Every device buffer must be 16-byte aligned.
+ *   - The caller owns every buffer.  The library allocates nothing and keeps no per-call
+ *     state; all work is enqueued on the CUDA stream given and the calls return without
+ *     synchronising.
+ *   - Token positions are 0-indexed.  Ls = l_sink, Lr = l_recent, K = topk, Lsr = Ls + Lr,
+ *     Sc = Ls + Lr + K, g = n_q_heads / n_kv_heads.
+ *   - Element type: all of q, k, v, caches and out share cfg->dtype.
+ *   - Return value: SNAP_OK (0) or a negative snap_status.  Nothing throws, aborts or traps.
+ *     Conditions only the device can see (a cache slot id out of range, a bounded wait that
+ *     ran out, a refinement band that overflowed) are OR-ed into *status_dev when given.
+ */
+#ifndef SNAPSTREAM_H_
+#define SNAPSTREAM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SNAP_F32 0
+#define SNAP_BF16 1
+
+#define SNAP_POOL_AVG 0
+#define SNAP_POOL_MAX 1
+
+typedef enum snap_status {
+  SNAP_OK = 0,
+  SNAP_ERR_INVALID_ARG = -1,        /* a value outside the documented domain */
+  SNAP_ERR_UNSUPPORTED = -2,        /* valid, but no kernel is built for this shape */
+  SNAP_ERR_WORKSPACE_TOO_SMALL = -3,
+  SNAP_ERR_NULL_POINTER = -4,
+  SNAP_ERR_CUDA = -5                /* a CUDA runtime call failed; see cudaGetLastError */
+} snap_status;
+
+/* bits of *status_dev */
+#define SNAP_DEV_BAD_SLOT 1u        /* a slot id was outside [0, max_seqs): that sequence was skipped */
+#define SNAP_DEV_WAIT_TIMEOUT 2u    /* a bounded wait on an async copy gave up: results invalid */
+#define SNAP_DEV_BAND_OVERFLOW 4u   /* more near-threshold candidates than the refinement can hold:
+                                       the single-precision order was kept for that head */
+
+/* One attention layer's shape and SnapStream hyper-parameters (appendix table
+ * "SnapStream Hyperparameters": sink, top-K, recent, observation window, pooling kernel). */
+typedef struct snap_config {
+  int32_t n_q_heads;      /* Hq */
+  int32_t n_kv_heads;     /* Hkv, divides Hq */
+  int32_t d_qk;           /* key/query row length, multiple of 16 */
+  int32_t d_v;            /* value row length, multiple of 16, <= 512 */
+  int32_t v_aliases_k;    /* 1: latent attention, V row = first d_v elements of the K row, no V buffers */
+  int32_t dtype;          /* SNAP_F32 or SNAP_BF16 */
+  int32_t l_sink;         /* Ls >= 0 */
+  int32_t l_recent;       /* Lr >= 1 */
+  int32_t topk;           /* K  >= 0 */
+  int32_t l_obs;          /* Lo, 1 <= Lo <= Lr (every candidate precedes every window query) */
+  int32_t pool_kernel;    /* w, odd >= 1 */
+  int32_t pool_mode;      /* SNAP_POOL_AVG (Eq. 2) or SNAP_POOL_MAX */
+  float softmax_scale;    /* Eq. 4's 1/sqrt(d), supplied by the caller */
+  int32_t max_seqs;       /* number of cache slots (sequences resident at once) */
+} snap_config_t;
+
+/* Section 3.1: where the three sections live, and the strides of the caches.
+ * K cache: [max_seqs][Hkv][Sc][d_qk], V cache: [max_seqs][Hkv][Sc][d_v], row-major, dense. */
+typedef struct snap_layout {
+  int32_t slots;          /* Sc = Ls + Lr + K  (L_snapstream, Section 3) */
+  int32_t sink_off;       /* 0 */
+  int32_t ring_off;       /* Ls */
+  int32_t topk_off;       /* Ls + Lr */
+  int64_t k_row_bytes, v_row_bytes;
+  int64_t k_head_stride_bytes, v_head_stride_bytes;   /* Sc * row bytes */
+  int64_t k_seq_stride_bytes, v_seq_stride_bytes;     /* Hkv * head stride */
+  int64_t k_cache_bytes, v_cache_bytes;               /* max_seqs * seq stride (v: 0 if aliased) */
+} snap_layout_t;
+
+/* Section 3.1.  Host only, pure arithmetic.  Validates cfg (INVALID_ARG / UNSUPPORTED). */
+int snap_cache_layout(const snap_config_t* cfg, snap_layout_t* out);
+
+/* Bytes of device scratch snap_compress needs for these prompt lengths (cu_seqlens_host has
+ * n_seq + 1 entries, prompt i is tokens [cu[i], cu[i+1])).  Negative snap_status on error. */
+int64_t snap_compress_workspace_bytes(const snap_config_t* cfg, const int32_t* cu_seqlens_host,
+                                      int32_t n_seq);
+
+/* Bytes of device scratch snap_decode_attn needs for n_active sequences. */
+int64_t snap_decode_workspace_bytes(const snap_config_t* cfg, int32_t n_active);
+
+/*
+ * Prefill compression of n_seq prompts (Section 3.2; appendix listing "SnapStream Prefill KV
+ * Cache Compression" describes the same inputs and outputs).
+ *
+ *   q_obs_dev   [n_seq][Hq][Lo][d_qk]  queries of each prompt's last Lo positions, after any
+ *               positional encoding (Section 3.2: encodings are applied before caching).
+ *               Ignored (may be NULL) when no prompt has more than Lsr + K tokens.
+ *   k_dev,v_dev prompt keys/values, token-major and ragged: element (t, h, c) of prompt i is at
+ *               k_dev[(cu[i] + t) * k_token_stride + h * k_head_stride + c]; strides in elements,
+ *               multiples of 16 bytes.  v_dev is ignored when cfg->v_aliases_k.
+ *   cu_seqlens_host, slot_ids_host   host arrays (n_seq + 1 and n_seq entries); slot_ids give the
+ *               cache slot each prompt is compressed into, distinct, in [0, max_seqs).
+ *   k_cache_dev, v_cache_dev   the caches (snap_layout_t strides).  For each prompt the whole slot
+ *               is rewritten: sinks [0, min(L, Ls)), ring rows of positions [max(Ls, L - Lr), L) at
+ *               slot Ls + (p - Ls) mod Lr, selected rows ascending by position from slot Lsr,
+ *               zeros elsewhere.
+ *   seq_len_dev, valid_topk_dev   [max_seqs] int32; entry slot_ids[i] is set to L_i and to
+ *               min(max(L_i - Lsr, 0), K).
+ *   topk_idx_dev  NULL, or [n_seq][Hkv][K] int32 receiving the selected absolute positions,
+ *               ascending, -1 after the valid ones.
+ *   A prompt with L <= Lsr + K is not scored: all its candidates are kept.  Otherwise the K
+ *   largest pooled scores win, ties to the lower position.
+ */
+int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout,
+                  const void* q_obs_dev,
+                  const void* k_dev, int64_t k_token_stride, int64_t k_head_stride,
+                  const void* v_dev, int64_t v_token_stride, int64_t v_head_stride,
+                  const int32_t* cu_seqlens_host, const int32_t* slot_ids_host, int32_t n_seq,
+                  void* k_cache_dev, void* v_cache_dev,
+                  int32_t* seq_len_dev, int32_t* valid_topk_dev,
+                  int32_t* topk_idx_dev,
+                  void* workspace_dev, size_t workspace_bytes,
+                  uint32_t* status_dev, void* cuda_stream);
+
+/*
+ * Eq. 3: for each of n_active sequences write the new token's K/V rows
+ * (k_new_dev [n_active][Hkv][d_qk], v_new_dev [n_active][Hkv][d_v], dense) into cache slot
+ *   L < Ls ? L : (L - Ls + Lr) mod Lr + Ls,   L = seq_len_dev[slot]  (tokens seen so far),
+ * then add one to seq_len_dev[slot].  slot_ids_dev: [n_active] int32 on the device, distinct.
+ */
+int snap_append_kv(const snap_config_t* cfg, const snap_layout_t* layout,
+                   const void* k_new_dev, const void* v_new_dev,
+                   const int32_t* slot_ids_dev, int32_t n_active,
+                   void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
+                   uint32_t* status_dev, void* cuda_stream);
+
+/*
+ * Section 3.3: one decode step.  With k_new_dev != NULL the new token is first written as in
+ * snap_append_kv (and seq_len advanced); then out[i][h] = softmax(scale * q[i][h] . K^T) V over
+ * the valid slots of sequence i: [0, min(len, Lsr)) and [Lsr, Lsr + valid_topk).
+ * With k_new_dev == NULL the cache is only read.
+ *   q_dev [n_active][Hq][d_qk], out_dev [n_active][Hq][d_v], dense.  A sequence with no valid
+ *   slot gets zeros.  Sequences in one call must use distinct slots.
+ */
+int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout,
+                     const void* q_dev, const void* k_new_dev, const void* v_new_dev,
+                     const int32_t* slot_ids_dev, int32_t n_active,
+                     void* k_cache_dev, void* v_cache_dev,
+                     int32_t* seq_len_dev, const int32_t* valid_topk_dev,
+                     void* out_dev,
+                     void* workspace_dev, size_t workspace_bytes,
+                     uint32_t* status_dev, void* cuda_stream);
+
+/* Text for a snap_status value (static storage). */
+const char* snap_status_string(int status);
+
+/* Number of kernels this library has launched in this process (for benchmarks' bookkeeping). */
+int64_t snap_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SNAPSTREAM_H_ */

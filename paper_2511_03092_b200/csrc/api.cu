@@ -1,0 +1,308 @@
+// Host side of the C ABI: argument validation, slot arithmetic, scratch planning and the
+// launch sequences.  No allocation, no synchronisation, no state besides the launch counter
+// and a cached SM count.
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "snap_internal.cuh"
+
+namespace snap {
+
+unsigned long long g_launches = 0;
+
+namespace {
+
+int sm_count() {
+  static int cached = 0;
+  if (cached > 0) return cached;
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) {
+    cached = n;
+    return n;
+  }
+  (void)cudaGetLastError();
+  return 148;   // B200; used only for sizing when no device is visible
+}
+
+int elt_bytes(int dtype) { return dtype == SNAP_F32 ? 4 : 2; }
+
+int validate(const snap_config_t* c) {
+  if (!c) return SNAP_ERR_NULL_POINTER;
+  if (c->dtype != SNAP_F32 && c->dtype != SNAP_BF16) return SNAP_ERR_INVALID_ARG;
+  if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads) return SNAP_ERR_INVALID_ARG;
+  if (c->d_qk < 16 || c->d_v < 16) return SNAP_ERR_INVALID_ARG;
+  if (c->l_sink < 0 || c->l_recent < 1 || c->topk < 0) return SNAP_ERR_INVALID_ARG;
+  if (c->l_obs < 1 || c->l_obs > c->l_recent) return SNAP_ERR_INVALID_ARG;
+  if (c->pool_kernel < 1 || c->pool_kernel % 2 == 0) return SNAP_ERR_INVALID_ARG;
+  if (c->pool_mode != SNAP_POOL_AVG && c->pool_mode != SNAP_POOL_MAX) return SNAP_ERR_INVALID_ARG;
+  if (!(c->softmax_scale > 0.f) || !std::isfinite(c->softmax_scale)) return SNAP_ERR_INVALID_ARG;
+  if (c->max_seqs < 1) return SNAP_ERR_INVALID_ARG;
+  if (c->v_aliases_k != 0 && c->v_aliases_k != 1) return SNAP_ERR_INVALID_ARG;
+  if (c->v_aliases_k && c->d_v > c->d_qk) return SNAP_ERR_INVALID_ARG;
+  if ((long long)c->l_sink + c->l_recent + c->topk > (1LL << 30)) return SNAP_ERR_INVALID_ARG;
+  if (c->d_qk % 16 || c->d_v % 16 || c->d_v > 512 || c->d_qk > 1024) return SNAP_ERR_UNSUPPORTED;
+  return SNAP_OK;
+}
+
+Shape make_shape(const snap_config_t* c) {
+  Shape s;
+  s.Hq = c->n_q_heads; s.Hkv = c->n_kv_heads; s.g = s.Hq / s.Hkv; s.d_qk = c->d_qk; s.d_v = c->d_v;
+  s.Ls = c->l_sink; s.Lr = c->l_recent; s.K = c->topk; s.Lo = c->l_obs; s.w = c->pool_kernel;
+  s.pool_mode = c->pool_mode; s.v_aliases_k = c->v_aliases_k; s.Sc = s.Ls + s.Lr + s.K;
+  s.max_seqs = c->max_seqs; s.scale = c->softmax_scale;
+  return s;
+}
+
+size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+// Scratch regions of one chunk of prompts (offsets relative to the chunk area).
+struct ChunkPlan {
+  int n_scored, max_le, nsplit, c_stride;
+  size_t part_off, stats_off, c_off, p_off, bytes;
+};
+
+ChunkPlan plan_chunk(const Shape& s, const int32_t* cu, int first, int n) {
+  ChunkPlan p;
+  std::memset(&p, 0, sizeof(p));
+  for (int i = 0; i < n; ++i) {
+    const int L = cu[first + i + 1] - cu[first + i];
+    const int Le = L - s.Ls - s.Lr;
+    if (s.K > 0 && Le > s.K) { ++p.n_scored; p.max_le = Le > p.max_le ? Le : p.max_le; }
+  }
+  if (p.n_scored == 0) return p;
+  const int R = s.g * s.Lo;
+  const int row_blocks = (R + 63) / 64;
+  const int tiles = (p.max_le + 63) / 64;
+  long long nsplit = (2LL * sm_count() + (long long)p.n_scored * s.Hkv * row_blocks - 1) /
+                     ((long long)p.n_scored * s.Hkv * row_blocks);
+  if (nsplit > tiles) nsplit = tiles;
+  if (nsplit > 64) nsplit = 64;
+  if (nsplit < 1) nsplit = 1;
+  p.nsplit = (int)nsplit;
+  p.c_stride = (int)align_up((size_t)p.max_le, 64);
+  const size_t nz = (size_t)p.n_scored * s.Hkv;
+  size_t off = 0;
+  p.part_off = off;  off += align_up(nz * p.nsplit * R * sizeof(float2));
+  p.stats_off = off; off += align_up(nz * R * sizeof(float2));
+  p.c_off = off;     off += align_up(nz * p.c_stride * sizeof(float));
+  p.p_off = off;     off += align_up(nz * p.c_stride * sizeof(float));
+  p.bytes = off;
+  return p;
+}
+
+int check_cu(const int32_t* cu, int n_seq) {
+  if (!cu) return SNAP_ERR_NULL_POINTER;
+  if (n_seq < 0) return SNAP_ERR_INVALID_ARG;
+  for (int i = 0; i < n_seq; ++i)
+    if (cu[i + 1] < cu[i]) return SNAP_ERR_INVALID_ARG;
+  return SNAP_OK;
+}
+
+size_t idx_bytes(const Shape& s, int n_seq) {
+  return align_up((size_t)n_seq * s.Hkv * (s.K > 0 ? s.K : 1) * sizeof(int));
+}
+
+}  // namespace
+}  // namespace snap
+
+using namespace snap;
+
+extern "C" {
+
+const char* snap_status_string(int status) {
+  switch (status) {
+    case SNAP_OK: return "ok";
+    case SNAP_ERR_INVALID_ARG: return "invalid argument";
+    case SNAP_ERR_UNSUPPORTED: return "unsupported shape";
+    case SNAP_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case SNAP_ERR_NULL_POINTER: return "null pointer";
+    case SNAP_ERR_CUDA: return "CUDA error";
+    default: return "unknown status";
+  }
+}
+
+int64_t snap_kernel_launch_count(void) { return (int64_t)g_launches; }
+
+int snap_cache_layout(const snap_config_t* cfg, snap_layout_t* out) {
+  if (!cfg || !out) return SNAP_ERR_NULL_POINTER;
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  const int eb = elt_bytes(cfg->dtype);
+  out->slots = cfg->l_sink + cfg->l_recent + cfg->topk;
+  out->sink_off = 0;
+  out->ring_off = cfg->l_sink;
+  out->topk_off = cfg->l_sink + cfg->l_recent;
+  out->k_row_bytes = (int64_t)cfg->d_qk * eb;
+  out->v_row_bytes = (int64_t)cfg->d_v * eb;
+  out->k_head_stride_bytes = out->k_row_bytes * out->slots;
+  out->v_head_stride_bytes = out->v_row_bytes * out->slots;
+  out->k_seq_stride_bytes = out->k_head_stride_bytes * cfg->n_kv_heads;
+  out->v_seq_stride_bytes = out->v_head_stride_bytes * cfg->n_kv_heads;
+  out->k_cache_bytes = out->k_seq_stride_bytes * cfg->max_seqs;
+  out->v_cache_bytes = cfg->v_aliases_k ? 0 : out->v_seq_stride_bytes * cfg->max_seqs;
+  return SNAP_OK;
+}
+
+int64_t snap_compress_workspace_bytes(const snap_config_t* cfg, const int32_t* cu_seqlens_host,
+                                      int32_t n_seq) {
+  int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  rc = check_cu(cu_seqlens_host, n_seq);
+  if (rc != SNAP_OK) return rc;
+  const Shape s = make_shape(cfg);
+  size_t worst = 0;
+  for (int first = 0; first < n_seq; first += kMaxBatchSeqs) {
+    const int n = n_seq - first < kMaxBatchSeqs ? n_seq - first : kMaxBatchSeqs;
+    const ChunkPlan p = plan_chunk(s, cu_seqlens_host, first, n);
+    worst = p.bytes > worst ? p.bytes : worst;
+  }
+  return (int64_t)(idx_bytes(s, n_seq) + worst + 256);
+}
+
+int64_t snap_decode_workspace_bytes(const snap_config_t* cfg, int32_t n_active) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (n_active < 0) return SNAP_ERR_INVALID_ARG;
+  const Shape s = make_shape(cfg);
+  const int nsplit = decode_generic_nsplit(s, n_active > 0 ? n_active : 1, sm_count());
+  return (int64_t)(decode_partial_floats(s, n_active, nsplit) * sizeof(float) + 256);
+}
+
+int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_obs_dev,
+                  const void* k_dev, int64_t k_token_stride, int64_t k_head_stride,
+                  const void* v_dev, int64_t v_token_stride, int64_t v_head_stride,
+                  const int32_t* cu_seqlens_host, const int32_t* slot_ids_host, int32_t n_seq,
+                  void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
+                  int32_t* valid_topk_dev, int32_t* topk_idx_dev, void* workspace_dev,
+                  size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
+  int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (!layout || !slot_ids_host) return SNAP_ERR_NULL_POINTER;
+  rc = check_cu(cu_seqlens_host, n_seq);
+  if (rc != SNAP_OK) return rc;
+  if (n_seq == 0) return SNAP_OK;
+  if (!k_dev || !k_cache_dev || !seq_len_dev || !valid_topk_dev) return SNAP_ERR_NULL_POINTER;
+  if (!cfg->v_aliases_k && (!v_dev || !v_cache_dev)) return SNAP_ERR_NULL_POINTER;
+  const Shape s = make_shape(cfg);
+  if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
+  const int eb = elt_bytes(cfg->dtype);
+  if ((k_token_stride * eb) % 16 || (k_head_stride * eb) % 16 || k_token_stride < s.d_qk)
+    return SNAP_ERR_INVALID_ARG;
+  if (!cfg->v_aliases_k && ((v_token_stride * eb) % 16 || (v_head_stride * eb) % 16 || v_token_stride < s.d_v))
+    return SNAP_ERR_INVALID_ARG;
+  {
+    std::vector<char> seen((size_t)cfg->max_seqs, 0);
+    for (int i = 0; i < n_seq; ++i) {
+      const int sl = slot_ids_host[i];
+      if (sl < 0 || sl >= cfg->max_seqs || seen[sl]) return SNAP_ERR_INVALID_ARG;
+      seen[sl] = 1;
+    }
+  }
+  const int64_t need = snap_compress_workspace_bytes(cfg, cu_seqlens_host, n_seq);
+  if (need < 0) return (int)need;
+  bool any_scored = false;
+  for (int i = 0; i < n_seq; ++i) {
+    const int L = cu_seqlens_host[i + 1] - cu_seqlens_host[i];
+    if (s.K > 0 && L - s.Ls - s.Lr > s.K) any_scored = true;
+  }
+  if (any_scored && !q_obs_dev) return SNAP_ERR_NULL_POINTER;
+  if ((any_scored || !topk_idx_dev) && s.K > 0) {
+    if (!workspace_dev) return SNAP_ERR_NULL_POINTER;
+    if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace_dev);
+  int* idx = topk_idx_dev ? topk_idx_dev : reinterpret_cast<int*>(ws);
+  char* chunk_ws = ws ? ws + idx_bytes(s, n_seq) : nullptr;
+
+  KVSource src;
+  src.k = k_dev; src.v = cfg->v_aliases_k ? nullptr : v_dev;
+  src.k_tok_stride = k_token_stride; src.k_head_stride = k_head_stride;
+  src.v_tok_stride = v_token_stride; src.v_head_stride = v_head_stride;
+
+  for (int first = 0; first < n_seq; first += kMaxBatchSeqs) {
+    const int n = n_seq - first < kMaxBatchSeqs ? n_seq - first : kMaxBatchSeqs;
+    const ChunkPlan p = plan_chunk(s, cu_seqlens_host, first, n);
+    SeqBatch b;
+    std::memset(&b, 0, sizeof(b));
+    b.n = n; b.first_seq = first;
+    for (int i = 0; i < n; ++i) {
+      b.tok_off[i] = cu_seqlens_host[first + i];
+      b.len[i] = cu_seqlens_host[first + i + 1] - cu_seqlens_host[first + i];
+      b.slot[i] = slot_ids_host[first + i];
+      b.score_idx[i] = -1;
+      if (s.K > 0 && b.len[i] - s.Ls - s.Lr > s.K) {
+        b.score_idx[i] = b.n_scored;
+        b.seq_of_score[b.n_scored++] = i;
+      }
+    }
+    ScoreBuffers buf;
+    std::memset(&buf, 0, sizeof(buf));
+    if (p.n_scored > 0) {
+      buf.part_stats = reinterpret_cast<float2*>(chunk_ws + p.part_off);
+      buf.stats = reinterpret_cast<float2*>(chunk_ws + p.stats_off);
+      buf.C = reinterpret_cast<float*>(chunk_ws + p.c_off);
+      buf.P = reinterpret_cast<float*>(chunk_ws + p.p_off);
+      buf.c_stride = p.c_stride; buf.nsplit = p.nsplit;
+      if (launch_score_simt(cfg->dtype, s, b, q_obs_dev, src, buf, st) != cudaSuccess) return SNAP_ERR_CUDA;
+    }
+    if (launch_pool_topk(s, b, buf, idx, status_dev, st) != cudaSuccess) return SNAP_ERR_CUDA;
+    if (launch_gather(cfg->dtype, s, b, src, idx, k_cache_dev, v_cache_dev, seq_len_dev,
+                      valid_topk_dev, status_dev, st) != cudaSuccess)
+      return SNAP_ERR_CUDA;
+  }
+  return SNAP_OK;
+}
+
+int snap_append_kv(const snap_config_t* cfg, const snap_layout_t* layout, const void* k_new_dev,
+                   const void* v_new_dev, const int32_t* slot_ids_dev, int32_t n_active,
+                   void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
+                   uint32_t* status_dev, void* cuda_stream) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (!layout) return SNAP_ERR_NULL_POINTER;
+  if (n_active < 0) return SNAP_ERR_INVALID_ARG;
+  if (n_active == 0) return SNAP_OK;
+  if (!k_new_dev || !slot_ids_dev || !k_cache_dev || !seq_len_dev) return SNAP_ERR_NULL_POINTER;
+  if (!cfg->v_aliases_k && (!v_new_dev || !v_cache_dev)) return SNAP_ERR_NULL_POINTER;
+  const Shape s = make_shape(cfg);
+  if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
+  if (launch_append(cfg->dtype, s, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
+                    v_cache_dev, seq_len_dev, status_dev,
+                    static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return SNAP_ERR_CUDA;
+  return SNAP_OK;
+}
+
+int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,
+                     const void* k_new_dev, const void* v_new_dev, const int32_t* slot_ids_dev,
+                     int32_t n_active, void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
+                     const int32_t* valid_topk_dev, void* out_dev, void* workspace_dev,
+                     size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (!layout) return SNAP_ERR_NULL_POINTER;
+  if (n_active < 0) return SNAP_ERR_INVALID_ARG;
+  if (n_active == 0) return SNAP_OK;
+  if (!q_dev || !slot_ids_dev || !k_cache_dev || !seq_len_dev || !valid_topk_dev || !out_dev ||
+      !workspace_dev)
+    return SNAP_ERR_NULL_POINTER;
+  if (!cfg->v_aliases_k && !v_cache_dev) return SNAP_ERR_NULL_POINTER;
+  if (k_new_dev && !cfg->v_aliases_k && !v_new_dev) return SNAP_ERR_NULL_POINTER;
+  const Shape s = make_shape(cfg);
+  if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
+  const int64_t need = snap_decode_workspace_bytes(cfg, n_active);
+  if (need < 0) return (int)need;
+  if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
+  const int nsplit = decode_generic_nsplit(s, n_active, sm_count());
+  if (launch_decode_generic(cfg->dtype, s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active,
+                            k_cache_dev, v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
+                            static_cast<float*>(workspace_dev), nsplit, status_dev,
+                            static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return SNAP_ERR_CUDA;
+  return SNAP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,87 @@
+// Internal declarations shared by the kernels and the host entry points of libsnapstream.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "snapstream.h"
+
+namespace snap {
+
+// Sequences handled by one group of compress launches; larger batches are chunked on the host.
+constexpr int kMaxBatchSeqs = 64;
+
+// Per-launch description of a chunk of prompts, passed to kernels by value.
+struct SeqBatch {
+  int n;                          // prompts in this chunk
+  int tok_off[kMaxBatchSeqs];     // index of each prompt's first token in k/v
+  int len[kMaxBatchSeqs];         // L
+  int slot[kMaxBatchSeqs];        // cache slot
+  int score_idx[kMaxBatchSeqs];   // index among the scored prompts of the chunk, -1 = not scored
+  int seq_of_score[kMaxBatchSeqs];// inverse map: scored index -> prompt index in the chunk
+  int n_scored;
+  int first_seq;                  // index of the chunk's first prompt in the caller's arrays
+};
+
+// Shape constants every kernel needs, derived from snap_config_t once on the host.
+struct Shape {
+  int Hq, Hkv, g, d_qk, d_v, Ls, Lr, K, Lo, w, pool_mode, v_aliases_k, Sc, max_seqs;
+  float scale;
+};
+
+struct KVSource {
+  const void* k;
+  const void* v;
+  long long k_tok_stride, k_head_stride, v_tok_stride, v_head_stride;   // elements
+};
+
+struct ScoreBuffers {
+  float2* part_stats;   // [n_scored*Hkv][nsplit][R]  (running max, sum of exp) per candidate split
+  float2* stats;        // [n_scored*Hkv][R]          (row max m_i, 1 / l_i)
+  float* C;             // [n_scored*Hkv][c_stride]   Eq. 1 scores summed over the head group
+  float* P;             // [n_scored*Hkv][c_stride]   pooled scores
+  int c_stride;         // floats per (prompt, kv head) row of C and P
+  int nsplit;
+};
+
+extern unsigned long long g_launches;
+inline void count_launch() { ++g_launches; }
+
+// --- launchers (each enqueues on `st` and returns cudaGetLastError()) ---
+cudaError_t launch_score_simt(int dtype, const Shape& s, const SeqBatch& b, const void* q_obs,
+                              const KVSource& src, const ScoreBuffers& buf, cudaStream_t st);
+cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffers& buf,
+                             int* idx_out, uint32_t* status, cudaStream_t st);
+cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KVSource& src,
+                          const int* idx, void* k_cache, void* v_cache, int* seq_len,
+                          int* valid_topk, uint32_t* status, cudaStream_t st);
+cudaError_t launch_append(int dtype, const Shape& s, const void* k_new, const void* v_new,
+                          const int* slot_ids, int n_active, void* k_cache, void* v_cache,
+                          int* seq_len, uint32_t* status, cudaStream_t st);
+cudaError_t launch_decode_generic(int dtype, const Shape& s, const void* q, const void* k_new,
+                                  const void* v_new, const int* slot_ids, int n_active,
+                                  void* k_cache, void* v_cache, int* seq_len,
+                                  const int* valid_topk, void* out, float* partials, int nsplit,
+                                  uint32_t* status, cudaStream_t st);
+int decode_generic_nsplit(const Shape& s, int n_active, int sm_count);
+size_t decode_partial_floats(const Shape& s, int n_active, int nsplit);
+
+// --- small device helpers ---
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) {
+  return __bfloat162float(x);
+}
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) {
+  return __float2bfloat16_rn(x);
+}
+
+// Eq. 3: cache slot written by the token at 0-indexed position t.
+__host__ __device__ __forceinline__ int ring_slot(int t, int Ls, int Lr) {
+  return t < Ls ? t : (t - Ls + Lr) % Lr + Ls;
+}
+
+}  // namespace snap

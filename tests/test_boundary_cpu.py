@@ -1,0 +1,98 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every declared
+symbol, its layout arithmetic matches the oracle's, and it rejects bad arguments."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from oracle import snapstream_oracle as orc
+from paper_2511_03092_b200 import binding as B
+from paper_2511_03092_b200 import build as snap_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    snap_build.build()
+
+
+def _cfg(**kw):
+    base = dict(n_q_heads=32, n_kv_heads=8, d_qk=128, d_v=128, dtype=B.SNAP_BF16, l_sink=4, l_recent=1024,
+                topk=4096, l_obs=64, pool_kernel=7, softmax_scale=0.088, max_seqs=3)
+    base.update(kw)
+    return B.make_config(**base)
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "snapstream.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(snap_[a-z_0-9]+)\s*\(", header))
+    assert {"snap_cache_layout", "snap_compress", "snap_append_kv", "snap_decode_attn"} <= declared
+    lib = B.lib()
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert set(B.EXPORTS) == declared
+
+
+def test_layout_matches_oracle_and_paper_totals():
+    for Ls, K, Lr, total in [(768, 6400, 1024, 8192), (512, 512, 31744, 32768), (4, 4096, 1024, 5124)]:
+        cfg = _cfg(l_sink=Ls, l_recent=Lr, topk=K, l_obs=32)
+        lay = B.snap_cache_layout(cfg)
+        ref = orc.cache_layout(Ls, Lr, K)
+        assert (lay.slots, lay.sink_off, lay.ring_off, lay.topk_off) == (
+            ref["slots"], ref["sink_off"], ref["ring_off"], ref["topk_off"])
+        assert lay.slots == total
+        assert lay.k_row_bytes == 256 and lay.k_head_stride_bytes == 256 * total
+        assert lay.k_seq_stride_bytes == 8 * 256 * total and lay.k_cache_bytes == 3 * 8 * 256 * total
+    lay = B.snap_cache_layout(_cfg(n_q_heads=128, n_kv_heads=1, d_qk=576, d_v=512, v_aliases_k=True,
+                                   l_recent=2048, topk=8192, l_obs=32))
+    assert lay.slots == 10244 and lay.k_row_bytes == 1152 and lay.v_cache_bytes == 0
+    lay = B.snap_cache_layout(_cfg(dtype=B.SNAP_F32))
+    assert lay.k_row_bytes == 512
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(n_q_heads=30), -1), (dict(l_recent=0), -1), (dict(l_obs=2000), -1), (dict(l_obs=0), -1),
+    (dict(pool_kernel=4), -1), (dict(pool_kernel=0), -1), (dict(topk=-1), -1), (dict(l_sink=-1), -1),
+    (dict(dtype=5), -1), (dict(pool_mode=3), -1), (dict(softmax_scale=0.0), -1), (dict(max_seqs=0), -1),
+    (dict(d_qk=120), -2), (dict(d_v=1024, d_qk=1024), -2), (dict(v_aliases_k=True, d_v=256), -1),
+])
+def test_invalid_configs_are_rejected(kw, code):
+    with pytest.raises(B.SnapError) as e:
+        B.snap_cache_layout(_cfg(**kw))
+    assert e.value.code == code
+    assert B.status_string(code) != "unknown status"
+
+
+def test_workspace_queries_and_argument_errors_without_gpu():
+    cfg = _cfg()
+    lay = B.snap_cache_layout(cfg)
+    assert B.snap_compress_workspace_bytes(cfg, [0, 100, 8000]) > 0
+    small = B.snap_compress_workspace_bytes(cfg, [0, 6000])
+    big = B.snap_compress_workspace_bytes(cfg, [0, 60000])
+    assert big > small
+    assert B.snap_decode_workspace_bytes(cfg, 32) >= 32 * 32 * 130 * 4
+    with pytest.raises(B.SnapError):
+        B.snap_compress_workspace_bytes(cfg, [0, 10, 5])            # decreasing offsets
+    lib = B.lib()
+    cu = (C.c_int32 * 2)(0, 9000)
+    bad_slot = (C.c_int32 * 1)(7)
+    ok_slot = (C.c_int32 * 1)(0)
+    one = C.c_void_p(256)   # never dereferenced: validation fails first
+    args = lambda slots, ws_bytes, kts=1024: (C.byref(cfg), C.byref(lay), one, one, kts, 128, one, 1024, 128,
+                                              cu, slots, 1, one, one, one, one, None, one, ws_bytes, None, None)
+    assert lib.snap_compress(*args(bad_slot, 1 << 40)) == -1                 # slot out of range
+    assert lib.snap_compress(*args(ok_slot, 16)) == -3                       # workspace too small
+    assert lib.snap_compress(*args(ok_slot, 1 << 40, kts=1023)) == -1        # stride not 16-byte multiple
+    assert lib.snap_compress(C.byref(cfg), C.byref(lay), one, None, 1024, 128, one, 1024, 128, cu, ok_slot, 1,
+                             one, one, one, one, None, one, 1 << 40, None, None) == -4
+    assert lib.snap_decode_attn(C.byref(cfg), C.byref(lay), one, None, None, one, 4, one, one, one, one, one,
+                                one, 8, None, None) == -3
+    assert lib.snap_decode_attn(C.byref(cfg), C.byref(lay), None, None, None, one, 4, one, one, one, one, one,
+                                one, 1 << 40, None, None) == -4
+    assert lib.snap_append_kv(C.byref(cfg), C.byref(lay), one, None, one, 2, one, one, one, None, None) == -4
+    assert lib.snap_append_kv(C.byref(cfg), C.byref(lay), one, one, one, -1, one, one, one, None, None) == -1
+    assert lib.snap_decode_attn(C.byref(cfg), C.byref(lay), one, None, None, one, 0, one, one, one, one, one,
+                                one, 0, None, None) == 0                     # nothing to do

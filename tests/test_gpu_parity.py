@@ -1,0 +1,189 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, element by
+element on the same seeded inputs.  Sizes span several tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import snapstream_oracle as orc
+from paper_2511_03092_b200 import binding as B
+from paper_2511_03092_b200 import synth
+from tests import _harness as H
+
+pytestmark = pytest.mark.gpu
+
+SMALL_F32 = synth.Workload("small_f32", 8, 2, 128, 128, "f32", 4, 48, 96, 16, 7, batch=1,
+                           prompt_len=(700, 700), decode_steps=8, salience="planted", n_planted=12)
+SMALL_BF16 = SMALL_F32.scaled(name="small_bf16", dtype="bf16", n_q_heads=16, n_kv_heads=4, salience="zipf")
+SMALL_MLA = synth.Workload("small_mla", 16, 1, 96, 64, "bf16", 3, 40, 64, 8, 5, batch=1,
+                           prompt_len=(500, 500), decode_steps=6, salience="planted", n_planted=8,
+                           v_aliases_k=True, softmax_scale=2.0 ** -0.5)
+
+
+def _run_compress_and_decode(wl, lengths, seed, steps, sharp=1.0, check_ring_every=1):
+    n = len(lengths)
+    layer = H.GpuLayer(wl, max_seqs=n + 2)
+    slots = [int(x) for x in np.random.default_rng(seed).permutation(n + 2)[:n]]   # not the identity map
+    prompts = [synth.make_prompt(wl, L, seed + i) for i, L in enumerate(lengths)]
+    idx = layer.compress(prompts, slots)
+    assert layer.status() == 0
+    seqs = [H.oracle_compress(wl, p) for p in prompts]
+    seq_len = layer.cache.seq_len.cpu().numpy()
+    vt = layer.cache.valid_topk.cpu().numpy()
+    for i, (seq, L) in enumerate(zip(seqs, lengths)):
+        assert seq_len[slots[i]] == L
+        assert vt[slots[i]] == orc.valid_topk(L, wl.l_sink, wl.l_recent, wl.topk)
+        if wl.topk > 0:
+            H.check_selection(idx[i], seq, wl)
+            seq.topk_pos = [idx[i][h][idx[i][h] >= 0].astype(np.int64) for h in range(wl.n_kv_heads)]
+        H.check_cache_image(layer, seq, slots[i], wl)
+    slots_dev = torch.tensor(slots, dtype=torch.int32, device="cuda")
+    for step in range(steps):
+        d = synth.make_decode_inputs(wl, n, seed, step)
+        q = (d["q"].float() * sharp).to(wl.torch_dtype)
+        out = layer.decode(q.cuda(), d["k_new"].cuda(), None if d["v_new"] is None else d["v_new"].cuda(),
+                           slots_dev)
+        for i, seq in enumerate(seqs):
+            ref = orc.decode_step(seq, synth.to_f64(q[i]), synth.to_f64(d["k_new"][i]),
+                                  synth.to_f64(d["v_new"][i]) if d["v_new"] is not None else None)
+            H.check_output(out[i], ref, wl, f"seq {i} step {step}")
+        if (step + 1) % check_ring_every == 0:
+            for i, seq in enumerate(seqs):
+                H.check_cache_image(layer, seq, slots[i], wl)
+    assert layer.status() == 0
+    np.testing.assert_array_equal(layer.cache.seq_len.cpu().numpy()[slots], [L + steps for L in lengths])
+    return layer, seqs
+
+
+@pytest.mark.parametrize("wl", [SMALL_F32, SMALL_BF16, SMALL_MLA], ids=lambda w: w.name)
+def test_compress_then_decode_matches_oracle(wl):
+    Lsr, K = wl.l_sink + wl.l_recent, wl.topk
+    # one prompt of every case: L<Ls, Ls<=L<Lsr, L==Lsr, Lsr<L<=Lsr+K, L==Lsr+K+1, long ragged ones
+    lengths = [2, wl.l_sink + 5, Lsr, Lsr + K // 2, Lsr + K, Lsr + K + 1, 333, wl.prompt_len[0], 1031]
+    _run_compress_and_decode(wl, lengths, seed=11, steps=wl.decode_steps)
+
+
+@pytest.mark.parametrize("wl", [SMALL_F32, SMALL_BF16], ids=lambda w: w.name)
+def test_sharp_softmax_outputs(wl):
+    """Queries scaled x4 make the decode softmax peaked, so outputs are O(1) and the absolute
+    tolerance bites."""
+    _run_compress_and_decode(wl, [wl.prompt_len[0], 260], seed=5, steps=4, sharp=4.0)
+
+
+def test_ring_wraps_many_times():
+    wl = SMALL_BF16.scaled(l_recent=9, l_obs=4, topk=20, l_sink=2)
+    _run_compress_and_decode(wl, [5, 11, 40, 300], seed=3, steps=40, check_ring_every=5)
+
+
+@pytest.mark.parametrize("kw", [dict(topk=0), dict(l_sink=0), dict(pool_kernel=1), dict(pool_mode="max"),
+                                dict(l_obs=1, pool_kernel=1), dict(pool_kernel=13, l_obs=32)],
+                         ids=lambda k: "-".join(f"{a}{b}" for a, b in k.items()))
+def test_degenerate_hyperparameters(kw):
+    wl = SMALL_BF16.scaled(**kw)
+    _run_compress_and_decode(wl, [wl.l_sink + wl.l_recent + wl.topk + 300, 77], seed=7, steps=3)
+
+
+@pytest.mark.parametrize("mode", ["avg", "max"])
+def test_all_equal_scores_tie_break(mode):
+    """Zero observation queries make every candidate score identical: average pooling then
+    favours candidates [r, r+K) (zero padding lowers the edges), max pooling [0, K)."""
+    wl = SMALL_BF16.scaled(pool_mode=mode)
+    L = 900
+    p = synth.make_prompt(wl, L, seed=1)
+    p["q_obs"] = torch.zeros_like(p["q_obs"])
+    layer = H.GpuLayer(wl, max_seqs=1)
+    idx = layer.compress([p], [0])
+    r = wl.pool_kernel // 2 if mode == "avg" else 0
+    for h in range(wl.n_kv_heads):
+        np.testing.assert_array_equal(idx[0][h], wl.l_sink + r + np.arange(wl.topk))
+    seq = H.oracle_compress(wl, p)
+    H.check_selection(idx[0], seq, wl)
+
+
+def test_duplicate_scores_and_exact_ties_at_the_boundary():
+    """Keys repeated verbatim give exactly equal scores; the lower index must win."""
+    wl = SMALL_BF16.scaled(pool_kernel=1, topk=50)
+    L = 600
+    p = synth.make_prompt(wl, L, seed=2)
+    lo = wl.l_sink
+    block = p["k"][lo:lo + 40].clone()
+    for rep in range(1, 12):                     # 12 identical copies of a 40-token block
+        p["k"][lo + 40 * rep: lo + 40 * (rep + 1)] = block
+    layer = H.GpuLayer(wl, max_seqs=1)
+    idx = layer.compress([p], [0])
+    seq = H.oracle_compress(wl, p)
+    for h in range(wl.n_kv_heads):
+        np.testing.assert_array_equal(idx[0][h], seq.topk_pos[h])
+
+
+def test_budget_covers_prompt_equals_dense_attention():
+    """K >= number of candidates and no new token: the compressed cache attends like the full one."""
+    wl = SMALL_F32.scaled(topk=1024)
+    L = 700
+    p = synth.make_prompt(wl, L, seed=9)
+    layer = H.GpuLayer(wl, max_seqs=1)
+    layer.compress([p], [0])
+    seq = H.oracle_compress(wl, p)
+    d = synth.make_decode_inputs(wl, 1, 9, 0)
+    slots_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = layer.decode(d["q"].cuda(), None, None, slots_dev)
+    H.check_output(out[0], orc.dense_attention(seq, synth.to_f64(d["q"][0])), wl, "dense")
+    assert int(layer.cache.seq_len[0]) == L          # attend-only leaves the length alone
+
+
+def test_append_kv_then_attend_equals_fused_step():
+    wl = SMALL_BF16
+    lengths = [3, 60, 400]
+    prompts = [synth.make_prompt(wl, L, 21 + i) for i, L in enumerate(lengths)]
+    a, b = H.GpuLayer(wl, 3), H.GpuLayer(wl, 3)
+    a.compress(prompts, [0, 1, 2]); b.compress(prompts, [0, 1, 2])
+    slots_dev = torch.arange(3, dtype=torch.int32, device="cuda")
+    for step in range(5):
+        d = synth.make_decode_inputs(wl, 3, 21, step)
+        q, kn, vn = d["q"].cuda(), d["k_new"].cuda(), d["v_new"].cuda()
+        out_a = a.decode(q, kn, vn, slots_dev)
+        B.snap_append_kv(b.cfg, b.layout, kn, vn, slots_dev, 3, b.cache.k_cache, b.cache.v_cache,
+                         b.cache.seq_len, b.cache.status)
+        out_b = b.decode(q, None, None, slots_dev)
+        torch.cuda.synchronize()
+        assert torch.equal(out_a, out_b)
+        assert torch.equal(a.cache.k_cache, b.cache.k_cache) and torch.equal(a.cache.v_cache, b.cache.v_cache)
+        assert torch.equal(a.cache.seq_len, b.cache.seq_len)
+
+
+def test_empty_sequence_and_bad_slot_are_reported_not_fatal():
+    wl = SMALL_BF16
+    layer = H.GpuLayer(wl, 2)
+    d = synth.make_decode_inputs(wl, 2, 1, 0)
+    slots_dev = torch.tensor([0, 5], dtype=torch.int32, device="cuda")      # slot 5 does not exist
+    out = layer.decode(d["q"].cuda(), None, None, slots_dev)
+    assert layer.status() & B.SNAP_DEV_BAD_SLOT
+    assert float(out.float().abs().max()) == 0.0                            # empty cache -> zeros
+
+
+def test_strided_prompt_layout():
+    """Prompt K/V that sit inside a fused [tokens, (Hq + 2 Hkv), d] QKV activation."""
+    wl = SMALL_BF16
+    L = 500
+    p = synth.make_prompt(wl, L, seed=4)
+    Hq, Hkv, d = wl.n_q_heads, wl.n_kv_heads, wl.d_qk
+    qkv = torch.zeros(L, Hq + 2 * Hkv, d, dtype=wl.torch_dtype, device="cuda")
+    qkv[:, Hq:Hq + Hkv] = p["k"].cuda(); qkv[:, Hq + Hkv:] = p["v"].cuda()
+    layer = H.GpuLayer(wl, 1)
+    cu = [0, L]
+    ws = torch.empty(B.snap_compress_workspace_bytes(layer.cfg, cu), dtype=torch.uint8, device="cuda")
+    c = layer.cache
+    B.snap_compress(layer.cfg, layer.layout, p["q_obs"].cuda(), qkv[:, Hq:Hq + Hkv], qkv[:, Hq + Hkv:], cu, [0],
+                    c.k_cache, c.v_cache, c.seq_len, c.valid_topk, None, ws, c.status)
+    ref = H.GpuLayer(wl, 1)
+    ref.compress([p], [0])
+    assert torch.equal(c.k_cache, ref.cache.k_cache) and torch.equal(c.v_cache, ref.cache.v_cache)
+
+
+def test_slot_reuse_overwrites_everything():
+    """A finished sequence's slot is simply compressed into again (continuous batching)."""
+    wl = SMALL_BF16
+    layer = H.GpuLayer(wl, 1)
+    layer.compress([synth.make_prompt(wl, 800, 1)], [0])
+    p = synth.make_prompt(wl, 30, 2)
+    layer.compress([p], [0])
+    H.check_cache_image(layer, H.oracle_compress(wl, p), 0, wl)
