@@ -1,0 +1,394 @@
+#!/usr/bin/env python
+"""Benchmark of the SnapStream hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Workload (config.workload): continuous batching of a Llama-3.1-8B-shaped attention layer in
+bf16 -- 32 resident sequences whose prompts (8k..128k tokens, seeded) were each compressed to
+a 4 + 1024 + 4096 slot cache.  One step = one pass of the whole hot path over the batch:
+sequences that finished after the previous step (seeded, 2 % per slot per step) are replaced
+by compressing a fresh prompt into their slot (scores, pooling, top-K, gather), then one
+decode step (ring append + attention over the compressed cache) runs for all 32 sequences.
+`value` counts decoded tokens per second over K such steps with every input resident in HBM;
+`e2e` repeats the steps with the step's inputs in pinned host memory and the outputs read back.
+All inputs are seeded synthetic tensors (paper_2511_03092_b200.synth).
+
+With N > 1 (torchrun) every rank runs its own 32 sequences (weak scaling, no data-path
+collective); time is the max over ranks.  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2511_03092_b200 import synth
+
+METRIC = "compressed-cache decode attn tokens/s (whole hot path: compress of replaced prompts + decode step)"
+UNIT = "tokens/s"
+SEED = 2511
+POOL_EXTRA = 16            # prompts beyond the initial batch that replacements cycle through
+DECODE_RING = 8            # distinct pre-generated decode inputs cycled through
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason sampling during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc = gpu_index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------
+
+class HotPath:
+    """Continuous-batching driver over the C ABI (argument marshalling + scheduling only)."""
+
+    def __init__(self, wl, device, seed):
+        from paper_2511_03092_b200 import binding as B
+        self.B, self.wl, self.dev = B, wl, device
+        self.cfg = B.make_config(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, d_qk=wl.d_qk, d_v=wl.d_v,
+                                 dtype=wl.torch_dtype, l_sink=wl.l_sink, l_recent=wl.l_recent, topk=wl.topk,
+                                 l_obs=wl.l_obs, pool_kernel=wl.pool_kernel, softmax_scale=wl.scale,
+                                 max_seqs=wl.batch, pool_mode=wl.pool_mode, v_aliases_k=wl.v_aliases_k)
+        self.layout = B.snap_cache_layout(self.cfg)
+        self.cache = B.alloc_cache(self.cfg, self.layout, device)
+        n_pool = wl.batch + POOL_EXTRA
+        self.lengths = synth.draw_prompt_lengths(wl, n_pool, seed)
+        self.pool = [synth.make_prompt(wl, L, seed + 17 * i, device) for i, L in enumerate(self.lengths)]
+        self.decode_in = [synth.make_decode_inputs(wl, wl.batch, seed, s, device) for s in range(DECODE_RING)]
+        ws_bytes = max(B.snap_compress_workspace_bytes(self.cfg, [0, max(self.lengths)]),
+                       B.snap_compress_workspace_bytes(self.cfg, [0] + list(np.cumsum(self.lengths[:wl.batch]))))
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+        self.dws = torch.empty(B.snap_decode_workspace_bytes(self.cfg, wl.batch), dtype=torch.uint8, device=device)
+        self.out = torch.empty(wl.batch, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device=device)
+        self.slots_dev = torch.arange(wl.batch, dtype=torch.int32, device=device)
+        self.next_prompt = wl.batch
+        self.resident = list(range(wl.batch))           # pool index held by each slot
+
+    def compress_prompt(self, p, slot):
+        c, L = self.cache, p["k"].shape[0]
+        self.B.snap_compress(self.cfg, self.layout, p["q_obs"].unsqueeze(0), p["k"], p["v"], [0, L], [slot],
+                             c.k_cache, c.v_cache, c.seq_len, c.valid_topk, None, self.ws, c.status)
+
+    def initial_fill(self):
+        for slot in range(self.wl.batch):
+            self.compress_prompt(self.pool[slot], slot)
+
+    def replace(self, slot):
+        i = self.next_prompt % len(self.pool)
+        self.next_prompt += 1
+        self.resident[slot] = i
+        self.compress_prompt(self.pool[i], slot)
+
+    def decode(self, d):
+        c = self.cache
+        self.B.snap_decode_attn(self.cfg, self.layout, d["q"], d["k_new"], d["v_new"], self.slots_dev,
+                                self.wl.batch, c.k_cache, c.v_cache, c.seq_len, c.valid_topk, self.out,
+                                self.dws, c.status)
+
+    def decode_bytes(self):
+        """Algorithmic bytes of one decode launch: every valid K and V row read once."""
+        wl = self.wl
+        eb = 2 if wl.dtype == "bf16" else 4
+        rows = sum(min(self.lengths[i] + 1, wl.slots) for i in self.resident)
+        per_row = (wl.d_qk + (0 if wl.v_aliases_k else wl.d_v)) * eb
+        return rows * wl.n_kv_heads * per_row
+
+
+def run_ours(args):
+    from paper_2511_03092_b200 import binding as B
+    B.lib()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    wl = synth.CONFIGS[2]
+    hp = HotPath(wl, dev, SEED + 1000 * rank)
+    sched = synth.continuous_batching_schedule(wl, args.warmup + args.steps + 1, SEED + rank)
+    hp.initial_fill()
+    torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def step(i, ev=None):
+        for slot in sched[i]:
+            hp.replace(slot)
+        d = hp.decode_in[i % DECODE_RING]
+        if ev is not None:
+            ev[0].record()
+        hp.decode(d)
+        if ev is not None:
+            ev[1].record()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = B.snap_kernel_launch_count()
+    bytes_acc = 0
+    n_replaced = 0
+    t0.record()
+    for i in range(args.steps):
+        step(args.warmup + i, evs[i])
+        bytes_acc += hp.decode_bytes()
+        n_replaced += len(sched[args.warmup + i])
+    t1.record()
+    barrier()
+    launches = B.snap_kernel_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms = t0.elapsed_time(t1)
+    dec_ms = [a.elapsed_time(b) for a, b in evs]
+    if world > 1:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    status = int(hp.cache.status.item())
+
+    # ---- end to end: inputs in pinned host memory, outputs read back, same steps ----
+    e2e_steps = min(args.steps, 64)
+    host_in = [{k: (v.cpu().pin_memory() if v is not None else None) for k, v in d.items()} for d in hp.decode_in]
+    host_prompts = []
+    for i in range(min(4, len(hp.pool))):
+        p = hp.pool[i]
+        host_prompts.append({k: (v.cpu().pin_memory() if torch.is_tensor(v) else v) for k, v in p.items()})
+    out_host = torch.empty(hp.out.shape, dtype=hp.out.dtype).pin_memory()
+    h2d = d2h = 0
+    hp_i = 0
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(e2e_steps):
+        for slot in sched[args.warmup + i]:
+            hpmt = host_prompts[hp_i % len(host_prompts)]; hp_i += 1
+            p = {k: (v.to(dev, non_blocking=True) if torch.is_tensor(v) else v) for k, v in hpmt.items()}
+            h2d += sum(v.numel() * v.element_size() for v in p.values() if torch.is_tensor(v))
+            hp.compress_prompt(p, slot)
+        hi = host_in[i % DECODE_RING]
+        d = {k: (v.to(dev, non_blocking=True) if v is not None else None) for k, v in hi.items()}
+        h2d += sum(v.numel() * v.element_size() for v in d.values() if v is not None)
+        hp.decode(d)
+        out_host.copy_(hp.out, non_blocking=True)
+        d2h += out_host.numel() * out_host.element_size()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_src = _peaks()
+    dec_avg_ms = sum(dec_ms) / len(dec_ms)
+    alg_bytes = bytes_acc / args.steps
+    achieved = alg_bytes / (dec_avg_ms * 1e-3) / 1e9
+    tokens = wl.batch * args.steps * world
+    line = {
+        "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "sequences_per_gpu": wl.batch, "prompt_tokens": "8192..131072 (seeded)",
+                   "cache_slots": wl.slots, "heads": f"{wl.n_q_heads}q/{wl.n_kv_heads}kv x {wl.d_qk}",
+                   "replace_prob_per_step": wl.replace_prob, "prompts_replaced_in_timed_region": n_replaced,
+                   "l2": "inputs larger than L2 (672 MB of cache read per step)", "parallelism": f"replicas x{world}"},
+        "clocks": clocks,
+        "e2e": {"value": wl.batch * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                "h2d_bytes_per_step": h2d / e2e_steps, "d2h_bytes_per_step": d2h / e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "decode attention (split + merge launches of one snap_decode_attn)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_source": peak_src, "algorithmic_bytes_per_launch": alg_bytes,
+                     "avg_launch_ms": dec_avg_ms, "traffic": None},
+        "device_status_word": status,
+    }
+    line["extra"] = {"decode_only_tokens_per_s": wl.batch / (dec_avg_ms * 1e-3),
+                     "decode_ms_median": statistics.median(dec_ms)}
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(wl, hp, sched)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------------------
+# CPU oracle legs
+# ----------------------------------------------------------------------------------------
+
+def _oracle_cfg(wl):
+    from oracle import snapstream_oracle as orc
+    return orc.OracleConfig(wl.n_q_heads, wl.n_kv_heads, wl.d_qk, wl.d_v, wl.l_sink, wl.l_recent, wl.topk,
+                            wl.l_obs, wl.pool_kernel, wl.scale, wl.pool_mode, wl.v_aliases_k)
+
+
+def _threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [t.get("num_threads", 1) for t in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(wl, hp, sched):
+    """The oracle, as it stands, on a bounded sample: the shortest pooled prompt is compressed once
+    and decoded for a few steps; per-token time = decode time + replace_prob x compress time scaled
+    to the mean prompt length."""
+    from oracle import snapstream_oracle as orc
+    i = int(np.argmin(hp.lengths))
+    p = hp.pool[i]
+    t0 = time.perf_counter()
+    seq = orc.compress(synth.to_f64(p["q_obs"]), synth.to_f64(p["k"]), synth.to_f64(p["v"]), _oracle_cfg(wl))
+    t_comp = time.perf_counter() - t0
+    n_dec = 4
+    t0 = time.perf_counter()
+    for s in range(n_dec):
+        d = hp.decode_in[s % DECODE_RING]
+        orc.decode_step(seq, synth.to_f64(d["q"][0]), synth.to_f64(d["k_new"][0]), synth.to_f64(d["v_new"][0]))
+    t_dec = (time.perf_counter() - t0) / n_dec
+    mean_len = float(np.mean(hp.lengths))
+    per_token = t_dec + wl.replace_prob * t_comp * mean_len / hp.lengths[i]
+    return {"value": 1.0 / per_token, "unit": UNIT, "cores": _threads(), "kind": "oracle",
+            "sample": f"one sequence: compress of its {hp.lengths[i]}-token prompt ({t_comp:.2f} s) and {n_dec} "
+                      f"decode steps ({t_dec * 1e3:.1f} ms each); per-token time = decode + "
+                      f"{wl.replace_prob} x compress scaled to the mean prompt length {mean_len:.0f}"}
+
+
+def run_reference(args):
+    """Times the CPU oracle on the same workload definition; each step decodes a bounded sample of
+    sequences (2 of the 32) whose prompts are shortened copies of the workload's shape."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import snapstream_oracle as orc
+    wl = synth.CONFIGS[2]
+    n_sample = 2
+    lengths = sorted(synth.draw_prompt_lengths(wl, wl.batch + POOL_EXTRA, SEED))[:n_sample]
+    cfg = _oracle_cfg(wl)
+    t0 = time.perf_counter()
+    seqs = []
+    for i, L in enumerate(lengths):
+        p = synth.make_prompt(wl, L, SEED + 17 * i)
+        seqs.append(orc.compress(synth.to_f64(p["q_obs"]), synth.to_f64(p["k"]), synth.to_f64(p["v"]), cfg))
+    t_comp = (time.perf_counter() - t0) / n_sample
+    ins = [synth.make_decode_inputs(wl, n_sample, SEED, s) for s in range(DECODE_RING)]
+
+    def step(i):
+        d = ins[i % DECODE_RING]
+        for j, seq in enumerate(seqs):
+            orc.decode_step(seq, synth.to_f64(d["q"][j]), synth.to_f64(d["k_new"][j]), synth.to_f64(d["v_new"][j]))
+
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    dt = time.perf_counter() - t0
+    mean_len = float(np.mean(synth.draw_prompt_lengths(wl, wl.batch + POOL_EXTRA, SEED)))
+    per_token = dt / (args.steps * n_sample) + wl.replace_prob * t_comp * mean_len / float(np.mean(lengths))
+    value = 1.0 / per_token
+    sample = (f"{n_sample} of {wl.batch} sequences per step (the two shortest prompts, {lengths} tokens); compress "
+              f"measured once per prompt ({t_comp:.2f} s) and charged at {wl.replace_prob} per token, scaled to "
+              f"the mean prompt length")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": _threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps > 64:
+            args.steps = 64
+        run_reference(args)
+    else:
+        if args.warmup < 3:
+            args.warmup = 3
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

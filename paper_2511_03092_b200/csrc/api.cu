@@ -100,6 +100,22 @@ int check_cu(const int32_t* cu, int n_seq) {
   return SNAP_OK;
 }
 
+struct DecodePlan { bool gqa; int nsplit; size_t floats; };
+
+DecodePlan plan_decode(int dtype, const Shape& s, int n_active) {
+  DecodePlan p;
+  const int n = n_active > 0 ? n_active : 1;
+  p.gqa = decode_gqa_supported(dtype, s);
+  if (p.gqa) {
+    p.nsplit = decode_gqa_nsplit(s, n, sm_count());
+    p.floats = decode_gqa_partial_floats(s, n_active, p.nsplit);
+  } else {
+    p.nsplit = decode_generic_nsplit(s, n, sm_count());
+    p.floats = decode_partial_floats(s, n_active, p.nsplit);
+  }
+  return p;
+}
+
 size_t idx_bytes(const Shape& s, int n_seq) {
   return align_up((size_t)n_seq * s.Hkv * (s.K > 0 ? s.K : 1) * sizeof(int));
 }
@@ -166,8 +182,8 @@ int64_t snap_decode_workspace_bytes(const snap_config_t* cfg, int32_t n_active) 
   if (rc != SNAP_OK) return rc;
   if (n_active < 0) return SNAP_ERR_INVALID_ARG;
   const Shape s = make_shape(cfg);
-  const int nsplit = decode_generic_nsplit(s, n_active > 0 ? n_active : 1, sm_count());
-  return (int64_t)(decode_partial_floats(s, n_active, nsplit) * sizeof(float) + 256);
+  const DecodePlan p = plan_decode(cfg->dtype, s, n_active);
+  return (int64_t)(p.floats * sizeof(float) + 256);
 }
 
 int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_obs_dev,
@@ -296,13 +312,18 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
   const int64_t need = snap_decode_workspace_bytes(cfg, n_active);
   if (need < 0) return (int)need;
   if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
-  const int nsplit = decode_generic_nsplit(s, n_active, sm_count());
-  if (launch_decode_generic(cfg->dtype, s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active,
-                            k_cache_dev, v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
-                            static_cast<float*>(workspace_dev), nsplit, status_dev,
-                            static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
-    return SNAP_ERR_CUDA;
-  return SNAP_OK;
+  const DecodePlan p = plan_decode(cfg->dtype, s, n_active);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e;
+  if (p.gqa)
+    e = launch_decode_gqa(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
+                          v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
+                          static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
+  else
+    e = launch_decode_generic(cfg->dtype, s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active,
+                              k_cache_dev, v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
+                              static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
+  return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
 }
 
 }  // extern "C"

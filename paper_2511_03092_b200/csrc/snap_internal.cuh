@@ -66,6 +66,14 @@ cudaError_t launch_decode_generic(int dtype, const Shape& s, const void* q, cons
                                   uint32_t* status, cudaStream_t st);
 int decode_generic_nsplit(const Shape& s, int n_active, int sm_count);
 size_t decode_partial_floats(const Shape& s, int n_active, int nsplit);
+// grouped-query bf16, 128-wide heads: bulk-async staged streaming kernel
+bool decode_gqa_supported(int dtype, const Shape& s);
+int decode_gqa_nsplit(const Shape& s, int n_active, int sm_count);
+size_t decode_gqa_partial_floats(const Shape& s, int n_active, int nsplit);
+cudaError_t launch_decode_gqa(const Shape& s, const void* q, const void* k_new, const void* v_new,
+                              const int* slot_ids, int n_active, void* k_cache, void* v_cache,
+                              int* seq_len, const int* valid_topk, void* out, float* partials,
+                              int nsplit, uint32_t* status, cudaStream_t st);
 
 // --- small device helpers ---
 template <typename T> __device__ __forceinline__ float to_f32(T x);

@@ -187,3 +187,17 @@ def test_slot_reuse_overwrites_everything():
     p = synth.make_prompt(wl, 30, 2)
     layer.compress([p], [0])
     H.check_cache_image(layer, H.oracle_compress(wl, p), 0, wl)
+
+
+@pytest.mark.parametrize("hq,hkv", [(8, 4), (32, 4), (4, 4)], ids=["g2", "g8", "g1"])
+def test_group_sizes(hq, hkv):
+    wl = SMALL_BF16.scaled(n_q_heads=hq, n_kv_heads=hkv)
+    _run_compress_and_decode(wl, [wl.prompt_len[0], 50, 3], seed=13, steps=5)
+
+
+def test_many_sequences_ragged_decode():
+    """More sequences than one launch chunk holds, lengths from empty-ish to several tiles."""
+    wl = SMALL_BF16.scaled(topk=64, l_recent=32)
+    rng = np.random.default_rng(0)
+    lengths = [int(x) for x in rng.integers(1, 400, size=70)]
+    _run_compress_and_decode(wl, lengths, seed=17, steps=3, check_ring_every=3)
