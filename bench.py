@@ -372,6 +372,72 @@ def run_reference(args):
     }), flush=True)
 
 
+def run_case(args):
+    """Small single-kernel-family cases for profiler captures (bounded device memory):
+    `decode`   32 sequences with 8192-token prompts compressed, then a few decode steps
+               (672 MB of cache read per step, ~1.5 GB resident);
+    `compress` one prompt of --case-len tokens compressed a few times."""
+    from paper_2511_03092_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    wl = synth.CONFIGS[2]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if args.case == "decode":
+        wl = wl.scaled(prompt_len=(8192, 8192))
+        hp = HotPath.__new__(HotPath)
+        hp.B, hp.wl, hp.dev = B, wl, dev
+        hp.cfg = B.make_config(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, d_qk=wl.d_qk, d_v=wl.d_v,
+                               dtype=wl.torch_dtype, l_sink=wl.l_sink, l_recent=wl.l_recent, topk=wl.topk,
+                               l_obs=wl.l_obs, pool_kernel=wl.pool_kernel, softmax_scale=wl.scale,
+                               max_seqs=wl.batch)
+        hp.layout = B.snap_cache_layout(hp.cfg)
+        hp.cache = B.alloc_cache(hp.cfg, hp.layout, dev)
+        hp.lengths = [8192] * wl.batch
+        hp.resident = list(range(wl.batch))
+        hp.ws = torch.empty(B.snap_compress_workspace_bytes(hp.cfg, [0, 8192]), dtype=torch.uint8, device=dev)
+        hp.dws = torch.empty(B.snap_decode_workspace_bytes(hp.cfg, wl.batch), dtype=torch.uint8, device=dev)
+        hp.out = torch.empty(wl.batch, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device=dev)
+        hp.slots_dev = torch.arange(wl.batch, dtype=torch.int32, device=dev)
+        for slot in range(wl.batch):
+            hp.compress_prompt(synth.make_prompt(wl, 8192, SEED + slot, dev), slot)
+        ins = [synth.make_decode_inputs(wl, wl.batch, SEED, s, dev) for s in range(2)]
+        for s in range(args.warmup):
+            hp.decode(ins[s % 2])
+        torch.cuda.synchronize()
+        t0.record()
+        for s in range(args.steps):
+            hp.decode(ins[s % 2])
+        t1.record()
+        torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / args.steps
+        print(json.dumps({"case": "decode", "ms_per_launch": ms, "bytes": hp.decode_bytes(),
+                          "GBps": hp.decode_bytes() / ms / 1e6, "status": int(hp.cache.status.item())}))
+    else:
+        L = args.case_len
+        wl = wl.scaled(prompt_len=(L, L), batch=1)
+        hp = HotPath.__new__(HotPath)
+        hp.B, hp.wl, hp.dev = B, wl, dev
+        hp.cfg = B.make_config(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, d_qk=wl.d_qk, d_v=wl.d_v,
+                               dtype=wl.torch_dtype, l_sink=wl.l_sink, l_recent=wl.l_recent, topk=wl.topk,
+                               l_obs=wl.l_obs, pool_kernel=wl.pool_kernel, softmax_scale=wl.scale, max_seqs=1)
+        hp.layout = B.snap_cache_layout(hp.cfg)
+        hp.cache = B.alloc_cache(hp.cfg, hp.layout, dev)
+        hp.ws = torch.empty(B.snap_compress_workspace_bytes(hp.cfg, [0, L]), dtype=torch.uint8, device=dev)
+        p = synth.make_prompt(wl, L, SEED, dev)
+        for s in range(args.warmup):
+            hp.compress_prompt(p, 0)
+        torch.cuda.synchronize()
+        t0.record()
+        for s in range(args.steps):
+            hp.compress_prompt(p, 0)
+        t1.record()
+        torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / args.steps
+        flops = 2 * 2.0 * wl.n_q_heads * wl.l_obs * (L - wl.l_sink - wl.l_recent) * wl.d_qk
+        print(json.dumps({"case": "compress", "prompt_tokens": L, "us_per_prompt": ms * 1e3,
+                          "score_TFLOPs": flops / ms / 1e9, "status": int(hp.cache.status.item())}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -379,10 +445,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", choices=["decode", "compress"], default=None,
+                    help="small single-kernel-family case for profiler captures")
+    ap.add_argument("--case-len", type=int, default=131072)
     args = ap.parse_args()
-    if args.impl == "reference":
-        if args.steps > 64:
-            args.steps = 64
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         if args.warmup < 3:

@@ -1,31 +1,38 @@
 // Decode attention over the compressed cache (Section 3.3) for grouped-query bf16 layers with
 // 128-wide heads -- the HBM-bound kernel of the decode step.
 //
-// Split-K flash decoding.  Grid = (splits, KV heads, sequences); a CTA of 4 warps streams its
-// share of the valid cache rows ([0, min(len, Lsr)) then [Lsr, Lsr + valid_topk)) through a
-// ring of shared-memory stages filled by bulk async copies (cp.async.bulk + mbarrier
-// transaction counts; rows of one KV head are contiguous, so a tile is one or two copies per
-// tensor).  K and V rows are each read from HBM exactly once.
+// Split-K flash decoding.  Grid = (splits, KV heads, sequences).  A CTA's share of the valid
+// cache rows ([0, min(len, Lsr)) then [Lsr, Lsr + valid_topk)) is cut into 16-row tiles that
+// are dealt round-robin to its warps.  Every warp runs its own pipeline: a private ring of
+// shared-memory stages filled by bulk async copies (cp.async.bulk completing on the warp's own
+// mbarriers; the rows of one KV head are contiguous, so a tile is one or two copies per
+// tensor), with no CTA-wide barrier in the loop.  K and V rows are read from HBM exactly once.
 //
-// Per 64-row tile each warp owns 16 rows.  A half-warp covers one 256-byte row with 128-bit
-// shared loads (lane = 8 dims); the lane-partial dot products of 8 rows x G heads are reduced
-// with a transposing shuffle network (each step halves the values a lane holds), which costs
-// ~4x fewer shuffles than reducing every dot product separately and leaves one row's logits in
-// each lane.  Online softmax is per warp (running max in the log2 domain, per-lane partial
-// sums), probabilities go through a small per-warp shared buffer and are re-read as broadcasts
-// for the P.V accumulation, where a lane owns 8 output dims of all G heads.  Warps are merged
-// once at the end; splits are merged by a second kernel, which also advances the sequence
-// length when a token was appended.
+// Within a tile a half-warp covers one 256-byte row with 128-bit shared loads (lane = 8 dims).
+// The lane-partial dot products of 8 rows x G heads are reduced with a transposing shuffle
+// network (each step halves the values a lane holds), which needs ~4x fewer shuffles than
+// reducing each dot product on its own and leaves one row's logits in each lane.  Online
+// softmax is per warp (running max in the log2 domain, per-lane partial sums); probabilities
+// go through a small per-half-warp shared buffer and come back as broadcasts for the P.V
+// accumulation, where a lane owns 8 output dims of all G heads.  All multiply-adds are packed
+// two-wide (fma.rn.f32x2), halving the issue slots of the arithmetic.  Warps are merged once at
+// the end; splits are merged by a second kernel, which also advances the sequence length when
+// a token was appended.
 //
 // Fused append (Eq. 3): the CTA whose range contains the new token's slot stores the new K/V
-// row to the cache and patches its staged tile, so the stale row is never used.
+// row to the cache, and the warp that stages that row patches its copy, so the stale row is
+// never used.
+#include <cstdlib>
+
 #include "snap_internal.cuh"
 
 namespace snap {
 namespace {
 
-constexpr int D = 128, TILE = 64, NSTAGE = 3, NT = 128, NWARP = 4;
-constexpr int ROW_B = D * 2, TILE_B = TILE * ROW_B, STAGE_B = 2 * TILE_B;
+typedef unsigned long long u64;
+
+constexpr int D = 128, WT = 16, NSTAGE = 2, NWARP = 4, NT = NWARP * 32;
+constexpr int ROW_B = D * 2, WT_B = WT * ROW_B, STAGE_B = 2 * WT_B;   // stage = K tile | V tile
 constexpr int PS = D + 2;                       // floats per partial: m, l, acc[D]
 constexpr unsigned kWaitLimit = 1u << 22;       // bounded spin on an mbarrier
 
@@ -80,32 +87,51 @@ __device__ __forceinline__ void issue_tile(uint32_t stage, uint32_t bar, const c
   if (va < e1) {
     const unsigned bytes = (unsigned)(e1 - va) * ROW_B;
     bulk_g2s(stage, kc + (long long)va * ROW_B, bytes, bar);
-    bulk_g2s(stage + TILE_B, vc + (long long)va * ROW_B, bytes, bar);
+    bulk_g2s(stage + WT_B, vc + (long long)va * ROW_B, bytes, bar);
   }
   const int s2 = max(va, n_low);
   if (s2 < vb) {
     const unsigned bytes = (unsigned)(vb - s2) * ROW_B, off = (unsigned)(s2 - va) * ROW_B;
     const long long src = (long long)(Lsr + s2 - n_low) * ROW_B;
     bulk_g2s(stage + off, kc + src, bytes, bar);
-    bulk_g2s(stage + TILE_B + off, vc + src, bytes, bar);
+    bulk_g2s(stage + WT_B + off, vc + src, bytes, bar);
   }
 }
 
-__device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
-  f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
-  f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
-  f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
-  f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
+// packed pairs of floats in one 64-bit register
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+  u64 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 mul2(u64 a, u64 b) {
+  u64 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 8 bf16 (one 128-bit load) -> 4 packed float pairs (elements 2c, 2c+1)
+__device__ __forceinline__ void unpack8(const uint4& u, u64 (&f)[4]) {
+  f[0] = pack2(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u));
+  f[1] = pack2(__uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+  f[2] = pack2(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u));
+  f[3] = pack2(__uint_as_float(u.w << 16), __uint_as_float(u.w & 0xffff0000u));
 }
 
 template <int G>
-__global__ void __launch_bounds__(NT, 2) decode_gqa_kernel(const FastArgs a) {
+__global__ void __launch_bounds__(NT, (G == 8 ? 2 : 3)) decode_gqa_kernel(const FastArgs a) {
   constexpr int VPL = G / 2;                    // logits a lane holds after the reduction
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  unsigned char* stages = smem_raw;                                   // NSTAGE x (K tile | V tile)
-  float* pbuf = reinterpret_cast<float*>(smem_raw + NSTAGE * STAGE_B);  // [NWARP][2][8][G]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(pbuf + NWARP * 16 * G);
-  __shared__ int abort_flag;
+  // [NWARP][NSTAGE] stages | [NWARP][2][8][G][2] probabilities | [NWARP][NSTAGE] mbarriers
+  float* pbuf = reinterpret_cast<float*>(smem_raw + NWARP * NSTAGE * STAGE_B);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(pbuf + NWARP * 2 * 8 * G * 2);
 
   const int sp = blockIdx.x, kvh = blockIdx.y, i = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, hw = lane >> 4, l16 = lane & 15;
@@ -122,100 +148,102 @@ __global__ void __launch_bounds__(NT, 2) decode_gqa_kernel(const FastArgs a) {
   } else if (tid == 0 && sp == 0 && kvh == 0 && a.status) {
     atomicOr(a.status, SNAP_DEV_BAD_SLOT);
   }
-  // even split of the tiles of this (sequence, KV head) over the splits
-  const int ntiles = (n_valid + TILE - 1) / TILE;
+  // even split of this (sequence, KV head)'s 16-row tiles over the splits
+  const int ntiles = (n_valid + WT - 1) / WT;
   const int t_begin = (int)((long long)ntiles * sp / a.nsplit);
   const int t_end = (int)((long long)ntiles * (sp + 1) / a.nsplit);
-  const int v0 = t_begin * TILE, v1 = min(n_valid, t_end * TILE);
-  const int T = t_end - t_begin;
+  const int v1 = min(n_valid, t_end * WT);
+  // this warp's tiles: t_begin + w, t_begin + w + NWARP, ...
+  const int T = t_end - t_begin > w ? (t_end - t_begin - w + NWARP - 1) / NWARP : 0;
 
   char* kc = a.kc + slot * a.seq_b + kvh * a.head_b;
   char* vc = a.vc + slot * a.seq_b + kvh * a.head_b;
   const __nv_bfloat16* kn = a.k_new ? a.k_new + ((long long)i * a.Hkv + kvh) * D : nullptr;
   const __nv_bfloat16* vn = a.v_new ? a.v_new + ((long long)i * a.Hkv + kvh) * D : nullptr;
 
-  const uint32_t stage0 = smem_u32(stages), bar0 = smem_u32(bars);
-  if (tid == 0) {
-    abort_flag = 0;
+  unsigned char* wstages = smem_raw + w * NSTAGE * STAGE_B;
+  const uint32_t stage0 = smem_u32(wstages), bar0 = smem_u32(bars + w * NSTAGE);
+  if (lane == 0) {
     for (int s = 0; s < NSTAGE; ++s) mbar_init(bar0 + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  __syncthreads();
-  if (tid == 0) {
-    for (int s = 0; s < NSTAGE && s < T; ++s)
-      issue_tile(stage0 + s * STAGE_B, bar0 + 8 * s, kc, vc, v0 + s * TILE, min(v1, v0 + (s + 1) * TILE),
-                 n_low, Lsr);
+  __syncwarp();
+  if (lane == 0) {
+    for (int s = 0; s < NSTAGE && s < T; ++s) {
+      const int va = (t_begin + w + s * NWARP) * WT;
+      issue_tile(stage0 + s * STAGE_B, bar0 + 8 * s, kc, vc, va, min(v1, va + WT), n_low, Lsr);
+    }
   }
-  // the owner of the new token's slot stores it (its staged copy is patched below)
-  const bool owns_new = new_slot >= v0 && new_slot < v1;
-  if (owns_new && w == 0) {
+  // the CTA that owns the new token's slot stores it (the staged copy is patched below)
+  if (new_slot >= t_begin * WT && new_slot < v1 && w == 0) {
     const uint4* srcp = reinterpret_cast<const uint4*>(hw == 0 ? kn : vn);
     char* dst = (hw == 0 ? kc : vc) + (long long)new_slot * ROW_B;
     reinterpret_cast<uint4*>(dst)[l16] = srcp[l16];
   }
 
   // query rows of the group, pre-scaled so that exp2 can be used directly
-  float q[G][8];
+  u64 q2[G][4];
   {
     const __nv_bfloat16* qp = a.q + ((long long)i * a.Hq + (long long)kvh * G) * D + l16 * 8;
+    const u64 sc2 = pack2(a.scale_log2, a.scale_log2);
 #pragma unroll
     for (int h = 0; h < G; ++h) {
       const uint4 u = *reinterpret_cast<const uint4*>(qp + h * D);
-      unpack8(u, q[h]);
+      unpack8(u, q2[h]);
 #pragma unroll
-      for (int c = 0; c < 8; ++c) q[h][c] *= a.scale_log2;
+      for (int c = 0; c < 4; ++c) q2[h][c] = mul2(q2[h][c], sc2);
     }
   }
-  float acc[G][8], m_run[G], l_lane[VPL];
+  u64 acc2[G][4];
+  float m_run[G], l_lane[VPL];
 #pragma unroll
   for (int h = 0; h < G; ++h) {
     m_run[h] = -INFINITY;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) acc[h][c] = 0.f;
+    for (int c = 0; c < 4; ++c) acc2[h][c] = 0ull;
   }
 #pragma unroll
   for (int e = 0; e < VPL; ++e) l_lane[e] = 0.f;
-  float* pw = pbuf + (w * 2 + hw) * 8 * G;      // this half-warp's probabilities [8][G]
+  float* pw = pbuf + (w * 2 + hw) * 8 * G * 2;  // this half-warp's probabilities [8][G][2]
+  bool timed_out = false;
 
-  for (int t = 0; t < T; ++t) {
-    const int s = t % NSTAGE;
-    const unsigned parity = (unsigned)(t / NSTAGE) & 1u;
-    if (!mbar_wait(bar0 + 8 * s, parity)) {
-      abort_flag = 1;
-      if (a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
-    }
-    const int va = v0 + t * TILE;
-    const int nrows = min(TILE, v1 - va);
-    unsigned char* sK = stages + s * STAGE_B;
-    unsigned char* sV = sK + TILE_B;
+  for (int n = 0; n < T; ++n) {
+    const int s = n % NSTAGE;
+    const unsigned parity = (unsigned)(n / NSTAGE) & 1u;
+    const bool landed = mbar_wait(bar0 + 8 * s, parity);
+    if (__any_sync(0xffffffffu, !landed)) { timed_out = true; break; }
+    const int va = (t_begin + w + n * NWARP) * WT;
+    const int nrows = min(WT, v1 - va);
+    unsigned char* sK = wstages + s * STAGE_B;
+    unsigned char* sV = sK + WT_B;
     const bool patch = new_slot >= va && new_slot < va + nrows;
-    if (patch || nrows < TILE) {                 // rare: new-token row, or the ragged last tile
-      if (patch && w == 0) {
-        const uint4* srcp = reinterpret_cast<const uint4*>(hw == 0 ? kn : vn);
-        reinterpret_cast<uint4*>((hw == 0 ? sK : sV) + (new_slot - va) * ROW_B)[l16] = srcp[l16];
-      }
-      for (int e = tid; e < (TILE - nrows) * (ROW_B / 16); e += NT) {      // zero rows past the end
+    if (patch || nrows < WT) {                   // rare: new-token row, or the ragged last tile
+      if (patch)
+        reinterpret_cast<uint4*>((hw == 0 ? sK : sV) + (new_slot - va) * ROW_B)[l16] =
+            reinterpret_cast<const uint4*>(hw == 0 ? kn : vn)[l16];
+      for (int e = lane; e < (WT - nrows) * (ROW_B / 16); e += 32) {      // zero rows past the end
         reinterpret_cast<uint4*>(sK + nrows * ROW_B)[e] = make_uint4(0, 0, 0, 0);
         reinterpret_cast<uint4*>(sV + nrows * ROW_B)[e] = make_uint4(0, 0, 0, 0);
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncthreads();
+      __syncwarp();
     }
 
     // ---- logits: lane-partial dot products of 8 rows x G heads ----
     float part[8 * G];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const int row = 16 * w + 2 * j + hw;
-      const uint4 u = *reinterpret_cast<const uint4*>(sK + row * ROW_B + l16 * 16);
-      float kf[8];
-      unpack8(u, kf);
+      const uint4 u = *reinterpret_cast<const uint4*>(sK + (2 * j + hw) * ROW_B + l16 * 16);
+      u64 k2[4];
+      unpack8(u, k2);
 #pragma unroll
       for (int h = 0; h < G; ++h) {
-        float sacc = q[h][0] * kf[0];
+        u64 s2 = mul2(q2[h][0], k2[0]);
 #pragma unroll
-        for (int c = 1; c < 8; ++c) sacc = fmaf(q[h][c], kf[c], sacc);
-        part[j * G + h] = sacc;
+        for (int c = 1; c < 4; ++c) s2 = fma2(q2[h][c], k2[c], s2);
+        float lo, hi;
+        unpack2(s2, lo, hi);
+        part[j * G + h] = lo + hi;
       }
     }
     // transposing reduction over the 16 lanes of a half-warp
@@ -229,119 +257,128 @@ __global__ void __launch_bounds__(NT, 2) decode_gqa_kernel(const FastArgs a) {
         part[e] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
       }
     }
-    // lane now holds row (16w + 2*jrow + hw), heads odd*VPL .. odd*VPL+VPL-1
-    const bool row_ok = 16 * w + 2 * jrow + hw < nrows;
-    float mx[VPL];
+    // lane now holds row 2*jrow + hw of the tile, heads odd*VPL .. odd*VPL + VPL-1
+    const bool row_ok = 2 * jrow + hw < nrows;
+    // The running maxima are only a reference point for exp2, so they are refreshed lazily:
+    // a warp vote detects a logit more than 8 (a factor 256) above the reference, and only then
+    // is the max reduced across the warp and the accumulators rescaled.
+    bool need = false;
 #pragma unroll
     for (int e = 0; e < VPL; ++e) {
       part[e] = row_ok ? part[e] : -INFINITY;
-      mx[e] = part[e];
-#pragma unroll
-      for (int o = 2; o <= 16; o <<= 1) mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], o));
+      need |= part[e] > (odd ? m_run[VPL + e] : m_run[e]) + 8.f;
     }
-    float m_use[G];
-    bool changed = false;
+    if (__any_sync(0xffffffffu, need)) {
+      float mx[VPL], m_use[G];
 #pragma unroll
-    for (int e = 0; e < VPL; ++e) {
-      const float other = __shfl_xor_sync(0xffffffffu, mx[e], 1);
-      const float lo = odd ? other : mx[e], hi = odd ? mx[e] : other;
-      const float n_lo = fmaxf(m_run[e], lo), n_hi = fmaxf(m_run[VPL + e], hi);
-      changed |= (n_lo > m_run[e]) | (n_hi > m_run[VPL + e]);
-      m_use[e] = n_lo; m_use[VPL + e] = n_hi;
-    }
-    if (changed) {                               // warp-uniform: every lane sees the same maxima
+      for (int e = 0; e < VPL; ++e) {
+        mx[e] = part[e];
+#pragma unroll
+        for (int o = 2; o <= 16; o <<= 1) mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], o));
+      }
+#pragma unroll
+      for (int e = 0; e < VPL; ++e) {
+        const float other = __shfl_xor_sync(0xffffffffu, mx[e], 1);
+        m_use[e] = fmaxf(m_run[e], odd ? other : mx[e]);
+        m_use[VPL + e] = fmaxf(m_run[VPL + e], odd ? mx[e] : other);
+      }
       float al[G];
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         al[h] = m_run[h] == -INFINITY ? 0.f : exp2f(m_run[h] - m_use[h]);
         m_run[h] = m_use[h];
+        const u64 al2 = pack2(al[h], al[h]);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) acc[h][c] *= al[h];
+        for (int c = 0; c < 4; ++c) acc2[h][c] = mul2(acc2[h][c], al2);
       }
 #pragma unroll
       for (int e = 0; e < VPL; ++e) l_lane[e] *= odd ? al[VPL + e] : al[e];
     }
-    float pv[VPL];
 #pragma unroll
     for (int e = 0; e < VPL; ++e) {
       const float mh = odd ? m_run[VPL + e] : m_run[e];
-      pv[e] = exp2f(part[e] - (mh == -INFINITY ? 0.f : mh));
-      l_lane[e] += pv[e];
-    }
-    if (VPL == 2) {
-      *reinterpret_cast<float2*>(pw + jrow * G + odd * VPL) = make_float2(pv[0], pv[VPL - 1]);
-    } else {
-#pragma unroll
-      for (int e = 0; e < VPL; ++e) pw[jrow * G + odd * VPL + e] = pv[e];
+      const float p = exp2f(part[e] - (mh == -INFINITY ? 0.f : mh));
+      l_lane[e] += p;
+      *reinterpret_cast<float2*>(pw + (jrow * G + odd * VPL + e) * 2) = make_float2(p, p);
     }
     __syncwarp();
     // ---- P.V: a lane owns 8 output dims of all G heads ----
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const int row = 16 * w + 2 * j + hw;
-      const uint4 u = *reinterpret_cast<const uint4*>(sV + row * ROW_B + l16 * 16);
-      float vf[8];
-      unpack8(u, vf);
-      float pj[G];
-      if (G == 4) {
-        const float4 p4 = *reinterpret_cast<const float4*>(pw + j * G);
-        pj[0] = p4.x; pj[1] = p4.y; pj[2] = p4.z; pj[G - 1] = p4.w;
-      } else {
+      const uint4 u = *reinterpret_cast<const uint4*>(sV + (2 * j + hw) * ROW_B + l16 * 16);
+      u64 v2[4];
+      unpack8(u, v2);
+      const ulonglong2* pp = reinterpret_cast<const ulonglong2*>(pw + j * G * 2);
 #pragma unroll
-        for (int h = 0; h < G; ++h) pj[h] = pw[j * G + h];
+      for (int hp = 0; hp < G / 2; ++hp) {
+        const ulonglong2 p2 = pp[hp];             // (p,p) of heads 2hp and 2hp+1
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          acc2[2 * hp][c] = fma2(p2.x, v2[c], acc2[2 * hp][c]);
+          acc2[2 * hp + 1][c] = fma2(p2.y, v2[c], acc2[2 * hp + 1][c]);
+        }
       }
-#pragma unroll
-      for (int h = 0; h < G; ++h)
-#pragma unroll
-        for (int c = 0; c < 8; ++c) acc[h][c] = fmaf(pj[h], vf[c], acc[h][c]);
     }
-    __syncthreads();
-    if (abort_flag) break;
-    if (tid == 0 && t + NSTAGE < T) {
-      const int nv = v0 + (t + NSTAGE) * TILE;
-      issue_tile(stage0 + s * STAGE_B, bar0 + 8 * s, kc, vc, nv, min(v1, nv + TILE), n_low, Lsr);
+    __syncwarp();
+    if (lane == 0 && n + NSTAGE < T) {
+      const int nv = (t_begin + w + (n + NSTAGE) * NWARP) * WT;
+      issue_tile(stage0 + s * STAGE_B, bar0 + 8 * s, kc, vc, nv, min(v1, nv + WT), n_low, Lsr);
     }
   }
+  if (timed_out) {
+    if (a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
+    // give copies still in flight a bounded chance to land before the stage memory is reused
+    for (int s = 0; s < NSTAGE; ++s) (void)mbar_wait(bar0 + 8 * s, 0u);
+  }
 
-  // ---- merge the two half-warps, then the four warps, and write the split's partial ----
+  // ---- merge the two half-warps, then the warps, and write the split's partial ----
+  float acc[G][8];
 #pragma unroll
   for (int h = 0; h < G; ++h)
 #pragma unroll
-    for (int c = 0; c < 8; ++c) acc[h][c] += __shfl_xor_sync(0xffffffffu, acc[h][c], 16);
+    for (int c = 0; c < 4; ++c) {
+      unpack2(acc2[h][c], acc[h][2 * c], acc[h][2 * c + 1]);
+      acc[h][2 * c] += __shfl_xor_sync(0xffffffffu, acc[h][2 * c], 16);
+      acc[h][2 * c + 1] += __shfl_xor_sync(0xffffffffu, acc[h][2 * c + 1], 16);
+    }
 #pragma unroll
   for (int e = 0; e < VPL; ++e)
 #pragma unroll
     for (int o = 2; o <= 16; o <<= 1) l_lane[e] += __shfl_xor_sync(0xffffffffu, l_lane[e], o);
-  float* wm = reinterpret_cast<float*>(stages);            // [NWARP][G]
-  float* wl = wm + NWARP * G;                              // [NWARP][G]
-  float* wacc = wl + NWARP * G;                            // [NWARP][G][D]
+  // every copy this warp issued has been consumed, so its own stage memory is free
+  float* wm = reinterpret_cast<float*>(wstages);           // [G] max, [G] sum, [G][D] acc
+  float* wl = wm + G;
+  float* wacc = wl + G;
+  __syncwarp();
   if (lane < 2) {
 #pragma unroll
     for (int e = 0; e < VPL; ++e) {
-      wm[w * G + lane * VPL + e] = lane ? m_run[VPL + e] : m_run[e];
-      wl[w * G + lane * VPL + e] = l_lane[e];
+      wm[lane * VPL + e] = lane ? m_run[VPL + e] : m_run[e];
+      wl[lane * VPL + e] = l_lane[e];
     }
   }
   if (hw == 0) {
 #pragma unroll
     for (int h = 0; h < G; ++h)
 #pragma unroll
-      for (int c = 0; c < 8; ++c) wacc[(w * G + h) * D + l16 * 8 + c] = acc[h][c];
+      for (int c = 0; c < 8; ++c) wacc[h * D + l16 * 8 + c] = acc[h][c];
   }
   __syncthreads();
   float* part_out = a.partials + (((long long)i * a.Hq + (long long)kvh * G) * a.nsplit + sp) * PS;
+  constexpr int WSTRIDE = NSTAGE * STAGE_B / 4;            // floats between two warps' regions
+  const float* base = reinterpret_cast<const float*>(smem_raw);
 #pragma unroll
   for (int h = 0; h < G; ++h) {
     float M = -INFINITY;
 #pragma unroll
-    for (int ww = 0; ww < NWARP; ++ww) M = fmaxf(M, wm[ww * G + h]);
+    for (int ww = 0; ww < NWARP; ++ww) M = fmaxf(M, base[ww * WSTRIDE + h]);
     float L = 0.f, O = 0.f;
 #pragma unroll
     for (int ww = 0; ww < NWARP; ++ww) {
-      const float mw = wm[ww * G + h];
+      const float mw = base[ww * WSTRIDE + h];
       const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
-      L += wl[ww * G + h] * f;
-      O += wacc[(ww * G + h) * D + tid] * f;
+      L += base[ww * WSTRIDE + G + h] * f;
+      O += base[ww * WSTRIDE + 2 * G + h * D + tid] * f;
     }
     float* ph = part_out + (long long)h * a.nsplit * PS;
     if (tid == 0) { ph[0] = M; ph[1] = L; }
@@ -375,7 +412,8 @@ __global__ void __launch_bounds__(D) decode_gqa_merge_kernel(const float* __rest
 template <int G>
 cudaError_t launch_g(const FastArgs& a, int n_active, __nv_bfloat16* out, int* seq_len, int bump,
                      cudaStream_t st) {
-  const size_t smem = (size_t)NSTAGE * STAGE_B + NWARP * 16 * G * sizeof(float) + NSTAGE * 8;
+  const size_t smem = (size_t)NWARP * NSTAGE * STAGE_B + NWARP * 2 * 8 * G * 2 * sizeof(float) +
+                      NWARP * NSTAGE * 8;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(decode_gqa_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -399,12 +437,17 @@ bool decode_gqa_supported(int dtype, const Shape& s) {
   return dtype == SNAP_BF16 && s.d_qk == D && s.d_v == D && !s.v_aliases_k && (s.g == 2 || s.g == 4 || s.g == 8);
 }
 
-// Splits per (sequence, KV head): enough CTAs to fill two per SM, preferring counts whose last
-// wave is nearly full, with at least one tile per split.
+// Splits per (sequence, KV head): enough CTAs to fill every resident slot (3 CTAs per SM, 2 for
+// g = 8), preferring counts whose last wave is nearly full, with at least one 64-row block per
+// split.  SNAP_DECODE_NSPLIT overrides the choice (tuning aid).
 int decode_gqa_nsplit(const Shape& s, int n_active, int sm_count) {
-  const int tiles = (s.Sc + TILE - 1) / TILE;
+  const int tiles = (s.Sc + 63) / 64;
+  if (const char* env = getenv("SNAP_DECODE_NSPLIT")) {
+    const int v = atoi(env);
+    if (v >= 1) return v < tiles ? v : tiles;
+  }
   const long long base = (long long)n_active * s.Hkv;
-  const double slots = 2.0 * sm_count;
+  const double slots = (s.g == 8 ? 2.0 : 3.0) * sm_count;
   int best = 1;
   double best_score = -1.0;
   const int max_ns = tiles < 64 ? tiles : 64;
