@@ -48,7 +48,9 @@ typedef enum snap_status {
   SNAP_ERR_UNSUPPORTED = -2,        /* valid, but no kernel is built for this shape */
   SNAP_ERR_WORKSPACE_TOO_SMALL = -3,
   SNAP_ERR_NULL_POINTER = -4,
-  SNAP_ERR_CUDA = -5                /* a CUDA runtime call failed; see cudaGetLastError */
+  SNAP_ERR_CUDA = -5,               /* a CUDA runtime call failed; see cudaGetLastError */
+  SNAP_ERR_STATIC_SCRATCH_EXCEEDED = -6  /* snap_decode_attn_static: the problem needs more than
+                                            SNAP_STATIC_SCRATCH_BYTES of scratch; nothing ran */
 } snap_status;
 
 /* bits of *status_dev */
@@ -162,6 +164,39 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout,
                      void* out_dev,
                      void* workspace_dev, size_t workspace_bytes,
                      uint32_t* status_dev, void* cuda_stream);
+
+/* Size of the scratch array built into the library for snap_decode_attn_static. */
+#define SNAP_STATIC_SCRATCH_BYTES (8u << 20)
+
+/*
+ * A decode step for callers that cannot allocate.  (The paper has no counterpart; this is a
+ * property of the library, not of the method.)
+ *
+ * Same operation, arguments and results as snap_decode_attn, but without the workspace
+ * arguments: the per-split partial results go to a fixed SNAP_STATIC_SCRATCH_BYTES array that
+ * lives inside the library, so the call performs no cudaMalloc/cudaFree and needs no buffer
+ * from the caller beyond the inputs and outputs.  It is meant for code that must not allocate
+ * where decode steps are issued: a serving loop whose device memory was partitioned up front
+ * and is full, a plugin running inside another runtime's callback, a process under a policy
+ * that treats late allocations as failures.
+ *
+ *   - Every GPU that loads this library holds the array from load until process exit.
+ *   - If n_active * n_q_heads * splits * (d_v + 2) floats exceed the array (splits is the
+ *     library's choice for that batch size, at most 64), the call returns
+ *     SNAP_ERR_STATIC_SCRATCH_EXCEEDED and launches nothing; use snap_decode_attn instead.
+ *     The 32-sequence, 32-head, d_v = 128 batch of a Llama-3.1-8B layer needs about 4.3 MB.
+ *   - All calls share the one array and it keeps the previous call's contents.  Nothing has to
+ *     be cleared (every partial that is read was written by the same call), but two calls
+ *     that can overlap on the GPU -- different streams without a dependency -- race.
+ *   - The first call on each device looks up the array's device address (no allocation);
+ *     make that first call outside any stream capture, with that device current.
+ */
+int snap_decode_attn_static(const snap_config_t* cfg, const snap_layout_t* layout,
+                            const void* q_dev, const void* k_new_dev, const void* v_new_dev,
+                            const int32_t* slot_ids_dev, int32_t n_active,
+                            void* k_cache_dev, void* v_cache_dev,
+                            int32_t* seq_len_dev, const int32_t* valid_topk_dev,
+                            void* out_dev, uint32_t* status_dev, void* cuda_stream);
 
 /* Text for a snap_status value (static storage). */
 const char* snap_status_string(int status);

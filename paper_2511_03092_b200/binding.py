@@ -70,12 +70,14 @@ def lib() -> C.CDLL:
     L.snap_append_kv.argtypes = [pcfg, play, vp, vp, vp, i32, vp, vp, vp, vp, vp]
     L.snap_decode_attn.restype = C.c_int
     L.snap_decode_attn.argtypes = [pcfg, play, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    L.snap_decode_attn_static.restype = C.c_int
+    L.snap_decode_attn_static.argtypes = [pcfg, play, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
     _lib = L
     return L
 
 
 EXPORTS = ("snap_cache_layout", "snap_compress_workspace_bytes", "snap_decode_workspace_bytes",
-           "snap_compress", "snap_append_kv", "snap_decode_attn", "snap_status_string",
+           "snap_compress", "snap_append_kv", "snap_decode_attn", "snap_decode_attn_static", "snap_status_string",
            "snap_kernel_launch_count")
 
 
@@ -170,6 +172,16 @@ def snap_decode_attn(cfg: SnapConfig, layout: SnapLayout, q, k_new, v_new, slot_
                                   _ptr(slot_ids_dev), int(n_active), _ptr(k_cache), _ptr(v_cache),
                                   _ptr(seq_len), _ptr(valid_topk), _ptr(out), _ptr(workspace), ws_bytes,
                                   _ptr(status), _stream(stream)), "snap_decode_attn")
+
+
+def snap_decode_attn_static(cfg: SnapConfig, layout: SnapLayout, q, k_new, v_new, slot_ids_dev, n_active: int,
+                            k_cache, v_cache, seq_len, valid_topk, out, status=None, stream=None) -> None:
+    """Decode step without a workspace argument: scratch is a fixed array inside the library, for
+    callers that must not allocate.  Raises SnapError(-6) when the batch does not fit that array."""
+    _check(lib().snap_decode_attn_static(C.byref(cfg), C.byref(layout), _ptr(q), _ptr(k_new), _ptr(v_new),
+                                         _ptr(slot_ids_dev), int(n_active), _ptr(k_cache), _ptr(v_cache),
+                                         _ptr(seq_len), _ptr(valid_topk), _ptr(out), _ptr(status),
+                                         _stream(stream)), "snap_decode_attn_static")
 
 
 @dataclass

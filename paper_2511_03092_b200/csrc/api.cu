@@ -135,6 +135,7 @@ const char* snap_status_string(int status) {
     case SNAP_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case SNAP_ERR_NULL_POINTER: return "null pointer";
     case SNAP_ERR_CUDA: return "CUDA error";
+    case SNAP_ERR_STATIC_SCRATCH_EXCEEDED: return "problem exceeds the built-in static scratch";
     default: return "unknown status";
   }
 }
