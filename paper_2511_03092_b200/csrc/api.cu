@@ -63,7 +63,7 @@ struct ChunkPlan {
   size_t part_off, stats_off, c_off, p_off, bytes;
 };
 
-ChunkPlan plan_chunk(const Shape& s, const int32_t* cu, int first, int n) {
+ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, int n) {
   ChunkPlan p;
   std::memset(&p, 0, sizeof(p));
   for (int i = 0; i < n; ++i) {
@@ -80,7 +80,7 @@ ChunkPlan plan_chunk(const Shape& s, const int32_t* cu, int first, int n) {
   if (nsplit > tiles) nsplit = tiles;
   if (nsplit > 64) nsplit = 64;
   if (nsplit < 1) nsplit = 1;
-  p.nsplit = (int)nsplit;
+  p.nsplit = score_mma_supported(dtype, s) ? score_mma_nsplit(s, p.n_scored, p.max_le, sm_count()) : (int)nsplit;
   p.c_stride = (int)align_up((size_t)p.max_le, 64);
   const size_t nz = (size_t)p.n_scored * s.Hkv;
   size_t off = 0;
@@ -172,7 +172,7 @@ int64_t snap_compress_workspace_bytes(const snap_config_t* cfg, const int32_t* c
   size_t worst = 0;
   for (int first = 0; first < n_seq; first += kMaxBatchSeqs) {
     const int n = n_seq - first < kMaxBatchSeqs ? n_seq - first : kMaxBatchSeqs;
-    const ChunkPlan p = plan_chunk(s, cu_seqlens_host, first, n);
+    const ChunkPlan p = plan_chunk(cfg->dtype, s, cu_seqlens_host, first, n);
     worst = p.bytes > worst ? p.bytes : worst;
   }
   return (int64_t)(idx_bytes(s, n_seq) + worst + 256);
@@ -241,7 +241,7 @@ int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout, const v
 
   for (int first = 0; first < n_seq; first += kMaxBatchSeqs) {
     const int n = n_seq - first < kMaxBatchSeqs ? n_seq - first : kMaxBatchSeqs;
-    const ChunkPlan p = plan_chunk(s, cu_seqlens_host, first, n);
+    const ChunkPlan p = plan_chunk(cfg->dtype, s, cu_seqlens_host, first, n);
     SeqBatch b;
     std::memset(&b, 0, sizeof(b));
     b.n = n; b.first_seq = first;
@@ -263,7 +263,10 @@ int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout, const v
       buf.C = reinterpret_cast<float*>(chunk_ws + p.c_off);
       buf.P = reinterpret_cast<float*>(chunk_ws + p.p_off);
       buf.c_stride = p.c_stride; buf.nsplit = p.nsplit;
-      if (launch_score_simt(cfg->dtype, s, b, q_obs_dev, src, buf, st) != cudaSuccess) return SNAP_ERR_CUDA;
+      const cudaError_t e = score_mma_supported(cfg->dtype, s)
+                                ? launch_score_mma(s, b, q_obs_dev, src, buf, st)
+                                : launch_score_simt(cfg->dtype, s, b, q_obs_dev, src, buf, st);
+      if (e != cudaSuccess) return SNAP_ERR_CUDA;
     }
     if (launch_pool_topk(s, b, buf, idx, status_dev, st) != cudaSuccess) return SNAP_ERR_CUDA;
     if (launch_gather(cfg->dtype, s, b, src, idx, k_cache_dev, v_cache_dev, seq_len_dev,

@@ -51,6 +51,11 @@ inline void count_launch() { ++g_launches; }
 // --- launchers (each enqueues on `st` and returns cudaGetLastError()) ---
 cudaError_t launch_score_simt(int dtype, const Shape& s, const SeqBatch& b, const void* q_obs,
                               const KVSource& src, const ScoreBuffers& buf, cudaStream_t st);
+// tensor-core version (bf16, 128-wide heads, g*Lo <= 256)
+bool score_mma_supported(int dtype, const Shape& s);
+int score_mma_nsplit(const Shape& s, int n_scored, int max_le, int sm_count);
+cudaError_t launch_score_mma(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
+                             const ScoreBuffers& buf, cudaStream_t st);
 cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffers& buf,
                              int* idx_out, uint32_t* status, cudaStream_t st);
 cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KVSource& src,
