@@ -1,0 +1,75 @@
+"""The benchmark configurations at their full sizes (where one sequence's oracle finishes in
+seconds) and sampled units of the larger ones, through the same C-ABI calls bench.py times."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import snapstream_oracle as orc
+from paper_2511_03092_b200 import synth
+from tests import _harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(wl, lengths, seed, steps, sample_steps=None):
+    n = len(lengths)
+    layer = H.GpuLayer(wl, max_seqs=n)
+    prompts = [synth.make_prompt(wl, L, seed + 101 * i) for i, L in enumerate(lengths)]
+    idx = layer.compress(prompts, list(range(n)))
+    assert layer.status() == 0
+    seqs = [H.oracle_compress(wl, p) for p in prompts]
+    swaps = 0
+    for i, seq in enumerate(seqs):
+        swaps += H.check_selection(idx[i], seq, wl)
+        seq.topk_pos = [idx[i][h][idx[i][h] >= 0].astype(np.int64) for h in range(wl.n_kv_heads)]
+        H.check_cache_image(layer, seq, i, wl)
+    slots_dev = torch.arange(n, dtype=torch.int32, device="cuda")
+    check = set(range(steps)) if sample_steps is None else set(sample_steps)
+    for step in range(steps):
+        d = synth.make_decode_inputs(wl, n, seed, step)
+        out = layer.decode(d["q"].cuda(), d["k_new"].cuda(), None if d["v_new"] is None else d["v_new"].cuda(),
+                           slots_dev)
+        for i, seq in enumerate(seqs):
+            ref = orc.decode_step(seq, synth.to_f64(d["q"][i]), synth.to_f64(d["k_new"][i]),
+                                  synth.to_f64(d["v_new"][i]) if d["v_new"] is not None else None)
+            if step in check:
+                H.check_output(out[i], ref, wl, f"seq {i} step {step}")
+    for i, seq in enumerate(seqs):
+        H.check_cache_image(layer, seq, i, wl)
+    assert layer.status() == 0
+    return swaps
+
+
+def test_config0_full():
+    """GQA 8/2 heads, fp32, prompt 4096, 16 decode steps."""
+    wl = synth.CONFIGS[0]
+    _run(wl, [4096], seed=100, steps=wl.decode_steps)
+
+
+def test_config1_full_size_prompt():
+    """Llama-shaped bf16 layer, prompt 32768; decode outputs checked on sampled steps."""
+    wl = synth.CONFIGS[1]
+    _run(wl, [32768], seed=200, steps=40, sample_steps=[0, 1, 7, 20, 39])
+
+
+def test_config2_ragged_batch_sample():
+    """Continuous-batching shape: a ragged batch (lengths drawn like config 2's, capped so the
+    oracle stays within seconds) compressed in one call and decoded together."""
+    wl = synth.CONFIGS[2]
+    lengths = [8192, 11000, 20011, 16384 + 5]
+    _run(wl, lengths, seed=300, steps=6)
+
+
+def test_config3_latent_sample():
+    """Latent-attention shape (128 heads over one 576-wide KV row, V = first 512 dims), prompt cut
+    to 16k tokens so that the oracle finishes in seconds."""
+    wl = synth.CONFIGS[3].scaled(topk=2048, l_recent=512)
+    _run(wl, [16384], seed=400, steps=3)
+
+
+def test_config4_one_sequence_layer_unit():
+    """One (sequence, layer) unit of the 32-layer, 128k-prompt configuration: units are independent,
+    so parity on a unit at full prompt length covers the kernels in the launch shape bench.py uses."""
+    wl = synth.CONFIGS[4]
+    swaps = _run(wl, [131072], seed=500, steps=4)
+    assert swaps <= 2
