@@ -2,6 +2,7 @@
 // launch sequences.  No allocation, no synchronisation, no state besides the launch counter
 // and a cached SM count.
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -57,6 +58,18 @@ Shape make_shape(const snap_config_t* c) {
 
 size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
+// SNAP_SCORE_PATH=mma|simt forces a slower score kernel (testing aid); default: the best one.
+bool use_umma(int dtype, const Shape& s) {
+  const char* env = getenv("SNAP_SCORE_PATH");
+  if (env && (!strcmp(env, "mma") || !strcmp(env, "simt"))) return false;
+  return score_umma_supported(dtype, s);
+}
+bool use_mma(int dtype, const Shape& s) {
+  const char* env = getenv("SNAP_SCORE_PATH");
+  if (env && !strcmp(env, "simt")) return false;
+  return score_mma_supported(dtype, s);
+}
+
 // Scratch regions of one chunk of prompts (offsets relative to the chunk area).
 struct ChunkPlan {
   int n_scored, max_le, nsplit, c_stride;
@@ -80,7 +93,9 @@ ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, in
   if (nsplit > tiles) nsplit = tiles;
   if (nsplit > 64) nsplit = 64;
   if (nsplit < 1) nsplit = 1;
-  p.nsplit = score_mma_supported(dtype, s) ? score_mma_nsplit(s, p.n_scored, p.max_le, sm_count()) : (int)nsplit;
+  if (use_umma(dtype, s)) p.nsplit = score_umma_nsplit(s, p.n_scored, p.max_le, sm_count());
+  else if (use_mma(dtype, s)) p.nsplit = score_mma_nsplit(s, p.n_scored, p.max_le, sm_count());
+  else p.nsplit = (int)nsplit;
   p.c_stride = (int)align_up((size_t)p.max_le, 64);
   const size_t nz = (size_t)p.n_scored * s.Hkv;
   size_t off = 0;
@@ -263,9 +278,9 @@ int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout, const v
       buf.C = reinterpret_cast<float*>(chunk_ws + p.c_off);
       buf.P = reinterpret_cast<float*>(chunk_ws + p.p_off);
       buf.c_stride = p.c_stride; buf.nsplit = p.nsplit;
-      const cudaError_t e = score_mma_supported(cfg->dtype, s)
-                                ? launch_score_mma(s, b, q_obs_dev, src, buf, st)
-                                : launch_score_simt(cfg->dtype, s, b, q_obs_dev, src, buf, st);
+      const cudaError_t e = use_umma(cfg->dtype, s)  ? launch_score_umma(s, b, q_obs_dev, src, buf, status_dev, st)
+                            : use_mma(cfg->dtype, s) ? launch_score_mma(s, b, q_obs_dev, src, buf, st)
+                                                     : launch_score_simt(cfg->dtype, s, b, q_obs_dev, src, buf, st);
       if (e != cudaSuccess) return SNAP_ERR_CUDA;
     }
     if (launch_pool_topk(s, b, buf, idx, status_dev, st) != cudaSuccess) return SNAP_ERR_CUDA;

@@ -257,20 +257,31 @@ __global__ void __launch_bounds__(256, 2) score_mma_kernel(const MmaArgs a) {
 // Merge the per-split statistics (log2 domain): m = max_s m_s, l = sum_s l_s 2^(m_s - m); keep (m, 1/l).
 __global__ void score_mma_combine_kernel(const float2* __restrict__ part, float2* __restrict__ stats,
                                          int nsplit, int R) {
-  const long long z = blockIdx.x;
-  for (int row = threadIdx.x; row < R; row += blockDim.x) {
-    float m = -INFINITY;
-    for (int s = 0; s < nsplit; ++s) m = fmaxf(m, part[(z * nsplit + s) * R + row].x);
-    double l = 0.0;
-    for (int s = 0; s < nsplit; ++s) {
-      const float2 p = part[(z * nsplit + s) * R + row];
-      if (p.y > 0.f) l += (double)p.y * exp2((double)p.x - (double)m);
-    }
-    stats[z * R + row] = make_float2(m, (float)(1.0 / l));
+  // one warp per query row, lanes over the splits
+  const long long z = blockIdx.y;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= R) return;
+  float m = -INFINITY;
+  for (int s = lane; s < nsplit; s += 32) m = fmaxf(m, part[(z * nsplit + s) * R + row].x);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  double l = 0.0;
+  for (int s = lane; s < nsplit; s += 32) {
+    const float2 p = part[(z * nsplit + s) * R + row];
+    if (p.y > 0.f) l += (double)p.y * exp2((double)p.x - (double)m);
   }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+  if (lane == 0) stats[z * R + row] = make_float2(m, (float)(1.0 / l));
 }
 
 }  // namespace
+
+cudaError_t launch_score_combine_log2(const ScoreBuffers& buf, int nz, int R, cudaStream_t st) {
+  score_mma_combine_kernel<<<dim3((R + 7) / 8, nz), 256, 0, st>>>(buf.part_stats, buf.stats, buf.nsplit, R);
+  count_launch();
+  return cudaGetLastError();
+}
 
 bool score_mma_supported(int dtype, const Shape& s) {
   return dtype == SNAP_BF16 && s.d_qk == D && s.g * s.Lo <= 256;
@@ -312,8 +323,7 @@ cudaError_t launch_score_mma(const Shape& s, const SeqBatch& b, const void* q_ob
   dim3 grid(buf.nsplit, nz);
   score_mma_kernel<1><<<grid, 32 * nrw, smem, st>>>(a);
   count_launch();
-  score_mma_combine_kernel<<<nz, 256, 0, st>>>(buf.part_stats, buf.stats, buf.nsplit, a.R);
-  count_launch();
+  if (launch_score_combine_log2(buf, nz, a.R, st) != cudaSuccess) return cudaGetLastError();
   score_mma_kernel<2><<<grid, 32 * nrw, smem, st>>>(a);
   count_launch();
   return cudaGetLastError();

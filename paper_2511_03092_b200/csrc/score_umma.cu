@@ -1,0 +1,408 @@
+// Observation-window scores on the 5th-generation tensor cores (Eq. 4 -> Eq. 1 with the GQA
+// group sum): tcgen05.mma with accumulators in tensor memory, operands staged by TMA.
+// Covers bf16 layers with 128-wide heads and 128 or 256 window rows per KV head (g * Lo).
+//
+// One CTA per SM, warp specialised, persistent over a run of 128-candidate tiles:
+//   warp 0   TMA producer: the query block once, then key tiles into a 4-stage ring
+//            (cp.async.bulk.tensor, 128-byte swizzle, two 64-element K halves per tile)
+//   warp 1   MMA issuer: one elected thread issues tcgen05.mma (M128, K16 steps) from shared
+//            memory descriptors into one of two TMEM accumulator buffers and commits to mbarriers
+//   warps 2-9  epilogue: read the accumulators with tcgen05.ld (thread = TMEM lane) while the
+//            next tile's MMAs run into the other buffer
+//
+// Pass 1 puts the query rows on M (two 128-row blocks share each key tile; N = 128 candidates),
+// so a thread owns one query row and keeps that row's running (reference max, sum of exp2) with
+// no cross-thread traffic.  Pass 2 puts the candidates on M (N = all query rows), so a thread
+// owns one candidate and sums exp2(s_ij - m_i) / l_i over the rows by itself and stores C[j].
+// The reference max of pass 1 is refreshed lazily (only when a tile's partial sum shows a logit
+// far above it).  Statistics are in the log2 domain.  Every mbarrier wait is bounded; a wait
+// that runs out raises SNAP_DEV_WAIT_TIMEOUT and the CTA drains and frees its tensor memory.
+#include <cuda.h>
+
+#include "snap_internal.cuh"
+
+namespace snap {
+namespace {
+
+constexpr int D = 128, TN = 128, NS = 4;
+constexpr int HALF_B = TN * 128;             // one K half of a 128-row tile: 128 rows x 128 bytes
+constexpr int STAGE_B = 2 * HALF_B;          // 32 KB
+constexpr int NTHREADS = 320;                // 10 warps
+constexpr unsigned kWaitLimit = 1u << 21;
+
+struct UmmaArgs {
+  int Hq, Hkv, g, Lo, Ls, Lr, R;
+  float scale_log2;
+  SeqBatch b;
+  ScoreBuffers buf;
+  uint32_t* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait; also gives up as soon as another role has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, unsigned parity, volatile int* abort_flag) {
+  for (unsigned it = 0; it < kWaitLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
+// K-major operand, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  return (uint64_t)((saddr >> 4) & 0x3fffu) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float fast_exp2(float x) {     // one MUFU op, relative error ~2^-22
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void merge_ml(float& m, float& l, float m2, float l2) {
+  const float mn = fmaxf(m, m2);
+  const float f1 = m == -INFINITY ? 0.f : exp2f(m - mn), f2 = m2 == -INFINITY ? 0.f : exp2f(m2 - mn);
+  l = l * f1 + l2 * f2;
+  m = mn;
+}
+
+// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(NTHREADS, 1)
+score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int R = a.R, MB = R / 128;
+  unsigned char* Qs = smem;                                   // [2 halves][R][128 B]
+  unsigned char* Ks = Qs + R * 256;                           // [NS][2 halves][128][128 B]
+  float2* stats_s = reinterpret_cast<float2*>(Ks + NS * STAGE_B);   // [R]  (pass 2: m_i, 1/l_i)
+  float2* xch = stats_s + 256;                                // [128] pass-1 exchange between epilogue groups
+  uint64_t* bars = reinterpret_cast<uint64_t*>(xch + 128);    // full[NS] empty[NS] tfull[2] tempty[2] qfull
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NS + 5);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int z = blockIdx.y, si = z / a.Hkv, kvh = z % a.Hkv;
+  const int seq = a.b.seq_of_score[si];
+  const int Le = a.b.len[seq] - a.Ls - a.Lr;
+  const int ntiles = (Le + TN - 1) / TN;
+  const int t0 = (int)((long long)ntiles * blockIdx.x / a.buf.nsplit);
+  const int t1 = (int)((long long)ntiles * (blockIdx.x + 1) / a.buf.nsplit);
+  const int nt = t1 - t0;
+  // both epilogue groups work on every tile (pass 1 with two row blocks) or they alternate tiles
+  const bool both = PASS == 1 && MB == 2;
+
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8 * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8 * (NS + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8 * (2 * NS + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8 * (2 * NS + 2 + b); };
+  const uint32_t qfull_bar = bar0 + 8 * (2 * NS + 4);
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), both ? 8 : 4); }
+    mbar_init(qfull_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (PASS == 2) {
+    for (int i = tid; i < R; i += NTHREADS) stats_s[i] = a.buf.stats[(long long)z * R + i];
+  }
+  if (warp == 0) {                                            // tensor memory: 512 columns (2 x 256)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  // epilogue threads: group, accumulator row, and (pass 1) the running statistics of that row
+  const int eg = warp >= 2 ? (warp - 2) >> 2 : 0;
+  const int lrow = 32 * (warp & 3) + lane;
+  float m_ref = -INFINITY, l_sum = 0.f;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0 && nt > 0) {
+      const int row0 = ((a.b.first_seq + seq) * a.Hq + kvh * a.g) * a.Lo;
+      mbar_expect_tx(qfull_bar, (unsigned)R * 256u);
+      for (int h = 0; h < 2; ++h)
+        for (int mb = 0; mb < MB; ++mb)
+          tma_load_2d(smem_u32(Qs) + h * (R * 128) + mb * HALF_B, &tmap_q, h * 64, row0 + 128 * mb, qfull_bar);
+      const int tok0 = a.b.tok_off[seq] + a.Ls;
+      for (int it = 0; it < nt; ++it) {
+        const int s = it % NS;
+        if (!mbar_wait(empty_bar(s), ((unsigned)(it / NS) & 1u) ^ 1u, abort_flag)) { *abort_flag = 1; break; }
+        mbar_expect_tx(full_bar(s), (unsigned)STAGE_B);
+        const uint32_t dst = smem_u32(Ks) + s * STAGE_B;
+        tma_load_3d(dst, &tmap_k, 0, kvh, tok0 + (t0 + it) * TN, full_bar(s));
+        tma_load_3d(dst + HALF_B, &tmap_k, 64, kvh, tok0 + (t0 + it) * TN, full_bar(s));
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0 && nt > 0) {
+      const uint32_t idesc = PASS == 1 ? make_idesc(128, 128) : make_idesc(128, R);
+      bool ok = mbar_wait(qfull_bar, 0u, abort_flag);
+      for (int it = 0; it < nt && ok; ++it) {
+        const int s = it % NS, b = it & 1;
+        ok = mbar_wait(full_bar(s), (unsigned)(it / NS) & 1u, abort_flag) &&
+             mbar_wait(tempty_bar(b), ((unsigned)(it / 2) & 1u) ^ 1u, abort_flag);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t kst = smem_u32(Ks) + s * STAGE_B, qst = smem_u32(Qs);
+        if (PASS == 1) {
+          for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+              umma_bf16(tmem_base + b * 256 + mb * 128,
+                        umma_desc(qst + (ks >> 2) * (R * 128) + mb * HALF_B + (ks & 3) * 32),
+                        umma_desc(kst + (ks >> 2) * HALF_B + (ks & 3) * 32), idesc, ks > 0);
+        } else {
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            umma_bf16(tmem_base + b * 256, umma_desc(kst + (ks >> 2) * HALF_B + (ks & 3) * 32),
+                      umma_desc(qst + (ks >> 2) * (R * 128) + (ks & 3) * 32), idesc, ks > 0);
+        }
+        umma_commit(empty_bar(s));        // the stage may be refilled once these MMAs have read it
+        umma_commit(tfull_bar(b));        // the accumulator buffer is complete
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    // a warp may read the TMEM lane quarter (warp id mod 4); thread = accumulator row lrow
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+    const int mb = both ? eg : 0;
+    bool ok = true;
+    for (int it = both ? 0 : eg; it < nt; it += both ? 1 : 2) {
+      const int b = it & 1;
+      if (!mbar_wait(tfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag)) { ok = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int cand0 = (t0 + it) * TN;
+      if (PASS == 1) {
+        const uint32_t col0 = lane_addr + b * 256 + mb * 128;
+        const bool full_tile = cand0 + TN <= Le;
+        float sum = 0.f;
+        float v[32];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          tmem_ld32(col0 + 32 * c, v);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float ex = fast_exp2(fmaf(v[i], a.scale_log2, -m_ref));
+            sum += (full_tile || cand0 + 32 * c + i < Le) ? ex : 0.f;
+          }
+        }
+        if (!(sum < 65536.f)) {                               // a logit far above the reference (or first tile)
+          float vmax = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(col0 + 32 * c, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (full_tile || cand0 + 32 * c + i < Le) vmax = fmaxf(vmax, v[i] * a.scale_log2);
+          }
+          const float mn = fmaxf(m_ref, vmax);
+          sum = 0.f;
+          if (mn != -INFINITY) {
+            l_sum *= m_ref == -INFINITY ? 0.f : exp2f(m_ref - mn);
+            m_ref = mn;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              tmem_ld32(col0 + 32 * c, v);
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (full_tile || cand0 + 32 * c + i < Le) sum += fast_exp2(fmaf(v[i], a.scale_log2, -mn));
+            }
+          }
+        }
+        l_sum += sum;
+      } else {
+        const uint32_t col0 = lane_addr + b * 256;
+        float s = 0.f;
+        float v[32];
+        for (int c = 0; c < R / 32; ++c) {
+          tmem_ld32(col0 + 32 * c, v);
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            const float4 st = *reinterpret_cast<const float4*>(&stats_s[32 * c + i]);
+            s = fmaf(fast_exp2(fmaf(v[i], a.scale_log2, -st.x)), st.y, s);
+            s = fmaf(fast_exp2(fmaf(v[i + 1], a.scale_log2, -st.z)), st.w, s);
+          }
+        }
+        if (cand0 + lrow < Le) a.buf.C[(long long)z * a.buf.c_stride + cand0 + lrow] = s;
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(b));
+    }
+    if (!ok) *abort_flag = 1;
+    if (PASS == 1) {
+      if (both)
+        a.buf.part_stats[((long long)z * a.buf.nsplit + blockIdx.x) * R + 128 * mb + lrow] = make_float2(m_ref, l_sum);
+      else if (eg == 1)
+        xch[lrow] = make_float2(m_ref, l_sum);                // merged by group 0 after the barrier below
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  if (PASS == 1 && !both && warp >= 2 && eg == 0) {          // one row block: the two groups took alternate tiles
+    const float2 o = xch[lrow];
+    merge_ml(m_ref, l_sum, o.x, o.y);
+    a.buf.part_stats[((long long)z * a.buf.nsplit + blockIdx.x) * R + lrow] = make_float2(m_ref, l_sum);
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+  if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+constexpr size_t kSmemBytes = 256 * 256 + NS * STAGE_B + 256 * sizeof(float2) + 128 * sizeof(float2) +
+                              (2 * NS + 5) * 8 + 16 + 1024;
+
+}  // namespace
+
+bool score_umma_supported(int dtype, const Shape& s) {
+  const int R = s.g * s.Lo;
+  return dtype == SNAP_BF16 && s.d_qk == D && (R == 128 || R == 256) && encode_fn() != nullptr;
+}
+
+// Candidate splits per (prompt, KV head): two CTAs per SM in sequence (one resident at a time).
+int score_umma_nsplit(const Shape& s, int n_scored, int max_le, int sm_count) {
+  const int tiles = (max_le + TN - 1) / TN;
+  const long long base = (long long)n_scored * s.Hkv;
+  long long ns = (2LL * sm_count + base / 2) / base;
+  if (ns > tiles) ns = tiles;
+  if (ns > 512) ns = 512;
+  if (ns < 1) ns = 1;
+  return (int)ns;
+}
+
+cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
+                              const ScoreBuffers& buf, uint32_t* status, cudaStream_t st) {
+  if (b.n_scored == 0) return cudaSuccess;
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  UmmaArgs a;
+  a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Lo = s.Lo; a.Ls = s.Ls; a.Lr = s.Lr; a.R = s.g * s.Lo;
+  a.scale_log2 = s.scale * 1.4426950408889634f;
+  a.b = b; a.buf = buf; a.status = status;
+
+  CUtensorMap tq, tk;
+  const cuuint32_t estr2[2] = {1, 1}, estr3[3] = {1, 1, 1};
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)(b.first_seq + b.n) * s.Hq * s.Lo};
+    const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    const cuuint32_t box[2] = {64, 128};
+    if (enc(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(q_obs), dims, strides, box, estr2,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  {
+    long long tokens = 0;
+    for (int i = 0; i < b.n; ++i) tokens = tokens > (long long)b.tok_off[i] + b.len[i] ? tokens : (long long)b.tok_off[i] + b.len[i];
+    const long long head_stride = src.k_head_stride >= D ? src.k_head_stride : D;
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)s.Hkv, (cuuint64_t)tokens};
+    const cuuint64_t strides[2] = {(cuuint64_t)head_stride * 2, (cuuint64_t)src.k_tok_stride * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)TN};
+    if (enc(&tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(src.k), dims, strides, box, estr3,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(score_umma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(score_umma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int nz = b.n_scored * s.Hkv;
+  dim3 grid(buf.nsplit, nz);
+  score_umma_kernel<1><<<grid, NTHREADS, kSmemBytes, st>>>(a, tq, tk);
+  count_launch();
+  cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
+  if (e != cudaSuccess) return e;
+  score_umma_kernel<2><<<grid, NTHREADS, kSmemBytes, st>>>(a, tq, tk);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace snap

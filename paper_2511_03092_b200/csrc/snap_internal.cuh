@@ -56,6 +56,12 @@ bool score_mma_supported(int dtype, const Shape& s);
 int score_mma_nsplit(const Shape& s, int n_scored, int max_le, int sm_count);
 cudaError_t launch_score_mma(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
                              const ScoreBuffers& buf, cudaStream_t st);
+cudaError_t launch_score_combine_log2(const ScoreBuffers& buf, int nz, int R, cudaStream_t st);
+// tcgen05 / TMEM / TMA version (bf16, 128-wide heads, g*Lo = 128 or 256)
+bool score_umma_supported(int dtype, const Shape& s);
+int score_umma_nsplit(const Shape& s, int n_scored, int max_le, int sm_count);
+cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
+                              const ScoreBuffers& buf, uint32_t* status, cudaStream_t st);
 cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffers& buf,
                              int* idx_out, uint32_t* status, cudaStream_t st);
 cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KVSource& src,

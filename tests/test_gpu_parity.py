@@ -75,7 +75,7 @@ def test_ring_wraps_many_times():
 
 
 @pytest.mark.parametrize("kw", [dict(topk=0), dict(l_sink=0), dict(pool_kernel=1), dict(pool_mode="max"),
-                                dict(l_obs=1, pool_kernel=1), dict(pool_kernel=13, l_obs=32)],
+                                dict(l_obs=1, pool_kernel=1), dict(pool_kernel=13, l_obs=32), dict(pool_kernel=19)],
                          ids=lambda k: "-".join(f"{a}{b}" for a, b in k.items()))
 def test_degenerate_hyperparameters(kw):
     wl = SMALL_BF16.scaled(**kw)
@@ -201,3 +201,9 @@ def test_many_sequences_ragged_decode():
     rng = np.random.default_rng(0)
     lengths = [int(x) for x in rng.integers(1, 400, size=70)]
     _run_compress_and_decode(wl, lengths, seed=17, steps=3, check_ring_every=3)
+
+
+def test_prompt_longer_than_the_register_resident_topk_path():
+    """More than 16 candidates per thread of the top-K cluster: keys are re-read from scratch."""
+    wl = SMALL_BF16.scaled(n_q_heads=4, n_kv_heads=2, topk=300)
+    _run_compress_and_decode(wl, [140000, 131072 + 60], seed=23, steps=2)
