@@ -13,7 +13,8 @@
 // Pass 1 puts the query rows on M (two 128-row blocks share each key tile; N = 128 candidates),
 // so a thread owns one query row and keeps that row's running (reference max, sum of exp2) with
 // no cross-thread traffic.  Pass 2 puts the candidates on M (N = all query rows), so a thread
-// owns one candidate and sums exp2(s_ij - m_i) / l_i over the rows by itself and stores C[j].
+// owns one candidate; the two epilogue groups each sum exp2(s_ij - m_i) / l_i over half of the
+// rows, group 1 hands its partial to group 0 through shared memory, and group 0 stores C[j].
 // The reference max of pass 1 is refreshed lazily (only when a tile's partial sum shows a logit
 // far above it).  Statistics are in the log2 domain.  Every mbarrier wait is bounded; a wait
 // that runs out raises SNAP_DEV_WAIT_TIMEOUT and the CTA drains and frees its tensor memory.
@@ -105,6 +106,41 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// Split form for software pipelining: issue the load, and wait later.  The wait lists the
+// registers as in/out operands so that no use of them can be scheduled above it.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :: "memory");
+}
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld16_wait(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :: "memory");
+}
 __device__ __forceinline__ float fast_exp2(float x) {     // one MUFU op, relative error ~2^-22
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -144,8 +180,9 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   const int t0 = (int)((long long)ntiles * blockIdx.x / a.buf.nsplit);
   const int t1 = (int)((long long)ntiles * (blockIdx.x + 1) / a.buf.nsplit);
   const int nt = t1 - t0;
-  // both epilogue groups work on every tile (pass 1 with two row blocks) or they alternate tiles
-  const bool both = PASS == 1 && MB == 2;
+  // Both epilogue groups work on every tile -- pass 1 with two row blocks (one block each) and
+  // pass 2 (half of the query-row columns each) -- or they alternate tiles (pass 1, one row block).
+  const bool both = PASS == 2 || MB == 2;
 
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8 * s; };
@@ -161,8 +198,12 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
     mbar_init(qfull_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  float* mu_s = reinterpret_cast<float*>(stats_s);            // pass 2: m_i + log2(l_i) per query row
   if (PASS == 2) {
-    for (int i = tid; i < R; i += NTHREADS) stats_s[i] = a.buf.stats[(long long)z * R + i];
+    for (int i = tid; i < R; i += NTHREADS) {
+      const float2 st = a.buf.stats[(long long)z * R + i];
+      mu_s[i] = st.x - log2f(st.y);
+    }
   }
   if (warp == 0) {                                            // tensor memory: 512 columns (2 x 256)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
@@ -231,9 +272,22 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
     const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
     const int mb = both ? eg : 0;
     bool ok = true;
+    // pass 2: minus the log-sum-exp (log2 domain) of each query row this group sums over, in
+    // registers, so that the inner loop is fma -> exp2 -> add with no memory operand
+    const int nc2 = R / 64;                                   // 32-column chunks per group: 2 or 4
+    float mu[128];
+    if (PASS == 2) {
+#pragma unroll
+      for (int i = 0; i < 128; ++i) mu[i] = i < 32 * nc2 ? -mu_s[32 * nc2 * eg + i] : 0.f;
+    }
     for (int it = both ? 0 : eg; it < nt; it += both ? 1 : 2) {
       const int b = it & 1;
-      if (!mbar_wait(tfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag)) { ok = false; break; }
+      const bool landed = mbar_wait(tfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag);
+      if (!landed) {
+        *abort_flag = 1;
+        ok = false;
+        if (PASS == 1) break;            // pass 2 leaves through the group barrier below
+      }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int cand0 = (t0 + it) * TN;
       if (PASS == 1) {
@@ -241,13 +295,38 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
         const bool full_tile = cand0 + TN <= Le;
         float sum = 0.f;
         float v[32];
+        if (full_tile) {
+          // software pipeline: the next 32 columns are in flight while these are exponentiated;
+          // four partial sums break the dependency chain of the additions
+          uint32_t ra[32], rb[32];
+          float s4[4] = {0.f, 0.f, 0.f, 0.f};
+          const float nm = -m_ref;
+          tmem_ld32_issue(col0, ra);
+          tmem_ld_wait(ra);
+          tmem_ld32_issue(col0 + 32, rb);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          tmem_ld32(col0 + 32 * c, v);
+          for (int i = 0; i < 32; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, nm));
+          tmem_ld_wait(rb);
+          tmem_ld32_issue(col0 + 64, ra);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float ex = fast_exp2(fmaf(v[i], a.scale_log2, -m_ref));
-            sum += (full_tile || cand0 + 32 * c + i < Le) ? ex : 0.f;
+          for (int i = 0; i < 32; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(rb[i]), a.scale_log2, nm));
+          tmem_ld_wait(ra);
+          tmem_ld32_issue(col0 + 96, rb);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, nm));
+          tmem_ld_wait(rb);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(rb[i]), a.scale_log2, nm));
+          sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(col0 + 32 * c, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float ex = fast_exp2(fmaf(v[i], a.scale_log2, -m_ref));
+              sum += (cand0 + 32 * c + i < Le) ? ex : 0.f;
+            }
           }
         }
         if (!(sum < 65536.f)) {                               // a logit far above the reference (or first tile)
@@ -275,23 +354,49 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
         }
         l_sum += sum;
       } else {
-        const uint32_t col0 = lane_addr + b * 256;
+        // this group's half of the query-row columns; group 1 hands its partial sum to group 0
+        const uint32_t col0 = lane_addr + b * 256 + 32 * (eg * nc2);
         float s = 0.f;
-        float v[32];
-        for (int c = 0; c < R / 32; ++c) {
-          tmem_ld32(col0 + 32 * c, v);
+        if (landed) {
+          // software pipeline over 16-column chunks (two small register buffers leave room for the
+          // 128 row constants); four partial sums break the dependency chain of the additions
+          uint32_t ra[16], rb[16];
+          float s4[4] = {0.f, 0.f, 0.f, 0.f};
+          const int nch = 2 * nc2;                             // 16-column chunks: 4 or 8
+          tmem_ld16_issue(col0, ra);
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            const float4 st = *reinterpret_cast<const float4*>(&stats_s[32 * c + i]);
-            s = fmaf(fast_exp2(fmaf(v[i], a.scale_log2, -st.x)), st.y, s);
-            s = fmaf(fast_exp2(fmaf(v[i + 1], a.scale_log2, -st.z)), st.w, s);
+          for (int c = 0; c < 8; c += 2) {
+            if (c < nch) {
+              tmem_ld16_wait(ra);
+              tmem_ld16_issue(col0 + 16 * (c + 1), rb);
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                s4[i & 3] += fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, mu[16 * c + i]));
+              tmem_ld16_wait(rb);
+              if (c + 2 < nch) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                s4[i & 3] += fast_exp2(fmaf(__uint_as_float(rb[i]), a.scale_log2, mu[16 * (c + 1) + i]));
+            }
           }
+          s = (s4[0] + s4[1]) + (s4[2] + s4[3]);
         }
-        if (cand0 + lrow < Le) a.buf.C[(long long)z * a.buf.c_stride + cand0 + lrow] = s;
+        float* xs = reinterpret_cast<float*>(xch) + b * 128;
+        if (eg == 1) xs[lrow] = s;
+        // barrier over the 8 epilogue warps that also agrees on whether anyone has given up
+        unsigned stop;
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+            "bar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(stop) : "r"((unsigned)(!landed || *abort_flag)) : "memory");
+        if (eg == 0 && !stop && cand0 + lrow < Le)
+          a.buf.C[(long long)z * a.buf.c_stride + cand0 + lrow] = s + xs[lrow];
+        if (stop) { *abort_flag = 1; ok = false; }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(b));
+      if (!ok) break;
     }
     if (!ok) *abort_flag = 1;
     if (PASS == 1) {
