@@ -329,7 +329,9 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
             }
           }
         }
-        if (!(sum < 65536.f)) {                               // a logit far above the reference (or first tile)
+        // A logit far above the reference (or the first tile): refresh the reference.  The TMEM
+        // loads below are warp-collective, so the whole warp takes the branch if any row needs it.
+        if (__any_sync(0xffffffffu, !(sum < 65536.f))) {
           float vmax = -INFINITY;
 #pragma unroll
           for (int c = 0; c < 4; ++c) {

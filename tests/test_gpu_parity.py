@@ -207,3 +207,25 @@ def test_prompt_longer_than_the_register_resident_topk_path():
     """More than 16 candidates per thread of the top-K cluster: keys are re-read from scratch."""
     wl = SMALL_BF16.scaled(n_q_heads=4, n_kv_heads=2, topk=300)
     _run_compress_and_decode(wl, [140000, 131072 + 60], seed=23, steps=2)
+
+
+def test_late_outlier_logits_refresh_the_running_reference():
+    """Keys far down the candidate range that give huge logits to single observation rows only:
+    the score kernels must refresh their per-row softmax reference mid-stream (rows of one warp
+    disagree about needing it)."""
+    wl = SMALL_BF16.scaled(l_obs=32, topk=200)          # 4 heads per KV head x 32 rows = 128 window rows
+    L = 5000
+    p = synth.make_prompt(wl, L, seed=41)
+    q = p["q_obs"].float()
+    k = p["k"].float()
+    for n, (hq, row, pos, c) in enumerate([(0, 0, 1500, 30.0), (5, 17, 2600, 45.0), (9, 31, 4000, 25.0), (14, 3, 4700, 60.0)]):
+        qv = q[hq, row]
+        k[pos, hq // 4] = qv * (c / (wl.scale * float(qv @ qv)))
+    p["k"] = k.to(wl.torch_dtype)
+    layer = H.GpuLayer(wl, max_seqs=1)
+    idx = layer.compress([p], [0])
+    assert layer.status() == 0
+    seq = H.oracle_compress(wl, p)
+    H.check_selection(idx[0], seq, wl)
+    for pos, kvh in [(1500, 0), (2600, 1), (4000, 2), (4700, 3)]:
+        assert pos in idx[0][kvh]
