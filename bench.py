@@ -52,45 +52,71 @@ def _peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason sampling during the timed region."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """SM clock / throttle-reason sampling during the timed region (NVML, read-only queries) from a
+    background thread every few milliseconds; samples are time-stamped and only those taken between
+    the two synchronisation points around the timed region are reported."""
 
-    def __init__(self, gpu_index: int):
-        self.gpu, self.proc = gpu_index, None
+    def __init__(self, gpu_index: int, period_s: float = 0.002):
+        self.gpu, self.period, self.samples, self.thread, self.stop_flag = gpu_index, period_s, [], None, False
+        self.nvml, self.handle, self.max_mhz = None, None, None
 
     def start(self):
+        import threading
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu)],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            idx = self.gpu
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            if vis:
+                try:
+                    idx = int(vis.split(",")[self.gpu])
+                except (ValueError, IndexError):
+                    idx = self.gpu
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.nvml = pynvml
+        except Exception:
+            self.nvml = None
+            return
 
-    def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-            out, _ = self.proc.communicate()
-        sm, smax, reasons = [], [], set()
-        for line in out.strip().splitlines():
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1])); smax.append(float(f[2]))
-            except ValueError:
-                continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        def loop():
+            nv = self.nvml
+            while not self.stop_flag:
+                try:
+                    mhz = nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)
+                    try:
+                        reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                    except Exception:
+                        reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
+                    self.samples.append((time.perf_counter(), float(mhz), int(reasons)))
+                except Exception:
+                    pass
+                time.sleep(self.period)
+
+        self.thread = threading.Thread(target=loop, daemon=True)
+        self.thread.start()
+
+    def stop(self, t_begin: float, t_end: float) -> dict:
+        if self.nvml is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["NVML unavailable"]}
+        self.stop_flag = True
+        self.thread.join(timeout=2)
+        inside = [x for x in self.samples if t_begin <= x[0] <= t_end]
+        note = None
+        if not inside:                      # region shorter than one sampling period: nearest samples
+            inside = sorted(self.samples, key=lambda x: min(abs(x[0] - t_begin), abs(x[0] - t_end)))[:3]
+            note = "timed region shorter than the sampling period; nearest samples used"
+        bits = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+        seen = set()
+        for _, _, r in inside:
+            for bit, name in bits.items():
+                if r & bit:
+                    seen.add(name)
+        out = {"sm_mhz": statistics.median([x[1] for x in inside]) if inside else None, "sm_max_mhz": self.max_mhz,
+               "samples": len(inside), "reasons": sorted(seen)}
+        if note:
+            out["note"] = note
+        return out
 
 
 # ----------------------------------------------------------------------------------------
@@ -196,6 +222,7 @@ def run_ours(args):
     launches0 = B.snap_kernel_launch_count()
     bytes_acc = 0
     n_replaced = 0
+    host_t0 = time.perf_counter()
     t0.record()
     for i in range(args.steps):
         step(args.warmup + i, evs[i])
@@ -203,8 +230,9 @@ def run_ours(args):
         n_replaced += len(sched[args.warmup + i])
     t1.record()
     barrier()
+    host_t1 = time.perf_counter()
     launches = B.snap_kernel_launch_count() - launches0
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(host_t0, host_t1) if rank == 0 else None
     ms = t0.elapsed_time(t1)
     dec_ms = [a.elapsed_time(b) for a, b in evs]
     if world > 1:
@@ -275,11 +303,66 @@ def run_ours(args):
     }
     line["extra"] = {"decode_only_tokens_per_s": wl.batch / (dec_avg_ms * 1e-3),
                      "decode_ms_median": statistics.median(dec_ms)}
+    if world == 1 and not args.no_extras:
+        line["extra"].update(extras(hp, wl, dev))
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl, hp, sched)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def extras(hp, wl, dev):
+    """Side measurements reported next to the headline: compress time of one 128k-token prompt, and
+    decode over the uncompressed (full) KV of the same resident sequences for the ratio."""
+    from paper_2511_03092_b200 import binding as B
+    out = {}
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    # (1) compress microseconds per 128k prefill (one sequence, one layer)
+    L = 131072
+    p = synth.make_prompt(wl, L, SEED + 99, dev)
+    times = []
+    for r in range(7):
+        a, b = ev(), ev()
+        a.record(); hp.compress_prompt(p, 0); b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b) * 1e3)
+    out["compress_us_per_128k_prefill"] = statistics.median(times[2:])
+    flops = 2 * 2.0 * wl.n_q_heads * wl.l_obs * (L - wl.l_sink - wl.l_recent) * wl.d_qk
+    out["compress_score_tflops_effective"] = flops / (out["compress_us_per_128k_prefill"] * 1e-6) / 1e12
+    hp.compress_prompt(hp.pool[hp.resident[0]], 0)          # restore slot 0
+    del p
+    # (2) full-KV decode over the same 32 sequences: the same library with Ls = 0, K = 0, Lr > every length
+    lens = [hp.lengths[i] for i in hp.resident]
+    lr = max(lens) + 64
+    cfg = B.make_config(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, d_qk=wl.d_qk, d_v=wl.d_v,
+                        dtype=wl.torch_dtype, l_sink=0, l_recent=lr, topk=0, l_obs=wl.l_obs,
+                        pool_kernel=wl.pool_kernel, softmax_scale=wl.scale, max_seqs=wl.batch)
+    lay = B.snap_cache_layout(cfg)
+    cache = B.alloc_cache(cfg, lay, dev)
+    for slot, i in enumerate(hp.resident):
+        q = hp.pool[i]
+        B.snap_compress(cfg, lay, None, q["k"], q["v"], [0, lens[slot]], [slot], cache.k_cache, cache.v_cache,
+                        cache.seq_len, cache.valid_topk, None, None, cache.status)
+    dws = torch.empty(B.snap_decode_workspace_bytes(cfg, wl.batch), dtype=torch.uint8, device=dev)
+    outb = torch.empty_like(hp.out)
+    times = []
+    for r in range(8):
+        d = hp.decode_in[r % DECODE_RING]
+        a, b = ev(), ev()
+        a.record()
+        B.snap_decode_attn(cfg, lay, d["q"], d["k_new"], d["v_new"], hp.slots_dev, wl.batch, cache.k_cache,
+                           cache.v_cache, cache.seq_len, cache.valid_topk, outb, dws, cache.status)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    full_ms = statistics.median(times[2:])
+    full_bytes = sum(lens) * wl.n_kv_heads * (wl.d_qk + wl.d_v) * 2
+    out["full_kv_decode_ms"] = full_ms
+    out["full_kv_decode_GBps"] = full_bytes / (full_ms * 1e-3) / 1e9
+    out["full_kv_bytes_over_compressed_bytes"] = full_bytes / hp.decode_bytes()
+    out["full_kv_status"] = int(cache.status.item())
+    return out
 
 
 # ----------------------------------------------------------------------------------------
@@ -445,6 +528,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the 128k-compress and full-KV side measurements")
     ap.add_argument("--case", choices=["decode", "compress"], default=None,
                     help="small single-kernel-family case for profiler captures")
     ap.add_argument("--case-len", type=int, default=131072)
