@@ -40,6 +40,9 @@ UNIT = "tokens/s"
 SEED = 2511
 POOL_EXTRA = 16            # prompts beyond the initial batch that replacements cycle through
 DECODE_RING = 8            # distinct pre-generated decode inputs cycled through
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_gqa_kernel launch on this launch shape (32 full
+# 5124-slot caches), from the ncu capture summarised in profiles/decode_gqa_kernel_32seq_llama_cache.md
+DECODE_TRAFFIC_BYTES = 672.11e6 + 5.82e6
 
 
 def _peaks():
@@ -298,7 +301,8 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "decode attention (split + merge launches of one snap_decode_attn)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": peak_src, "algorithmic_bytes_per_launch": alg_bytes,
-                     "avg_launch_ms": dec_avg_ms, "traffic": None},
+                     "avg_launch_ms": dec_avg_ms, "traffic": DECODE_TRAFFIC_BYTES,
+                     "traffic_source": "one ncu capture of the same launch shape (profiles/)"},
         "device_status_word": status,
     }
     line["extra"] = {"decode_only_tokens_per_s": wl.batch / (dec_avg_ms * 1e-3),
