@@ -115,13 +115,17 @@ int check_cu(const int32_t* cu, int n_seq) {
   return SNAP_OK;
 }
 
-struct DecodePlan { bool gqa; int nsplit; size_t floats; };
+struct DecodePlan { bool gqa, mla; int nsplit; size_t floats; };
 
 DecodePlan plan_decode(int dtype, const Shape& s, int n_active) {
   DecodePlan p;
   const int n = n_active > 0 ? n_active : 1;
   p.gqa = decode_gqa_supported(dtype, s);
-  if (p.gqa) {
+  p.mla = !p.gqa && decode_mla_supported(dtype, s);
+  if (p.mla) {
+    p.nsplit = decode_mla_nsplit(s, n, sm_count());
+    p.floats = decode_mla_partial_floats(s, n_active, p.nsplit);
+  } else if (p.gqa) {
     p.nsplit = decode_gqa_nsplit(s, n, sm_count());
     p.floats = decode_gqa_partial_floats(s, n_active, p.nsplit);
   } else {
@@ -334,7 +338,10 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
   const DecodePlan p = plan_decode(cfg->dtype, s, n_active);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e;
-  if (p.gqa)
+  if (p.mla)
+    e = launch_decode_mla(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev,
+                          valid_topk_dev, out_dev, static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
+  else if (p.gqa)
     e = launch_decode_gqa(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
                           v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
                           static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);

@@ -86,6 +86,14 @@ cudaError_t launch_decode_gqa(const Shape& s, const void* q, const void* k_new, 
                               int* seq_len, const int* valid_topk, void* out, float* partials,
                               int nsplit, uint32_t* status, cudaStream_t st);
 
+// latent attention (one 576-wide KV row shared by all heads, V = its first 512 dims): mma.sync kernel
+bool decode_mla_supported(int dtype, const Shape& s);
+int decode_mla_nsplit(const Shape& s, int n_active, int sm_count);
+size_t decode_mla_partial_floats(const Shape& s, int n_active, int nsplit);
+cudaError_t launch_decode_mla(const Shape& s, const void* q, const void* k_new, const int* slot_ids,
+                              int n_active, void* k_cache, int* seq_len, const int* valid_topk, void* out,
+                              float* partials, int nsplit, uint32_t* status, cudaStream_t st);
+
 // --- small device helpers ---
 template <typename T> __device__ __forceinline__ float to_f32(T x);
 template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }

@@ -229,3 +229,14 @@ def test_late_outlier_logits_refresh_the_running_reference():
     H.check_selection(idx[0], seq, wl)
     for pos, kvh in [(1500, 0), (2600, 1), (4000, 2), (4700, 3)]:
         assert pos in idx[0][kvh]
+
+
+@pytest.mark.parametrize("hq", [64, 128])
+def test_latent_attention_kernel_shapes(hq):
+    """The 576/512 latent layout (tensor-core decode kernel): short and ragged sequences, ring wrap,
+    sharp softmax."""
+    wl = synth.Workload("mla_small", hq, 1, 576, 512, "bf16", 3, 40, 64, 8, 5, batch=1,
+                        prompt_len=(500, 500), decode_steps=6, salience="planted", n_planted=8,
+                        v_aliases_k=True, softmax_scale=2.0 ** -0.5)
+    _run_compress_and_decode(wl, [2, 30, 43, 44, 107, 500, 333], seed=29, steps=6)
+    _run_compress_and_decode(wl, [500, 70], seed=31, steps=45, sharp=3.0, check_ring_every=9)
