@@ -47,14 +47,26 @@ __device__ __forceinline__ void copy_rows(const char* __restrict__ src_base, lon
                                           char* __restrict__ dst_base, int row_b, int s0, int Sc,
                                           int L, int Ls, int Lr, int vt,
                                           const int* __restrict__ idx_row) {
-  const int vecs = row_b / 16;
-  for (int item = threadIdx.x; item < ROWS * vecs; item += NT) {
-    const int s = s0 + item / vecs, c = item % vecs;
-    if (s >= Sc) break;
-    const int p = source_position(s, L, Ls, Lr, vt, idx_row);
-    uint4 val = make_uint4(0u, 0u, 0u, 0u);
-    if (p >= 0) val = __ldg(reinterpret_cast<const uint4*>(src_base + (long long)p * tok_b) + c);
-    reinterpret_cast<uint4*>(dst_base + (long long)s * row_b)[c] = val;
+  const int vecs = row_b / 16, total = ROWS * vecs;
+  // four independent 16-byte loads are in flight per thread before anything is stored
+  for (int base = threadIdx.x; base < total; base += 4 * NT) {
+    uint4 val[4];
+    int slot_of[4], chunk_of[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int item = base + u * NT;
+      const int s = s0 + item / vecs;
+      slot_of[u] = item < total && s < Sc ? s : -1;
+      chunk_of[u] = item % vecs;
+      val[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (slot_of[u] >= 0) {
+        const int p = source_position(s, L, Ls, Lr, vt, idx_row);
+        if (p >= 0) val[u] = __ldg(reinterpret_cast<const uint4*>(src_base + (long long)p * tok_b) + chunk_of[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (slot_of[u] >= 0) reinterpret_cast<uint4*>(dst_base + (long long)slot_of[u] * row_b)[chunk_of[u]] = val[u];
   }
 }
 

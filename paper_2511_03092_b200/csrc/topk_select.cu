@@ -42,6 +42,7 @@ struct TopkShared {
   int bins[2][256];      // this CTA's histogram (double buffered), read by the whole cluster
   int counts[2];         // this CTA's (greater, equal) counts, read by the whole cluster
   int warp_tot[NW + 1];
+  int tot[256];          // cluster-wide histogram of the current pass
   unsigned prefix;
   int remaining;
 };
@@ -142,17 +143,19 @@ __device__ __forceinline__ void cluster_select_digit(cg::cluster_group& cluster,
     mybins[tid] = s;
   }
   cluster.sync();
+  if (tid < 256) {                                   // one bin per thread, eight independent remote reads
+    int s = 0;
+#pragma unroll
+    for (int rr = 0; rr < CL; ++rr) s += cluster.map_shared_rank(mybins, rr)[tid];
+    sh.tot[tid] = s;
+  }
+  __syncthreads();
   if (wid == 0) {
     // lane l owns bins 255-8l .. 248-8l (descending)
     const int remaining = sh.remaining;
     int loc[8], csum = 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) loc[i] = 0;
-    for (int rr = 0; rr < CL; ++rr) {
-      const int* rb = cluster.map_shared_rank(mybins, rr);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) loc[i] += rb[255 - 8 * lane - i];
-    }
+    for (int i = 0; i < 8; ++i) loc[i] = sh.tot[255 - 8 * lane - i];
 #pragma unroll
     for (int i = 0; i < 8; ++i) csum += loc[i];
     int inc = csum;
