@@ -525,6 +525,75 @@ def run_case(args):
                           "score_TFLOPs": flops / ms / 1e9, "status": int(hp.cache.status.item())}))
 
 
+def run_config(args):
+    """The other benchmark configurations (0, 1, 3, 4), reported as context next to the default
+    workload: compress time per prompt and decode time per step with the prompts' caches resident.
+    Config 4's 32 layers share one set of 16 synthetic prompts (layers are independent for timing);
+    a decode step is 32 launches, one per layer."""
+    from paper_2511_03092_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    wl = synth.CONFIGS[args.workload]
+    n_layers, nseq, L = wl.n_layers, wl.batch, wl.prompt_len[1]
+    cfg = B.make_config(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, d_qk=wl.d_qk, d_v=wl.d_v,
+                        dtype=wl.torch_dtype, l_sink=wl.l_sink, l_recent=wl.l_recent, topk=wl.topk,
+                        l_obs=wl.l_obs, pool_kernel=wl.pool_kernel, softmax_scale=wl.scale,
+                        max_seqs=nseq * n_layers, pool_mode=wl.pool_mode, v_aliases_k=wl.v_aliases_k)
+    lay = B.snap_cache_layout(cfg)
+    cache = B.alloc_cache(cfg, lay, dev)
+    ws = torch.empty(B.snap_compress_workspace_bytes(cfg, [0, L]), dtype=torch.uint8, device=dev)
+    prompts = [synth.make_prompt(wl, L, SEED + 31 * i, dev) for i in range(nseq)]
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def compress(p, slot):
+        B.snap_compress(cfg, lay, p["q_obs"].unsqueeze(0), p["k"], p["v"], [0, L], [slot], cache.k_cache,
+                        cache.v_cache, cache.seq_len, cache.valid_topk, None, ws, cache.status)
+
+    compress(prompts[0], 0)                                  # untimed: first-call set-up
+    torch.cuda.synchronize()
+    comp = []
+    for layer in range(n_layers):
+        for i, p in enumerate(prompts):
+            a, b = ev(), ev()
+            a.record(); compress(p, layer * nseq + i); b.record()
+            comp.append((a, b))
+    torch.cuda.synchronize()
+    comp_us = [a.elapsed_time(b) * 1e3 for a, b in comp]
+    dws = torch.empty(B.snap_decode_workspace_bytes(cfg, nseq), dtype=torch.uint8, device=dev)
+    out = torch.empty(nseq, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device=dev)
+    slots = [torch.arange(l * nseq, (l + 1) * nseq, dtype=torch.int32, device=dev) for l in range(n_layers)]
+    ins = [synth.make_decode_inputs(wl, nseq, SEED, s, dev) for s in range(4)]
+
+    def step(s):
+        d = ins[s % 4]
+        for l in range(n_layers):
+            B.snap_decode_attn(cfg, lay, d["q"], d["k_new"], d["v_new"], slots[l], nseq, cache.k_cache, cache.v_cache,
+                               cache.seq_len, cache.valid_topk, out, dws, cache.status)
+
+    steps = min(args.steps, wl.decode_steps)
+    for s in range(args.warmup):
+        step(s)
+    torch.cuda.synchronize()
+    t0, t1 = ev(), ev()
+    t0.record()
+    for s in range(steps):
+        step(s)
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / steps
+    eb = 2 if wl.dtype == "bf16" else 4
+    rows = min(L + 1, wl.slots)
+    step_bytes = n_layers * nseq * wl.n_kv_heads * rows * (wl.d_qk + (0 if wl.v_aliases_k else wl.d_v)) * eb
+    peak, _ = _peaks()
+    print(json.dumps({
+        "workload": wl.name, "n_layers": n_layers, "sequences": nseq, "prompt_tokens": L, "cache_slots": wl.slots,
+        "compress_us_per_prompt_layer_median": statistics.median(comp_us),
+        "compress_ms_total": sum(comp_us) / 1e3, "decode_steps_timed": steps, "decode_us_per_step": ms * 1e3,
+        "decode_tokens_per_s": nseq / (ms * 1e-3), "decode_bytes_per_step": step_bytes,
+        "decode_GBps": step_bytes / (ms * 1e-3) / 1e9, "decode_frac_of_measured_hbm": step_bytes / (ms * 1e-3) / 1e9 / peak,
+        "status": int(cache.status.item())}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -536,9 +605,13 @@ def main():
     ap.add_argument("--case", choices=["decode", "compress"], default=None,
                     help="small single-kernel-family case for profiler captures")
     ap.add_argument("--case-len", type=int, default=131072)
+    ap.add_argument("--workload", type=int, choices=[0, 1, 3, 4], default=None,
+                    help="report compress and decode times of another benchmark configuration (context only)")
     args = ap.parse_args()
     if args.case:
         run_case(args)
+    elif args.workload is not None:
+        run_config(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
