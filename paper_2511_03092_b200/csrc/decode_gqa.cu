@@ -384,6 +384,7 @@ __global__ void __launch_bounds__(NT, (G == 8 ? 2 : 3)) decode_gqa_kernel(const 
     if (tid == 0) { ph[0] = M; ph[1] = L; }
     ph[2 + tid] = O;
   }
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
 // Merge the splits of one (sequence, query head); maxima are in the log2 domain.
@@ -393,6 +394,9 @@ __global__ void __launch_bounds__(D) decode_gqa_merge_kernel(const float* __rest
                                                              int* seq_len, int max_seqs, int bump) {
   const int h = blockIdx.x, i = blockIdx.y, t = threadIdx.x;
   const float* p = partials + ((long long)i * Hq + h) * nsplit * PS;
+  // launched with programmatic stream serialisation: the grid may start while the split kernel
+  // drains; everything the split kernel wrote is visible after this wait
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   float M = -INFINITY;
   for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * PS]);
   float L = 0.f, O = 0.f;
@@ -424,11 +428,23 @@ cudaError_t launch_g(const FastArgs& a, int n_active, __nv_bfloat16* out, int* s
   dim3 grid(a.nsplit, a.Hkv, n_active);
   decode_gqa_kernel<G><<<grid, NT, smem, st>>>(a);
   count_launch();
-  dim3 mgrid(a.Hq, n_active);
-  decode_gqa_merge_kernel<<<mgrid, D, 0, st>>>(a.partials, out, a.Hq, a.nsplit, a.slot_ids, seq_len,
-                                               a.max_seqs, bump);
+  // the merge kernel is a programmatic dependent launch: its launch latency overlaps the split kernel's tail
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(a.Hq, n_active);
+  lc.blockDim = dim3(D);
+  lc.dynamicSmemBytes = 0;
+  lc.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  const float* parts = a.partials;
+  const int* slots = a.slot_ids;
+  cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_merge_kernel, parts, out, a.Hq, a.nsplit, slots, seq_len,
+                                     a.max_seqs, bump);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
