@@ -184,24 +184,22 @@ class HotPath:
 def run_ours(args):
     from paper_2511_03092_b200 import binding as B
     B.lib()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2511_03092_b200 import replicas
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    grp = replicas.init_from_env("nccl", dev)
+    rank, world = grp.rank, grp.world
     wl = synth.CONFIGS[2]
-    hp = HotPath(wl, dev, SEED + 1000 * rank)
-    sched = synth.continuous_batching_schedule(wl, args.warmup + args.steps + 1, SEED + rank)
+    hp = HotPath(wl, dev, grp.seed_for(SEED))
+    sched = synth.continuous_batching_schedule(wl, args.warmup + args.steps + 1, grp.seed_for(SEED, 1))
     hp.initial_fill()
     torch.cuda.synchronize()
 
     def barrier():
         torch.cuda.synchronize()
         if world > 1:
-            dist.barrier()
+            grp.barrier()
             torch.cuda.synchronize()
 
     def step(i, ev=None):
@@ -238,10 +236,7 @@ def run_ours(args):
     clocks = sampler.stop(host_t0, host_t1) if rank == 0 else None
     ms = t0.elapsed_time(t1)
     dec_ms = [a.elapsed_time(b) for a, b in evs]
-    if world > 1:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = grp.max_over_ranks(ms, dev)
     status = int(hp.cache.status.item())
 
     # ---- end to end: inputs in pinned host memory, outputs read back, same steps ----
@@ -272,14 +267,10 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = grp.max_over_ranks(e2e_ms, dev)
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        grp.close()
         return
     peak, peak_src = _peaks()
     dec_avg_ms = sum(dec_ms) / len(dec_ms)
@@ -312,8 +303,7 @@ def run_ours(args):
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl, hp, sched)
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    grp.close()
 
 
 def extras(hp, wl, dev):
