@@ -64,6 +64,11 @@ bool use_umma(int dtype, const Shape& s) {
   if (env && (!strcmp(env, "mma") || !strcmp(env, "simt"))) return false;
   return score_umma_supported(dtype, s);
 }
+bool use_umma_wide(int dtype, const Shape& s) {
+  const char* env = getenv("SNAP_SCORE_PATH");
+  if (env && (!strcmp(env, "mma") || !strcmp(env, "simt"))) return false;
+  return !score_umma_supported(dtype, s) && score_umma_wide_supported(dtype, s);
+}
 bool use_mma(int dtype, const Shape& s) {
   const char* env = getenv("SNAP_SCORE_PATH");
   if (env && !strcmp(env, "simt")) return false;
@@ -73,7 +78,7 @@ bool use_mma(int dtype, const Shape& s) {
 // Scratch regions of one chunk of prompts (offsets relative to the chunk area).
 struct ChunkPlan {
   int n_scored, max_le, nsplit, c_stride;
-  size_t part_off, stats_off, c_off, p_off, bytes;
+  size_t part_off, stats_off, c_off, p_off, cpart_off, bytes;
 };
 
 ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, int n) {
@@ -94,6 +99,7 @@ ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, in
   if (nsplit > 64) nsplit = 64;
   if (nsplit < 1) nsplit = 1;
   if (use_umma(dtype, s)) p.nsplit = score_umma_nsplit(s, p.n_scored, p.max_le, sm_count());
+  else if (use_umma_wide(dtype, s)) p.nsplit = score_umma_wide_nsplit(s, p.n_scored, p.max_le, sm_count());
   else if (use_mma(dtype, s)) p.nsplit = score_mma_nsplit(s, p.n_scored, p.max_le, sm_count());
   else p.nsplit = (int)nsplit;
   p.c_stride = (int)align_up((size_t)p.max_le, 64);
@@ -103,6 +109,8 @@ ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, in
   p.stats_off = off; off += align_up(nz * R * sizeof(float2));
   p.c_off = off;     off += align_up(nz * p.c_stride * sizeof(float));
   p.p_off = off;     off += align_up(nz * p.c_stride * sizeof(float));
+  p.cpart_off = off;
+  if (use_umma_wide(dtype, s)) off += align_up(nz * score_umma_wide_row_blocks(s) * p.c_stride * sizeof(float));
   p.bytes = off;
   return p;
 }
@@ -283,6 +291,9 @@ int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout, const v
       buf.P = reinterpret_cast<float*>(chunk_ws + p.p_off);
       buf.c_stride = p.c_stride; buf.nsplit = p.nsplit;
       const cudaError_t e = use_umma(cfg->dtype, s)  ? launch_score_umma(s, b, q_obs_dev, src, buf, status_dev, st)
+                            : use_umma_wide(cfg->dtype, s)
+                                ? launch_score_umma_wide(s, b, q_obs_dev, src, buf,
+                                                         reinterpret_cast<float*>(chunk_ws + p.cpart_off), status_dev, st)
                             : use_mma(cfg->dtype, s) ? launch_score_mma(s, b, q_obs_dev, src, buf, st)
                                                      : launch_score_simt(cfg->dtype, s, b, q_obs_dev, src, buf, st);
       if (e != cudaSuccess) return SNAP_ERR_CUDA;

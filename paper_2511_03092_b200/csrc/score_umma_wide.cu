@@ -1,0 +1,352 @@
+// Observation-window scores (Eq. 4 -> Eq. 1) on tcgen05 for wide rows and many window rows --
+// the latent-attention shape: 128 query heads x Lo rows (4096 window rows) against 576-wide keys.
+//
+// Same roles as the 128-wide kernel (TMA producer warp, single-thread MMA issuer, eight epilogue
+// warps reading TMEM), but the contraction dimension is streamed: grid = (candidate splits,
+// blocks of 128 window rows, prompts).  A CTA keeps its 128-row query block resident in shared
+// memory (one 16 KB swizzled slab per 64 dims) and, for every candidate tile, pulls the keys
+// through a 2-stage ring one 64-dim slab at a time, accumulating in tensor memory; two
+// accumulator buffers let the next tile's MMAs overlap the epilogue of the current one.
+//   pass 1  M = 128 query rows, N = 256 candidates; thread = query row; the two epilogue groups
+//           take 128 candidates each and their (reference max, sum) pairs are merged at the end.
+//   pass 2  M = 128 candidates, N = 128 query rows; thread = candidate; each group sums
+//           exp2(s_ij - m_i - log2 l_i) over 64 rows (constants in registers); the per-row-block
+//           partial column sums go to scratch and a small kernel adds the row blocks in a fixed
+//           order (deterministic, no atomics).
+// Every mbarrier wait is bounded; a wait that runs out raises SNAP_DEV_WAIT_TIMEOUT.
+#include "snap_internal.cuh"
+#include "umma_helpers.cuh"
+
+namespace snap {
+namespace {
+
+using namespace umma;
+
+constexpr int NTHREADS = 320, NS = 2, STAGE_B = 32768, QH_B = 16384, MAXH = 9;
+
+struct WideArgs {
+  int Hq, Hkv, g, Lo, Ls, Lr, R, NH, RB;
+  float scale_log2;
+  SeqBatch b;
+  ScoreBuffers buf;
+  float* cpart;          // [nz][RB][c_stride] partial column sums of pass 2
+  uint32_t* status;
+};
+
+template <int PASS>
+__global__ void __launch_bounds__(NTHREADS, 1)
+score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tmap_q,
+                       const __grid_constant__ CUtensorMap tmap_k) {
+  constexpr int TNP = PASS == 1 ? 256 : 128;                  // candidates per tile
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int NH = a.NH;
+  unsigned char* Qs = smem;                                   // [NH][128 rows][128 B]
+  unsigned char* Ks = Qs + NH * QH_B;                         // [NS][up to 256 rows][128 B]
+  float* mu_s = reinterpret_cast<float*>(Ks + NS * STAGE_B);  // [128] pass 2: m_i + log2 l_i of this row block
+  float2* xch = reinterpret_cast<float2*>(mu_s + 128);        // [128] exchange between the epilogue groups
+  uint64_t* bars = reinterpret_cast<uint64_t*>(xch + 128);    // full[NS] empty[NS] tfull[2] tempty[2] qfull
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NS + 5);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rb = blockIdx.y, z = blockIdx.z, si = z / a.Hkv, kvh = z % a.Hkv;
+  const int seq = a.b.seq_of_score[si];
+  const int Le = a.b.len[seq] - a.Ls - a.Lr;
+  const int R = a.R;
+  const int ntiles = (Le + TNP - 1) / TNP;
+  const int t0 = (int)((long long)ntiles * blockIdx.x / a.buf.nsplit);
+  const int t1 = (int)((long long)ntiles * (blockIdx.x + 1) / a.buf.nsplit);
+  const int nt = t1 - t0;
+
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8 * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8 * (NS + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8 * (2 * NS + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8 * (2 * NS + 2 + b); };
+  const uint32_t qfull_bar = bar0 + 8 * (2 * NS + 4);
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+    mbar_init(qfull_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (PASS == 2 && tid < 128) {
+    const float2 st = a.buf.stats[(long long)z * R + rb * 128 + tid];
+    mu_s[tid] = st.x - log2f(st.y);
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int eg = warp >= 2 ? (warp - 2) >> 2 : 0;             // epilogue group
+  const int lrow = 32 * (warp & 3) + lane;                    // accumulator row = TMEM lane
+  float m_ref = -INFINITY, l_sum = 0.f;                       // pass 1: statistics of query row rb*128 + lrow
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0 && nt > 0) {
+      const int row0 = ((a.b.first_seq + seq) * a.Hq + kvh * a.g) * a.Lo + rb * 128;
+      mbar_expect_tx(qfull_bar, (unsigned)NH * QH_B);
+      for (int h = 0; h < NH; ++h) tma_load_2d(smem_u32(Qs) + h * QH_B, &tmap_q, h * 64, row0, qfull_bar);
+      const int tok0 = a.b.tok_off[seq] + a.Ls;
+      bool ok = true;
+      for (int it = 0; it < nt && ok; ++it)
+        for (int h = 0; h < NH; ++h) {
+          const int q = it * NH + h, s = q % NS;
+          if (!mbar_wait(empty_bar(s), ((unsigned)(q / NS) & 1u) ^ 1u, abort_flag)) { *abort_flag = 1; ok = false; break; }
+          mbar_expect_tx(full_bar(s), (unsigned)TNP * 128u);
+          tma_load_3d(smem_u32(Ks) + s * STAGE_B, &tmap_k, h * 64, kvh, tok0 + (t0 + it) * TNP, full_bar(s));
+        }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0 && nt > 0) {
+      const uint32_t idesc = PASS == 1 ? idesc_bf16(128, 256) : idesc_bf16(128, 128);
+      bool ok = mbar_wait(qfull_bar, 0u, abort_flag);
+      for (int it = 0; it < nt && ok; ++it) {
+        const int b = it & 1;
+        ok = mbar_wait(tempty_bar(b), ((unsigned)(it / 2) & 1u) ^ 1u, abort_flag);
+        for (int h = 0; h < NH && ok; ++h) {
+          const int q = it * NH + h, s = q % NS;
+          ok = mbar_wait(full_bar(s), (unsigned)(q / NS) & 1u, abort_flag);
+          if (!ok) break;
+          fence_after();
+          const uint32_t kst = smem_u32(Ks) + s * STAGE_B, qst = smem_u32(Qs) + h * QH_B;
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            if (PASS == 1)
+              mma_bf16(tmem_base + b * 256, smem_desc(qst + ks * 32), smem_desc(kst + ks * 32), idesc, (h | ks) != 0);
+            else
+              mma_bf16(tmem_base + b * 256, smem_desc(kst + ks * 32), smem_desc(qst + ks * 32), idesc, (h | ks) != 0);
+          }
+          mma_commit(empty_bar(s));                            // slab may be refilled once these MMAs have read it
+        }
+        if (ok) mma_commit(tfull_bar(b));                      // accumulator buffer complete
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+    bool ok = true;
+    float mu[64];
+    if (PASS == 2) {
+#pragma unroll
+      for (int i = 0; i < 64; ++i) mu[i] = -mu_s[64 * eg + i];
+    }
+    for (int it = 0; it < nt; ++it) {
+      const int b = it & 1;
+      const bool landed = mbar_wait(tfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag);
+      if (!landed) {
+        *abort_flag = 1;
+        ok = false;
+        if (PASS == 1) break;                                  // pass 2 leaves through the group barrier below
+      }
+      fence_after();
+      uint32_t ra[16], rb16[16];
+      if (PASS == 1) {
+        const uint32_t col0 = lane_addr + b * 256 + eg * 128;
+        const int cand0 = (t0 + it) * TNP + eg * 128;         // first candidate of this group's columns
+        const bool full_tile = cand0 + 128 <= Le;
+        // sum of exp2 over this group's 128 columns relative to reference `ref`
+        auto sweep = [&](float ref, bool want_max, float& vmax) -> float {
+          float s4[4] = {0.f, 0.f, 0.f, 0.f};
+          tmem_ld16_issue(col0, ra);
+#pragma unroll
+          for (int c = 0; c < 8; c += 2) {
+            tmem_ld16_wait(ra);
+            tmem_ld16_issue(col0 + 16 * (c + 1), rb16);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float v = __uint_as_float(ra[i]) * a.scale_log2;
+              const bool in = full_tile || cand0 + 16 * c + i < Le;
+              if (want_max) { if (in) vmax = fmaxf(vmax, v); }
+              else s4[i & 3] += in ? fast_exp2(v - ref) : 0.f;
+            }
+            tmem_ld16_wait(rb16);
+            if (c + 2 < 8) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float v = __uint_as_float(rb16[i]) * a.scale_log2;
+              const bool in = full_tile || cand0 + 16 * (c + 1) + i < Le;
+              if (want_max) { if (in) vmax = fmaxf(vmax, v); }
+              else s4[i & 3] += in ? fast_exp2(v - ref) : 0.f;
+            }
+          }
+          return (s4[0] + s4[1]) + (s4[2] + s4[3]);
+        };
+        float dummy = 0.f;
+        float sum = sweep(m_ref, false, dummy);
+        // a logit far above the reference (or the first tile): refresh it; the TMEM loads are
+        // warp-collective, so the whole warp takes the branch if any row needs it
+        if (__any_sync(0xffffffffu, !(sum < 65536.f))) {
+          float vmax = -INFINITY;
+          (void)sweep(0.f, true, vmax);
+          const float mn = fmaxf(m_ref, vmax);
+          sum = 0.f;
+          if (mn != -INFINITY) {
+            l_sum *= m_ref == -INFINITY ? 0.f : fast_exp2(m_ref - mn);
+            m_ref = mn;
+          }
+          const float s2 = sweep(mn == -INFINITY ? 0.f : mn, false, dummy);
+          if (mn != -INFINITY) sum = s2;
+        }
+        l_sum += sum;
+      } else {
+        const uint32_t col0 = lane_addr + b * 256 + eg * 64;
+        const int cand = (t0 + it) * TNP + lrow;
+        float s = 0.f;
+        if (landed) {
+          float s4[4] = {0.f, 0.f, 0.f, 0.f};
+          tmem_ld16_issue(col0, ra);
+#pragma unroll
+          for (int c = 0; c < 4; c += 2) {
+            tmem_ld16_wait(ra);
+            tmem_ld16_issue(col0 + 16 * (c + 1), rb16);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, mu[16 * c + i]));
+            tmem_ld16_wait(rb16);
+            if (c + 2 < 4) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(rb16[i]), a.scale_log2, mu[16 * (c + 1) + i]));
+          }
+          s = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+        }
+        float* xs = reinterpret_cast<float*>(xch) + b * 128;
+        if (eg == 1) xs[lrow] = s;
+        unsigned stop;                                         // barrier over the 8 epilogue warps + agreement on giving up
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+            "bar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(stop) : "r"((unsigned)(!landed || *abort_flag)) : "memory");
+        if (eg == 0 && !stop && cand < Le)
+          a.cpart[((long long)z * a.RB + rb) * a.buf.c_stride + cand] = s + xs[lrow];
+        if (stop) { *abort_flag = 1; ok = false; }
+      }
+      fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(b));
+      if (!ok) break;
+    }
+    if (!ok) *abort_flag = 1;
+    if (PASS == 1 && eg == 1) xch[lrow] = make_float2(m_ref, l_sum);
+  }
+
+  fence_before();
+  __syncthreads();
+  fence_after();
+  if (PASS == 1 && warp >= 2 && eg == 0) {                     // the two groups took different candidates of each tile
+    const float2 o = xch[lrow];
+    merge_ml(m_ref, l_sum, o.x, o.y);
+    a.buf.part_stats[((long long)z * a.buf.nsplit + blockIdx.x) * R + rb * 128 + lrow] = make_float2(m_ref, l_sum);
+  }
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
+}
+
+// C[z][j] = sum over the row blocks of the partial column sums, in a fixed order.
+__global__ void score_rowblock_reduce_kernel(const float* __restrict__ cpart, float* __restrict__ C, int RB,
+                                             int c_stride, SeqBatch b, int Hkv, int Ls, int Lr) {
+  const int z = blockIdx.y, si = z / Hkv;
+  const int Le = b.len[b.seq_of_score[si]] - Ls - Lr;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= Le) return;
+  float s = 0.f;
+  for (int rb = 0; rb < RB; ++rb) s += cpart[((long long)z * RB + rb) * c_stride + j];
+  C[(long long)z * c_stride + j] = s;
+}
+
+size_t wide_smem_bytes(int NH) {
+  return (size_t)NH * QH_B + NS * STAGE_B + 128 * sizeof(float) + 128 * sizeof(float2) + (2 * NS + 5) * 8 + 16 + 1024;
+}
+
+}  // namespace
+
+bool score_umma_wide_supported(int dtype, const Shape& s) {
+  const int R = s.g * s.Lo;
+  return dtype == SNAP_BF16 && s.d_qk % 64 == 0 && s.d_qk / 64 <= MAXH && R % 128 == 0 &&
+         umma::encode_tiled_fn() != nullptr;
+}
+
+int score_umma_wide_row_blocks(const Shape& s) { return s.g * s.Lo / 128; }
+
+// Candidate splits: about two CTAs per SM in sequence over (splits x row blocks x prompts x KV heads).
+int score_umma_wide_nsplit(const Shape& s, int n_scored, int max_le, int sm_count) {
+  const int tiles = (max_le + 255) / 256;
+  const long long base = (long long)n_scored * s.Hkv * score_umma_wide_row_blocks(s);
+  long long ns = (2LL * sm_count + base / 2) / base;
+  if (ns > tiles) ns = tiles;
+  if (ns > 512) ns = 512;
+  if (ns < 1) ns = 1;
+  return (int)ns;
+}
+
+cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
+                                   const ScoreBuffers& buf, float* cpart, uint32_t* status, cudaStream_t st) {
+  if (b.n_scored == 0) return cudaSuccess;
+  umma::EncodeTiledFn enc = umma::encode_tiled_fn();
+  if (!enc) return cudaErrorNotSupported;
+  WideArgs a;
+  a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Lo = s.Lo; a.Ls = s.Ls; a.Lr = s.Lr; a.R = s.g * s.Lo;
+  a.NH = s.d_qk / 64; a.RB = a.R / 128;
+  a.scale_log2 = s.scale * 1.4426950408889634f;
+  a.b = b; a.buf = buf; a.cpart = cpart; a.status = status;
+
+  CUtensorMap tq, tk1, tk2;
+  const cuuint32_t estr2[2] = {1, 1}, estr3[3] = {1, 1, 1};
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)s.d_qk, (cuuint64_t)(b.first_seq + b.n) * s.Hq * s.Lo};
+    const cuuint64_t strides[1] = {(cuuint64_t)s.d_qk * 2};
+    const cuuint32_t box[2] = {64, 128};
+    if (enc(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(q_obs), dims, strides, box, estr2,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  long long tokens = 0;
+  for (int i = 0; i < b.n; ++i) tokens = tokens > (long long)b.tok_off[i] + b.len[i] ? tokens : (long long)b.tok_off[i] + b.len[i];
+  const long long head_stride = src.k_head_stride >= s.d_qk ? src.k_head_stride : s.d_qk;
+  const cuuint64_t kdims[3] = {(cuuint64_t)s.d_qk, (cuuint64_t)s.Hkv, (cuuint64_t)tokens};
+  const cuuint64_t kstrides[2] = {(cuuint64_t)head_stride * 2, (cuuint64_t)src.k_tok_stride * 2};
+  for (int pass = 1; pass <= 2; ++pass) {
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)(pass == 1 ? 256 : 128)};
+    if (enc(pass == 1 ? &tk1 : &tk2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(src.k), kdims, kstrides,
+            box, estr3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  const size_t smem = wide_smem_bytes(a.NH);
+  static size_t attr_bytes = 0;
+  if (smem > attr_bytes) {
+    cudaError_t e = cudaFuncSetAttribute(score_umma_wide_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(score_umma_wide_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_bytes = smem;
+  }
+  const int nz = b.n_scored * s.Hkv;
+  int max_le = 0;
+  for (int i = 0; i < b.n; ++i)
+    if (b.score_idx[i] >= 0) max_le = max_le > b.len[i] - s.Ls - s.Lr ? max_le : b.len[i] - s.Ls - s.Lr;
+  dim3 grid(buf.nsplit, a.RB, nz);
+  score_umma_wide_kernel<1><<<grid, NTHREADS, smem, st>>>(a, tq, tk1);
+  count_launch();
+  cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
+  if (e != cudaSuccess) return e;
+  score_umma_wide_kernel<2><<<grid, NTHREADS, smem, st>>>(a, tq, tk2);
+  count_launch();
+  score_rowblock_reduce_kernel<<<dim3((max_le + 255) / 256, nz), 256, 0, st>>>(cpart, buf.C, a.RB, buf.c_stride, b,
+                                                                            s.Hkv, s.Ls, s.Lr);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace snap

@@ -62,6 +62,12 @@ bool score_umma_supported(int dtype, const Shape& s);
 int score_umma_nsplit(const Shape& s, int n_scored, int max_le, int sm_count);
 cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
                               const ScoreBuffers& buf, uint32_t* status, cudaStream_t st);
+// tcgen05 version for wide rows / many window rows (d_qk up to 576, g*Lo a multiple of 128)
+bool score_umma_wide_supported(int dtype, const Shape& s);
+int score_umma_wide_row_blocks(const Shape& s);
+int score_umma_wide_nsplit(const Shape& s, int n_scored, int max_le, int sm_count);
+cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
+                                   const ScoreBuffers& buf, float* cpart, uint32_t* status, cudaStream_t st);
 cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffers& buf,
                              int* idx_out, uint32_t* status, cudaStream_t st);
 cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KVSource& src,

@@ -240,3 +240,25 @@ def test_latent_attention_kernel_shapes(hq):
                         v_aliases_k=True, softmax_scale=2.0 ** -0.5)
     _run_compress_and_decode(wl, [2, 30, 43, 44, 107, 500, 333], seed=29, steps=6)
     _run_compress_and_decode(wl, [500, 70], seed=31, steps=45, sharp=3.0, check_ring_every=9)
+
+
+def test_late_outlier_logits_latent_shape():
+    """Same hazard as above on the wide-row score kernel (576-wide keys, 512 window rows)."""
+    wl = synth.Workload("mla_outlier", 64, 1, 576, 512, "bf16", 3, 40, 100, 8, 5, batch=1,
+                        prompt_len=(3000, 3000), decode_steps=2, salience="planted", n_planted=8,
+                        v_aliases_k=True, softmax_scale=2.0 ** -0.5)
+    L = 3000
+    p = synth.make_prompt(wl, L, seed=43)
+    q = p["q_obs"].float()
+    k = p["k"].float()
+    for hq, row, pos, c in [(0, 0, 900, 30.0), (17, 5, 1700, 45.0), (40, 7, 2500, 25.0), (63, 3, 2900, 60.0)]:
+        qv = q[hq, row]
+        k[pos, 0] = qv * (c / (wl.scale * float(qv @ qv)))
+    p["k"] = k.to(wl.torch_dtype)
+    layer = H.GpuLayer(wl, max_seqs=1)
+    idx = layer.compress([p], [0])
+    assert layer.status() == 0
+    seq = H.oracle_compress(wl, p)
+    H.check_selection(idx[0], seq, wl)
+    for pos in (900, 1700, 2500, 2900):
+        assert pos in idx[0][0]
