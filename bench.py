@@ -356,6 +356,27 @@ def extras(hp, wl, dev):
     out["full_kv_decode_GBps"] = full_bytes / (full_ms * 1e-3) / 1e9
     out["full_kv_bytes_over_compressed_bytes"] = full_bytes / hp.decode_bytes()
     out["full_kv_status"] = int(cache.status.item())
+    del cache, dws
+    # (3) the slice-and-concatenate update the ring buffer replaces (Section 3.2.1): whole cache rewritten per step
+    c = hp.cache
+    bufs = [(torch.empty_like(c.k_cache), torch.empty_like(c.v_cache)) for _ in range(2)]
+    seq_len = c.seq_len.clone()
+    src = (c.k_cache, c.v_cache)
+    times = []
+    for r in range(8):
+        d = hp.decode_in[r % DECODE_RING]
+        dst = bufs[r % 2]
+        a, b = ev(), ev()
+        a.record()
+        B.snap_append_kv_concat(hp.cfg, hp.layout, d["k_new"], d["v_new"], hp.slots_dev, wl.batch, src[0], src[1],
+                                dst[0], dst[1], seq_len, c.status)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+        src = dst
+    out["concat_update_ms"] = statistics.median(times[2:])
+    out["concat_update_bytes"] = 2 * wl.batch * wl.n_kv_heads * hp.layout.slots * (wl.d_qk + wl.d_v) * 2
+    out["ring_append_bytes"] = 2 * wl.batch * wl.n_kv_heads * (wl.d_qk + wl.d_v) * 2
     return out
 
 

@@ -198,6 +198,28 @@ int snap_decode_attn_static(const snap_config_t* cfg, const snap_layout_t* layou
                             int32_t* seq_len_dev, const int32_t* valid_topk_dev,
                             void* out_dev, uint32_t* status_dev, void* cuda_stream);
 
+/*
+ * Section 3.2.1's counter-example, as a measured baseline: the rolling window kept in position
+ * order and updated by slicing and concatenating, which yields a NEW cache every step.
+ * For each active sequence (L = seq_len_dev[slot]), rows of the output cache are
+ *   L <  Ls + Lr:  the input rows, with row L replaced by the new token (a plain scatter);
+ *   L >= Ls + Lr:  sinks [0, Ls) and selected rows [Ls+Lr, Sc) copied, window row r takes input
+ *                  row r + 1 for Ls <= r < Ls+Lr-1, and the new token goes to row Ls+Lr-1.
+ * Then seq_len_dev[slot] += 1.  Slots that are not listed in slot_ids_dev are not copied.
+ * The output buffers must differ from the input buffers (SNAP_ERR_INVALID_ARG otherwise); both
+ * have the cache layout of snap_cache_layout and are owned by the caller.  A cache that
+ * snap_compress built has its window in ring order (Eq. 3); it is in position order as well
+ * exactly when (L - Ls) is a multiple of Lr or L <= Ls + Lr.  snap_decode_attn with
+ * k_new_dev == NULL reads either order, since attention does not depend on the row order.
+ * Traffic per step: the whole cache read and written, against one row for snap_append_kv.
+ */
+int snap_append_kv_concat(const snap_config_t* cfg, const snap_layout_t* layout,
+                          const void* k_new_dev, const void* v_new_dev,
+                          const int32_t* slot_ids_dev, int32_t n_active,
+                          const void* k_cache_in_dev, const void* v_cache_in_dev,
+                          void* k_cache_out_dev, void* v_cache_out_dev,
+                          int32_t* seq_len_dev, uint32_t* status_dev, void* cuda_stream);
+
 /* Text for a snap_status value (static storage). */
 const char* snap_status_string(int status);
 

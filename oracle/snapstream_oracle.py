@@ -333,3 +333,29 @@ def expected_cache(seq: OracleSequence):
                 Kc[kvh, s] = seq.k_hist[p][kvh]
                 Vc[kvh, s] = seq.v_hist[p][kvh]
     return Kc, (None if cfg.v_aliases_k else Vc), pos_map
+
+
+def expected_cache_position_order(seq: OracleSequence):
+    """Cache image under the slice-and-concatenate update that Section 3.2.1 describes as the
+    naive alternative to the ring: sinks at [0, Ls), the rolling window in position order
+    (its i-th oldest entry at Ls + i), the i-th selected position at Lsr + i, zeros elsewhere.
+    Same return values as expected_cache."""
+    cfg = seq.cfg
+    lay = cache_layout(cfg.l_sink, cfg.l_recent, cfg.topk)
+    Sc = lay["slots"]
+    Kc = np.zeros((cfg.n_kv_heads, Sc, cfg.d_qk), dtype=np.float64)
+    Vc = np.zeros((cfg.n_kv_heads, Sc, cfg.d_v), dtype=np.float64)
+    pos_map = -np.ones((cfg.n_kv_heads, Sc), dtype=np.int64)
+    for kvh in range(cfg.n_kv_heads):
+        for p in seq.sinks:
+            pos_map[kvh, p] = p
+        for i, p in enumerate(seq.recents):
+            pos_map[kvh, cfg.l_sink + i] = p
+        for i, p in enumerate(seq.topk_pos[kvh]):
+            pos_map[kvh, lay["topk_off"] + i] = int(p)
+        for s in range(Sc):
+            p = pos_map[kvh, s]
+            if p >= 0:
+                Kc[kvh, s] = seq.k_hist[p][kvh]
+                Vc[kvh, s] = seq.v_hist[p][kvh]
+    return Kc, (None if cfg.v_aliases_k else Vc), pos_map

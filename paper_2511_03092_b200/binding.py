@@ -68,6 +68,8 @@ def lib() -> C.CDLL:
                                 vp, vp, vp, vp, vp, vp, sz, vp, vp]
     L.snap_append_kv.restype = C.c_int
     L.snap_append_kv.argtypes = [pcfg, play, vp, vp, vp, i32, vp, vp, vp, vp, vp]
+    L.snap_append_kv_concat.restype = C.c_int
+    L.snap_append_kv_concat.argtypes = [pcfg, play, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
     L.snap_decode_attn.restype = C.c_int
     L.snap_decode_attn.argtypes = [pcfg, play, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     L.snap_decode_attn_static.restype = C.c_int
@@ -77,7 +79,7 @@ def lib() -> C.CDLL:
 
 
 EXPORTS = ("snap_cache_layout", "snap_compress_workspace_bytes", "snap_decode_workspace_bytes",
-           "snap_compress", "snap_append_kv", "snap_decode_attn", "snap_decode_attn_static", "snap_status_string",
+           "snap_compress", "snap_append_kv", "snap_append_kv_concat", "snap_decode_attn", "snap_decode_attn_static", "snap_status_string",
            "snap_kernel_launch_count")
 
 
@@ -163,6 +165,16 @@ def snap_append_kv(cfg: SnapConfig, layout: SnapLayout, k_new, v_new, slot_ids_d
     _check(lib().snap_append_kv(C.byref(cfg), C.byref(layout), _ptr(k_new), _ptr(v_new), _ptr(slot_ids_dev),
                                 int(n_active), _ptr(k_cache), _ptr(v_cache), _ptr(seq_len), _ptr(status),
                                 _stream(stream)), "snap_append_kv")
+
+
+def snap_append_kv_concat(cfg: SnapConfig, layout: SnapLayout, k_new, v_new, slot_ids_dev, n_active: int,
+                          k_cache_in, v_cache_in, k_cache_out, v_cache_out, seq_len, status=None,
+                          stream=None) -> None:
+    """Baseline update by slicing and concatenating into a second cache (position-ordered window)."""
+    _check(lib().snap_append_kv_concat(C.byref(cfg), C.byref(layout), _ptr(k_new), _ptr(v_new),
+                                       _ptr(slot_ids_dev), int(n_active), _ptr(k_cache_in), _ptr(v_cache_in),
+                                       _ptr(k_cache_out), _ptr(v_cache_out), _ptr(seq_len), _ptr(status),
+                                       _stream(stream)), "snap_append_kv_concat")
 
 
 def snap_decode_attn(cfg: SnapConfig, layout: SnapLayout, q, k_new, v_new, slot_ids_dev, n_active: int,

@@ -262,3 +262,53 @@ def test_late_outlier_logits_latent_shape():
     H.check_selection(idx[0], seq, wl)
     for pos in (900, 1700, 2500, 2900):
         assert pos in idx[0][0]
+
+
+@pytest.mark.parametrize("wl,lengths", [(SMALL_BF16, [3, 30, 4 + 5 * 48]), (SMALL_MLA, [2, 3 + 2 * 40])])
+def test_concat_update_baseline_matches_oracle(wl, lengths):
+    """The slice-and-concatenate update (position-ordered window, new cache every step) gives
+    the oracle's outputs and, row for row, the oracle's position-ordered cache image."""
+    n = len(lengths)
+    prompts = [synth.make_prompt(wl, L, 51 + i) for i, L in enumerate(lengths)]
+    layer = H.GpuLayer(wl, n)
+    layer.compress(prompts, list(range(n)))
+    seqs = [H.oracle_compress(wl, p) for p in prompts]
+    c = layer.cache
+    cur_k, cur_v = c.k_cache, c.v_cache
+    alt_k = torch.zeros_like(cur_k)
+    alt_v = None if cur_v is None else torch.zeros_like(cur_v)
+    slots_dev = torch.arange(n, dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.snap_decode_workspace_bytes(layer.cfg, n), dtype=torch.uint8, device="cuda")
+    for step in range(wl.l_recent + 12):
+        d = synth.make_decode_inputs(wl, n, 51, step)
+        q, kn = d["q"].cuda(), d["k_new"].cuda()
+        vn = None if wl.v_aliases_k else d["v_new"].cuda()
+        B.snap_append_kv_concat(layer.cfg, layer.layout, kn, vn, slots_dev, n, cur_k, cur_v, alt_k, alt_v,
+                                c.seq_len, c.status)
+        cur_k, alt_k, cur_v, alt_v = alt_k, cur_k, alt_v, cur_v
+        out = torch.empty(n, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device="cuda")
+        B.snap_decode_attn(layer.cfg, layer.layout, q, None, None, slots_dev, n, cur_k, cur_v, c.seq_len,
+                           c.valid_topk, out, ws, c.status)
+        for i in range(n):
+            ref = orc.decode_step(seqs[i], synth.to_f64(d["q"][i]), synth.to_f64(d["k_new"][i]),
+                                  None if wl.v_aliases_k else synth.to_f64(d["v_new"][i]))
+            if step % 8 == 0 or step >= wl.l_recent:
+                H.check_output(out[i], ref, wl, f"step {step} seq {i}")
+    assert layer.status() == 0
+    for i in range(n):
+        assert int(c.seq_len[i]) == seqs[i].n_tokens
+        Kc, Vc, _ = orc.expected_cache_position_order(seqs[i])
+        np.testing.assert_array_equal(cur_k[i].to("cpu", torch.float64).numpy(), Kc)
+        if Vc is not None:
+            np.testing.assert_array_equal(cur_v[i].to("cpu", torch.float64).numpy(), Vc)
+
+
+def test_concat_update_refuses_in_place():
+    wl = SMALL_BF16
+    layer = H.GpuLayer(wl, 1)
+    c = layer.cache
+    d = synth.make_decode_inputs(wl, 1, 1, 0)
+    slots_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.SnapError):
+        B.snap_append_kv_concat(layer.cfg, layer.layout, d["k_new"].cuda(), d["v_new"].cuda(), slots_dev, 1,
+                                c.k_cache, c.v_cache, c.k_cache, c.v_cache, c.seq_len, c.status)

@@ -415,3 +415,34 @@ def test_planted_heavy_hitters_are_selected():
     for h in range(wl.n_kv_heads):
         hit = len(set(p["planted"][h]) & set(idx[h])) / len(p["planted"][h])
         assert hit >= 0.7          # chance level would be topk / candidates = 0.13
+
+
+def test_position_order_image_equals_repeated_array_concatenation():
+    """Section 3.2.1's slice-and-concatenate update, done literally on arrays, step by step,
+    gives the position-ordered cache image; it holds the same rows as the ring image, and the
+    two images coincide when the ring's write pointer is back at the window start."""
+    cfg = _cfg()
+    Ls, Lr, Lsr = cfg.l_sink, cfg.l_recent, cfg.l_sr
+    L = Ls + 3 * Lr                              # ring pointer at the window start
+    q, k, v = _rand_prompt(cfg, L, seed=21)
+    seq = orc.compress(q, k, v, cfg)
+    K0, V0, _ = orc.expected_cache(seq)
+    Kp, Vp, _ = orc.expected_cache_position_order(seq)
+    np.testing.assert_array_equal(K0, Kp)
+    np.testing.assert_array_equal(V0, Vp)
+    rng = np.random.default_rng(5)
+    Kc, Vc = K0.copy(), V0.copy()
+    for step in range(2 * Lr + 3):
+        kn = rng.standard_normal((cfg.n_kv_heads, cfg.d_qk))
+        vn = rng.standard_normal((cfg.n_kv_heads, cfg.d_v))
+        orc.decode_step(seq, rng.standard_normal((cfg.n_q_heads, cfg.d_qk)), kn, vn)
+        Kc = np.concatenate([Kc[:, :Ls], Kc[:, Ls + 1:Lsr], kn[:, None], Kc[:, Lsr:]], axis=1)
+        Vc = np.concatenate([Vc[:, :Ls], Vc[:, Ls + 1:Lsr], vn[:, None], Vc[:, Lsr:]], axis=1)
+        Kp, Vp, pm = orc.expected_cache_position_order(seq)
+        np.testing.assert_array_equal(Kc, Kp)
+        np.testing.assert_array_equal(Vc, Vp)
+        Kr, Vr, pr = orc.expected_cache(seq)
+        for kvh in range(cfg.n_kv_heads):
+            assert sorted(pm[kvh].tolist()) == sorted(pr[kvh].tolist())
+        if (seq.n_tokens - Ls) % Lr == 0:
+            np.testing.assert_array_equal(Kr, Kp)
