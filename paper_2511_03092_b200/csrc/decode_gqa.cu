@@ -136,6 +136,7 @@ __global__ void __launch_bounds__(NT, (G == 8 ? 2 : 3)) decode_gqa_kernel(const 
   const int sp = blockIdx.x, kvh = blockIdx.y, i = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, hw = lane >> 4, l16 = lane & 15;
   const int odd = l16 & 1, jrow = l16 >> 1;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int slot = a.slot_ids[i];
   const bool bad = slot < 0 || slot >= a.max_seqs;
   const int Lsr = a.Ls + a.Lr;
@@ -393,6 +394,7 @@ __global__ void __launch_bounds__(D) decode_gqa_merge_kernel(const float* __rest
                                                              int nsplit, const int* __restrict__ slot_ids,
                                                              int* seq_len, int max_seqs, int bump) {
   const int h = blockIdx.x, i = blockIdx.y, t = threadIdx.x;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const float* p = partials + ((long long)i * Hq + h) * nsplit * PS;
   // launched with programmatic stream serialisation: the grid may start while the split kernel
   // drains; everything the split kernel wrote is visible after this wait
@@ -425,20 +427,24 @@ cudaError_t launch_g(const FastArgs& a, int n_active, __nv_bfloat16* out, int* s
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  dim3 grid(a.nsplit, a.Hkv, n_active);
-  decode_gqa_kernel<G><<<grid, NT, smem, st>>>(a);
-  count_launch();
-  // the merge kernel is a programmatic dependent launch: its launch latency overlaps the split kernel's tail
-  cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(a.Hq, n_active);
-  lc.blockDim = dim3(D);
-  lc.dynamicSmemBytes = 0;
-  lc.stream = st;
+  // Both kernels are programmatic dependent launches: each may become resident while its
+  // predecessor in the stream drains, and waits (griddepcontrol.wait) before touching memory.
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(a.nsplit, a.Hkv, n_active);
+  lc.blockDim = dim3(NT);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
   lc.attrs = attr;
   lc.numAttrs = 1;
+  cudaError_t e0 = cudaLaunchKernelEx(&lc, decode_gqa_kernel<G>, a);
+  count_launch();
+  if (e0 != cudaSuccess) return e0;
+  lc.gridDim = dim3(a.Hq, n_active);
+  lc.blockDim = dim3(D);
+  lc.dynamicSmemBytes = 0;
   const float* parts = a.partials;
   const int* slots = a.slot_ids;
   cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_merge_kernel, parts, out, a.Hq, a.nsplit, slots, seq_len,
