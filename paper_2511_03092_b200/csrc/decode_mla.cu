@@ -270,6 +270,14 @@ __global__ void __launch_bounds__(256) decode_mla_merge_kernel(const float* __re
 
 }  // namespace
 
+cudaError_t launch_decode_mla_merge(const float* partials, void* out, int n_active, int Hq, int nsplit,
+                                    const int* slot_ids, int* seq_len, int max_seqs, int bump, cudaStream_t st) {
+  decode_mla_merge_kernel<<<dim3(Hq, (unsigned)n_active), 256, 0, st>>>(partials, static_cast<__nv_bfloat16*>(out), Hq, nsplit,
+                                                                       slot_ids, seq_len, max_seqs, bump);
+  count_launch();
+  return cudaGetLastError();
+}
+
 bool decode_mla_supported(int dtype, const Shape& s) {
   return dtype == SNAP_BF16 && s.v_aliases_k && s.d_qk == DQK && s.d_v == DV && s.Hkv == 1 && s.Hq % HB == 0;
 }

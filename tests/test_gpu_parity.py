@@ -242,6 +242,17 @@ def test_latent_attention_kernel_shapes(hq):
     _run_compress_and_decode(wl, [500, 70], seed=31, steps=45, sharp=3.0, check_ring_every=9)
 
 
+def test_latent_attention_tcgen05_decode_kernel(monkeypatch):
+    """The opt-in tcgen05 decode kernel for the latent layout (queries and probabilities as
+    tensor-memory operands, V read as an MN-major operand from the staged tile): same cases."""
+    monkeypatch.setenv("SNAP_DECODE_MLA", "umma")
+    wl = synth.Workload("mla_small", 128, 1, 576, 512, "bf16", 3, 40, 64, 8, 5, batch=1,
+                        prompt_len=(500, 500), decode_steps=6, salience="planted", n_planted=8,
+                        v_aliases_k=True, softmax_scale=2.0 ** -0.5)
+    _run_compress_and_decode(wl, [2, 30, 43, 44, 107, 500, 333], seed=29, steps=6)
+    _run_compress_and_decode(wl, [500, 70], seed=31, steps=45, sharp=3.0, check_ring_every=9)
+
+
 def test_late_outlier_logits_latent_shape():
     """Same hazard as above on the wide-row score kernel (576-wide keys, 512 window rows)."""
     wl = synth.Workload("mla_outlier", 64, 1, 576, 512, "bf16", 3, 40, 100, 8, 5, batch=1,
