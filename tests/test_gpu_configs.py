@@ -60,6 +60,40 @@ def test_config2_ragged_batch_sample():
     _run(wl, lengths, seed=300, steps=6)
 
 
+def test_config2_decode_in_the_benchmark_launch_shape():
+    """32 resident sequences with full caches: the decode launch bench.py times (same grid, same
+    number of splits).  The oracle follows a sample of the sequences; the others only have to
+    leave the status word clean."""
+    wl = synth.CONFIGS[2]
+    n = wl.batch
+    assert n == 32
+    lengths = [8192] * n
+    lengths[17], lengths[29], lengths[31] = 12000, 20000, 32768
+    sample = [0, 17, 29, 31]
+    layer = H.GpuLayer(wl, max_seqs=n)
+    prompts = [synth.make_prompt(wl, L, 600 + 7 * i) for i, L in enumerate(lengths)]
+    idx = layer.compress(prompts, list(range(n)))
+    assert layer.status() == 0
+    seqs = {}
+    for i in sample:
+        seqs[i] = H.oracle_compress(wl, prompts[i])
+        H.check_selection(idx[i], seqs[i], wl)
+        seqs[i].topk_pos = [idx[i][h][idx[i][h] >= 0].astype(np.int64) for h in range(wl.n_kv_heads)]
+        H.check_cache_image(layer, seqs[i], i, wl)
+    slots_dev = torch.arange(n, dtype=torch.int32, device="cuda")
+    for step in range(3):
+        d = synth.make_decode_inputs(wl, n, 600, step)
+        out = layer.decode(d["q"].cuda(), d["k_new"].cuda(), d["v_new"].cuda(), slots_dev)
+        for i in sample:
+            ref = orc.decode_step(seqs[i], synth.to_f64(d["q"][i]), synth.to_f64(d["k_new"][i]),
+                                  synth.to_f64(d["v_new"][i]))
+            H.check_output(out[i], ref, wl, f"seq {i} step {step}")
+    for i in sample:
+        H.check_cache_image(layer, seqs[i], i, wl)
+    assert layer.status() == 0
+    assert [int(x) for x in layer.cache.seq_len.cpu()] == [L + 3 for L in lengths]
+
+
 def test_config3_latent_sample():
     """Latent-attention shape (128 heads over one 576-wide KV row, V = first 512 dims), prompt cut
     to 16k tokens so that the oracle finishes in seconds."""
