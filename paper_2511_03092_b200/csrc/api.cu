@@ -125,12 +125,11 @@ int check_cu(const int32_t* cu, int n_seq) {
 
 struct DecodePlan { bool gqa, mla, mla_umma; int nsplit; size_t floats; };
 
-// The latent layout decodes on the mma.sync kernel; SNAP_DECODE_MLA=umma selects the tcgen05 kernel
-// with tensor-memory operands instead (correct, but slower at this shape: its 32-row tiles make
-// every MMA latency-bound).
+// The latent layout decodes on the tcgen05 kernel when the head count allows (multiples of 128);
+// SNAP_DECODE_MLA=mma keeps it on the mma.sync kernel (testing aid).
 bool use_mla_umma(int dtype, const Shape& s) {
   const char* env = getenv("SNAP_DECODE_MLA");
-  if (!env || env[0] != 'u') return false;
+  if (env && env[0] == 'm') return false;
   return decode_mla_umma_supported(dtype, s);
 }
 

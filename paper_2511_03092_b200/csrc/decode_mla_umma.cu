@@ -3,18 +3,21 @@
 //
 // With 128 heads sharing every cache row the step is a pair of dense contractions per tile
 // (S = Q K^T over 576 dims, O += P V over the tile's rows), so it belongs on the tensor cores.
-// What shapes the kernel is that the stationary operand, the 128 x 576 query block, must not be
-// re-read from shared memory for every tile (that alone would saturate shared-memory bandwidth):
-// it lives in tensor memory and is the TMEM-sourced A operand of the MMAs, as are the
-// probabilities.  Tensor memory then holds, per CTA,
-//     O 128 | S 2 x 32 | P 2 x 16 (bf16 pairs) | Q 288 (bf16 pairs)    = 512 columns,
-// which leaves room for 128 output dims: the 512 value dims are split over four CTAs that each
-// recompute S.  Grid = (row splits, 4 x head blocks, sequences), one CTA per SM:
-//   warp 0      TMA producer: 32-row cache tiles (nine 64-dim slabs, 128-byte swizzle) into a
-//               5-stage ring;
-//   warp 1      MMA issuer: S(t+1) = Q K^T is queued before O += P(t) V so that the tensor pipe
-//               works while the softmax warps handle tile t; V is the same staged tile read as
-//               an MN-major operand;
+// Two facts shape the kernel.  The stationary operand, the 128 x 576 query block, would fill
+// most of shared memory, so it lives in tensor memory and is the TMEM-sourced A operand of the
+// MMAs, as are the probabilities.  And an MMA instruction occupies the tensor pipe for a fixed
+// minimum time however few columns it produces (measured: about 110 clocks at N = 32 or 64, from
+// either operand source), so tiles are as wide as tensor memory allows:
+//     O 128 | S 64 | P 32 (bf16 pairs) | Q 288 (bf16 pairs)    = 512 columns.
+// That leaves room for 128 output dims, so the 512 value dims are split over four CTAs that each
+// recompute S, and S and P are single-buffered.  Grid = (row splits, 4 x head blocks,
+// sequences), one CTA per SM:
+//   warp 0      TMA producer: 64-row cache tiles (nine 64-dim slabs, 128-byte swizzle) into a
+//               3-stage ring;
+//   warp 1      MMA issuer (whole warp converged, instructions predicated on one lane):
+//               S(t) = Q K(t)^T is issued as soon as the softmax warps have taken S(t-1) out of
+//               tensor memory and runs while they do their arithmetic; O += P(t-1) V(t-1) is
+//               queued behind it; V is the same staged tile read as an MN-major operand;
 //   warps 2-5   thread = head: read S from TMEM, online softmax in the log2 domain with a lazily
 //               refreshed reference (O is rescaled in TMEM only when a logit exceeds it by 8),
 //               write P back to TMEM as bf16.
@@ -28,10 +31,10 @@ namespace {
 
 using namespace umma;
 
-constexpr int DQK = 576, DV = 512, HBLK = 128, TR = 32, NSTG = 5, NTH = 192, DVQ = 128, NQ = DV / DVQ;
-constexpr int NSLAB = DQK / 64, SLAB_B = TR * 128, STAGE_B = NSLAB * SLAB_B;        // 9 x 4096 = 36864
+constexpr int DQK = 576, DV = 512, HBLK = 128, TR = 64, NSTG = 3, NTH = 192, DVQ = 128, NQ = DV / DVQ;
+constexpr int NSLAB = DQK / 64, SLAB_B = TR * 128, STAGE_B = NSLAB * SLAB_B;        // 9 x 8192 = 73728
 constexpr int PSM = DV + 2;
-constexpr uint32_t COL_O = 0, COL_S = 128, COL_P = 192, COL_Q = 224;                // tensor-memory columns
+constexpr uint32_t COL_O = 0, COL_S = 128, COL_P = 192, COL_Q = 224;                // tensor-memory columns: O 128 | S 64 | P 32 | Q 288
 
 struct UArgs {
   const __nv_bfloat16* q;
@@ -59,6 +62,21 @@ __device__ __forceinline__ void mma_ts_bf16(uint32_t d_tmem, uint32_t a_tmem, ui
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+// The same, executed by a whole (converged) warp with the instruction predicated on one lane, so
+// that the operands are computed on the warp-uniform path instead of inside a divergent branch.
+__device__ __forceinline__ void mma_ts_bf16_pred(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t acc, uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void mma_commit_pred(uint32_t bar, uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar), "r"(leader) : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
@@ -94,8 +112,8 @@ __global__ void __launch_bounds__(NTH, 1) decode_mla_umma_kernel(const UArgs a, 
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* Ks = smem;                                                   // [NSTG][9 slabs][32 rows][128 B]
   uint64_t* bars = reinterpret_cast<uint64_t*>(Ks + NSTG * STAGE_B);
-  // full[NSTG] empty[NSTG] s_full[2] p_ready[2] pv_done[2] q_ready
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTG + 7);
+  // full[NSTG] empty[NSTG] s_full s_free p_ready pv_done q_ready
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTG + 5);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -118,15 +136,14 @@ __global__ void __launch_bounds__(NTH, 1) decode_mla_umma_kernel(const UArgs a, 
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8 * s; };
   auto empty_bar = [&](int s) { return bar0 + 8 * (NSTG + s); };
-  auto sfull_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + b); };
-  auto pready_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 2 + b); };
-  auto pvdone_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 4 + b); };
-  const uint32_t qready_bar = bar0 + 8 * (2 * NSTG + 6);
+  const uint32_t sfull_bar = bar0 + 8 * (2 * NSTG), sfree_bar = bar0 + 8 * (2 * NSTG + 1);
+  const uint32_t pready_bar = bar0 + 8 * (2 * NSTG + 2), pvdone_bar = bar0 + 8 * (2 * NSTG + 3);
+  const uint32_t qready_bar = bar0 + 8 * (2 * NSTG + 4);
 
   if (tid == 0) {
     *abort_flag = 0;
     for (int s = 0; s < NSTG; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(sfull_bar(b), 1); mbar_init(pready_bar(b), 4); mbar_init(pvdone_bar(b), 1); }
+    mbar_init(sfull_bar, 1); mbar_init(sfree_bar, 4); mbar_init(pready_bar, 4); mbar_init(pvdone_bar, 1);
     mbar_init(qready_bar, 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -154,39 +171,44 @@ __global__ void __launch_bounds__(NTH, 1) decode_mla_umma_kernel(const UArgs a, 
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0 && nt > 0) {
+    if (nt > 0) {                                              // whole warp, MMAs and commits predicated on lane 0
+      const uint32_t leader = lane == 0;
       const uint32_t idesc_s = idesc_ts(128, TR, false), idesc_pv = idesc_ts(128, DVQ, true);
-      bool ok = mbar_wait(qready_bar, 0u, abort_flag);
+      bool ok = wait_warp(qready_bar, 0u, abort_flag);
       fence_after();
-      auto issue_s = [&](int it) -> bool {                    // S[it & 1] = Q K(it)^T
+      // S, P and the one set of barriers around them are single-buffered: tile it's logits are
+      // computed once the softmax warps have taken tile it-1's out of tensor memory, and run on the
+      // tensor pipe while those warps do their arithmetic; O += P(it-1) V(it-1) is queued behind.
+      auto issue_pv = [&](int it) -> bool {                   // O += P(it) V(it): V = rows of the staged tile, MN-major
+        if (!wait_warp(pready_bar, (unsigned)it & 1u, abort_flag)) return false;
+        fence_after();
         const int s = it % NSTG;
-        if (!mbar_wait(full_bar(s), (unsigned)(it / NSTG) & 1u, abort_flag)) return false;
+        const uint32_t vst = smem_u32(Ks) + s * STAGE_B + (2 * qd) * SLAB_B;
+#pragma unroll
+        for (int ks = 0; ks < TR / 16; ++ks)
+          mma_ts_bf16_pred(tmem_base + COL_O, tmem_base + COL_P + 8 * ks, smem_desc_mn(vst + ks * 16 * 128, SLAB_B),
+                           idesc_pv, (it | ks) != 0, leader);
+        mma_commit_pred(pvdone_bar, leader);
+        mma_commit_pred(empty_bar(s), leader);                 // the stage may be refilled once these MMAs have read it
+        return true;
+      };
+      for (int it = 0; it < nt && ok; ++it) {
+        const int s = it % NSTG;
+        ok = wait_warp(full_bar(s), (unsigned)(it / NSTG) & 1u, abort_flag);
+        if (ok && it > 0) ok = wait_warp(sfree_bar, (unsigned)(it - 1) & 1u, abort_flag);
+        if (!ok) break;
         fence_after();
         // descriptors differ from the stage's first one only by compile-time constants (16-byte units)
         const uint64_t kd0 = smem_desc(smem_u32(Ks) + s * STAGE_B);
-        const uint32_t sd = tmem_base + COL_S + (it & 1) * TR, qa = tmem_base + COL_Q;
+        const uint32_t sd = tmem_base + COL_S, qa = tmem_base + COL_Q;
 #pragma unroll
-        for (int k = 0; k < NSLAB * 4; ++k)
-          mma_ts_bf16(sd, qa + 8 * k, kd0 + (uint64_t)(((k >> 2) * SLAB_B + (k & 3) * 32) >> 4), idesc_s, k != 0);
-        mma_commit(sfull_bar(it & 1));
-        return true;
-      };
-      if (ok) ok = issue_s(0);
-      for (int it = 0; it < nt && ok; ++it) {
-        const int b = it & 1, s = it % NSTG;
-        if (it + 1 < nt) { ok = issue_s(it + 1); if (!ok) break; }
-        ok = mbar_wait(pready_bar(b), (unsigned)(it / 2) & 1u, abort_flag);
-        if (!ok) break;
-        fence_after();
-        const uint32_t vst = smem_u32(Ks) + s * STAGE_B + (2 * qd) * SLAB_B;
-#pragma unroll
-        for (int ks = 0; ks < TR / 16; ++ks)                  // O += P(it) V(it): V = rows of the staged tile, MN-major
-          mma_ts_bf16(tmem_base + COL_O, tmem_base + COL_P + b * 16 + 8 * ks,
-                      smem_desc_mn(vst + ks * 16 * 128, SLAB_B), idesc_pv, (it | ks) != 0);
-        mma_commit(pvdone_bar(b));
-        mma_commit(empty_bar(s));                              // the stage may be refilled once these MMAs have read it
+        for (int k = 0; k < NSLAB * 4; ++k)                    // S = Q K(it)^T
+          mma_ts_bf16_pred(sd, qa + 8 * k, kd0 + (uint64_t)(((k >> 2) * SLAB_B + (k & 3) * 32) >> 4), idesc_s, k != 0, leader);
+        mma_commit_pred(sfull_bar, leader);
+        if (it > 0) ok = issue_pv(it - 1);
       }
-      if (!ok) *abort_flag = 1;
+      if (ok) ok = issue_pv(nt - 1);
+      if (!ok && lane == 0) *abort_flag = 1;
     }
   } else {
     // ---------------- softmax warps: thread = head ----------------
@@ -220,31 +242,38 @@ __global__ void __launch_bounds__(NTH, 1) decode_mla_umma_kernel(const UArgs a, 
       if (lane == 0) mbar_arrive(qready_bar);
     }
     for (int it = 0; it < nt; ++it) {
-      const int b = it & 1;
-      if (!wait_warp(sfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag)) { ok = false; break; }
+      if (!wait_warp(sfull_bar, (unsigned)it & 1u, abort_flag)) { ok = false; break; }
       fence_after();
-      uint32_t ra[16], rb[16];
-      tmem_ld16_issue(lane_addr + COL_S + b * TR, ra);
-      tmem_ld16_issue(lane_addr + COL_S + b * TR + 16, rb);
+      uint32_t r0[16], r1[16], r2[16], r3[16];
+      tmem_ld16_issue(lane_addr + COL_S, r0);
+      tmem_ld16_issue(lane_addr + COL_S + 16, r1);
+      tmem_ld16_issue(lane_addr + COL_S + 32, r2);
+      tmem_ld16_issue(lane_addr + COL_S + 48, r3);
       const TileRows tr = tile_rows(g0 + it, nA, n_low, Lsr, n_top);
       const int nrows = tr.row_end - tr.row0;                  // >= 1; columns at or past it are masked
-      tmem_ld16_wait(ra);
-      tmem_ld16_wait(rb);
+      tmem_ld16_wait(r0); tmem_ld16_wait(r1); tmem_ld16_wait(r2); tmem_ld16_wait(r3);
+      fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sfree_bar);                   // the next tile's logits may overwrite S
       float v[TR];
       float mx = -INFINITY;
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        v[j] = j < nrows ? __uint_as_float(ra[j]) * a.scale_log2 : -INFINITY;
-        v[16 + j] = 16 + j < nrows ? __uint_as_float(rb[j]) * a.scale_log2 : -INFINITY;
-        mx = fmaxf(mx, fmaxf(v[j], v[16 + j]));
+        v[j] = j < nrows ? __uint_as_float(r0[j]) * a.scale_log2 : -INFINITY;
+        v[16 + j] = 16 + j < nrows ? __uint_as_float(r1[j]) * a.scale_log2 : -INFINITY;
+        v[32 + j] = 32 + j < nrows ? __uint_as_float(r2[j]) * a.scale_log2 : -INFINITY;
+        v[48 + j] = 48 + j < nrows ? __uint_as_float(r3[j]) * a.scale_log2 : -INFINITY;
+        mx = fmaxf(fmaxf(mx, fmaxf(v[j], v[16 + j])), fmaxf(v[32 + j], v[48 + j]));
       }
       // Lazy reference: refreshed (and O rescaled) only when some head of the warp sees a logit 8
       // above its reference; the tensor-memory accesses are warp-collective, so the warp votes.
+      bool pv_waited = it == 0;
       if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
         const float m_new = fmaxf(m_ref, mx);
         const float alpha = m_ref == -INFINITY ? 0.f : exp2f(m_ref - m_new);
         if (it > 0) {
-          if (!wait_warp(pvdone_bar((it - 1) & 1), (unsigned)((it - 1) / 2) & 1u, abort_flag)) { ok = false; break; }
+          if (!wait_warp(pvdone_bar, (unsigned)(it - 1) & 1u, abort_flag)) { ok = false; break; }
+          pv_waited = true;
           fence_after();
 #pragma unroll 1
           for (int c = 0; c < DVQ / 16; ++c) {
@@ -260,30 +289,34 @@ __global__ void __launch_bounds__(NTH, 1) decode_mla_umma_kernel(const UArgs a, 
         l_sum *= alpha;
         m_ref = m_new;
       }
-      uint32_t pk[16];
+      uint32_t pk0[16], pk1[16];
       const float mr = m_ref == -INFINITY ? 0.f : m_ref;
-      float ls = 0.f;
+      float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
         const float p0 = fast_exp2(v[2 * j] - mr), p1 = fast_exp2(v[2 * j + 1] - mr);
-        ls += p0 + p1;
-        pk[j] = pack_bf16(p0, p1);
+        const float p2 = fast_exp2(v[32 + 2 * j] - mr), p3 = fast_exp2(v[33 + 2 * j] - mr);
+        ls0 += p0 + p1;
+        ls1 += p2 + p3;
+        pk0[j] = pack_bf16(p0, p1);
+        pk1[j] = pack_bf16(p2, p3);
       }
-      l_sum += ls;
-      if (it >= 2) {                                           // P[b] was last read by the MMAs of tile it - 2
-        if (!wait_warp(pvdone_bar(b), (unsigned)((it - 2) / 2) & 1u, abort_flag)) { ok = false; break; }
+      l_sum += ls0 + ls1;
+      if (!pv_waited) {                                        // P was last read by the MMAs of tile it - 1
+        if (!wait_warp(pvdone_bar, (unsigned)(it - 1) & 1u, abort_flag)) { ok = false; break; }
         fence_after();
       }
-      tmem_st16(lane_addr + COL_P + b * 16, pk);
+      tmem_st16(lane_addr + COL_P, pk0);
+      tmem_st16(lane_addr + COL_P + 16, pk1);
       tmem_st_wait();
       fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(pready_bar(b));
+      if (lane == 0) mbar_arrive(pready_bar);
     }
     if (!ok) *abort_flag = 1;
     // ---------------- this split's partial result ----------------
     float* ph = a.partials + (((long long)i * a.Hq + head) * a.nsplit + sp) * PSM;
-    if (ok && nt > 0) ok = wait_warp(pvdone_bar((nt - 1) & 1), (unsigned)((nt - 1) / 2) & 1u, abort_flag);
+    if (ok && nt > 0) ok = wait_warp(pvdone_bar, (unsigned)(nt - 1) & 1u, abort_flag);
     if (!ok) *abort_flag = 1;
     fence_after();
     if (qd == 0) { ph[0] = nt > 0 && ok ? m_ref : -INFINITY; ph[1] = nt > 0 && ok ? l_sum : 0.f; }

@@ -233,8 +233,8 @@ def test_late_outlier_logits_refresh_the_running_reference():
 
 @pytest.mark.parametrize("hq", [64, 128])
 def test_latent_attention_kernel_shapes(hq):
-    """The 576/512 latent layout (tensor-core decode kernel): short and ragged sequences, ring wrap,
-    sharp softmax."""
+    """The 576/512 latent layout (tensor-core decode kernels: tcgen05 for 128 heads, mma.sync for
+    64): short and ragged sequences, ring wrap, sharp softmax."""
     wl = synth.Workload("mla_small", hq, 1, 576, 512, "bf16", 3, 40, 64, 8, 5, batch=1,
                         prompt_len=(500, 500), decode_steps=6, salience="planted", n_planted=8,
                         v_aliases_k=True, softmax_scale=2.0 ** -0.5)
@@ -242,10 +242,10 @@ def test_latent_attention_kernel_shapes(hq):
     _run_compress_and_decode(wl, [500, 70], seed=31, steps=45, sharp=3.0, check_ring_every=9)
 
 
-def test_latent_attention_tcgen05_decode_kernel(monkeypatch):
-    """The opt-in tcgen05 decode kernel for the latent layout (queries and probabilities as
-    tensor-memory operands, V read as an MN-major operand from the staged tile): same cases."""
-    monkeypatch.setenv("SNAP_DECODE_MLA", "umma")
+def test_latent_attention_mma_sync_decode_kernel_with_128_heads(monkeypatch):
+    """The mma.sync decode kernel for the latent layout stays selectable at 128 heads, where the
+    tcgen05 kernel is the default: same cases."""
+    monkeypatch.setenv("SNAP_DECODE_MLA", "mma")
     wl = synth.Workload("mla_small", 128, 1, 576, 512, "bf16", 3, 40, 64, 8, 5, batch=1,
                         prompt_len=(500, 500), decode_steps=6, salience="planted", n_planted=8,
                         v_aliases_k=True, softmax_scale=2.0 ** -0.5)
