@@ -592,6 +592,19 @@ def run_config(args):
     t1.record()
     torch.cuda.synchronize()
     ms = t0.elapsed_time(t1) / steps
+    # the same step captured once as a CUDA graph (all layers' launches) and replayed
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step(0)
+    for s in range(args.warmup):
+        graph.replay()
+    torch.cuda.synchronize()
+    t0.record()
+    for s in range(steps):
+        graph.replay()
+    t1.record()
+    torch.cuda.synchronize()
+    ms_graph = t0.elapsed_time(t1) / steps
     eb = 2 if wl.dtype == "bf16" else 4
     rows = min(L + 1, wl.slots)
     step_bytes = n_layers * nseq * wl.n_kv_heads * rows * (wl.d_qk + (0 if wl.v_aliases_k else wl.d_v)) * eb
@@ -600,6 +613,7 @@ def run_config(args):
         "workload": wl.name, "n_layers": n_layers, "sequences": nseq, "prompt_tokens": L, "cache_slots": wl.slots,
         "compress_us_per_prompt_layer_median": statistics.median(comp_us),
         "compress_ms_total": sum(comp_us) / 1e3, "decode_steps_timed": steps, "decode_us_per_step": ms * 1e3,
+        "decode_us_per_step_cuda_graph": ms_graph * 1e3,
         "decode_tokens_per_s": nseq / (ms * 1e-3), "decode_bytes_per_step": step_bytes,
         "decode_GBps": step_bytes / (ms * 1e-3) / 1e9, "decode_frac_of_measured_hbm": step_bytes / (ms * 1e-3) / 1e9 / peak,
         "status": int(cache.status.item())}), flush=True)

@@ -323,3 +323,44 @@ def test_concat_update_refuses_in_place():
     with pytest.raises(B.SnapError):
         B.snap_append_kv_concat(layer.cfg, layer.layout, d["k_new"].cuda(), d["v_new"].cuda(), slots_dev, 1,
                                 c.k_cache, c.v_cache, c.k_cache, c.v_cache, c.seq_len, c.status)
+
+
+LATENT_128 = synth.Workload("mla_graph", 128, 1, 576, 512, "bf16", 3, 40, 64, 8, 5, batch=1,
+                            prompt_len=(500, 500), decode_steps=6, salience="planted", n_planted=8,
+                            v_aliases_k=True, softmax_scale=2.0 ** -0.5)
+
+
+@pytest.mark.parametrize("wl", [SMALL_BF16, LATENT_128], ids=lambda w: w.name)
+def test_decode_step_replayed_from_a_cuda_graph(wl):
+    """A decode step (append + attention + merge, programmatic dependent launches included) is
+    captured once into a CUDA graph and replayed with new inputs: same outputs, cache and
+    lengths as issuing the calls directly.  The first call happens before the capture."""
+    lengths = [60, 400, 150]
+    n = len(lengths)
+    prompts = [synth.make_prompt(wl, L, 71 + i) for i, L in enumerate(lengths)]
+    a, b = H.GpuLayer(wl, n), H.GpuLayer(wl, n)
+    a.compress(prompts, list(range(n))); b.compress(prompts, list(range(n)))
+    slots_dev = torch.arange(n, dtype=torch.int32, device="cuda")
+    d0 = synth.make_decode_inputs(wl, n, 71, 0)
+    q_s, kn_s = d0["q"].cuda(), d0["k_new"].cuda()
+    vn_s = None if wl.v_aliases_k else d0["v_new"].cuda()
+    a.decode(q_s, kn_s, vn_s, slots_dev); b.decode(q_s, kn_s, vn_s, slots_dev)      # step 0, direct on both
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        out_s = b.decode(q_s, kn_s, vn_s, slots_dev)
+    for step in range(1, 6):
+        d = synth.make_decode_inputs(wl, n, 71, step)
+        q, kn = d["q"].cuda(), d["k_new"].cuda()
+        vn = None if wl.v_aliases_k else d["v_new"].cuda()
+        q_s.copy_(q); kn_s.copy_(kn)
+        if vn is not None:
+            vn_s.copy_(vn)
+        graph.replay()
+        out_a = a.decode(q, kn, vn, slots_dev)
+        torch.cuda.synchronize()
+        assert torch.equal(out_a, out_s)
+        assert torch.equal(a.cache.k_cache, b.cache.k_cache)
+        assert torch.equal(a.cache.seq_len, b.cache.seq_len)
+    assert a.status() == 0 and b.status() == 0
+    assert [int(x) for x in b.cache.seq_len.cpu()] == [L + 6 for L in lengths]
