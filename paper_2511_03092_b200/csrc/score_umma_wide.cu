@@ -5,7 +5,7 @@
 // warps reading TMEM), but the contraction dimension is streamed: grid = (candidate splits,
 // blocks of 128 window rows, prompts).  A CTA keeps its 128-row query block resident in shared
 // memory (one 16 KB swizzled slab per 64 dims) and, for every candidate tile, pulls the keys
-// through a 2-stage ring one 64-dim slab at a time, accumulating in tensor memory; two
+// through a ring of 2 to 6 stages (whatever fits beside the query block) one 64-dim slab at a time, accumulating in tensor memory; two
 // accumulator buffers let the next tile's MMAs overlap the epilogue of the current one.
 //   pass 1  M = 128 query rows, N = 256 candidates; thread = query row; the two epilogue groups
 //           take 128 candidates each and their (reference max, sum) pairs are merged at the end.
@@ -14,6 +14,8 @@
 //           partial column sums go to scratch and a small kernel adds the row blocks in a fixed
 //           order (deterministic, no atomics).
 // Every mbarrier wait is bounded; a wait that runs out raises SNAP_DEV_WAIT_TIMEOUT.
+#include <cstdlib>
+
 #include "snap_internal.cuh"
 #include "umma_helpers.cuh"
 
@@ -22,10 +24,11 @@ namespace {
 
 using namespace umma;
 
-constexpr int NTHREADS = 320, NS = 2, STAGE_B = 32768, QH_B = 16384, MAXH = 9;
+constexpr int NTHREADS = 320, MAXNS = 6, STAGE_B = 32768, QH_B = 16384, MAXH = 9;
 
 struct WideArgs {
   int Hq, Hkv, g, Lo, Ls, Lr, R, NH, RB;
+  int NS;                // key-slab stages: as many as fit beside the query block (2..MAXNS)
   float scale_log2;
   SeqBatch b;
   ScoreBuffers buf;
@@ -40,7 +43,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
   constexpr int TNP = PASS == 1 ? 256 : 128;                  // candidates per tile
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int NH = a.NH;
+  const int NH = a.NH, NS = a.NS;
   unsigned char* Qs = smem;                                   // [NH][128 rows][128 B]
   unsigned char* Ks = Qs + NH * QH_B;                         // [NS][up to 256 rows][128 B]
   float* mu_s = reinterpret_cast<float*>(Ks + NS * STAGE_B);  // [128] pass 2: m_i + log2 l_i of this row block
@@ -264,8 +267,19 @@ __global__ void score_rowblock_reduce_kernel(const float* __restrict__ cpart, fl
   C[(long long)z * c_stride + j] = s;
 }
 
-size_t wide_smem_bytes(int NH) {
+size_t wide_smem_bytes(int NH, int NS) {
   return (size_t)NH * QH_B + NS * STAGE_B + 128 * sizeof(float) + 128 * sizeof(float2) + (2 * NS + 5) * 8 + 16 + 1024;
+}
+
+// SNAP_WIDE_STAGES caps the ring depth (tuning aid).
+int wide_stages(int NH) {
+  int ns = MAXNS;
+  if (const char* env = getenv("SNAP_WIDE_STAGES")) {
+    const int v = atoi(env);
+    if (v >= 2 && v < ns) ns = v;
+  }
+  while (ns > 2 && wide_smem_bytes(NH, ns) > 227u * 1024u) --ns;
+  return ns;
 }
 
 }  // namespace
@@ -296,7 +310,7 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   if (!enc) return cudaErrorNotSupported;
   WideArgs a;
   a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Lo = s.Lo; a.Ls = s.Ls; a.Lr = s.Lr; a.R = s.g * s.Lo;
-  a.NH = s.d_qk / 64; a.RB = a.R / 128;
+  a.NH = s.d_qk / 64; a.RB = a.R / 128; a.NS = wide_stages(a.NH);
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.b = b; a.buf = buf; a.cpart = cpart; a.status = status;
 
@@ -323,7 +337,7 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
   }
-  const size_t smem = wide_smem_bytes(a.NH);
+  const size_t smem = wide_smem_bytes(a.NH, a.NS);
   static size_t attr_bytes = 0;
   if (smem > attr_bytes) {
     cudaError_t e = cudaFuncSetAttribute(score_umma_wide_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -96,3 +96,10 @@ def test_workspace_queries_and_argument_errors_without_gpu():
     assert lib.snap_append_kv(C.byref(cfg), C.byref(lay), one, one, one, -1, one, one, one, None, None) == -1
     assert lib.snap_decode_attn(C.byref(cfg), C.byref(lay), one, None, None, one, 0, one, one, one, one, one,
                                 one, 0, None, None) == 0                     # nothing to do
+    two = C.c_void_p(512)
+    cc = lambda *a: lib.snap_append_kv_concat(C.byref(cfg), C.byref(lay), *a)
+    assert cc(one, one, one, 2, one, one, one, one, one, None, None) == -1   # in place: output must differ from input
+    assert cc(one, one, one, 2, one, one, None, two, one, None, None) == -4  # missing output buffer
+    assert cc(one, None, one, 2, one, one, two, two, one, None, None) == -4  # missing new values
+    assert cc(one, one, one, -3, one, one, two, two, one, None, None) == -1
+    assert cc(one, one, one, 0, one, one, two, two, one, None, None) == 0    # nothing to do
