@@ -420,13 +420,8 @@ cudaError_t launch_g(const FastArgs& a, int n_active, __nv_bfloat16* out, int* s
                      cudaStream_t st) {
   const size_t smem = (size_t)NWARP * NSTAGE * STAGE_B + NWARP * 2 * 8 * G * 2 * sizeof(float) +
                       NWARP * NSTAGE * 8;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(decode_gqa_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static SmemLimit limit = {};
+  if (cudaError_t e0 = ensure_dyn_smem(decode_gqa_kernel<G>, smem, limit)) return e0;
   // Both kernels are programmatic dependent launches: each may become resident while its
   // predecessor in the stream drains, and waits (griddepcontrol.wait) before touching memory.
   cudaLaunchAttribute attr[1];

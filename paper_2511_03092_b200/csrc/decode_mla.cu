@@ -311,12 +311,8 @@ cudaError_t launch_decode_mla(const Shape& s, const void* q, const void* k_new, 
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.seq_len = seq_len; a.valid_topk = valid_topk; a.partials = partials; a.status = status;
   const size_t smem = QS_B + NSTG * KT_B;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(decode_mla_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static SmemLimit limit = {};
+  if (cudaError_t e = ensure_dyn_smem(decode_mla_kernel, smem, limit)) return e;
   dim3 grid(nsplit, s.Hq / HB, n_active);
   decode_mla_kernel<<<grid, NT, smem, st>>>(a);
   count_launch();

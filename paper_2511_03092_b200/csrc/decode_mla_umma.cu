@@ -400,12 +400,8 @@ cudaError_t launch_decode_mla_umma(const Shape& s, const void* q, const void* k_
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.partials = partials; a.status = status;
   const size_t smem = umma_smem_bytes();
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(decode_mla_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static SmemLimit limit = {};
+  if (cudaError_t e = ensure_dyn_smem(decode_mla_umma_kernel, smem, limit)) return e;
   dim3 grid(nsplit, NQ * (s.Hq / HBLK), n_active);
   decode_mla_umma_kernel<<<grid, NTH, smem, st>>>(a, tc);
   count_launch();

@@ -24,7 +24,6 @@ namespace snap {
 namespace {
 
 constexpr size_t kStaticFloats = SNAP_STATIC_SCRATCH_BYTES / sizeof(float);
-constexpr int kMaxDevices = 64;
 
 // The scratch itself.  In host code this name is only a handle for the runtime, not an address
 // the GPU can use; the usable address comes from cudaGetSymbolAddress below.

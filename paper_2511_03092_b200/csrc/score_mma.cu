@@ -311,14 +311,9 @@ cudaError_t launch_score_mma(const Shape& s, const SeqBatch& b, const void* q_ob
   a.b = b; a.buf = buf;
   const int nrw = a.RP / 32;
   const size_t smem = (size_t)a.RP * ROW_B + 2 * KT_B + 2 * nrw * TN * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(score_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(score_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static SmemLimit limit1 = {}, limit2 = {};
+  if (cudaError_t e = ensure_dyn_smem(score_mma_kernel<1>, 110 * 1024, limit1)) return e;
+  if (cudaError_t e = ensure_dyn_smem(score_mma_kernel<2>, 110 * 1024, limit2)) return e;
   const int nz = b.n_scored * s.Hkv;
   dim3 grid(buf.nsplit, nz);
   score_mma_kernel<1><<<grid, 32 * nrw, smem, st>>>(a);

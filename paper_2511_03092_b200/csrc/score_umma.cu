@@ -493,14 +493,9 @@ cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_o
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(score_umma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(score_umma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static SmemLimit limit1 = {}, limit2 = {};
+  if (cudaError_t e = ensure_dyn_smem(score_umma_kernel<1>, kSmemBytes, limit1)) return e;
+  if (cudaError_t e = ensure_dyn_smem(score_umma_kernel<2>, kSmemBytes, limit2)) return e;
   const int nz = b.n_scored * s.Hkv;
   dim3 grid(buf.nsplit, nz);
   score_umma_kernel<1><<<grid, NTHREADS, kSmemBytes, st>>>(a, tq, tk);

@@ -338,14 +338,9 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
       return cudaErrorInvalidValue;
   }
   const size_t smem = wide_smem_bytes(a.NH, a.NS);
-  static size_t attr_bytes = 0;
-  if (smem > attr_bytes) {
-    cudaError_t e = cudaFuncSetAttribute(score_umma_wide_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(score_umma_wide_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_bytes = smem;
-  }
+  static SmemLimit limit1 = {}, limit2 = {};
+  if (cudaError_t e = ensure_dyn_smem(score_umma_wide_kernel<1>, smem, limit1)) return e;
+  if (cudaError_t e = ensure_dyn_smem(score_umma_wide_kernel<2>, smem, limit2)) return e;
   const int nz = b.n_scored * s.Hkv;
   int max_le = 0;
   for (int i = 0; i < b.n; ++i)

@@ -48,6 +48,22 @@ struct ScoreBuffers {
 extern unsigned long long g_launches;
 inline void count_launch() { ++g_launches; }
 
+// A kernel's dynamic shared-memory limit is a per-device attribute: raise it once on every
+// device the library is used on.  `done` is the caller's per-kernel record (static storage).
+constexpr int kMaxDevices = 64;
+struct SmemLimit { size_t bytes[kMaxDevices]; };
+template <typename Kernel>
+inline cudaError_t ensure_dyn_smem(Kernel kernel, size_t bytes, SmemLimit& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (done.bytes[dev] >= bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) done.bytes[dev] = bytes;
+  return e;
+}
+
 // --- launchers (each enqueues on `st` and returns cudaGetLastError()) ---
 cudaError_t launch_score_simt(int dtype, const Shape& s, const SeqBatch& b, const void* q_obs,
                               const KVSource& src, const ScoreBuffers& buf, cudaStream_t st);
