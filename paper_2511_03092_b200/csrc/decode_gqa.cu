@@ -1,5 +1,5 @@
-// Decode attention over the compressed cache (Section 3.3) for grouped-query bf16 layers with
-// 128-wide heads -- the HBM-bound kernel of the decode step.
+// Decode attention over the compressed cache (Section 3.3) for bf16 layers with 128-wide heads
+// and 1 to 8 query heads per KV head -- the HBM-bound kernel of the decode step.
 //
 // Split-K flash decoding.  Grid = (splits, KV heads, sequences).  A CTA's share of the valid
 // cache rows ([0, min(len, Lsr)) then [Lsr, Lsr + valid_topk)) is cut into 16-row tiles that
@@ -42,6 +42,7 @@ struct FastArgs {
   char* kc; char* vc;
   long long seq_b, head_b;                      // cache strides in bytes (K and V alike)
   int Hq, Hkv, Ls, Lr, max_seqs, nsplit;
+  int g;                                        // real group size (<= the kernel's G, which is even)
   float scale_log2;                             // softmax_scale * log2(e)
   const int* seq_len; const int* valid_topk;
   float* partials;                              // [n_active][Hq][nsplit][PS]
@@ -126,7 +127,7 @@ __device__ __forceinline__ void unpack8(const uint4& u, u64 (&f)[4]) {
 }
 
 template <int G>
-__global__ void __launch_bounds__(NT, (G == 8 ? 2 : 3)) decode_gqa_kernel(const FastArgs a) {
+__global__ void __launch_bounds__(NT, (G > 4 ? 2 : 3)) decode_gqa_kernel(const FastArgs a) {
   constexpr int VPL = G / 2;                    // logits a lane holds after the reduction
   extern __shared__ __align__(128) unsigned char smem_raw[];
   // [NWARP][NSTAGE] stages | [NWARP][2][8][G][2] probabilities | [NWARP][NSTAGE] mbarriers
@@ -185,11 +186,12 @@ __global__ void __launch_bounds__(NT, (G == 8 ? 2 : 3)) decode_gqa_kernel(const 
   // query rows of the group, pre-scaled so that exp2 can be used directly
   u64 q2[G][4];
   {
-    const __nv_bfloat16* qp = a.q + ((long long)i * a.Hq + (long long)kvh * G) * D + l16 * 8;
+    const __nv_bfloat16* qp = a.q + ((long long)i * a.Hq + (long long)kvh * a.g) * D + l16 * 8;
     const u64 sc2 = pack2(a.scale_log2, a.scale_log2);
 #pragma unroll
     for (int h = 0; h < G; ++h) {
-      const uint4 u = *reinterpret_cast<const uint4*>(qp + h * D);
+      // groups of odd size run with one all-zero query row; its result is never written
+      const uint4 u = h < a.g ? *reinterpret_cast<const uint4*>(qp + h * D) : make_uint4(0, 0, 0, 0);
       unpack8(u, q2[h]);
 #pragma unroll
       for (int c = 0; c < 4; ++c) q2[h][c] = mul2(q2[h][c], sc2);
@@ -365,7 +367,7 @@ __global__ void __launch_bounds__(NT, (G == 8 ? 2 : 3)) decode_gqa_kernel(const 
       for (int c = 0; c < 8; ++c) wacc[h * D + l16 * 8 + c] = acc[h][c];
   }
   __syncthreads();
-  float* part_out = a.partials + (((long long)i * a.Hq + (long long)kvh * G) * a.nsplit + sp) * PS;
+  float* part_out = a.partials + (((long long)i * a.Hq + (long long)kvh * a.g) * a.nsplit + sp) * PS;
   constexpr int WSTRIDE = NSTAGE * STAGE_B / 4;            // floats between two warps' regions
   const float* base = reinterpret_cast<const float*>(smem_raw);
 #pragma unroll
@@ -381,9 +383,11 @@ __global__ void __launch_bounds__(NT, (G == 8 ? 2 : 3)) decode_gqa_kernel(const 
       L += base[ww * WSTRIDE + G + h] * f;
       O += base[ww * WSTRIDE + 2 * G + h * D + tid] * f;
     }
-    float* ph = part_out + (long long)h * a.nsplit * PS;
-    if (tid == 0) { ph[0] = M; ph[1] = L; }
-    ph[2 + tid] = O;
+    if (h < a.g) {
+      float* ph = part_out + (long long)h * a.nsplit * PS;
+      if (tid == 0) { ph[0] = M; ph[1] = L; }
+      ph[2 + tid] = O;
+    }
   }
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
@@ -451,7 +455,7 @@ cudaError_t launch_g(const FastArgs& a, int n_active, __nv_bfloat16* out, int* s
 }  // namespace
 
 bool decode_gqa_supported(int dtype, const Shape& s) {
-  return dtype == SNAP_BF16 && s.d_qk == D && s.d_v == D && !s.v_aliases_k && (s.g == 2 || s.g == 4 || s.g == 8);
+  return dtype == SNAP_BF16 && s.d_qk == D && s.d_v == D && !s.v_aliases_k && s.g >= 1 && s.g <= 8;
 }
 
 // Splits per (sequence, KV head): enough CTAs to fill every resident slot (3 CTAs per SM, 2 for
@@ -464,7 +468,7 @@ int decode_gqa_nsplit(const Shape& s, int n_active, int sm_count) {
     if (v >= 1) return v < tiles ? v : tiles;
   }
   const long long base = (long long)n_active * s.Hkv;
-  const double slots = (s.g == 8 ? 2.0 : 3.0) * sm_count;
+  const double slots = (s.g > 4 ? 2.0 : 3.0) * sm_count;
   int best = 1;
   double best_score = -1.0;
   const int max_ns = tiles < 64 ? tiles : 64;
@@ -495,15 +499,17 @@ cudaError_t launch_decode_gqa(const Shape& s, const void* q, const void* k_new, 
   a.slot_ids = slot_ids;
   a.kc = static_cast<char*>(k_cache); a.vc = static_cast<char*>(v_cache);
   a.head_b = (long long)s.Sc * ROW_B; a.seq_b = a.head_b * s.Hkv;
-  a.Hq = s.Hq; a.Hkv = s.Hkv; a.Ls = s.Ls; a.Lr = s.Lr; a.max_seqs = s.max_seqs; a.nsplit = nsplit;
+  a.Hq = s.Hq; a.Hkv = s.Hkv; a.Ls = s.Ls; a.Lr = s.Lr; a.max_seqs = s.max_seqs; a.nsplit = nsplit; a.g = s.g;
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.seq_len = seq_len; a.valid_topk = valid_topk; a.partials = partials; a.status = status;
   __nv_bfloat16* o = static_cast<__nv_bfloat16*>(out);
   const int bump = k_new != nullptr;
   switch (s.g) {
-    case 2: return launch_g<2>(a, n_active, o, seq_len, bump, st);
-    case 4: return launch_g<4>(a, n_active, o, seq_len, bump, st);
-    case 8: return launch_g<8>(a, n_active, o, seq_len, bump, st);
+    // the kernel handles an even number of heads per KV head; odd group sizes run padded by one
+    case 1: case 2: return launch_g<2>(a, n_active, o, seq_len, bump, st);
+    case 3: case 4: return launch_g<4>(a, n_active, o, seq_len, bump, st);
+    case 5: case 6: return launch_g<6>(a, n_active, o, seq_len, bump, st);
+    case 7: case 8: return launch_g<8>(a, n_active, o, seq_len, bump, st);
     default: return cudaErrorInvalidValue;
   }
 }

@@ -189,8 +189,10 @@ def test_slot_reuse_overwrites_everything():
     H.check_cache_image(layer, H.oracle_compress(wl, p), 0, wl)
 
 
-@pytest.mark.parametrize("hq,hkv", [(8, 4), (32, 4), (4, 4)], ids=["g2", "g8", "g1"])
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 4), (12, 4), (20, 4), (24, 4), (28, 4), (32, 4)],
+                         ids=["g1", "g2", "g3", "g5", "g6", "g7", "g8"])
 def test_group_sizes(hq, hkv):
+    """Every number of query heads per KV head from 1 to 8 (odd sizes run padded by one head)."""
     wl = SMALL_BF16.scaled(n_q_heads=hq, n_kv_heads=hkv)
     _run_compress_and_decode(wl, [wl.prompt_len[0], 50, 3], seed=13, steps=5)
 
