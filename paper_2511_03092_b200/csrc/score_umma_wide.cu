@@ -1,5 +1,7 @@
 // Observation-window scores (Eq. 4 -> Eq. 1) on tcgen05 for wide rows and many window rows --
-// the latent-attention shape: 128 query heads x Lo rows (4096 window rows) against 576-wide keys.
+// the latent-attention shape: 128 query heads x Lo rows (4096 window rows) against 576-wide keys;
+// also every other bf16 shape with rows of 64 to 576 dims in steps of 64 (a partly filled last
+// block of window rows is masked).
 //
 // Same roles as the 128-wide kernel (TMA producer warp, single-thread MMA issuer, eight epilogue
 // warps reading TMEM), but the contraction dimension is streamed: grid = (candidate splits,
@@ -77,8 +79,14 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (PASS == 2 && tid < 128) {
-    const float2 st = a.buf.stats[(long long)z * R + rb * 128 + tid];
-    mu_s[tid] = st.x - log2f(st.y);
+    // rows past the group's last one (a partly filled row block) get an infinite offset: weight 0
+    const int row = rb * 128 + tid;
+    float mu = INFINITY;
+    if (row < a.R) {
+      const float2 st = a.buf.stats[(long long)z * a.R + row];
+      mu = st.x - log2f(st.y);
+    }
+    mu_s[tid] = mu;
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
@@ -245,7 +253,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
   fence_before();
   __syncthreads();
   fence_after();
-  if (PASS == 1 && warp >= 2 && eg == 0) {                     // the two groups took different candidates of each tile
+  if (PASS == 1 && warp >= 2 && eg == 0 && rb * 128 + lrow < R) {   // the two groups took different candidates of each tile
     const float2 o = xch[lrow];
     merge_ml(m_ref, l_sum, o.x, o.y);
     a.buf.part_stats[((long long)z * a.buf.nsplit + blockIdx.x) * R + rb * 128 + lrow] = make_float2(m_ref, l_sum);
@@ -286,11 +294,11 @@ int wide_stages(int NH) {
 
 bool score_umma_wide_supported(int dtype, const Shape& s) {
   const int R = s.g * s.Lo;
-  return dtype == SNAP_BF16 && s.d_qk % 64 == 0 && s.d_qk / 64 <= MAXH && R % 128 == 0 &&
+  return dtype == SNAP_BF16 && s.d_qk % 64 == 0 && s.d_qk / 64 <= MAXH && R >= 1 &&
          umma::encode_tiled_fn() != nullptr;
 }
 
-int score_umma_wide_row_blocks(const Shape& s) { return s.g * s.Lo / 128; }
+int score_umma_wide_row_blocks(const Shape& s) { return (s.g * s.Lo + 127) / 128; }
 
 // Candidate splits: about two CTAs per SM in sequence over (splits x row blocks x prompts x KV heads).
 int score_umma_wide_nsplit(const Shape& s, int n_scored, int max_le, int sm_count) {
@@ -310,7 +318,7 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   if (!enc) return cudaErrorNotSupported;
   WideArgs a;
   a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Lo = s.Lo; a.Ls = s.Ls; a.Lr = s.Lr; a.R = s.g * s.Lo;
-  a.NH = s.d_qk / 64; a.RB = a.R / 128; a.NS = wide_stages(a.NH);
+  a.NH = s.d_qk / 64; a.RB = (a.R + 127) / 128; a.NS = wide_stages(a.NH);
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.b = b; a.buf = buf; a.cpart = cpart; a.status = status;
 
