@@ -124,25 +124,25 @@ int check_cu(const int32_t* cu, int n_seq) {
   return SNAP_OK;
 }
 
-struct DecodePlan { bool gqa, mla, mla_umma; int nsplit; size_t floats; };
+struct DecodePlan { bool gqa, mla, mla_stream; int nsplit; size_t floats; };
 
-// The latent layout decodes on the tcgen05 kernel when the head count allows (multiples of 128);
-// SNAP_DECODE_MLA=mma keeps it on the mma.sync kernel (testing aid).
-bool use_mla_umma(int dtype, const Shape& s) {
+// Kernel for the latent layout: the streamed tcgen05 kernel when the head count allows (multiples
+// of 128), else the mma.sync kernel; SNAP_DECODE_MLA=mma forces the latter (testing aid).
+bool use_mla_stream(int dtype, const Shape& s) {
   const char* env = getenv("SNAP_DECODE_MLA");
   if (env && env[0] == 'm') return false;
-  return decode_mla_umma_supported(dtype, s);
+  return decode_mla_stream_supported(dtype, s);
 }
 
 DecodePlan plan_decode(int dtype, const Shape& s, int n_active) {
   DecodePlan p;
   const int n = n_active > 0 ? n_active : 1;
   p.gqa = decode_gqa_supported(dtype, s);
-  p.mla_umma = !p.gqa && use_mla_umma(dtype, s);
-  p.mla = !p.gqa && !p.mla_umma && decode_mla_supported(dtype, s);
-  if (p.mla_umma) {
-    p.nsplit = decode_mla_umma_nsplit(s, n, sm_count());
-    p.floats = decode_mla_umma_partial_floats(s, n_active, p.nsplit);
+  p.mla_stream = !p.gqa && use_mla_stream(dtype, s);
+  p.mla = !p.gqa && !p.mla_stream && decode_mla_supported(dtype, s);
+  if (p.mla_stream) {
+    p.nsplit = decode_mla_stream_nsplit(s, n, sm_count());
+    p.floats = decode_mla_stream_partial_floats(s, n_active, p.nsplit);
   } else if (p.mla) {
     p.nsplit = decode_mla_nsplit(s, n, sm_count());
     p.floats = decode_mla_partial_floats(s, n_active, p.nsplit);
@@ -362,9 +362,9 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
   const DecodePlan p = plan_decode(cfg->dtype, s, n_active);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e;
-  if (p.mla_umma)
-    e = launch_decode_mla_umma(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev,
-                               valid_topk_dev, out_dev, static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
+  if (p.mla_stream)
+    e = launch_decode_mla_stream(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev,
+                                 valid_topk_dev, out_dev, static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
   else if (p.mla)
     e = launch_decode_mla(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev,
                           valid_topk_dev, out_dev, static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);

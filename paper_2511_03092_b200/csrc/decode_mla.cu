@@ -246,6 +246,8 @@ __global__ void __launch_bounds__(256) decode_mla_merge_kernel(const float* __re
                                                                int max_seqs, int bump) {
   const int h = blockIdx.x, i = blockIdx.y;
   const float* p = partials + ((long long)i * Hq + h) * nsplit * PSM;
+  // when launched as a programmatic dependent, wait for the split kernel's results (no-op otherwise)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   float M = -INFINITY;
   for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * PSM]);
   float L = 0.f;
@@ -271,11 +273,21 @@ __global__ void __launch_bounds__(256) decode_mla_merge_kernel(const float* __re
 }  // namespace
 
 cudaError_t launch_decode_mla_merge(const float* partials, void* out, int n_active, int Hq, int nsplit,
-                                    const int* slot_ids, int* seq_len, int max_seqs, int bump, cudaStream_t st) {
-  decode_mla_merge_kernel<<<dim3(Hq, (unsigned)n_active), 256, 0, st>>>(partials, static_cast<__nv_bfloat16*>(out), Hq, nsplit,
-                                                                       slot_ids, seq_len, max_seqs, bump);
+                                    const int* slot_ids, int* seq_len, int max_seqs, int bump, cudaStream_t st,
+                                    bool programmatic) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(Hq, (unsigned)n_active);
+  lc.blockDim = dim3(256);
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = programmatic ? 1 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&lc, decode_mla_merge_kernel, partials, static_cast<__nv_bfloat16*>(out), Hq, nsplit,
+                                     slot_ids, seq_len, max_seqs, bump);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 bool decode_mla_supported(int dtype, const Shape& s) {

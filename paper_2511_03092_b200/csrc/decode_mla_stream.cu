@@ -1,0 +1,446 @@
+// Decode attention over the compressed cache (Section 3.3) for the latent-attention layout on
+// tcgen05, streamed version: one 576-wide cache row shared by all heads, V = its first 512 dims.
+//
+// An MMA instruction occupies the tensor pipe for a fixed minimum time however few columns it
+// produces, so this kernel is built around wide instructions: S = Q K^T in 128-row tiles
+// (N = 128) and O += P V over 256 value dims at a time (N = 256).  The 128 x 576 query block
+// stays in shared memory (nine 64-dim slabs, 128-byte swizzle) as the A operand of S; what is
+// left of shared memory is a ring of four 16 KB stages through which the cache rows stream
+// twice: as key slabs (128 rows x 64 dims, K-major B operand of S) and, once the tile's
+// probabilities exist, as value chunks (32 rows x 256 dims, MN-major B operand of P V).  The
+// second pass costs 0.44 of the first in L2 traffic and buys a tile four times as wide as one
+// that has to stay resident.  Tensor memory holds S twice (2 x 128 columns, so that the next
+// tile's logits are computed while the softmax warps work on this one) and O (256 columns: the
+// 512 value dims are split over two CTAs that each compute S); the probabilities overwrite
+// their own logits as bf16 pairs and are the TMEM-sourced A operand of P V.
+//
+// Grid = (row splits, 2 x head blocks, sequences), one CTA per SM:
+//   warp 0      TMA producer, in the order the MMAs consume: K(0), K(1), V(0), K(2), V(1), ...
+//   warp 1      MMA issuer (whole warp converged, instructions predicated on one lane)
+//   warps 2-5   thread = head: S from TMEM, online softmax in the log2 domain with a lazily
+//               refreshed reference (O is rescaled in TMEM only when a logit exceeds it by 8),
+//               P back to TMEM.
+// The new token, if any, is appended by a separate launch before this kernel (Eq. 3).  Every
+// mbarrier wait is bounded; one that runs out raises SNAP_DEV_WAIT_TIMEOUT.
+#include "snap_internal.cuh"
+#include "umma_helpers.cuh"
+
+namespace snap {
+namespace {
+
+using namespace umma;
+
+constexpr int DQK = 576, DV = 512, HBLK = 128, TR = 128, NSTG = 4, NTH = 192, DVH = 256, NHALF = DV / DVH;
+constexpr int NSLAB = DQK / 64, QSLAB_B = HBLK * 128, STAGE_B = 16384;   // key slab = 128 rows x 128 B = one stage
+constexpr int VROWS = 32, VSUB_B = VROWS * 128, NVCH = TR / VROWS;       // value chunk = 4 sub-slabs of 32 rows x 64 dims
+constexpr int PSM = DV + 2;
+constexpr uint32_t COL_S = 0, COL_O = 256;                               // tensor memory: S0 128 | S1 128 | O 256
+
+struct SArgs {
+  const int* slot_ids; const int* seq_len; const int* valid_topk;
+  int Hq, Ls, Lr, Sc, max_seqs, nsplit;
+  float scale_log2;
+  float* partials;                             // [n_active][Hq][nsplit][PSM], maxima in the log2 domain
+  uint32_t* status;
+};
+
+__host__ __device__ constexpr uint32_t idesc_f16(int M, int N, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
+}
+// MN-major operand, 128-byte swizzle: 64 contiguous elements per row of the contraction dim,
+// 8-row groups 1024 bytes apart, the next 64 elements `lbo_bytes` further on.
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t saddr, uint32_t lbo_bytes) {
+  return (uint64_t)((saddr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+         ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// MMAs and commits executed by a whole converged warp, predicated on one lane.
+__device__ __forceinline__ void mma_ss_pred(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc,
+                                            uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void mma_ts_pred(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc,
+                                            uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void commit_pred(uint32_t bar, uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// Bounded wait whose outcome is the same for every lane (what follows is warp-collective).
+__device__ __forceinline__ bool wait_warp(uint32_t bar, unsigned parity, volatile int* abort_flag) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+}
+
+// Tile g of a sequence: rows [row0, row0 + TR) of the cache, valid below row_end.  Tiles cover
+// [0, n_low) first, then [Lsr, Lsr + n_top).
+struct TileRows { int row0, row_end; };
+__device__ __forceinline__ TileRows tile_rows(int g, int nA, int n_low, int Lsr, int n_top) {
+  TileRows t;
+  if (g < nA) { t.row0 = g * TR; t.row_end = n_low; }
+  else { t.row0 = Lsr + (g - nA) * TR; t.row_end = Lsr + n_top; }
+  return t;
+}
+
+__global__ void __launch_bounds__(NTH, 1)
+decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                         const __grid_constant__ CUtensorMap tmap_v) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* Qs = smem;                                                   // [9 slabs][128 heads][128 B]
+  unsigned char* Rs = Qs + NSLAB * QSLAB_B;                                   // [NSTG][16 KB] ring
+  uint64_t* bars = reinterpret_cast<uint64_t*>(Rs + NSTG * STAGE_B);
+  // full[NSTG] empty[NSTG] s_full[2] p_ready[2] pv_done[2] q_full
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTG + 7);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int sp = blockIdx.x, hb = blockIdx.y / NHALF, hd = blockIdx.y % NHALF, i = blockIdx.z;
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8 * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8 * (NSTG + s); };
+  auto sfull_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + b); };
+  auto pready_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 2 + b); };
+  auto pvdone_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 4 + b); };
+  const uint32_t qfull_bar = bar0 + 8 * (2 * NSTG + 6);
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < NSTG; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(sfull_bar(b), 1); mbar_init(pready_bar(b), 4); mbar_init(pvdone_bar(b), 1); }
+    mbar_init(qfull_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // launched as a programmatic dependent of the append kernel: the set-up above overlaps it; wait
+  // for it before reading lengths or rows
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int slot = a.slot_ids[i];
+  const bool bad = slot < 0 || slot >= a.max_seqs;
+  const int Lsr = a.Ls + a.Lr;
+  int n_low = 0, n_top = 0;
+  if (!bad) {
+    n_low = min(a.seq_len[slot], Lsr);
+    n_top = a.valid_topk[slot];
+  } else if (tid == 0 && sp == 0 && blockIdx.y == 0 && a.status) {
+    atomicOr(a.status, SNAP_DEV_BAD_SLOT);
+  }
+  const int nA = (n_low + TR - 1) / TR, ntiles = nA + (n_top + TR - 1) / TR;
+  const int g0 = (int)((long long)ntiles * sp / a.nsplit);
+  const int g1 = (int)((long long)ntiles * (sp + 1) / a.nsplit);
+  const int nt = g1 - g0;
+
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0 && nt > 0) {
+      mbar_expect_tx(qfull_bar, (unsigned)NSLAB * QSLAB_B);
+      for (int h = 0; h < NSLAB; ++h)
+        tma_load_2d(smem_u32(Qs) + h * QSLAB_B, &tmap_q, h * 64, i * a.Hq + hb * HBLK, qfull_bar);
+      int q = 0;                                               // stages issued so far
+      bool ok = true;
+      auto stage_wait = [&]() -> bool {
+        const int s = q % NSTG;
+        if (!mbar_wait(empty_bar(s), ((unsigned)(q / NSTG) & 1u) ^ 1u, abort_flag)) { *abort_flag = 1; return false; }
+        mbar_expect_tx(full_bar(s), (unsigned)STAGE_B);
+        return true;
+      };
+      auto load_k = [&](int it) {                              // nine key slabs of tile it
+        const TileRows tr = tile_rows(g0 + it, nA, n_low, Lsr, n_top);
+        for (int h = 0; h < NSLAB && ok; ++h) {
+          ok = stage_wait();
+          if (!ok) break;
+          const int s = q % NSTG;
+          tma_load_3d(smem_u32(Rs) + s * STAGE_B, &tmap_k, h * 64, tr.row0, slot, full_bar(s));
+          ++q;
+        }
+      };
+      auto load_v = [&](int it) {                              // four value chunks of tile it (this CTA's 256 dims)
+        const TileRows tr = tile_rows(g0 + it, nA, n_low, Lsr, n_top);
+        for (int c = 0; c < NVCH && ok; ++c) {
+          ok = stage_wait();
+          if (!ok) break;
+          const int s = q % NSTG;
+          for (int j = 0; j < DVH / 64; ++j)
+            tma_load_3d(smem_u32(Rs) + s * STAGE_B + j * VSUB_B, &tmap_v, hd * DVH + j * 64, tr.row0 + c * VROWS, slot, full_bar(s));
+          ++q;
+        }
+      };
+      load_k(0);
+      for (int it = 0; it < nt && ok; ++it) {
+        if (it + 1 < nt) load_k(it + 1);
+        if (ok) load_v(it);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (nt > 0) {
+      const uint32_t leader = lane == 0;
+      const uint32_t idesc_s = idesc_f16(128, TR, false), idesc_pv = idesc_f16(128, DVH, true);
+      const uint64_t qd0 = smem_desc(smem_u32(Qs));
+      int q = 0;                                               // stages consumed so far
+      bool ok = wait_warp(qfull_bar, 0u, abort_flag);
+      fence_after();
+      auto issue_s = [&](int it) -> bool {                    // S[it & 1] = Q K(it)^T, one key slab per stage
+        const uint32_t sd = tmem_base + COL_S + (it & 1) * TR;
+#pragma unroll 1
+        for (int h = 0; h < NSLAB; ++h) {
+          const int s = q % NSTG;
+          if (!wait_warp(full_bar(s), (unsigned)(q / NSTG) & 1u, abort_flag)) return false;
+          fence_after();
+          const uint64_t kd = smem_desc(smem_u32(Rs) + s * STAGE_B), qd = qd0 + (uint64_t)((h * QSLAB_B) >> 4);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            mma_ss_pred(sd, qd + (uint64_t)(ks * 2), kd + (uint64_t)(ks * 2), idesc_s, (h | ks) != 0, leader);
+          commit_pred(empty_bar(s), leader);
+          ++q;
+        }
+        commit_pred(sfull_bar(it & 1), leader);
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      for (int it = 0; it < nt && ok; ++it) {
+        const int b = it & 1;
+        if (it + 1 < nt) { ok = issue_s(it + 1); if (!ok) break; }
+        ok = wait_warp(pready_bar(b), (unsigned)(it / 2) & 1u, abort_flag);
+        if (!ok) break;
+        fence_after();
+        const uint32_t pa = tmem_base + COL_S + b * TR;       // P(it) lies over the first 64 columns of S(it)
+#pragma unroll 1
+        for (int c = 0; c < NVCH; ++c) {                      // O += P(it) V(it), one 32-row value chunk per stage
+          const int s = q % NSTG;
+          ok = wait_warp(full_bar(s), (unsigned)(q / NSTG) & 1u, abort_flag);
+          if (!ok) break;
+          fence_after();
+          const uint32_t vst = smem_u32(Rs) + s * STAGE_B;
+#pragma unroll
+          for (int ks = 0; ks < VROWS / 16; ++ks)
+            mma_ts_pred(tmem_base + COL_O, pa + 8 * (c * (VROWS / 16) + ks), smem_desc_mn(vst + ks * 16 * 128, VSUB_B),
+                        idesc_pv, (it | c | ks) != 0, leader);
+          commit_pred(empty_bar(s), leader);
+          ++q;
+        }
+        if (ok) commit_pred(pvdone_bar(b), leader);
+      }
+      if (!ok && lane == 0) *abort_flag = 1;
+    }
+  } else {
+    // ---------------- softmax warps: thread = head ----------------
+    const int hrow = 32 * (warp & 3) + lane;                   // TMEM lane = head within the block
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+    const int head = hb * HBLK + hrow;
+    float m_ref = -INFINITY, l_sum = 0.f;
+    bool ok = true;
+    for (int it = 0; it < nt; ++it) {
+      const int b = it & 1;
+      if (!wait_warp(sfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag)) { ok = false; break; }
+      fence_after();
+      const uint32_t s_addr = lane_addr + COL_S + b * TR;
+      const TileRows tr = tile_rows(g0 + it, nA, n_low, Lsr, n_top);
+      const int nrows = tr.row_end - tr.row0;                  // >= 1; columns at or past it are masked
+      float v[TR];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < TR / 32; ++c) {
+        uint32_t r0[16], r1[16];
+        tmem_ld16_issue(s_addr + 32 * c, r0);
+        tmem_ld16_issue(s_addr + 32 * c + 16, r1);
+        tmem_ld16_wait(r0);
+        tmem_ld16_wait(r1);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          v[32 * c + j] = 32 * c + j < nrows ? __uint_as_float(r0[j]) * a.scale_log2 : -INFINITY;
+          v[32 * c + 16 + j] = 32 * c + 16 + j < nrows ? __uint_as_float(r1[j]) * a.scale_log2 : -INFINITY;
+          mx = fmaxf(mx, fmaxf(v[32 * c + j], v[32 * c + 16 + j]));
+        }
+      }
+      // Lazy reference: refreshed (and O rescaled) only when some head of the warp sees a logit 8
+      // above its reference; the tensor-memory accesses are warp-collective, so the warp votes.
+      if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+        const float m_new = fmaxf(m_ref, mx);
+        const float alpha = m_ref == -INFINITY ? 0.f : exp2f(m_ref - m_new);
+        if (it > 0) {
+          if (!wait_warp(pvdone_bar((it - 1) & 1), (unsigned)((it - 1) / 2) & 1u, abort_flag)) { ok = false; break; }
+          fence_after();
+#pragma unroll 1
+          for (int c = 0; c < DVH / 16; ++c) {
+            uint32_t o[16];
+            tmem_ld16_issue(lane_addr + COL_O + 16 * c, o);
+            tmem_ld16_wait(o);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st16(lane_addr + COL_O + 16 * c, o);
+          }
+          tmem_st_wait();
+        }
+        l_sum *= alpha;
+        m_ref = m_new;
+      }
+      const float mr = m_ref == -INFINITY ? 0.f : m_ref;
+      float ls0 = 0.f, ls1 = 0.f;
+      // the logits of this tile are all in registers, so the probabilities may overwrite them
+#pragma unroll
+      for (int c = 0; c < TR / 32; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float p0 = fast_exp2(v[32 * c + 2 * j] - mr), p1 = fast_exp2(v[32 * c + 2 * j + 1] - mr);
+          ls0 += p0;
+          ls1 += p1;
+          pk[j] = pack_bf16(p0, p1);
+        }
+        tmem_st16(s_addr + 16 * c, pk);
+      }
+      l_sum += ls0 + ls1;
+      tmem_st_wait();
+      fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pready_bar(b));
+    }
+    if (!ok) *abort_flag = 1;
+    // ---------------- this split's partial result ----------------
+    float* ph = a.partials + (((long long)i * a.Hq + head) * a.nsplit + sp) * PSM;
+    if (ok && nt > 0) ok = wait_warp(pvdone_bar((nt - 1) & 1), (unsigned)((nt - 1) / 2) & 1u, abort_flag);
+    if (!ok) *abort_flag = 1;
+    fence_after();
+    if (hd == 0) { ph[0] = nt > 0 && ok ? m_ref : -INFINITY; ph[1] = nt > 0 && ok ? l_sum : 0.f; }
+    const bool have = __all_sync(0xffffffffu, ok && nt > 0);
+#pragma unroll 1
+    for (int c = 0; c < DVH / 16; ++c) {
+      uint32_t o[16];
+      if (have) {
+        tmem_ld16_issue(lane_addr + COL_O + 16 * c, o);
+        tmem_ld16_wait(o);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) o[e] = 0u;
+      }
+      float2* d2 = reinterpret_cast<float2*>(ph + 2 + hd * DVH + 16 * c);   // ph + 2 is 8-byte aligned only
+#pragma unroll
+      for (int e = 0; e < 8; ++e) d2[e] = make_float2(__uint_as_float(o[2 * e]), __uint_as_float(o[2 * e + 1]));
+    }
+  }
+
+  fence_before();
+  __syncthreads();
+  fence_after();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+size_t stream_smem_bytes() { return (size_t)NSLAB * QSLAB_B + NSTG * STAGE_B + (2 * NSTG + 7) * 8 + 16 + 1024; }
+
+}  // namespace
+
+bool decode_mla_stream_supported(int dtype, const Shape& s) {
+  return dtype == SNAP_BF16 && s.v_aliases_k && s.d_qk == DQK && s.d_v == DV && s.Hkv == 1 && s.Hq % HBLK == 0 &&
+         umma::encode_tiled_fn() != nullptr;
+}
+
+// Row splits per sequence: the grid (splits x 2 value halves x head blocks x sequences) should
+// fill the SMs once or twice over, with at least two tiles per split.
+int decode_mla_stream_nsplit(const Shape& s, int n_active, int sm_count) {
+  const int tiles = (s.Sc + TR - 1) / TR + 1;
+  const long long base = (long long)n_active * NHALF * (s.Hq / HBLK);
+  int best = 1;
+  double best_fill = -1.0;
+  for (int ns = 1; ns <= 64 && ns <= (tiles / 2 > 1 ? tiles / 2 : 1); ++ns) {
+    const long long ctas = base * ns;
+    const long long waves = (ctas + sm_count - 1) / sm_count;
+    if (waves > 2 && ns > 1) break;
+    const double fill = (double)ctas / (double)(waves * sm_count);
+    if (fill > best_fill + 1e-9) { best_fill = fill; best = ns; }
+  }
+  return best;
+}
+
+size_t decode_mla_stream_partial_floats(const Shape& s, int n_active, int nsplit) {
+  return (size_t)n_active * s.Hq * nsplit * PSM;
+}
+
+cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* k_new, const int* slot_ids,
+                                     int n_active, void* k_cache, int* seq_len, const int* valid_topk, void* out,
+                                     float* partials, int nsplit, uint32_t* status, cudaStream_t st) {
+  if (n_active == 0) return cudaSuccess;
+  umma::EncodeTiledFn enc = umma::encode_tiled_fn();
+  if (!enc) return cudaErrorNotSupported;
+  if (k_new) {                                                 // Eq. 3 append (also advances the lengths)
+    cudaError_t e = launch_append(SNAP_BF16, s, k_new, nullptr, slot_ids, n_active, k_cache, nullptr, seq_len, status, st);
+    if (e != cudaSuccess) return e;
+  }
+  CUtensorMap tq, tk, tv;
+  const cuuint32_t estr2[2] = {1, 1}, estr3[3] = {1, 1, 1};
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)DQK, (cuuint64_t)n_active * s.Hq};
+    const cuuint64_t strides[1] = {(cuuint64_t)DQK * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)HBLK};
+    if (enc(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(q), dims, strides, box, estr2,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  const cuuint64_t dims[3] = {(cuuint64_t)DQK, (cuuint64_t)s.Sc, (cuuint64_t)s.max_seqs};
+  const cuuint64_t strides[2] = {(cuuint64_t)DQK * 2, (cuuint64_t)s.Sc * DQK * 2};
+  const cuuint32_t kbox[3] = {64, (cuuint32_t)TR, 1}, vbox[3] = {64, (cuuint32_t)VROWS, 1};
+  if (enc(&tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, k_cache, dims, strides, kbox, estr3, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+      enc(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, k_cache, dims, strides, vbox, estr3, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  SArgs a;
+  a.slot_ids = slot_ids; a.seq_len = seq_len; a.valid_topk = valid_topk;
+  a.Hq = s.Hq; a.Ls = s.Ls; a.Lr = s.Lr; a.Sc = s.Sc; a.max_seqs = s.max_seqs; a.nsplit = nsplit;
+  a.scale_log2 = s.scale * 1.4426950408889634f;
+  a.partials = partials; a.status = status;
+  const size_t smem = stream_smem_bytes();
+  static SmemLimit limit = {};
+  if (cudaError_t e = ensure_dyn_smem(decode_mla_stream_kernel, smem, limit)) return e;
+  // a programmatic dependent launch: the CTAs may become resident while the append kernel drains
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(nsplit, NHALF * (s.Hq / HBLK), n_active);
+  lc.blockDim = dim3(NTH);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&lc, decode_mla_stream_kernel, a, tq, tk, tv);
+  count_launch();
+  if (e != cudaSuccess) return e;
+  return launch_decode_mla_merge(partials, out, n_active, s.Hq, nsplit, slot_ids, seq_len, s.max_seqs, 0, st, true);
+}
+
+}  // namespace snap

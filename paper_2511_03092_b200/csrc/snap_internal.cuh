@@ -117,14 +117,15 @@ cudaError_t launch_decode_mla(const Shape& s, const void* q, const void* k_new, 
                               float* partials, int nsplit, uint32_t* status, cudaStream_t st);
 
 cudaError_t launch_decode_mla_merge(const float* partials, void* out, int n_active, int Hq, int nsplit,
-                                    const int* slot_ids, int* seq_len, int max_seqs, int bump, cudaStream_t st);
-// latent attention on tcgen05: queries and probabilities as tensor-memory operands (heads % 128 == 0)
-bool decode_mla_umma_supported(int dtype, const Shape& s);
-int decode_mla_umma_nsplit(const Shape& s, int n_active, int sm_count);
-size_t decode_mla_umma_partial_floats(const Shape& s, int n_active, int nsplit);
-cudaError_t launch_decode_mla_umma(const Shape& s, const void* q, const void* k_new, const int* slot_ids,
-                                   int n_active, void* k_cache, int* seq_len, const int* valid_topk, void* out,
-                                   float* partials, int nsplit, uint32_t* status, cudaStream_t st);
+                                    const int* slot_ids, int* seq_len, int max_seqs, int bump, cudaStream_t st,
+                                    bool programmatic = false);
+// latent attention on tcgen05, streamed: queries in shared memory, cache rows streamed as key slabs and value chunks
+bool decode_mla_stream_supported(int dtype, const Shape& s);
+int decode_mla_stream_nsplit(const Shape& s, int n_active, int sm_count);
+size_t decode_mla_stream_partial_floats(const Shape& s, int n_active, int nsplit);
+cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* k_new, const int* slot_ids,
+                                     int n_active, void* k_cache, int* seq_len, const int* valid_topk, void* out,
+                                     float* partials, int nsplit, uint32_t* status, cudaStream_t st);
 
 // --- small device helpers ---
 template <typename T> __device__ __forceinline__ float to_f32(T x);
