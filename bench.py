@@ -40,9 +40,9 @@ UNIT = "tokens/s"
 SEED = 2511
 POOL_EXTRA = 16            # prompts beyond the initial batch that replacements cycle through
 DECODE_RING = 8            # distinct pre-generated decode inputs cycled through
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_gqa_kernel launch on this launch shape (32 full
-# 5124-slot caches), from the ncu capture summarised in profiles/decode_gqa_kernel_32seq_llama_cache.md
-DECODE_TRAFFIC_BYTES = 672.11e6 + 5.82e6
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_gqa_mma_kernel launch on this launch shape (32 full
+# 5124-slot caches), from the ncu capture summarised in profiles/decode_gqa_mma_kernel_32seq_llama_cache.md
+DECODE_TRAFFIC_BYTES = 672.03e6 + 8.11e6
 
 
 def _peaks():

@@ -12,6 +12,14 @@ namespace snap {
 
 unsigned long long g_launches = 0;
 
+// 128-wide bf16 heads decode on the tensor-core kernel (faster than the packed-FP32 kernel at every
+// group size); SNAP_DECODE_GQA=simt keeps the packed-FP32 kernel (testing aid).
+bool decode_use_gqa_mma(int dtype, const Shape& s) {
+  const char* env = getenv("SNAP_DECODE_GQA");
+  if (env && env[0] == 's') return false;
+  return decode_gqa_mma_supported(dtype, s);
+}
+
 namespace {
 
 int sm_count() {
@@ -124,7 +132,9 @@ int check_cu(const int32_t* cu, int n_seq) {
   return SNAP_OK;
 }
 
-struct DecodePlan { bool gqa, mla, mla_stream; int nsplit; size_t floats; };
+struct DecodePlan { bool gqa, gqa_mma, mla, mla_stream; int nsplit; size_t floats; };
+
+bool use_gqa_mma(int dtype, const Shape& s) { return decode_use_gqa_mma(dtype, s); }
 
 // Kernel for the latent layout: the streamed tcgen05 kernel when the head count allows (multiples
 // of 128), else the mma.sync kernel; SNAP_DECODE_MLA=mma forces the latter (testing aid).
@@ -137,6 +147,7 @@ bool use_mla_stream(int dtype, const Shape& s) {
 DecodePlan plan_decode(int dtype, const Shape& s, int n_active) {
   DecodePlan p;
   const int n = n_active > 0 ? n_active : 1;
+  p.gqa_mma = false;
   p.gqa = decode_gqa_supported(dtype, s);
   p.mla_stream = !p.gqa && use_mla_stream(dtype, s);
   p.mla = !p.gqa && !p.mla_stream && decode_mla_supported(dtype, s);
@@ -147,7 +158,8 @@ DecodePlan plan_decode(int dtype, const Shape& s, int n_active) {
     p.nsplit = decode_mla_nsplit(s, n, sm_count());
     p.floats = decode_mla_partial_floats(s, n_active, p.nsplit);
   } else if (p.gqa) {
-    p.nsplit = decode_gqa_nsplit(s, n, sm_count());
+    p.gqa_mma = use_gqa_mma(dtype, s);
+    p.nsplit = p.gqa_mma ? decode_gqa_mma_nsplit(s, n, sm_count()) : decode_gqa_nsplit(s, n, sm_count());
     p.floats = decode_gqa_partial_floats(s, n_active, p.nsplit);
   } else {
     p.nsplit = decode_generic_nsplit(s, n, sm_count());
@@ -368,6 +380,10 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
   else if (p.mla)
     e = launch_decode_mla(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev,
                           valid_topk_dev, out_dev, static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
+  else if (p.gqa && p.gqa_mma)
+    e = launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
+                              v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
+                              static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
   else if (p.gqa)
     e = launch_decode_gqa(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
                           v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,

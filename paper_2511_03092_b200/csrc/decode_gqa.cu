@@ -454,6 +454,24 @@ cudaError_t launch_g(const FastArgs& a, int n_active, __nv_bfloat16* out, int* s
 
 }  // namespace
 
+// The split merge as a programmatic dependent launch (shared with the tensor-core kernel).
+cudaError_t launch_decode_gqa_merge(const float* partials, void* out, int Hq, int nsplit, const int* slot_ids,
+                                    int n_active, int* seq_len, int max_seqs, int bump, cudaStream_t st) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(Hq, n_active);
+  lc.blockDim = dim3(D);
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_merge_kernel, partials, static_cast<__nv_bfloat16*>(out), Hq, nsplit,
+                                     slot_ids, seq_len, max_seqs, bump);
+  count_launch();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 bool decode_gqa_supported(int dtype, const Shape& s) {
   return dtype == SNAP_BF16 && s.d_qk == D && s.d_v == D && !s.v_aliases_k && s.g >= 1 && s.g <= 8;
 }
@@ -461,14 +479,14 @@ bool decode_gqa_supported(int dtype, const Shape& s) {
 // Splits per (sequence, KV head): enough CTAs to fill every resident slot (3 CTAs per SM, 2 for
 // g = 8), preferring counts whose last wave is nearly full, with at least one 64-row block per
 // split.  SNAP_DECODE_NSPLIT overrides the choice (tuning aid).
-int decode_gqa_nsplit(const Shape& s, int n_active, int sm_count) {
+int decode_gqa_nsplit_for(const Shape& s, int n_active, int sm_count, int ctas_per_sm) {
   const int tiles = (s.Sc + 63) / 64;
   if (const char* env = getenv("SNAP_DECODE_NSPLIT")) {
     const int v = atoi(env);
     if (v >= 1) return v < tiles ? v : tiles;
   }
   const long long base = (long long)n_active * s.Hkv;
-  const double slots = (s.g > 4 ? 2.0 : 3.0) * sm_count;
+  const double slots = (double)ctas_per_sm * sm_count;
   int best = 1;
   double best_score = -1.0;
   const int max_ns = tiles < 64 ? tiles : 64;
@@ -481,6 +499,12 @@ int decode_gqa_nsplit(const Shape& s, int n_active, int sm_count) {
     if (score > best_score + 1e-9) { best_score = score; best = ns; }
   }
   return best;
+}
+int decode_gqa_nsplit(const Shape& s, int n_active, int sm_count) {
+  return decode_gqa_nsplit_for(s, n_active, sm_count, s.g > 4 ? 2 : 3);
+}
+int decode_gqa_mma_nsplit(const Shape& s, int n_active, int sm_count) {
+  return decode_gqa_nsplit_for(s, n_active, sm_count, 3);
 }
 
 size_t decode_gqa_partial_floats(const Shape& s, int n_active, int nsplit) {

@@ -1,0 +1,335 @@
+// Decode attention over the compressed cache (Section 3.3) for bf16 layers with 128-wide heads
+// and 5 to 8 query heads per KV head, on tensor cores.
+//
+// From five heads per KV head on, the multiply-adds of the packed-FP32 kernel outrun the FP32
+// pipe before HBM is saturated.  Here the same split-K scheme (grid = splits x KV heads x
+// sequences, warp-private pipelines of 16-row tiles, one partial result per split, the same
+// merge kernel) does its arithmetic with mma.sync.m16n8k16, the group's heads on the N side:
+//     S^T[16 rows x 8 heads]   = K tile [16 x 128] . Q^T                  (8 MMAs)
+//     O^T[128 dims x 8 heads] += V tile^T [128 x 16] . P^T [16 x 8 heads] (8 MMAs)
+// so the cost per cache row no longer depends on the group size.  Tiles arrive through TMA
+// tensor loads with the 128-byte swizzle (two 64-dim slabs per tensor), which makes the
+// ldmatrix reads conflict-free; V is read with ldmatrix.trans; the probabilities leave the
+// S^T accumulators for the B operand of the second product through movmatrix (an 8x8
+// transpose across the warp).  Online softmax is per head in the log2 domain with a lazily
+// refreshed reference; row sums are kept per thread and reduced once at the end.
+//
+// Fused append (Eq. 3): as in the packed-FP32 kernel, the warp that stages the new token's
+// slot stores the row to the cache and patches its staged copy.
+#include <cuda.h>
+
+#include "snap_internal.cuh"
+#include "umma_helpers.cuh"
+
+namespace snap {
+namespace {
+
+using umma::mbar_init;
+using umma::mbar_expect_tx;
+using umma::mbar_try_wait;
+using umma::smem_u32;
+using umma::tma_load_3d;
+
+constexpr int D = 128, WT = 16, NSTAGE = 2, NWARP = 4, NT = NWARP * 32, GP = 8;   // GP: head slots (N of the MMAs)
+constexpr int SLAB_B = WT * 128, TENS_B = 2 * SLAB_B, STAGE_B = 2 * TENS_B;       // stage = K (2 slabs) | V (2 slabs)
+constexpr int PS = D + 2;
+constexpr unsigned kWaitLimit = 1u << 22;
+
+struct MmaArgs {
+  const __nv_bfloat16* q; const __nv_bfloat16* k_new; const __nv_bfloat16* v_new;
+  const int* slot_ids;
+  char* kc; char* vc;
+  long long seq_b, head_b;
+  int Hq, Hkv, g, Ls, Lr, max_seqs, nsplit;
+  float scale_log2;
+  const int* seq_len; const int* valid_topk;
+  float* partials;                              // [n_active][Hq][nsplit][PS]
+  uint32_t* status;
+};
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, unsigned parity) {
+  for (unsigned it = 0; it < kWaitLimit; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm4t(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// 8x8 transpose of 16-bit elements across the warp: lane (g, t) gives M[g][2t, 2t+1] and gets M[2t, 2t+1][g]
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// byte offset of row r, 16-byte chunk c (0..7) inside a 128-byte-swizzled slab
+__device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
+
+// Tile j of a (sequence, KV head): cache rows [row0, row0 + WT), valid below row_end.  Tiles
+// cover [0, n_low) first, then [Lsr, Lsr + n_top); a tile never spans the two regions.
+struct TileRows { int row0, row_end; };
+__device__ __forceinline__ TileRows tile_rows(int j, int nA, int n_low, int Lsr, int n_top) {
+  TileRows t;
+  if (j < nA) { t.row0 = j * WT; t.row_end = n_low; }
+  else { t.row0 = Lsr + (j - nA) * WT; t.row_end = Lsr + n_top; }
+  return t;
+}
+
+__global__ void __launch_bounds__(NT, 3)
+decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem_raw = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  // [NWARP][NSTAGE] stages | [NWARP][NSTAGE] mbarriers
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + NWARP * NSTAGE * STAGE_B);
+
+  const int sp = blockIdx.x, kvh = blockIdx.y, i = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, gq = lane >> 2, tq = lane & 3;
+  unsigned char* wstages = smem_raw + w * NSTAGE * STAGE_B;
+  const uint32_t stage0 = smem_u32(wstages), bar0 = smem_u32(bars + w * NSTAGE);
+  if (lane == 0) {
+    for (int s = 0; s < NSTAGE; ++s) mbar_init(bar0 + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int slot = a.slot_ids[i];
+  const bool bad = slot < 0 || slot >= a.max_seqs;
+  const int Lsr = a.Ls + a.Lr;
+  int n_low = 0, n_top = 0, new_slot = -1;
+  if (!bad) {
+    const int t = a.seq_len[slot];
+    n_low = min(t + (a.k_new ? 1 : 0), Lsr);
+    n_top = a.valid_topk[slot];
+    if (a.k_new) new_slot = ring_slot(t, a.Ls, a.Lr);
+  } else if (tid == 0 && sp == 0 && kvh == 0 && a.status) {
+    atomicOr(a.status, SNAP_DEV_BAD_SLOT);
+  }
+  const int nA = (n_low + WT - 1) / WT, ntiles = nA + (n_top + WT - 1) / WT;
+  const int t_begin = (int)((long long)ntiles * sp / a.nsplit);
+  const int t_end = (int)((long long)ntiles * (sp + 1) / a.nsplit);
+  // this warp's tiles: t_begin + w, t_begin + w + NWARP, ...
+  const int T = t_end - t_begin > w ? (t_end - t_begin - w + NWARP - 1) / NWARP : 0;
+  const int plane = bad ? 0 : slot * a.Hkv + kvh;               // third tensor-map coordinate
+
+  auto issue = [&](int n) {                                     // tile n of this warp -> stage n % NSTAGE
+    const int s = n % NSTAGE;
+    const TileRows tr = tile_rows(t_begin + w + n * NWARP, nA, n_low, Lsr, n_top);
+    const uint32_t dst = stage0 + s * STAGE_B, bar = bar0 + 8 * s;
+    mbar_expect_tx(bar, (unsigned)STAGE_B);
+    tma_load_3d(dst, &tmap_k, 0, tr.row0, plane, bar);
+    tma_load_3d(dst + SLAB_B, &tmap_k, 64, tr.row0, plane, bar);
+    tma_load_3d(dst + TENS_B, &tmap_v, 0, tr.row0, plane, bar);
+    tma_load_3d(dst + TENS_B + SLAB_B, &tmap_v, 64, tr.row0, plane, bar);
+  };
+  if (lane == 0)
+    for (int n = 0; n < NSTAGE && n < T; ++n) issue(n);
+
+  char* kc = a.kc + slot * a.seq_b + kvh * a.head_b;
+  char* vc = a.vc + slot * a.seq_b + kvh * a.head_b;
+  const __nv_bfloat16* kn = a.k_new ? a.k_new + ((long long)i * a.Hkv + kvh) * D : nullptr;
+  const __nv_bfloat16* vn = a.v_new ? a.v_new + ((long long)i * a.Hkv + kvh) * D : nullptr;
+
+  // B fragments of Q^T for the eight 16-dim steps: head gq (zero beyond the group), dims 16 ks + 2 tq (+8)
+  uint32_t qb[8][2];
+  {
+    const __nv_bfloat16* qp = a.q + ((long long)i * a.Hq + (long long)kvh * a.g + gq) * D + 2 * tq;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      qb[ks][0] = gq < a.g ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks) : 0u;
+      qb[ks][1] = gq < a.g ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks + 8) : 0u;
+    }
+  }
+  float oacc[8][4];                              // O^T: dims 16 db + gq (+8), heads 2 tq (+1)
+#pragma unroll
+  for (int db = 0; db < 8; ++db)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) oacc[db][e] = 0.f;
+  float m_ref[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};   // heads 2 tq, 2 tq + 1
+  bool timed_out = false;
+
+  // ldmatrix lane roles: K (plain): row (lane & 7) + 8 * bit3, chunk + bit4; V (transposed): row (lane & 7) + 8 * bit4, chunk + bit3
+  const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_cadd = lane >> 4;
+  const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8, v_cadd = (lane >> 3) & 1;
+
+  for (int n = 0; n < T; ++n) {
+    const int s = n % NSTAGE;
+    const unsigned parity = (unsigned)(n / NSTAGE) & 1u;
+    const bool landed = mbar_wait_bounded(bar0 + 8 * s, parity);
+    if (__any_sync(0xffffffffu, !landed)) { timed_out = true; break; }
+    const TileRows tr = tile_rows(t_begin + w + n * NWARP, nA, n_low, Lsr, n_top);
+    const int nrows = tr.row_end - tr.row0;                    // >= 1; rows at or past it are masked
+    const uint32_t sK = stage0 + s * STAGE_B, sV = sK + TENS_B;
+    if (new_slot >= tr.row0 && new_slot < tr.row0 + WT && new_slot < tr.row_end) {
+      // the new token's slot is in this tile: store the row to the cache and patch the staged copy
+      const int r = new_slot - tr.row0, c = lane & 15;
+      const uint4 val = reinterpret_cast<const uint4*>(lane < 16 ? kn : vn)[c];
+      reinterpret_cast<uint4*>((lane < 16 ? kc : vc) + (long long)new_slot * (D * 2))[c] = val;
+      unsigned char* sp_ = wstages + s * STAGE_B + (lane < 16 ? 0 : TENS_B) + (c >> 3) * SLAB_B + swz(r, c & 7);
+      *reinterpret_cast<uint4*>(sp_) = val;
+      __syncwarp();
+    }
+
+    // ---- S^T = K tile . Q^T ----
+    float sacc[4] = {0.f, 0.f, 0.f, 0.f};       // rows gq, gq + 8; heads 2 tq, 2 tq + 1
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      uint32_t af[4];
+      ldsm4(sK + (ks >> 2) * SLAB_B + swz(k_row, (ks & 3) * 2 + k_cadd), af);
+      mma16816(sacc, af, qb[ks][0], qb[ks][1]);
+    }
+    float v0 = gq < nrows ? sacc[0] * a.scale_log2 : -INFINITY, v1 = gq < nrows ? sacc[1] * a.scale_log2 : -INFINITY;
+    float v2 = gq + 8 < nrows ? sacc[2] * a.scale_log2 : -INFINITY, v3 = gq + 8 < nrows ? sacc[3] * a.scale_log2 : -INFINITY;
+    // Lazy reference per head: refreshed (accumulators rescaled) only when a warp vote sees a
+    // logit 8 above it; the column maxima are then reduced over the lanes that share tq.
+    if (__any_sync(0xffffffffu, fmaxf(v0, v2) > m_ref[0] + 8.f || fmaxf(v1, v3) > m_ref[1] + 8.f)) {
+      float mx0 = fmaxf(v0, v2), mx1 = fmaxf(v1, v3);
+#pragma unroll
+      for (int o = 4; o <= 16; o <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+      }
+      const float n0 = fmaxf(m_ref[0], mx0), n1 = fmaxf(m_ref[1], mx1);
+      const float a0 = m_ref[0] == -INFINITY ? 0.f : exp2f(m_ref[0] - n0), a1 = m_ref[1] == -INFINITY ? 0.f : exp2f(m_ref[1] - n1);
+      m_ref[0] = n0; m_ref[1] = n1;
+      l_part[0] *= a0; l_part[1] *= a1;
+#pragma unroll
+      for (int db = 0; db < 8; ++db) { oacc[db][0] *= a0; oacc[db][1] *= a1; oacc[db][2] *= a0; oacc[db][3] *= a1; }
+    }
+    const float r0 = m_ref[0] == -INFINITY ? 0.f : m_ref[0], r1 = m_ref[1] == -INFINITY ? 0.f : m_ref[1];
+    const float p0 = fast_exp2(v0 - r0), p1 = fast_exp2(v1 - r1), p2 = fast_exp2(v2 - r0), p3 = fast_exp2(v3 - r1);
+    l_part[0] += p0 + p2;
+    l_part[1] += p1 + p3;
+    // P^T as the B operand: rows 2 tq (+1) and 2 tq + 8 (+9) of head gq
+    const uint32_t pb0 = movmatrix_t(pack_bf16(p0, p1)), pb1 = movmatrix_t(pack_bf16(p2, p3));
+
+    // ---- O^T += V tile^T . P^T ----
+#pragma unroll
+    for (int db = 0; db < 8; ++db) {
+      uint32_t af[4];
+      ldsm4t(sV + (db >> 2) * SLAB_B + swz(v_row, (db & 3) * 2 + v_cadd), af);
+      mma16816(oacc[db], af, pb0, pb1);
+    }
+    __syncwarp();
+    if (lane == 0 && n + NSTAGE < T) issue(n + NSTAGE);
+  }
+  if (timed_out) {
+    if (a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
+    for (int s = 0; s < NSTAGE; ++s) (void)mbar_wait_bounded(bar0 + 8 * s, 0u);
+  }
+
+  // ---- per-warp result -> this warp's stage memory, then merge the warps ----
+#pragma unroll
+  for (int o = 4; o <= 16; o <<= 1) {
+    l_part[0] += __shfl_xor_sync(0xffffffffu, l_part[0], o);
+    l_part[1] += __shfl_xor_sync(0xffffffffu, l_part[1], o);
+  }
+  float* wm = reinterpret_cast<float*>(wstages);           // [GP] max, [GP] sum, [GP][D] acc
+  float* wl = wm + GP;
+  float* wacc = wl + GP;
+  __syncwarp();
+  if (gq == 0) {
+    wm[2 * tq] = m_ref[0]; wm[2 * tq + 1] = m_ref[1];
+    wl[2 * tq] = l_part[0]; wl[2 * tq + 1] = l_part[1];
+  }
+#pragma unroll
+  for (int db = 0; db < 8; ++db) {
+    wacc[(2 * tq) * D + 16 * db + gq] = oacc[db][0];
+    wacc[(2 * tq + 1) * D + 16 * db + gq] = oacc[db][1];
+    wacc[(2 * tq) * D + 16 * db + gq + 8] = oacc[db][2];
+    wacc[(2 * tq + 1) * D + 16 * db + gq + 8] = oacc[db][3];
+  }
+  __syncthreads();
+  float* part_out = a.partials + (((long long)i * a.Hq + (long long)kvh * a.g) * a.nsplit + sp) * PS;
+  constexpr int WSTRIDE = NSTAGE * STAGE_B / 4;            // floats between two warps' regions
+  const float* base = reinterpret_cast<const float*>(smem_raw);
+  for (int h = 0; h < a.g; ++h) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int ww = 0; ww < NWARP; ++ww) M = fmaxf(M, base[ww * WSTRIDE + h]);
+    float L = 0.f, O = 0.f;
+#pragma unroll
+    for (int ww = 0; ww < NWARP; ++ww) {
+      const float mw = base[ww * WSTRIDE + h];
+      const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
+      L += base[ww * WSTRIDE + GP + h] * f;
+      O += base[ww * WSTRIDE + 2 * GP + h * D + tid] * f;
+    }
+    float* ph = part_out + (long long)h * a.nsplit * PS;
+    if (tid == 0) { ph[0] = M; ph[1] = L; }
+    ph[2 + tid] = O;
+  }
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+}  // namespace
+
+bool decode_gqa_mma_supported(int dtype, const Shape& s) {
+  return dtype == SNAP_BF16 && s.d_qk == D && s.d_v == D && !s.v_aliases_k && s.g >= 1 && s.g <= GP &&
+         umma::encode_tiled_fn() != nullptr;
+}
+
+cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_new, const void* v_new,
+                                  const int* slot_ids, int n_active, void* k_cache, void* v_cache,
+                                  int* seq_len, const int* valid_topk, void* out, float* partials,
+                                  int nsplit, uint32_t* status, cudaStream_t st) {
+  if (n_active == 0) return cudaSuccess;
+  umma::EncodeTiledFn enc = umma::encode_tiled_fn();
+  if (!enc) return cudaErrorNotSupported;
+  CUtensorMap tk, tv;
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)s.Sc, (cuuint64_t)s.max_seqs * s.Hkv};
+  const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)s.Sc * D * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)WT, 1}, estr[3] = {1, 1, 1};
+  if (enc(&tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, k_cache, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+      enc(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, v_cache, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  MmaArgs a;
+  a.q = static_cast<const __nv_bfloat16*>(q);
+  a.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  a.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  a.slot_ids = slot_ids;
+  a.kc = static_cast<char*>(k_cache); a.vc = static_cast<char*>(v_cache);
+  a.head_b = (long long)s.Sc * D * 2; a.seq_b = a.head_b * s.Hkv;
+  a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Ls = s.Ls; a.Lr = s.Lr; a.max_seqs = s.max_seqs; a.nsplit = nsplit;
+  a.scale_log2 = s.scale * 1.4426950408889634f;
+  a.seq_len = seq_len; a.valid_topk = valid_topk; a.partials = partials; a.status = status;
+  const size_t smem = (size_t)NWARP * NSTAGE * STAGE_B + NWARP * NSTAGE * 8 + 1024;
+  static SmemLimit limit = {};
+  if (cudaError_t e = ensure_dyn_smem(decode_gqa_mma_kernel, smem, limit)) return e;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(nsplit, s.Hkv, n_active);
+  lc.blockDim = dim3(NT);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_mma_kernel, a, tk, tv);
+  count_launch();
+  if (e != cudaSuccess) return e;
+  return launch_decode_gqa_merge(partials, out, s.Hq, nsplit, slot_ids, n_active, seq_len, s.max_seqs, k_new != nullptr, st);
+}
+
+}  // namespace snap

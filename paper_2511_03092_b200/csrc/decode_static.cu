@@ -87,14 +87,21 @@ extern "C" int snap_decode_attn_static(const snap_config_t* cfg, const snap_layo
   if (src != SNAP_OK) return src;
 
   const bool gqa = decode_gqa_supported(cfg->dtype, s);
-  const int nsplit = gqa ? decode_gqa_nsplit(s, n_active, sms) : decode_generic_nsplit(s, n_active, sms);
+  const bool gqa_mma = gqa && decode_use_gqa_mma(cfg->dtype, s);
+  const int nsplit = gqa_mma ? decode_gqa_mma_nsplit(s, n_active, sms)
+                     : gqa   ? decode_gqa_nsplit(s, n_active, sms)
+                             : decode_generic_nsplit(s, n_active, sms);
   const size_t need = gqa ? decode_gqa_partial_floats(s, n_active, nsplit)
                           : decode_partial_floats(s, n_active, nsplit);
   if (need > kStaticFloats) return SNAP_ERR_STATIC_SCRATCH_EXCEEDED;
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e;
-  if (gqa)
+  if (gqa_mma)
+    e = launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
+                              v_cache_dev, seq_len_dev, valid_topk_dev, out_dev, scratch, nsplit,
+                              status_dev, st);
+  else if (gqa)
     e = launch_decode_gqa(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
                           v_cache_dev, seq_len_dev, valid_topk_dev, out_dev, scratch, nsplit,
                           status_dev, st);

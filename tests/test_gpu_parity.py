@@ -197,6 +197,15 @@ def test_group_sizes(hq, hkv):
     _run_compress_and_decode(wl, [wl.prompt_len[0], 50, 3], seed=13, steps=5)
 
 
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (16, 4), (20, 4), (32, 4)], ids=["g1", "g4", "g5", "g8"])
+def test_packed_fp32_decode_kernel_stays_selectable(hq, hkv, monkeypatch):
+    """The packed-FP32 decode kernel (the default before the tensor-core one) on the same cases."""
+    monkeypatch.setenv("SNAP_DECODE_GQA", "simt")
+    wl = SMALL_BF16.scaled(n_q_heads=hq, n_kv_heads=hkv)
+    _run_compress_and_decode(wl, [wl.prompt_len[0], 50, 3], seed=13, steps=5)
+    _run_compress_and_decode(wl, [300], seed=17, steps=2 * wl.l_recent + 5, check_ring_every=16)
+
+
 def test_many_sequences_ragged_decode():
     """More sequences than one launch chunk holds, lengths from empty-ish to several tiles."""
     wl = SMALL_BF16.scaled(topk=64, l_recent=32)
