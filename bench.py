@@ -375,6 +375,27 @@ def extras(hp, wl, dev):
         times.append(a.elapsed_time(b))
         src = dst
     out["concat_update_ms"] = statistics.median(times[2:])
+    del bufs
+    # (4) two new tokens per sequence and step (multi-token prediction, Section 5) in one pass over the cache
+    q_len = 2
+    mws = torch.empty(B.snap_decode_multi_workspace_bytes(hp.cfg, wl.batch, q_len), dtype=torch.uint8, device=dev)
+    mout = torch.empty(wl.batch, q_len, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device=dev)
+    stack = lambda key, r: torch.stack([hp.decode_in[(r + u) % DECODE_RING][key] for u in range(q_len)], dim=1).contiguous()
+    ins2 = [(stack("q", r), stack("k_new", r), stack("v_new", r)) for r in range(2)]
+    times = []
+    for r in range(8):
+        q2, k2, v2 = ins2[r % 2]
+        a, b = ev(), ev()
+        a.record()
+        B.snap_decode_attn_multi(hp.cfg, hp.layout, q2, k2, v2, hp.slots_dev, wl.batch, q_len, c.k_cache, c.v_cache,
+                                 c.seq_len, c.valid_topk, mout, mws, c.status)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    out["multi_token_q_len"] = q_len
+    out["multi_token_decode_ms"] = statistics.median(times[2:])
+    out["multi_token_tokens_per_s"] = wl.batch * q_len / (out["multi_token_decode_ms"] * 1e-3)
+    out["multi_token_status"] = int(c.status.item())
     out["concat_update_bytes"] = 2 * wl.batch * wl.n_kv_heads * hp.layout.slots * (wl.d_qk + wl.d_v) * 2
     out["ring_append_bytes"] = 2 * wl.batch * wl.n_kv_heads * (wl.d_qk + wl.d_v) * 2
     return out

@@ -165,6 +165,30 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout,
                      void* workspace_dev, size_t workspace_bytes,
                      uint32_t* status_dev, void* cuda_stream);
 
+/*
+ * A decode step with q_len new tokens per sequence (the multi-token prediction that the
+ * throughput evaluation of Section 5 assumes: several tokens per forward pass over the same
+ * cache).  Defined as q_len steps of
+ * snap_decode_attn: token u is appended as in Eq. 3, then query u attends over the cache as it
+ * is after tokens 0..u -- a window row that token u evicts is still seen by the queries before
+ * u and by none from u on.  One pass over the cache serves all q_len queries.
+ *   q_dev     [n_active][q_len][Hq][d_qk]
+ *   k_new_dev [n_active][q_len][Hkv][d_qk], v_new_dev [n_active][q_len][Hkv][d_v]   (required)
+ *   out_dev   [n_active][q_len][Hq][d_v];  seq_len_dev[slot] += q_len
+ * Built for bf16 layers with 128-wide heads and q_len * (Hq / Hkv) <= 8, 1 <= q_len <= Lr
+ * (SNAP_ERR_UNSUPPORTED / SNAP_ERR_INVALID_ARG otherwise).  Scratch:
+ * snap_decode_multi_workspace_bytes(cfg, n_active, q_len).
+ */
+int64_t snap_decode_multi_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t q_len);
+int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout,
+                           const void* q_dev, const void* k_new_dev, const void* v_new_dev,
+                           const int32_t* slot_ids_dev, int32_t n_active, int32_t q_len,
+                           void* k_cache_dev, void* v_cache_dev,
+                           int32_t* seq_len_dev, const int32_t* valid_topk_dev,
+                           void* out_dev,
+                           void* workspace_dev, size_t workspace_bytes,
+                           uint32_t* status_dev, void* cuda_stream);
+
 /* Size of the scratch array built into the library for snap_decode_attn_static. */
 #define SNAP_STATIC_SCRATCH_BYTES (8u << 20)
 

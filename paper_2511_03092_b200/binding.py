@@ -72,6 +72,10 @@ def lib() -> C.CDLL:
     L.snap_append_kv_concat.argtypes = [pcfg, play, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
     L.snap_decode_attn.restype = C.c_int
     L.snap_decode_attn.argtypes = [pcfg, play, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    L.snap_decode_multi_workspace_bytes.restype = i64
+    L.snap_decode_multi_workspace_bytes.argtypes = [pcfg, i32, i32]
+    L.snap_decode_attn_multi.restype = C.c_int
+    L.snap_decode_attn_multi.argtypes = [pcfg, play, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     L.snap_decode_attn_static.restype = C.c_int
     L.snap_decode_attn_static.argtypes = [pcfg, play, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
     _lib = L
@@ -79,7 +83,8 @@ def lib() -> C.CDLL:
 
 
 EXPORTS = ("snap_cache_layout", "snap_compress_workspace_bytes", "snap_decode_workspace_bytes",
-           "snap_compress", "snap_append_kv", "snap_append_kv_concat", "snap_decode_attn", "snap_decode_attn_static", "snap_status_string",
+           "snap_compress", "snap_append_kv", "snap_append_kv_concat", "snap_decode_attn",
+           "snap_decode_multi_workspace_bytes", "snap_decode_attn_multi", "snap_decode_attn_static", "snap_status_string",
            "snap_kernel_launch_count")
 
 
@@ -184,6 +189,25 @@ def snap_decode_attn(cfg: SnapConfig, layout: SnapLayout, q, k_new, v_new, slot_
                                   _ptr(slot_ids_dev), int(n_active), _ptr(k_cache), _ptr(v_cache),
                                   _ptr(seq_len), _ptr(valid_topk), _ptr(out), _ptr(workspace), ws_bytes,
                                   _ptr(status), _stream(stream)), "snap_decode_attn")
+
+
+def snap_decode_multi_workspace_bytes(cfg: SnapConfig, n_active: int, q_len: int) -> int:
+    n = lib().snap_decode_multi_workspace_bytes(C.byref(cfg), int(n_active), int(q_len))
+    if n < 0:
+        raise SnapError(int(n), "snap_decode_multi_workspace_bytes")
+    return int(n)
+
+
+def snap_decode_attn_multi(cfg: SnapConfig, layout: SnapLayout, q, k_new, v_new, slot_ids_dev, n_active: int,
+                           q_len: int, k_cache, v_cache, seq_len, valid_topk, out, workspace, status=None,
+                           stream=None) -> None:
+    """q_len new tokens per sequence in one pass over the cache (q [n][q_len][Hq][d], out alike)."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().snap_decode_attn_multi(C.byref(cfg), C.byref(layout), _ptr(q), _ptr(k_new), _ptr(v_new),
+                                        _ptr(slot_ids_dev), int(n_active), int(q_len), _ptr(k_cache),
+                                        _ptr(v_cache), _ptr(seq_len), _ptr(valid_topk), _ptr(out),
+                                        _ptr(workspace), ws_bytes, _ptr(status), _stream(stream)),
+           "snap_decode_attn_multi")
 
 
 def snap_decode_attn_static(cfg: SnapConfig, layout: SnapLayout, q, k_new, v_new, slot_ids_dev, n_active: int,

@@ -395,4 +395,52 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
   return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
 }
 
+// Several query tokens per sequence in one step: only the tensor-core kernel for 128-wide bf16
+// heads takes them (the tokens' heads share the N side of its MMAs, so q_len * group <= 8).
+static int multi_supported(const snap_config_t* cfg, const Shape& s, int q_len) {
+  if (q_len < 1 || q_len > s.Lr) return SNAP_ERR_INVALID_ARG;
+  if (!decode_gqa_supported(cfg->dtype, s) || !decode_use_gqa_mma(cfg->dtype, s) || q_len * s.g > 8)
+    return SNAP_ERR_UNSUPPORTED;
+  return SNAP_OK;
+}
+
+int64_t snap_decode_multi_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t q_len) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (n_active < 0) return SNAP_ERR_INVALID_ARG;
+  const Shape s = make_shape(cfg);
+  const int ms = multi_supported(cfg, s, q_len);
+  if (ms != SNAP_OK) return ms;
+  const int nsplit = decode_gqa_mma_nsplit(s, n_active > 0 ? n_active : 1, sm_count());
+  return (int64_t)(decode_gqa_partial_floats(s, n_active * q_len, nsplit) * sizeof(float) + 256);
+}
+
+int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,
+                           const void* k_new_dev, const void* v_new_dev, const int32_t* slot_ids_dev,
+                           int32_t n_active, int32_t q_len, void* k_cache_dev, void* v_cache_dev,
+                           int32_t* seq_len_dev, const int32_t* valid_topk_dev, void* out_dev,
+                           void* workspace_dev, size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (!layout) return SNAP_ERR_NULL_POINTER;
+  if (n_active < 0) return SNAP_ERR_INVALID_ARG;
+  const Shape s = make_shape(cfg);
+  const int ms = multi_supported(cfg, s, q_len);
+  if (ms != SNAP_OK) return ms;
+  if (n_active == 0) return SNAP_OK;
+  if (!q_dev || !k_new_dev || !v_new_dev || !slot_ids_dev || !k_cache_dev || !v_cache_dev || !seq_len_dev ||
+      !valid_topk_dev || !out_dev || !workspace_dev)
+    return SNAP_ERR_NULL_POINTER;
+  if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
+  const int64_t need = snap_decode_multi_workspace_bytes(cfg, n_active, q_len);
+  if (need < 0) return (int)need;
+  if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
+  const int nsplit = decode_gqa_mma_nsplit(s, n_active, sm_count());
+  const cudaError_t e = launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
+                                              v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
+                                              static_cast<float*>(workspace_dev), nsplit, status_dev,
+                                              static_cast<cudaStream_t>(cuda_stream), q_len);
+  return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+}
+
 }  // extern "C"

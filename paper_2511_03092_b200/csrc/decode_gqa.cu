@@ -392,11 +392,13 @@ __global__ void __launch_bounds__(NT, (G > 4 ? 2 : 3)) decode_gqa_kernel(const F
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
-// Merge the splits of one (sequence, query head); maxima are in the log2 domain.
+// Merge the splits of one (sequence, query token, query head); maxima are in the log2 domain.
+// With q_len query tokens per sequence the rows of `partials` and `out` are indexed by
+// sequence * q_len + token, and every token's block advances the sequence length by one.
 __global__ void __launch_bounds__(D) decode_gqa_merge_kernel(const float* __restrict__ partials,
                                                              __nv_bfloat16* __restrict__ out, int Hq,
                                                              int nsplit, const int* __restrict__ slot_ids,
-                                                             int* seq_len, int max_seqs, int bump) {
+                                                             int* seq_len, int max_seqs, int bump, int q_len) {
   const int h = blockIdx.x, i = blockIdx.y, t = threadIdx.x;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const float* p = partials + ((long long)i * Hq + h) * nsplit * PS;
@@ -414,8 +416,8 @@ __global__ void __launch_bounds__(D) decode_gqa_merge_kernel(const float* __rest
   }
   out[((long long)i * Hq + h) * D + t] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
   if (bump && h == 0 && t == 0) {
-    const int slot = slot_ids[i];
-    if (slot >= 0 && slot < max_seqs) seq_len[slot] += 1;
+    const int slot = slot_ids[i / q_len];
+    if (slot >= 0 && slot < max_seqs) atomicAdd(&seq_len[slot], 1);
   }
 }
 
@@ -447,27 +449,28 @@ cudaError_t launch_g(const FastArgs& a, int n_active, __nv_bfloat16* out, int* s
   const float* parts = a.partials;
   const int* slots = a.slot_ids;
   cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_merge_kernel, parts, out, a.Hq, a.nsplit, slots, seq_len,
-                                     a.max_seqs, bump);
+                                     a.max_seqs, bump, 1);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
 
-// The split merge as a programmatic dependent launch (shared with the tensor-core kernel).
+// The split merge as a programmatic dependent launch (shared with the tensor-core kernel);
+// n_rows = sequences * q_len.
 cudaError_t launch_decode_gqa_merge(const float* partials, void* out, int Hq, int nsplit, const int* slot_ids,
-                                    int n_active, int* seq_len, int max_seqs, int bump, cudaStream_t st) {
+                                    int n_rows, int q_len, int* seq_len, int max_seqs, int bump, cudaStream_t st) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(Hq, n_active);
+  lc.gridDim = dim3(Hq, n_rows);
   lc.blockDim = dim3(D);
   lc.stream = st;
   lc.attrs = attr;
   lc.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_merge_kernel, partials, static_cast<__nv_bfloat16*>(out), Hq, nsplit,
-                                     slot_ids, seq_len, max_seqs, bump);
+                                     slot_ids, seq_len, max_seqs, bump, q_len);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }

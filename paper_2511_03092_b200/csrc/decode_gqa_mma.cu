@@ -41,9 +41,10 @@ struct MmaArgs {
   char* kc; char* vc;
   long long seq_b, head_b;
   int Hq, Hkv, g, Ls, Lr, max_seqs, nsplit;
+  int T;                                        // query tokens per sequence in this step (T * g <= 8)
   float scale_log2;
   const int* seq_len; const int* valid_topk;
-  float* partials;                              // [n_active][Hq][nsplit][PS]
+  float* partials;                              // [n_active][T][Hq][nsplit][PS]
   uint32_t* status;
 };
 
@@ -113,17 +114,26 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int slot = a.slot_ids[i];
   const bool bad = slot < 0 || slot >= a.max_seqs;
-  const int Lsr = a.Ls + a.Lr;
-  int n_low = 0, n_top = 0, new_slot = -1;
+  const int Lsr = a.Ls + a.Lr, TQ = a.T;
+  // One new token (the usual step): its row is patched into the staged tile, so it counts as valid.
+  // Several new tokens: query t must see the cache as it is after tokens 0..t, so the old rows
+  // are attended as they are (the rows that tokens evict masked per query) and the new rows
+  // form a tile of their own; n_low_st then only extends the tile list to the slots they fill.
+  int L0 = 0, n_low = 0, n_low_st = 0, n_top = 0, new_slot = -1;
   if (!bad) {
-    const int t = a.seq_len[slot];
-    n_low = min(t + (a.k_new ? 1 : 0), Lsr);
+    L0 = a.seq_len[slot];
     n_top = a.valid_topk[slot];
-    if (a.k_new) new_slot = ring_slot(t, a.Ls, a.Lr);
+    if (TQ == 1) {
+      n_low = n_low_st = min(L0 + (a.k_new ? 1 : 0), Lsr);
+      if (a.k_new) new_slot = ring_slot(L0, a.Ls, a.Lr);
+    } else {
+      n_low = min(L0, Lsr);
+      n_low_st = min(L0 + TQ, Lsr);
+    }
   } else if (tid == 0 && sp == 0 && kvh == 0 && a.status) {
     atomicOr(a.status, SNAP_DEV_BAD_SLOT);
   }
-  const int nA = (n_low + WT - 1) / WT, ntiles = nA + (n_top + WT - 1) / WT;
+  const int nA = (n_low_st + WT - 1) / WT, ntiles = nA + (n_top + WT - 1) / WT;
   const int t_begin = (int)((long long)ntiles * sp / a.nsplit);
   const int t_end = (int)((long long)ntiles * (sp + 1) / a.nsplit);
   // this warp's tiles: t_begin + w, t_begin + w + NWARP, ...
@@ -145,60 +155,51 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
 
   char* kc = a.kc + slot * a.seq_b + kvh * a.head_b;
   char* vc = a.vc + slot * a.seq_b + kvh * a.head_b;
-  const __nv_bfloat16* kn = a.k_new ? a.k_new + ((long long)i * a.Hkv + kvh) * D : nullptr;
-  const __nv_bfloat16* vn = a.v_new ? a.v_new + ((long long)i * a.Hkv + kvh) * D : nullptr;
+  // new rows of this KV head: token u at kn + u * Hkv * D
+  const __nv_bfloat16* kn = a.k_new ? a.k_new + ((long long)i * TQ * a.Hkv + kvh) * D : nullptr;
+  const __nv_bfloat16* vn = a.v_new ? a.v_new + ((long long)i * TQ * a.Hkv + kvh) * D : nullptr;
+  const long long new_stride = (long long)a.Hkv * D;
 
-  // B fragments of Q^T for the eight 16-dim steps: head gq (zero beyond the group), dims 16 ks + 2 tq (+8)
+  // Column n of the MMAs is query token n / g, head n % g of the group (zero beyond T * g).
+  // B fragments of Q^T for the eight 16-dim steps: column gq, dims 16 ks + 2 tq (+8)
+  const int ncols = TQ * a.g;
   uint32_t qb[8][2];
   {
-    const __nv_bfloat16* qp = a.q + ((long long)i * a.Hq + (long long)kvh * a.g + gq) * D + 2 * tq;
+    const int tcol = gq / a.g, hcol = gq - tcol * a.g;
+    const __nv_bfloat16* qp = a.q + (((long long)i * TQ + tcol) * a.Hq + (long long)kvh * a.g + hcol) * D + 2 * tq;
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
-      qb[ks][0] = gq < a.g ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks) : 0u;
-      qb[ks][1] = gq < a.g ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks + 8) : 0u;
+      qb[ks][0] = gq < ncols ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks) : 0u;
+      qb[ks][1] = gq < ncols ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks + 8) : 0u;
     }
   }
-  float oacc[8][4];                              // O^T: dims 16 db + gq (+8), heads 2 tq (+1)
+  const int tc0 = (2 * tq) / a.g, tc1 = (2 * tq + 1) / a.g;     // query tokens of this thread's two columns
+  float oacc[8][4];                              // O^T: dims 16 db + gq (+8), columns 2 tq (+1)
 #pragma unroll
   for (int db = 0; db < 8; ++db)
 #pragma unroll
     for (int e = 0; e < 4; ++e) oacc[db][e] = 0.f;
-  float m_ref[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};   // heads 2 tq, 2 tq + 1
+  float m_ref[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};   // columns 2 tq, 2 tq + 1
   bool timed_out = false;
 
   // ldmatrix lane roles: K (plain): row (lane & 7) + 8 * bit3, chunk + bit4; V (transposed): row (lane & 7) + 8 * bit4, chunk + bit3
   const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_cadd = lane >> 4;
   const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8, v_cadd = (lane >> 3) & 1;
 
-  for (int n = 0; n < T; ++n) {
-    const int s = n % NSTAGE;
-    const unsigned parity = (unsigned)(n / NSTAGE) & 1u;
-    const bool landed = mbar_wait_bounded(bar0 + 8 * s, parity);
-    if (__any_sync(0xffffffffu, !landed)) { timed_out = true; break; }
-    const TileRows tr = tile_rows(t_begin + w + n * NWARP, nA, n_low, Lsr, n_top);
-    const int nrows = tr.row_end - tr.row0;                    // >= 1; rows at or past it are masked
-    const uint32_t sK = stage0 + s * STAGE_B, sV = sK + TENS_B;
-    if (new_slot >= tr.row0 && new_slot < tr.row0 + WT && new_slot < tr.row_end) {
-      // the new token's slot is in this tile: store the row to the cache and patch the staged copy
-      const int r = new_slot - tr.row0, c = lane & 15;
-      const uint4 val = reinterpret_cast<const uint4*>(lane < 16 ? kn : vn)[c];
-      reinterpret_cast<uint4*>((lane < 16 ? kc : vc) + (long long)new_slot * (D * 2))[c] = val;
-      unsigned char* sp_ = wstages + s * STAGE_B + (lane < 16 ? 0 : TENS_B) + (c >> 3) * SLAB_B + swz(r, c & 7);
-      *reinterpret_cast<uint4*>(sp_) = val;
-      __syncwarp();
-    }
-
+  // One staged tile: okN says whether this thread's value N (rows gq, gq, gq + 8, gq + 8 x columns
+  // 2 tq, 2 tq + 1, 2 tq, 2 tq + 1) takes part.
+  auto process = [&](uint32_t sK, uint32_t sV, bool ok0, bool ok1, bool ok2, bool ok3) {
     // ---- S^T = K tile . Q^T ----
-    float sacc[4] = {0.f, 0.f, 0.f, 0.f};       // rows gq, gq + 8; heads 2 tq, 2 tq + 1
+    float sacc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       uint32_t af[4];
       ldsm4(sK + (ks >> 2) * SLAB_B + swz(k_row, (ks & 3) * 2 + k_cadd), af);
       mma16816(sacc, af, qb[ks][0], qb[ks][1]);
     }
-    float v0 = gq < nrows ? sacc[0] * a.scale_log2 : -INFINITY, v1 = gq < nrows ? sacc[1] * a.scale_log2 : -INFINITY;
-    float v2 = gq + 8 < nrows ? sacc[2] * a.scale_log2 : -INFINITY, v3 = gq + 8 < nrows ? sacc[3] * a.scale_log2 : -INFINITY;
-    // Lazy reference per head: refreshed (accumulators rescaled) only when a warp vote sees a
+    const float v0 = ok0 ? sacc[0] * a.scale_log2 : -INFINITY, v1 = ok1 ? sacc[1] * a.scale_log2 : -INFINITY;
+    const float v2 = ok2 ? sacc[2] * a.scale_log2 : -INFINITY, v3 = ok3 ? sacc[3] * a.scale_log2 : -INFINITY;
+    // Lazy reference per column: refreshed (accumulators rescaled) only when a warp vote sees a
     // logit 8 above it; the column maxima are then reduced over the lanes that share tq.
     if (__any_sync(0xffffffffu, fmaxf(v0, v2) > m_ref[0] + 8.f || fmaxf(v1, v3) > m_ref[1] + 8.f)) {
       float mx0 = fmaxf(v0, v2), mx1 = fmaxf(v1, v3);
@@ -218,9 +219,8 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     const float p0 = fast_exp2(v0 - r0), p1 = fast_exp2(v1 - r1), p2 = fast_exp2(v2 - r0), p3 = fast_exp2(v3 - r1);
     l_part[0] += p0 + p2;
     l_part[1] += p1 + p3;
-    // P^T as the B operand: rows 2 tq (+1) and 2 tq + 8 (+9) of head gq
+    // P^T as the B operand: rows 2 tq (+1) and 2 tq + 8 (+9) of column gq
     const uint32_t pb0 = movmatrix_t(pack_bf16(p0, p1)), pb1 = movmatrix_t(pack_bf16(p2, p3));
-
     // ---- O^T += V tile^T . P^T ----
 #pragma unroll
     for (int db = 0; db < 8; ++db) {
@@ -228,12 +228,61 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
       ldsm4t(sV + (db >> 2) * SLAB_B + swz(v_row, (db & 3) * 2 + v_cadd), af);
       mma16816(oacc[db], af, pb0, pb1);
     }
+  };
+
+  for (int n = 0; n < T; ++n) {
+    const int s = n % NSTAGE;
+    const unsigned parity = (unsigned)(n / NSTAGE) & 1u;
+    const bool landed = mbar_wait_bounded(bar0 + 8 * s, parity);
+    if (__any_sync(0xffffffffu, !landed)) { timed_out = true; break; }
+    const int j = t_begin + w + n * NWARP;
+    const TileRows tr = tile_rows(j, nA, n_low, Lsr, n_top);
+    const int nrows = tr.row_end - tr.row0;                    // rows at or past it are masked (may be <= 0)
+    const uint32_t sK = stage0 + s * STAGE_B, sV = sK + TENS_B;
+    bool ok0 = gq < nrows, ok1 = ok0, ok2 = gq + 8 < nrows, ok3 = ok2;
+    if (TQ == 1) {
+      if (new_slot >= tr.row0 && new_slot < tr.row0 + WT && new_slot < tr.row_end) {
+        // the new token's slot is in this tile: store the row to the cache and patch the staged copy
+        const int r = new_slot - tr.row0, c = lane & 15;
+        const uint4 val = reinterpret_cast<const uint4*>(lane < 16 ? kn : vn)[c];
+        reinterpret_cast<uint4*>((lane < 16 ? kc : vc) + (long long)new_slot * (D * 2))[c] = val;
+        unsigned char* sp_ = wstages + s * STAGE_B + (lane < 16 ? 0 : TENS_B) + (c >> 3) * SLAB_B + swz(r, c & 7);
+        *reinterpret_cast<uint4*>(sp_) = val;
+        __syncwarp();
+      }
+    } else if (j < nA) {
+      // new tokens whose slot lies in this tile: the old row (if the token evicts one) stays visible to
+      // the queries before that token only; the new row goes to the cache now that the old one is staged
+      for (int u = 0; u < TQ; ++u) {
+        const int ru = ring_slot(L0 + u, a.Ls, a.Lr);
+        if (ru < tr.row0 || ru >= tr.row0 + WT) continue;
+        const int r = ru - tr.row0, c = lane & 15;
+        if (gq == r) { ok0 = ok0 && tc0 < u; ok1 = ok1 && tc1 < u; }
+        if (gq + 8 == r) { ok2 = ok2 && tc0 < u; ok3 = ok3 && tc1 < u; }
+        const uint4 val = reinterpret_cast<const uint4*>((lane < 16 ? kn : vn) + u * new_stride)[c];
+        reinterpret_cast<uint4*>((lane < 16 ? kc : vc) + (long long)ru * (D * 2))[c] = val;
+      }
+    }
+    process(sK, sV, ok0, ok1, ok2, ok3);
     __syncwarp();
     if (lane == 0 && n + NSTAGE < T) issue(n + NSTAGE);
   }
   if (timed_out) {
     if (a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
     for (int s = 0; s < NSTAGE; ++s) (void)mbar_wait_bounded(bar0 + 8 * s, 0u);
+  }
+  if (TQ > 1 && sp == 0 && w == 0 && !bad && !timed_out) {
+    // the new tokens as a tile of their own (this warp's pipeline has drained): row u is token u,
+    // visible to the queries from token u on; rows past the last token are zero and masked
+    for (int e = lane; e < 2 * WT * 16; e += 32) {
+      const int tens = e / (WT * 16), r = (e / 16) % WT, c = e % 16;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if (r < TQ) val = reinterpret_cast<const uint4*>((tens ? vn : kn) + r * new_stride)[c];
+      *reinterpret_cast<uint4*>(wstages + tens * TENS_B + (c >> 3) * SLAB_B + swz(r, c & 7)) = val;
+    }
+    __syncwarp();
+    process(stage0, stage0 + TENS_B, gq < TQ && gq <= tc0, gq < TQ && gq <= tc1, false, false);
+    __syncwarp();
   }
 
   // ---- per-warp result -> this warp's stage memory, then merge the warps ----
@@ -258,10 +307,9 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     wacc[(2 * tq + 1) * D + 16 * db + gq + 8] = oacc[db][3];
   }
   __syncthreads();
-  float* part_out = a.partials + (((long long)i * a.Hq + (long long)kvh * a.g) * a.nsplit + sp) * PS;
   constexpr int WSTRIDE = NSTAGE * STAGE_B / 4;            // floats between two warps' regions
   const float* base = reinterpret_cast<const float*>(smem_raw);
-  for (int h = 0; h < a.g; ++h) {
+  for (int h = 0; h < ncols; ++h) {
     float M = -INFINITY;
 #pragma unroll
     for (int ww = 0; ww < NWARP; ++ww) M = fmaxf(M, base[ww * WSTRIDE + h]);
@@ -273,7 +321,8 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
       L += base[ww * WSTRIDE + GP + h] * f;
       O += base[ww * WSTRIDE + 2 * GP + h * D + tid] * f;
     }
-    float* ph = part_out + (long long)h * a.nsplit * PS;
+    const int tcol = h / a.g, hcol = h - tcol * a.g;
+    float* ph = a.partials + ((((long long)i * TQ + tcol) * a.Hq + (long long)kvh * a.g + hcol) * a.nsplit + sp) * PS;
     if (tid == 0) { ph[0] = M; ph[1] = L; }
     ph[2 + tid] = O;
   }
@@ -290,8 +339,9 @@ bool decode_gqa_mma_supported(int dtype, const Shape& s) {
 cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_new, const void* v_new,
                                   const int* slot_ids, int n_active, void* k_cache, void* v_cache,
                                   int* seq_len, const int* valid_topk, void* out, float* partials,
-                                  int nsplit, uint32_t* status, cudaStream_t st) {
+                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len) {
   if (n_active == 0) return cudaSuccess;
+  if (q_len < 1 || q_len * s.g > GP || (q_len > 1 && (!k_new || q_len > s.Lr))) return cudaErrorInvalidValue;
   umma::EncodeTiledFn enc = umma::encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
   CUtensorMap tk, tv;
@@ -311,6 +361,7 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   a.kc = static_cast<char*>(k_cache); a.vc = static_cast<char*>(v_cache);
   a.head_b = (long long)s.Sc * D * 2; a.seq_b = a.head_b * s.Hkv;
   a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Ls = s.Ls; a.Lr = s.Lr; a.max_seqs = s.max_seqs; a.nsplit = nsplit;
+  a.T = q_len;
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.seq_len = seq_len; a.valid_topk = valid_topk; a.partials = partials; a.status = status;
   const size_t smem = (size_t)NWARP * NSTAGE * STAGE_B + NWARP * NSTAGE * 8 + 1024;
@@ -329,7 +380,8 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_mma_kernel, a, tk, tv);
   count_launch();
   if (e != cudaSuccess) return e;
-  return launch_decode_gqa_merge(partials, out, s.Hq, nsplit, slot_ids, n_active, seq_len, s.max_seqs, k_new != nullptr, st);
+  return launch_decode_gqa_merge(partials, out, s.Hq, nsplit, slot_ids, n_active * q_len, q_len, seq_len, s.max_seqs,
+                                 k_new != nullptr, st);
 }
 
 }  // namespace snap

@@ -109,7 +109,7 @@ cudaError_t launch_decode_gqa(const Shape& s, const void* q, const void* k_new, 
                               int nsplit, uint32_t* status, cudaStream_t st);
 
 cudaError_t launch_decode_gqa_merge(const float* partials, void* out, int Hq, int nsplit, const int* slot_ids,
-                                    int n_active, int* seq_len, int max_seqs, int bump, cudaStream_t st);
+                                    int n_rows, int q_len, int* seq_len, int max_seqs, int bump, cudaStream_t st);
 // the same on tensor cores (mma.sync, the group's heads on the N side): cost independent of the group size
 bool decode_gqa_mma_supported(int dtype, const Shape& s);
 bool decode_use_gqa_mma(int dtype, const Shape& s);     // the choice between the two, shared by all entry points
@@ -117,7 +117,7 @@ int decode_gqa_mma_nsplit(const Shape& s, int n_active, int sm_count);
 cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_new, const void* v_new,
                                   const int* slot_ids, int n_active, void* k_cache, void* v_cache,
                                   int* seq_len, const int* valid_topk, void* out, float* partials,
-                                  int nsplit, uint32_t* status, cudaStream_t st);
+                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len = 1);
 
 // latent attention (one 576-wide KV row shared by all heads, V = its first 512 dims): mma.sync kernel
 bool decode_mla_supported(int dtype, const Shape& s);

@@ -375,3 +375,57 @@ def test_decode_step_replayed_from_a_cuda_graph(wl):
         assert torch.equal(a.cache.seq_len, b.cache.seq_len)
     assert a.status() == 0 and b.status() == 0
     assert [int(x) for x in b.cache.seq_len.cpu()] == [L + 6 for L in lengths]
+
+
+def _run_multi(wl, lengths, q_len, steps, seed):
+    """Multi-token steps through snap_decode_attn_multi against q_len oracle steps each."""
+    n = len(lengths)
+    layer = H.GpuLayer(wl, max_seqs=n)
+    prompts = [synth.make_prompt(wl, L, seed + i) for i, L in enumerate(lengths)]
+    layer.compress(prompts, list(range(n)))
+    seqs = [H.oracle_compress(wl, p) for p in prompts]
+    slots_dev = torch.arange(n, dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.snap_decode_multi_workspace_bytes(layer.cfg, n, q_len), dtype=torch.uint8, device="cuda")
+    c = layer.cache
+    for step in range(steps):
+        ds = [synth.make_decode_inputs(wl, n, seed, step * q_len + u) for u in range(q_len)]
+        q = torch.stack([d["q"] for d in ds], dim=1).contiguous().cuda()            # [n][q_len][Hq][d]
+        kn = torch.stack([d["k_new"] for d in ds], dim=1).contiguous().cuda()
+        vn = torch.stack([d["v_new"] for d in ds], dim=1).contiguous().cuda()
+        out = torch.empty(n, q_len, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device="cuda")
+        B.snap_decode_attn_multi(layer.cfg, layer.layout, q, kn, vn, slots_dev, n, q_len, c.k_cache, c.v_cache,
+                                 c.seq_len, c.valid_topk, out, ws, c.status)
+        for i in range(n):
+            for u in range(q_len):
+                ref = orc.decode_step(seqs[i], synth.to_f64(ds[u]["q"][i]), synth.to_f64(ds[u]["k_new"][i]),
+                                      synth.to_f64(ds[u]["v_new"][i]))
+                H.check_output(out[i, u], ref, wl, f"step {step} seq {i} token {u}")
+    assert layer.status() == 0
+    for i in range(n):
+        assert int(c.seq_len[i]) == seqs[i].n_tokens
+        H.check_cache_image(layer, seqs[i], i, wl)
+
+
+@pytest.mark.parametrize("hq,hkv,q_len", [(16, 4, 2), (8, 4, 4), (8, 4, 3), (4, 4, 8), (32, 4, 1)],
+                         ids=["g4x2", "g2x4", "g2x3", "g1x8", "g8x1"])
+def test_multi_token_decode_steps(hq, hkv, q_len):
+    """q_len tokens per step: each query sees the cache as it is after its own token -- window rows
+    evicted by later tokens of the step included, those evicted by earlier ones not.  Sequences that
+    are still filling the sinks, filling the window, and wrapping the ring."""
+    wl = SMALL_BF16.scaled(n_q_heads=hq, n_kv_heads=hkv)
+    _run_multi(wl, [1, 3, 45, 50, 51, 52, 300, wl.prompt_len[0]], q_len, steps=max(4, 60 // q_len), seed=83)
+
+
+def test_multi_token_decode_rejects_what_it_cannot_do():
+    wl = SMALL_BF16                                   # 4 heads per KV head
+    layer = H.GpuLayer(wl, 1)
+    with pytest.raises(B.SnapError) as e:
+        B.snap_decode_multi_workspace_bytes(layer.cfg, 1, 3)          # 3 tokens x 4 heads > 8 columns
+    assert e.value.code == -2
+    with pytest.raises(B.SnapError) as e:
+        B.snap_decode_multi_workspace_bytes(layer.cfg, 1, 0)
+    assert e.value.code == -1
+    f32 = H.GpuLayer(SMALL_F32, 1)
+    with pytest.raises(B.SnapError) as e:
+        B.snap_decode_multi_workspace_bytes(f32.cfg, 1, 2)            # no fp32 kernel for it
+    assert e.value.code == -2
