@@ -240,6 +240,16 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     const int nrows = tr.row_end - tr.row0;                    // rows at or past it are masked (may be <= 0)
     const uint32_t sK = stage0 + s * STAGE_B, sV = sK + TENS_B;
     bool ok0 = gq < nrows, ok1 = ok0, ok2 = gq + 8 < nrows, ok3 = ok2;
+    if (nrows < WT) {
+      // ragged tile: rows past the end may hold anything (memory the caller never wrote), and a
+      // zero probability does not silence a NaN in V: clear those V rows
+      const int first = max(nrows, 0);
+      for (int e = lane; e < (WT - first) * 16; e += 32) {
+        const int r = first + e / 16, c = e % 16;
+        *reinterpret_cast<uint4*>(wstages + s * STAGE_B + TENS_B + (c >> 3) * SLAB_B + swz(r, c & 7)) = make_uint4(0, 0, 0, 0);
+      }
+      __syncwarp();
+    }
     if (TQ == 1) {
       if (new_slot >= tr.row0 && new_slot < tr.row0 + WT && new_slot < tr.row_end) {
         // the new token's slot is in this tile: store the row to the cache and patch the staged copy

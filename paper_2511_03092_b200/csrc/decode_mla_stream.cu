@@ -235,6 +235,8 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
         if (!ok) break;
         fence_after();
         const uint32_t pa = tmem_base + COL_S + b * TR;       // P(it) lies over the first 64 columns of S(it)
+        const TileRows ptr_ = tile_rows(g0 + it, nA, n_low, Lsr, n_top);
+        const int tile_nrows = ptr_.row_end - ptr_.row0;
 #pragma unroll 1
         for (int c = 0; c < NVCH; ++c) {                      // O += P(it) V(it), one 32-row value chunk per stage
           const int s = q % NSTG;
@@ -242,6 +244,17 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
           if (!ok) break;
           fence_after();
           const uint32_t vst = smem_u32(Rs) + s * STAGE_B;
+          if (tile_nrows < (c + 1) * VROWS) {
+            // ragged chunk: rows past the end may hold anything (memory the caller never wrote), and a
+            // zero probability does not silence a NaN in V: clear them before the tensor core reads
+            const int first = max(tile_nrows - c * VROWS, 0);
+            for (int e = lane; e < (VROWS - first) * (DVH / 64) * 8; e += 32) {
+              const int r = first + e / ((DVH / 64) * 8), j = (e / 8) % (DVH / 64), ch = e % 8;
+              *reinterpret_cast<uint4*>(Rs + s * STAGE_B + j * VSUB_B + r * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+          }
 #pragma unroll
           for (int ks = 0; ks < VROWS / 16; ++ks)
             mma_ts_pred(tmem_base + COL_O, pa + 8 * (c * (VROWS / 16) + ks), smem_desc_mn(vst + ks * 16 * 128, VSUB_B),

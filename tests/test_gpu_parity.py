@@ -429,3 +429,32 @@ def test_multi_token_decode_rejects_what_it_cannot_do():
     with pytest.raises(B.SnapError) as e:
         B.snap_decode_multi_workspace_bytes(f32.cfg, 1, 2)            # no fp32 kernel for it
     assert e.value.code == -2
+
+
+@pytest.mark.parametrize("wl", [SMALL_BF16, LATENT_128, SMALL_F32], ids=lambda w: w.name)
+def test_decode_from_empty_slots_in_memory_full_of_nans(wl):
+    """Sequences built by decode steps alone, in cache memory that was never cleared: rows past
+    the end of a ragged tile must not leak into the result (0 x NaN is NaN)."""
+    n = 2
+    layer = H.GpuLayer(wl, n)
+    c = layer.cache
+    c.k_cache.fill_(float("nan"))
+    if c.v_cache is not None:
+        c.v_cache.fill_(float("nan"))
+    ocfg = H.oracle_config(wl)
+    seqs = []
+    for _ in range(n):
+        seq = orc.OracleSequence(ocfg)
+        seq.topk_pos = [np.zeros(0, dtype=np.int64) for _ in range(wl.n_kv_heads)]
+        seqs.append(seq)
+    slots_dev = torch.arange(n, dtype=torch.int32, device="cuda")
+    for step in range(wl.l_sink + wl.l_recent + 9):
+        d = synth.make_decode_inputs(wl, n, 91, step)
+        vn = None if wl.v_aliases_k else d["v_new"].cuda()
+        out = layer.decode(d["q"].cuda(), d["k_new"].cuda(), vn, slots_dev)
+        for i in range(n):
+            ref = orc.decode_step(seqs[i], synth.to_f64(d["q"][i]), synth.to_f64(d["k_new"][i]),
+                                  None if wl.v_aliases_k else synth.to_f64(d["v_new"][i]))
+            if step < 20 or step % 7 == 0:
+                H.check_output(out[i], ref, wl, f"step {step} seq {i}")
+    assert layer.status() == 0
