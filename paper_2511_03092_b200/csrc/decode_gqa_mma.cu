@@ -1,21 +1,28 @@
 // Decode attention over the compressed cache (Section 3.3) for bf16 layers with 128-wide heads
-// and 5 to 8 query heads per KV head, on tensor cores.
+// and 1 to 8 query heads per KV head, on tensor cores -- the HBM-bound kernel of the decode step.
 //
-// From five heads per KV head on, the multiply-adds of the packed-FP32 kernel outrun the FP32
-// pipe before HBM is saturated.  Here the same split-K scheme (grid = splits x KV heads x
-// sequences, warp-private pipelines of 16-row tiles, one partial result per split, the same
-// merge kernel) does its arithmetic with mma.sync.m16n8k16, the group's heads on the N side:
-//     S^T[16 rows x 8 heads]   = K tile [16 x 128] . Q^T                  (8 MMAs)
-//     O^T[128 dims x 8 heads] += V tile^T [128 x 16] . P^T [16 x 8 heads] (8 MMAs)
-// so the cost per cache row no longer depends on the group size.  Tiles arrive through TMA
-// tensor loads with the 128-byte swizzle (two 64-dim slabs per tensor), which makes the
-// ldmatrix reads conflict-free; V is read with ldmatrix.trans; the probabilities leave the
-// S^T accumulators for the B operand of the second product through movmatrix (an 8x8
-// transpose across the warp).  Online softmax is per head in the log2 domain with a lazily
-// refreshed reference; row sums are kept per thread and reduced once at the end.
+// Split-K flash decoding: grid = splits x KV heads x sequences, warp-private pipelines of 16-row
+// tiles, one partial result per split, a merge kernel.  The arithmetic is mma.sync.m16n8k16
+// with the group's heads on the N side:
+//     S^T[16 rows x 8 columns]   = K tile [16 x 128] . Q^T                    (8 MMAs)
+//     O^T[128 dims x 8 columns] += V tile^T [128 x 16] . P^T [16 x 8 columns] (8 MMAs)
+// so the cost per cache row does not depend on the group size (with packed FP32 arithmetic the
+// multiply-adds outrun the FP32 pipe from five heads per KV head on, and cost issue slots
+// before that).  Tiles arrive through TMA tensor loads with the 128-byte swizzle (two 64-dim
+// slabs per tensor, per-warp mbarriers), which makes the ldmatrix reads conflict-free; V is read
+// with ldmatrix.trans; the probabilities leave the S^T accumulators for the B operand of the
+// second product through movmatrix (an 8x8 transpose across the warp).  Online softmax is per
+// column in the log2 domain with a lazily refreshed reference; row sums are kept per thread
+// and reduced once at the end.
 //
-// Fused append (Eq. 3): as in the packed-FP32 kernel, the warp that stages the new token's
-// slot stores the row to the cache and patches its staged copy.
+// Fused append (Eq. 3): the warp that stages the new token's slot stores the row to the cache
+// and patches its staged copy.
+//
+// Several new tokens per step (multi-token prediction): the eight columns are then (token,
+// head) pairs, T x g <= 8.  Query t must see the cache as it is after tokens 0..t: the old rows
+// are attended as staged, a window row that token u evicts is masked for the queries from u
+// on, the new rows form one extra tile with a causal mask, and each new row is written to the
+// cache by the warp that has just staged the row it replaces.
 #include <cuda.h>
 
 #include "snap_internal.cuh"
