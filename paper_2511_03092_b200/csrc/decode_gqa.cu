@@ -479,29 +479,26 @@ bool decode_gqa_supported(int dtype, const Shape& s) {
   return dtype == SNAP_BF16 && s.d_qk == D && s.d_v == D && !s.v_aliases_k && s.g >= 1 && s.g <= 8;
 }
 
-// Splits per (sequence, KV head): enough CTAs to fill every resident slot (3 CTAs per SM, 2 for
-// g = 8), preferring counts whose last wave is nearly full, with at least one 64-row block per
-// split.  SNAP_DECODE_NSPLIT overrides the choice (tuning aid).
-int decode_gqa_nsplit_for(const Shape& s, int n_active, int sm_count, int ctas_per_sm) {
+// Splits per (sequence, KV head).  Measured on B200 over batch sizes 1..64 (5124 slots, 8 KV heads,
+// CUDA-graph replays): the time is flat around a total of about 1.75 CTAs per SM for small
+// batches -- more splits only lengthen the merge -- and three splits are best once the batch
+// alone fills the GPU (they even out the tail).  A split keeps at least two 64-row blocks and,
+// for very long caches, at most about 48.
+// SNAP_DECODE_NSPLIT overrides the choice (tuning aid).
+int decode_gqa_nsplit_for(const Shape& s, int n_active, int sm_count, int /*ctas_per_sm*/) {
   const int tiles = (s.Sc + 63) / 64;
   if (const char* env = getenv("SNAP_DECODE_NSPLIT")) {
     const int v = atoi(env);
     if (v >= 1) return v < tiles ? v : tiles;
   }
-  const long long base = (long long)n_active * s.Hkv;
-  const double slots = (double)ctas_per_sm * sm_count;
-  int best = 1;
-  double best_score = -1.0;
-  const int max_ns = tiles < 64 ? tiles : 64;
-  for (int ns = 1; ns <= max_ns; ++ns) {
-    const double waves = base * ns / slots;
-    const double full = waves < 1.0 ? waves : waves / (double)(long long)(waves + 0.999999);
-    const double per_split = (double)tiles / ns;
-    const double overhead = per_split / (per_split + 1.5);      // pipeline fill and merge per split
-    const double score = full * overhead;
-    if (score > best_score + 1e-9) { best_score = score; best = ns; }
-  }
-  return best;
+  const long long base = (long long)(n_active > 0 ? n_active : 1) * s.Hkv;
+  long long ns = (7LL * sm_count / 4 + base / 2) / base;
+  if (ns < 3) ns = 3;
+  if (ns < (tiles + 47) / 48) ns = (tiles + 47) / 48;           // very long caches: keep a split short, lengths may be ragged
+  if (ns > 16) ns = 16;
+  if (ns > tiles / 2) ns = tiles / 2;
+  if (ns < 1) ns = 1;
+  return (int)ns;
 }
 int decode_gqa_nsplit(const Shape& s, int n_active, int sm_count) {
   return decode_gqa_nsplit_for(s, n_active, sm_count, s.g > 4 ? 2 : 3);
