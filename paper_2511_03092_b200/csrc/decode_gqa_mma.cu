@@ -361,15 +361,36 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   if (q_len < 1 || q_len * s.g > GP || (q_len > 1 && (!k_new || q_len > s.Lr))) return cudaErrorInvalidValue;
   umma::EncodeTiledFn enc = umma::encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
-  CUtensorMap tk, tv;
-  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)s.Sc, (cuuint64_t)s.max_seqs * s.Hkv};
-  const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)s.Sc * D * 2};
-  const cuuint32_t box[3] = {64, (cuuint32_t)WT, 1}, estr[3] = {1, 1, 1};
-  if (enc(&tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, k_cache, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
-      enc(&tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, v_cache, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return cudaErrorInvalidValue;
+  // The two tensor maps depend only on the cache buffers and their shape: keep the last few per
+  // host thread instead of encoding them on every decode step.
+  struct MapEntry { const void* k; const void* v; int Sc; long long planes; CUtensorMap tk, tv; };
+  constexpr int kMapCache = 8;
+  thread_local MapEntry cache[kMapCache] = {};
+  thread_local int cache_next = 0;
+  const long long planes = (long long)s.max_seqs * s.Hkv;
+  const MapEntry* hit = nullptr;
+  for (int e = 0; e < kMapCache; ++e)
+    if (cache[e].k == k_cache && cache[e].v == v_cache && cache[e].Sc == s.Sc && cache[e].planes == planes && cache[e].k) {
+      hit = &cache[e];
+      break;
+    }
+  if (!hit) {
+    MapEntry& m = cache[cache_next];
+    cache_next = (cache_next + 1) % kMapCache;
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)s.Sc, (cuuint64_t)planes};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)s.Sc * D * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)WT, 1}, estr[3] = {1, 1, 1};
+    m.k = nullptr;
+    if (enc(&m.tk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, k_cache, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+        enc(&m.tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, v_cache, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    m.k = k_cache; m.v = v_cache; m.Sc = s.Sc; m.planes = planes;
+    hit = &m;
+  }
+  const CUtensorMap& tk = hit->tk;
+  const CUtensorMap& tv = hit->tv;
   MmaArgs a;
   a.q = static_cast<const __nv_bfloat16*>(q);
   a.k_new = static_cast<const __nv_bfloat16*>(k_new);
