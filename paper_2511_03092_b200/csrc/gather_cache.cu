@@ -71,6 +71,7 @@ __device__ __forceinline__ void copy_rows(const char* __restrict__ src_base, lon
 }
 
 __global__ void __launch_bounds__(NT) gather_kernel(const GatherArgs a) {
+  pdl_wait();
   const int seq = blockIdx.z, kvh = blockIdx.y;
   const int L = a.b.len[seq], slot = a.b.slot[seq];
   if (slot < 0 || slot >= a.max_seqs) {
@@ -150,9 +151,9 @@ cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KV
   a.b = b; a.idx = s.K > 0 ? idx : nullptr;
   a.seq_len = seq_len; a.valid_topk = valid_topk; a.status = status;
   dim3 grid((s.Sc + ROWS - 1) / ROWS, s.Hkv, b.n);
-  gather_kernel<<<grid, NT, 0, st>>>(a);
+  const cudaError_t e = launch_pdl(gather_kernel, grid, dim3(NT), 0, st, a);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_append(int dtype, const Shape& s, const void* k_new, const void* v_new,

@@ -258,6 +258,7 @@ __global__ void __launch_bounds__(256, 2) score_mma_kernel(const MmaArgs a) {
 __global__ void score_mma_combine_kernel(const float2* __restrict__ part, float2* __restrict__ stats,
                                          int nsplit, int R) {
   // one warp per query row, lanes over the splits
+  pdl_wait();
   const long long z = blockIdx.y;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (row >= R) return;
@@ -278,9 +279,10 @@ __global__ void score_mma_combine_kernel(const float2* __restrict__ part, float2
 }  // namespace
 
 cudaError_t launch_score_combine_log2(const ScoreBuffers& buf, int nz, int R, cudaStream_t st) {
-  score_mma_combine_kernel<<<dim3((R + 7) / 8, nz), 256, 0, st>>>(buf.part_stats, buf.stats, buf.nsplit, R);
+  const cudaError_t e = launch_pdl(score_mma_combine_kernel, dim3((R + 7) / 8, nz), dim3(256), 0, st,
+                                   static_cast<const float2*>(buf.part_stats), buf.stats, buf.nsplit, R);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 bool score_mma_supported(int dtype, const Shape& s) {

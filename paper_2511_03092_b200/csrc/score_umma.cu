@@ -198,6 +198,7 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
     mbar_init(qfull_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  pdl_wait();                                                 // everything above overlaps the previous kernel's tail
   float* mu_s = reinterpret_cast<float*>(stats_s);            // pass 2: m_i + log2(l_i) per query row
   if (PASS == 2) {
     for (int i = tid; i < R; i += NTHREADS) {
@@ -498,11 +499,11 @@ cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_o
   if (cudaError_t e = ensure_dyn_smem(score_umma_kernel<2>, kSmemBytes, limit2)) return e;
   const int nz = b.n_scored * s.Hkv;
   dim3 grid(buf.nsplit, nz);
-  score_umma_kernel<1><<<grid, NTHREADS, kSmemBytes, st>>>(a, tq, tk);
+  if (launch_pdl(score_umma_kernel<1>, grid, dim3(NTHREADS), kSmemBytes, st, a, tq, tk) != cudaSuccess) return cudaGetLastError();
   count_launch();
   cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
   if (e != cudaSuccess) return e;
-  score_umma_kernel<2><<<grid, NTHREADS, kSmemBytes, st>>>(a, tq, tk);
+  if (launch_pdl(score_umma_kernel<2>, grid, dim3(NTHREADS), kSmemBytes, st, a, tq, tk) != cudaSuccess) return cudaGetLastError();
   count_launch();
   return cudaGetLastError();
 }

@@ -64,6 +64,25 @@ inline cudaError_t ensure_dyn_smem(Kernel kernel, size_t bytes, SmemLimit& done)
   return e;
 }
 
+// Launch as a programmatic dependent of whatever precedes it in the stream: the grid may become
+// resident (and run whatever it has before its griddepcontrol.wait) while the predecessor drains.
+// The kernel must execute griddepcontrol.wait before it touches memory a predecessor may write.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = grid;
+  lc.blockDim = block;
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // --- launchers (each enqueues on `st` and returns cudaGetLastError()) ---
 cudaError_t launch_score_simt(int dtype, const Shape& s, const SeqBatch& b, const void* q_obs,
                               const KVSource& src, const ScoreBuffers& buf, cudaStream_t st);

@@ -203,6 +203,7 @@ __device__ __forceinline__ bool trivial_case(const TopkArgs& a, int seq, int Le,
 
 // ---- register-resident kernel: thread t of rank r owns candidates [j0 + 16t, j0 + 16t + 16) ----
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_regs_kernel(const TopkArgs a) {
+  pdl_wait();
   __shared__ TopkShared sh;
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
@@ -289,6 +290,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_regs_
 
 // ---- streaming kernel: any length and pooling width; pooled scores live in scratch ----
 __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_stream_kernel(const TopkArgs a) {
+  pdl_wait();
   __shared__ TopkShared sh;
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
@@ -376,12 +378,13 @@ cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffe
   int max_le = 0;
   for (int i = 0; i < b.n; ++i) max_le = max(max_le, b.len[i] - s.Ls - s.Lr);
   dim3 grid(CL, s.Hkv, b.n);
+  cudaError_t e;
   if ((max_le + CL - 1) / CL + 1 <= MAXE * NT && s.w / 2 <= MAXR)
-    pool_topk_regs_kernel<<<grid, NT, 0, st>>>(a);
+    e = launch_pdl(pool_topk_regs_kernel, grid, dim3(NT), 0, st, a);
   else
-    pool_topk_stream_kernel<<<grid, NT, 0, st>>>(a);
+    e = launch_pdl(pool_topk_stream_kernel, grid, dim3(NT), 0, st, a);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace snap
