@@ -147,8 +147,8 @@ bool use_mla_stream(int dtype, const Shape& s) {
 DecodePlan plan_decode(int dtype, const Shape& s, int n_active) {
   DecodePlan p;
   const int n = n_active > 0 ? n_active : 1;
-  p.gqa_mma = false;
-  p.gqa = decode_gqa_supported(dtype, s);
+  p.gqa_mma = use_gqa_mma(dtype, s);
+  p.gqa = p.gqa_mma || decode_gqa_supported(dtype, s);
   p.mla_stream = !p.gqa && use_mla_stream(dtype, s);
   p.mla = !p.gqa && !p.mla_stream && decode_mla_supported(dtype, s);
   if (p.mla_stream) {
@@ -157,9 +157,11 @@ DecodePlan plan_decode(int dtype, const Shape& s, int n_active) {
   } else if (p.mla) {
     p.nsplit = decode_mla_nsplit(s, n, sm_count());
     p.floats = decode_mla_partial_floats(s, n_active, p.nsplit);
+  } else if (p.gqa_mma) {
+    p.nsplit = decode_gqa_mma_nsplit(s, n, sm_count());
+    p.floats = decode_gqa_mma_partial_floats(s, n_active, p.nsplit);
   } else if (p.gqa) {
-    p.gqa_mma = use_gqa_mma(dtype, s);
-    p.nsplit = p.gqa_mma ? decode_gqa_mma_nsplit(s, n, sm_count()) : decode_gqa_nsplit(s, n, sm_count());
+    p.nsplit = decode_gqa_nsplit(s, n, sm_count());
     p.floats = decode_gqa_partial_floats(s, n_active, p.nsplit);
   } else {
     p.nsplit = decode_generic_nsplit(s, n, sm_count());
@@ -399,7 +401,7 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
 // heads takes them (the tokens' heads share the N side of its MMAs, so q_len * group <= 8).
 static int multi_supported(const snap_config_t* cfg, const Shape& s, int q_len) {
   if (q_len < 1 || q_len > s.Lr) return SNAP_ERR_INVALID_ARG;
-  if (!decode_gqa_supported(cfg->dtype, s) || !decode_use_gqa_mma(cfg->dtype, s) || q_len * s.g > 8)
+  if (!decode_use_gqa_mma(cfg->dtype, s) || q_len * s.g > 8)
     return SNAP_ERR_UNSUPPORTED;
   return SNAP_OK;
 }
@@ -412,7 +414,7 @@ int64_t snap_decode_multi_workspace_bytes(const snap_config_t* cfg, int32_t n_ac
   const int ms = multi_supported(cfg, s, q_len);
   if (ms != SNAP_OK) return ms;
   const int nsplit = decode_gqa_mma_nsplit(s, n_active > 0 ? n_active : 1, sm_count());
-  return (int64_t)(decode_gqa_partial_floats(s, n_active * q_len, nsplit) * sizeof(float) + 256);
+  return (int64_t)(decode_gqa_mma_partial_floats(s, n_active * q_len, nsplit) * sizeof(float) + 256);
 }
 
 int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,

@@ -37,9 +37,8 @@ using umma::mbar_try_wait;
 using umma::smem_u32;
 using umma::tma_load_3d;
 
-constexpr int D = 128, WT = 16, NSTAGE = 2, NWARP = 4, NT = NWARP * 32, GP = 8;   // GP: head slots (N of the MMAs)
-constexpr int SLAB_B = WT * 128, TENS_B = 2 * SLAB_B, STAGE_B = 2 * TENS_B;       // stage = K (2 slabs) | V (2 slabs)
-constexpr int PS = D + 2;
+constexpr int WT = 16, NSTAGE = 2, GP = 8;     // 16-row tiles, two stages per warp, GP: column slots (N of the MMAs)
+constexpr int SLAB_B = WT * 128;                // one 64-dim slab of a tile: 16 rows x 128 bytes
 constexpr unsigned kWaitLimit = 1u << 22;
 
 struct MmaArgs {
@@ -102,8 +101,12 @@ __device__ __forceinline__ TileRows tile_rows(int j, int nA, int n_low, int Lsr,
   return t;
 }
 
-__global__ void __launch_bounds__(NT, 3)
+// D: head size (64, 128 or 256); NWARP: warps per CTA (fewer for wide heads, whose stages are larger)
+template <int D, int NWARP>
+__global__ void __launch_bounds__(NWARP * 32, 3)
 decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
+  constexpr int NT = NWARP * 32, NSL = D / 64, CPR = D / 8, KS = D / 16;   // slabs per tensor, 16-byte chunks per row, 16-dim steps
+  constexpr int TENS_B = NSL * SLAB_B, STAGE_B = 2 * TENS_B, PS = D + 2;   // stage = K slabs | V slabs
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem_raw = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   // [NWARP][NSTAGE] stages | [NWARP][NSTAGE] mbarriers
@@ -152,10 +155,11 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     const TileRows tr = tile_rows(t_begin + w + n * NWARP, nA, n_low, Lsr, n_top);
     const uint32_t dst = stage0 + s * STAGE_B, bar = bar0 + 8 * s;
     mbar_expect_tx(bar, (unsigned)STAGE_B);
-    tma_load_3d(dst, &tmap_k, 0, tr.row0, plane, bar);
-    tma_load_3d(dst + SLAB_B, &tmap_k, 64, tr.row0, plane, bar);
-    tma_load_3d(dst + TENS_B, &tmap_v, 0, tr.row0, plane, bar);
-    tma_load_3d(dst + TENS_B + SLAB_B, &tmap_v, 64, tr.row0, plane, bar);
+#pragma unroll
+    for (int h = 0; h < NSL; ++h) {
+      tma_load_3d(dst + h * SLAB_B, &tmap_k, 64 * h, tr.row0, plane, bar);
+      tma_load_3d(dst + TENS_B + h * SLAB_B, &tmap_v, 64 * h, tr.row0, plane, bar);
+    }
   };
   if (lane == 0)
     for (int n = 0; n < NSTAGE && n < T; ++n) issue(n);
@@ -170,20 +174,20 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
   // Column n of the MMAs is query token n / g, head n % g of the group (zero beyond T * g).
   // B fragments of Q^T for the eight 16-dim steps: column gq, dims 16 ks + 2 tq (+8)
   const int ncols = TQ * a.g;
-  uint32_t qb[8][2];
+  uint32_t qb[KS][2];
   {
     const int tcol = gq / a.g, hcol = gq - tcol * a.g;
     const __nv_bfloat16* qp = a.q + (((long long)i * TQ + tcol) * a.Hq + (long long)kvh * a.g + hcol) * D + 2 * tq;
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
+    for (int ks = 0; ks < KS; ++ks) {
       qb[ks][0] = gq < ncols ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks) : 0u;
       qb[ks][1] = gq < ncols ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks + 8) : 0u;
     }
   }
   const int tc0 = (2 * tq) / a.g, tc1 = (2 * tq + 1) / a.g;     // query tokens of this thread's two columns
-  float oacc[8][4];                              // O^T: dims 16 db + gq (+8), columns 2 tq (+1)
+  float oacc[KS][4];                             // O^T: dims 16 db + gq (+8), columns 2 tq (+1)
 #pragma unroll
-  for (int db = 0; db < 8; ++db)
+  for (int db = 0; db < KS; ++db)
 #pragma unroll
     for (int e = 0; e < 4; ++e) oacc[db][e] = 0.f;
   float m_ref[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};   // columns 2 tq, 2 tq + 1
@@ -199,7 +203,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     // ---- S^T = K tile . Q^T ----
     float sacc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
+    for (int ks = 0; ks < KS; ++ks) {
       uint32_t af[4];
       ldsm4(sK + (ks >> 2) * SLAB_B + swz(k_row, (ks & 3) * 2 + k_cadd), af);
       mma16816(sacc, af, qb[ks][0], qb[ks][1]);
@@ -220,7 +224,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
       m_ref[0] = n0; m_ref[1] = n1;
       l_part[0] *= a0; l_part[1] *= a1;
 #pragma unroll
-      for (int db = 0; db < 8; ++db) { oacc[db][0] *= a0; oacc[db][1] *= a1; oacc[db][2] *= a0; oacc[db][3] *= a1; }
+      for (int db = 0; db < KS; ++db) { oacc[db][0] *= a0; oacc[db][1] *= a1; oacc[db][2] *= a0; oacc[db][3] *= a1; }
     }
     const float r0 = m_ref[0] == -INFINITY ? 0.f : m_ref[0], r1 = m_ref[1] == -INFINITY ? 0.f : m_ref[1];
     const float p0 = fast_exp2(v0 - r0), p1 = fast_exp2(v1 - r1), p2 = fast_exp2(v2 - r0), p3 = fast_exp2(v3 - r1);
@@ -230,7 +234,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     const uint32_t pb0 = movmatrix_t(pack_bf16(p0, p1)), pb1 = movmatrix_t(pack_bf16(p2, p3));
     // ---- O^T += V tile^T . P^T ----
 #pragma unroll
-    for (int db = 0; db < 8; ++db) {
+    for (int db = 0; db < KS; ++db) {
       uint32_t af[4];
       ldsm4t(sV + (db >> 2) * SLAB_B + swz(v_row, (db & 3) * 2 + v_cadd), af);
       mma16816(oacc[db], af, pb0, pb1);
@@ -251,8 +255,8 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
       // ragged tile: rows past the end may hold anything (memory the caller never wrote), and a
       // zero probability does not silence a NaN in V: clear those V rows
       const int first = max(nrows, 0);
-      for (int e = lane; e < (WT - first) * 16; e += 32) {
-        const int r = first + e / 16, c = e % 16;
+      for (int e = lane; e < (WT - first) * CPR; e += 32) {
+        const int r = first + e / CPR, c = e % CPR;
         *reinterpret_cast<uint4*>(wstages + s * STAGE_B + TENS_B + (c >> 3) * SLAB_B + swz(r, c & 7)) = make_uint4(0, 0, 0, 0);
       }
       __syncwarp();
@@ -260,11 +264,13 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     if (TQ == 1) {
       if (new_slot >= tr.row0 && new_slot < tr.row0 + WT && new_slot < tr.row_end) {
         // the new token's slot is in this tile: store the row to the cache and patch the staged copy
-        const int r = new_slot - tr.row0, c = lane & 15;
-        const uint4 val = reinterpret_cast<const uint4*>(lane < 16 ? kn : vn)[c];
-        reinterpret_cast<uint4*>((lane < 16 ? kc : vc) + (long long)new_slot * (D * 2))[c] = val;
-        unsigned char* sp_ = wstages + s * STAGE_B + (lane < 16 ? 0 : TENS_B) + (c >> 3) * SLAB_B + swz(r, c & 7);
-        *reinterpret_cast<uint4*>(sp_) = val;
+        const int r = new_slot - tr.row0;
+        for (int e = lane; e < 2 * CPR; e += 32) {             // K chunks, then V chunks of the row
+          const int tens = e / CPR, c = e % CPR;
+          const uint4 val = reinterpret_cast<const uint4*>(tens ? vn : kn)[c];
+          reinterpret_cast<uint4*>((tens ? vc : kc) + (long long)new_slot * (D * 2))[c] = val;
+          *reinterpret_cast<uint4*>(wstages + s * STAGE_B + tens * TENS_B + (c >> 3) * SLAB_B + swz(r, c & 7)) = val;
+        }
         __syncwarp();
       }
     } else if (j < nA) {
@@ -273,11 +279,14 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
       for (int u = 0; u < TQ; ++u) {
         const int ru = ring_slot(L0 + u, a.Ls, a.Lr);
         if (ru < tr.row0 || ru >= tr.row0 + WT) continue;
-        const int r = ru - tr.row0, c = lane & 15;
+        const int r = ru - tr.row0;
         if (gq == r) { ok0 = ok0 && tc0 < u; ok1 = ok1 && tc1 < u; }
         if (gq + 8 == r) { ok2 = ok2 && tc0 < u; ok3 = ok3 && tc1 < u; }
-        const uint4 val = reinterpret_cast<const uint4*>((lane < 16 ? kn : vn) + u * new_stride)[c];
-        reinterpret_cast<uint4*>((lane < 16 ? kc : vc) + (long long)ru * (D * 2))[c] = val;
+        for (int e = lane; e < 2 * CPR; e += 32) {
+          const int tens = e / CPR, c = e % CPR;
+          reinterpret_cast<uint4*>((tens ? vc : kc) + (long long)ru * (D * 2))[c] =
+              reinterpret_cast<const uint4*>((tens ? vn : kn) + u * new_stride)[c];
+        }
       }
     }
     process(sK, sV, ok0, ok1, ok2, ok3);
@@ -291,8 +300,8 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
   if (TQ > 1 && sp == 0 && w == 0 && !bad && !timed_out) {
     // the new tokens as a tile of their own (this warp's pipeline has drained): row u is token u,
     // visible to the queries from token u on; rows past the last token are zero and masked
-    for (int e = lane; e < 2 * WT * 16; e += 32) {
-      const int tens = e / (WT * 16), r = (e / 16) % WT, c = e % 16;
+    for (int e = lane; e < 2 * WT * CPR; e += 32) {
+      const int tens = e / (WT * CPR), r = (e / CPR) % WT, c = e % CPR;
       uint4 val = make_uint4(0, 0, 0, 0);
       if (r < TQ) val = reinterpret_cast<const uint4*>((tens ? vn : kn) + r * new_stride)[c];
       *reinterpret_cast<uint4*>(wstages + tens * TENS_B + (c >> 3) * SLAB_B + swz(r, c & 7)) = val;
@@ -317,7 +326,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     wl[2 * tq] = l_part[0]; wl[2 * tq + 1] = l_part[1];
   }
 #pragma unroll
-  for (int db = 0; db < 8; ++db) {
+  for (int db = 0; db < KS; ++db) {
     wacc[(2 * tq) * D + 16 * db + gq] = oacc[db][0];
     wacc[(2 * tq + 1) * D + 16 * db + gq] = oacc[db][1];
     wacc[(2 * tq) * D + 16 * db + gq + 8] = oacc[db][2];
@@ -330,27 +339,79 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     float M = -INFINITY;
 #pragma unroll
     for (int ww = 0; ww < NWARP; ++ww) M = fmaxf(M, base[ww * WSTRIDE + h]);
-    float L = 0.f, O = 0.f;
+    float L = 0.f, f[NWARP];
 #pragma unroll
     for (int ww = 0; ww < NWARP; ++ww) {
       const float mw = base[ww * WSTRIDE + h];
-      const float f = mw == -INFINITY ? 0.f : exp2f(mw - M);
-      L += base[ww * WSTRIDE + GP + h] * f;
-      O += base[ww * WSTRIDE + 2 * GP + h * D + tid] * f;
+      f[ww] = mw == -INFINITY ? 0.f : exp2f(mw - M);
+      L += base[ww * WSTRIDE + GP + h] * f[ww];
     }
     const int tcol = h / a.g, hcol = h - tcol * a.g;
     float* ph = a.partials + ((((long long)i * TQ + tcol) * a.Hq + (long long)kvh * a.g + hcol) * a.nsplit + sp) * PS;
     if (tid == 0) { ph[0] = M; ph[1] = L; }
-    ph[2 + tid] = O;
+    for (int dv = tid; dv < D; dv += NT) {
+      float O = 0.f;
+#pragma unroll
+      for (int ww = 0; ww < NWARP; ++ww) O += base[ww * WSTRIDE + 2 * GP + h * D + dv] * f[ww];
+      ph[2 + dv] = O;
+    }
   }
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// Merge the splits of one (sequence, query token, query head) for any head size; maxima are in
+// the log2 domain.  Rows of `partials` and `out` are indexed by sequence * q_len + token, and every
+// token's block advances the sequence length by one.
+__global__ void __launch_bounds__(128) decode_gqa_mma_merge_kernel(const float* __restrict__ partials,
+                                                                   __nv_bfloat16* __restrict__ out, int Hq, int d,
+                                                                   int nsplit, const int* __restrict__ slot_ids,
+                                                                   int* seq_len, int max_seqs, int bump, int q_len) {
+  const int h = blockIdx.x, i = blockIdx.y, ps = d + 2;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const float* p = partials + ((long long)i * Hq + h) * nsplit * ps;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  float M = -INFINITY;
+  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * ps]);
+  float L = 0.f;
+  for (int s = 0; s < nsplit; ++s) {
+    const float ms = p[s * ps];
+    if (ms != -INFINITY) L += p[s * ps + 1] * exp2f(ms - M);
+  }
+  const float inv = L > 0.f ? 1.f / L : 0.f;
+  for (int t = threadIdx.x; t < d; t += blockDim.x) {
+    float O = 0.f;
+    for (int s = 0; s < nsplit; ++s) {
+      const float ms = p[s * ps];
+      if (ms != -INFINITY) O += p[s * ps + 2 + t] * exp2f(ms - M);
+    }
+    out[((long long)i * Hq + h) * d + t] = __float2bfloat16_rn(O * inv);
+  }
+  if (bump && h == 0 && threadIdx.x == 0) {
+    const int slot = slot_ids[i / q_len];
+    if (slot >= 0 && slot < max_seqs) atomicAdd(&seq_len[slot], 1);
+  }
+}
+
+template <int D, int NWARP>
+cudaError_t launch_d(const MmaArgs& a, const CUtensorMap& tk, const CUtensorMap& tv, int n_active, cudaStream_t st) {
+  constexpr size_t smem = (size_t)NWARP * NSTAGE * (2 * (D / 64) * SLAB_B) + NWARP * NSTAGE * 8 + 1024;
+  static SmemLimit limit = {};
+  if (cudaError_t e = ensure_dyn_smem(decode_gqa_mma_kernel<D, NWARP>, smem, limit)) return e;
+  const cudaError_t e = launch_pdl(decode_gqa_mma_kernel<D, NWARP>, dim3(a.nsplit, a.Hkv, n_active), dim3(NWARP * 32), smem, st,
+                                   a, tk, tv);
+  count_launch();
+  return e;
 }
 
 }  // namespace
 
 bool decode_gqa_mma_supported(int dtype, const Shape& s) {
-  return dtype == SNAP_BF16 && s.d_qk == D && s.d_v == D && !s.v_aliases_k && s.g >= 1 && s.g <= GP &&
-         umma::encode_tiled_fn() != nullptr;
+  return dtype == SNAP_BF16 && s.d_qk == s.d_v && (s.d_qk == 64 || s.d_qk == 128 || s.d_qk == 256) && !s.v_aliases_k &&
+         s.g >= 1 && s.g <= GP && umma::encode_tiled_fn() != nullptr;
+}
+
+size_t decode_gqa_mma_partial_floats(const Shape& s, int n_rows, int nsplit) {
+  return (size_t)n_rows * s.Hq * nsplit * (s.d_v + 2);
 }
 
 cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_new, const void* v_new,
@@ -361,16 +422,18 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   if (q_len < 1 || q_len * s.g > GP || (q_len > 1 && (!k_new || q_len > s.Lr))) return cudaErrorInvalidValue;
   umma::EncodeTiledFn enc = umma::encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
+  const int D = s.d_qk;
   // The two tensor maps depend only on the cache buffers and their shape: keep the last few per
   // host thread instead of encoding them on every decode step.
-  struct MapEntry { const void* k; const void* v; int Sc; long long planes; CUtensorMap tk, tv; };
+  struct MapEntry { const void* k; const void* v; int Sc, d; long long planes; CUtensorMap tk, tv; };
   constexpr int kMapCache = 8;
   thread_local MapEntry cache[kMapCache] = {};
   thread_local int cache_next = 0;
   const long long planes = (long long)s.max_seqs * s.Hkv;
   const MapEntry* hit = nullptr;
   for (int e = 0; e < kMapCache; ++e)
-    if (cache[e].k == k_cache && cache[e].v == v_cache && cache[e].Sc == s.Sc && cache[e].planes == planes && cache[e].k) {
+    if (cache[e].k == k_cache && cache[e].v == v_cache && cache[e].Sc == s.Sc && cache[e].d == D && cache[e].planes == planes &&
+        cache[e].k) {
       hit = &cache[e];
       break;
     }
@@ -386,11 +449,9 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
         enc(&m.tv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, v_cache, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
-    m.k = k_cache; m.v = v_cache; m.Sc = s.Sc; m.planes = planes;
+    m.k = k_cache; m.v = v_cache; m.Sc = s.Sc; m.d = D; m.planes = planes;
     hit = &m;
   }
-  const CUtensorMap& tk = hit->tk;
-  const CUtensorMap& tv = hit->tv;
   MmaArgs a;
   a.q = static_cast<const __nv_bfloat16*>(q);
   a.k_new = static_cast<const __nv_bfloat16*>(k_new);
@@ -402,24 +463,19 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   a.T = q_len;
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.seq_len = seq_len; a.valid_topk = valid_topk; a.partials = partials; a.status = status;
-  const size_t smem = (size_t)NWARP * NSTAGE * STAGE_B + NWARP * NSTAGE * 8 + 1024;
-  static SmemLimit limit = {};
-  if (cudaError_t e = ensure_dyn_smem(decode_gqa_mma_kernel, smem, limit)) return e;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(nsplit, s.Hkv, n_active);
-  lc.blockDim = dim3(NT);
-  lc.dynamicSmemBytes = smem;
-  lc.stream = st;
-  lc.attrs = attr;
-  lc.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_mma_kernel, a, tk, tv);
-  count_launch();
+  cudaError_t e;
+  if (D == 128) e = launch_d<128, 4>(a, hit->tk, hit->tv, n_active, st);
+  else if (D == 64) e = launch_d<64, 4>(a, hit->tk, hit->tv, n_active, st);
+  else e = launch_d<256, 2>(a, hit->tk, hit->tv, n_active, st);
   if (e != cudaSuccess) return e;
-  return launch_decode_gqa_merge(partials, out, s.Hq, nsplit, slot_ids, n_active * q_len, q_len, seq_len, s.max_seqs,
-                                 k_new != nullptr, st);
+  if (D == 128)
+    return launch_decode_gqa_merge(partials, out, s.Hq, nsplit, slot_ids, n_active * q_len, q_len, seq_len, s.max_seqs,
+                                   k_new != nullptr, st);
+  e = launch_pdl(decode_gqa_mma_merge_kernel, dim3(s.Hq, n_active * q_len), dim3(128), 0, st,
+                 static_cast<const float*>(partials), static_cast<__nv_bfloat16*>(out), s.Hq, D, nsplit, slot_ids, seq_len,
+                 s.max_seqs, (int)(k_new != nullptr), q_len);
+  count_launch();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace snap

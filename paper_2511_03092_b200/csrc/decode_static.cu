@@ -86,13 +86,14 @@ extern "C" int snap_decode_attn_static(const snap_config_t* cfg, const snap_layo
   const int src = static_scratch(&scratch, &sms);
   if (src != SNAP_OK) return src;
 
-  const bool gqa = decode_gqa_supported(cfg->dtype, s);
-  const bool gqa_mma = gqa && decode_use_gqa_mma(cfg->dtype, s);
+  const bool gqa_mma = decode_use_gqa_mma(cfg->dtype, s);
+  const bool gqa = gqa_mma || decode_gqa_supported(cfg->dtype, s);
   const int nsplit = gqa_mma ? decode_gqa_mma_nsplit(s, n_active, sms)
                      : gqa   ? decode_gqa_nsplit(s, n_active, sms)
                              : decode_generic_nsplit(s, n_active, sms);
-  const size_t need = gqa ? decode_gqa_partial_floats(s, n_active, nsplit)
-                          : decode_partial_floats(s, n_active, nsplit);
+  const size_t need = gqa_mma ? decode_gqa_mma_partial_floats(s, n_active, nsplit)
+                      : gqa   ? decode_gqa_partial_floats(s, n_active, nsplit)
+                              : decode_partial_floats(s, n_active, nsplit);
   if (need > kStaticFloats) return SNAP_ERR_STATIC_SCRATCH_EXCEEDED;
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

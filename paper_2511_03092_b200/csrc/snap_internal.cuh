@@ -129,10 +129,11 @@ cudaError_t launch_decode_gqa(const Shape& s, const void* q, const void* k_new, 
 
 cudaError_t launch_decode_gqa_merge(const float* partials, void* out, int Hq, int nsplit, const int* slot_ids,
                                     int n_rows, int q_len, int* seq_len, int max_seqs, int bump, cudaStream_t st);
-// the same on tensor cores (mma.sync, the group's heads on the N side): cost independent of the group size
+// the same on tensor cores (mma.sync, the group's heads on the N side; head sizes 64, 128, 256): cost independent of the group size
 bool decode_gqa_mma_supported(int dtype, const Shape& s);
 bool decode_use_gqa_mma(int dtype, const Shape& s);     // the choice between the two, shared by all entry points
 int decode_gqa_mma_nsplit(const Shape& s, int n_active, int sm_count);
+size_t decode_gqa_mma_partial_floats(const Shape& s, int n_rows, int nsplit);
 cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_new, const void* v_new,
                                   const int* slot_ids, int n_active, void* k_cache, void* v_cache,
                                   int* seq_len, const int* valid_topk, void* out, float* partials,

@@ -458,3 +458,17 @@ def test_decode_from_empty_slots_in_memory_full_of_nans(wl):
             if step < 20 or step % 7 == 0:
                 H.check_output(out[i], ref, wl, f"step {step} seq {i}")
     assert layer.status() == 0
+
+
+@pytest.mark.parametrize("d,hq,hkv", [(64, 16, 4), (64, 4, 4), (256, 8, 4), (256, 32, 4)],
+                         ids=["d64g4", "d64g1", "d256g2", "d256g8"])
+def test_head_sizes_64_and_256(d, hq, hkv):
+    """The tensor-core decode kernel and the wide score kernel at the other common head sizes."""
+    wl = SMALL_BF16.scaled(d_qk=d, d_v=d, n_q_heads=hq, n_kv_heads=hkv)
+    _run_compress_and_decode(wl, [wl.prompt_len[0], 50, 3], seed=19, steps=5)
+    _run_compress_and_decode(wl, [300], seed=23, steps=2 * wl.l_recent + 5, check_ring_every=16)
+
+
+def test_multi_token_decode_with_64_wide_heads():
+    wl = SMALL_BF16.scaled(d_qk=64, d_v=64, n_q_heads=8, n_kv_heads=4)
+    _run_multi(wl, [3, 50, 52, 300], 3, steps=20, seed=89)
