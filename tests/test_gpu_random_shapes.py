@@ -1,0 +1,95 @@
+"""Seeded random small configurations through the C ABI against the oracle: head size, group size,
+sink / window / budget sizes, pooling width, ragged prompt lengths, one or several tokens per step,
+and the latent layout with 64, 128 and 256 heads.  Every case checks the selected indices, every
+decode output, the sequence lengths and the final cache image."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import snapstream_oracle as orc
+from paper_2511_03092_b200 import binding as B
+from paper_2511_03092_b200 import synth
+from tests import _harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _compress_and_check(wl, lengths, seed):
+    n = len(lengths)
+    layer = H.GpuLayer(wl, n)
+    prompts = [synth.make_prompt(wl, L, seed + i) for i, L in enumerate(lengths)]
+    idx = layer.compress(prompts, list(range(n)))
+    seqs = [H.oracle_compress(wl, p) for p in prompts]
+    for i in range(n):
+        H.check_selection(idx[i], seqs[i], wl)
+        seqs[i].topk_pos = [idx[i][h][idx[i][h] >= 0].astype(np.int64) for h in range(wl.n_kv_heads)]
+    return layer, seqs
+
+
+def _finish(layer, seqs, wl):
+    assert layer.status() == 0
+    for i, seq in enumerate(seqs):
+        assert int(layer.cache.seq_len[i]) == seq.n_tokens
+        H.check_cache_image(layer, seq, i, wl)
+
+
+@pytest.mark.parametrize("seed", [3, 4])
+def test_random_grouped_query_configurations(seed):
+    rng = np.random.default_rng(seed)
+    for case in range(40):
+        d = int(rng.choice([64, 128, 256]))
+        hkv = int(rng.choice([1, 2, 4]))
+        g = int(rng.integers(1, 9))
+        Ls, Lr, K = int(rng.integers(0, 6)), int(rng.integers(1, 40)), int(rng.choice([0, 5, 16, 33, 64]))
+        Lo, w = int(rng.integers(1, min(Lr, 16) + 1)), int(rng.choice([1, 3, 7]))
+        wl = synth.Workload("rnd", g * hkv, hkv, d, d, "bf16", Ls, Lr, K, Lo, w, batch=1, prompt_len=(100, 100),
+                            decode_steps=4, salience="zipf")
+        n = int(rng.integers(1, 4))
+        lengths = [int(rng.integers(1, 200)) for _ in range(n)]
+        q_len = int(rng.integers(1, max(1, min(8 // g, Lr)) + 1))
+        steps = int(rng.integers(1, 2 * Lr // q_len + 4))
+        what = f"case {case}: d{d} hkv{hkv} g{g} Ls{Ls} Lr{Lr} K{K} Lo{Lo} w{w} L{lengths} q_len{q_len}"
+        layer, seqs = _compress_and_check(wl, lengths, 1000 * case + seed)
+        c = layer.cache
+        slots = torch.arange(n, dtype=torch.int32, device="cuda")
+        ws = torch.empty(B.snap_decode_multi_workspace_bytes(layer.cfg, n, q_len), dtype=torch.uint8, device="cuda")
+        for st in range(steps):
+            ds = [synth.make_decode_inputs(wl, n, case, st * q_len + u) for u in range(q_len)]
+            if q_len == 1:
+                out = layer.decode(ds[0]["q"].cuda(), ds[0]["k_new"].cuda(), ds[0]["v_new"].cuda(), slots).unsqueeze(1)
+            else:
+                q = torch.stack([x["q"] for x in ds], 1).contiguous().cuda()
+                kn = torch.stack([x["k_new"] for x in ds], 1).contiguous().cuda()
+                vn = torch.stack([x["v_new"] for x in ds], 1).contiguous().cuda()
+                out = torch.empty(n, q_len, wl.n_q_heads, d, dtype=torch.bfloat16, device="cuda")
+                B.snap_decode_attn_multi(layer.cfg, layer.layout, q, kn, vn, slots, n, q_len, c.k_cache, c.v_cache,
+                                         c.seq_len, c.valid_topk, out, ws, c.status)
+            for i in range(n):
+                for u in range(q_len):
+                    ref = orc.decode_step(seqs[i], synth.to_f64(ds[u]["q"][i]), synth.to_f64(ds[u]["k_new"][i]),
+                                          synth.to_f64(ds[u]["v_new"][i]))
+                    H.check_output(out[i, u], ref, wl, f"{what} step {st} seq {i} token {u}")
+        _finish(layer, seqs, wl)
+
+
+def test_random_latent_configurations():
+    rng = np.random.default_rng(5)
+    for case in range(16):
+        hq = int(rng.choice([64, 128, 256]))
+        Ls, Lr, K = int(rng.integers(0, 6)), int(rng.integers(1, 300)), int(rng.choice([0, 7, 64, 200]))
+        Lo, w = int(rng.integers(1, min(Lr, 8) + 1)), int(rng.choice([1, 5]))
+        wl = synth.Workload("rnd_latent", hq, 1, 576, 512, "bf16", Ls, Lr, K, Lo, w, batch=1, prompt_len=(100, 100),
+                            decode_steps=4, salience="planted", n_planted=4, v_aliases_k=True,
+                            softmax_scale=2.0 ** -0.5)
+        n = int(rng.integers(1, 3))
+        lengths = [int(rng.integers(1, 700)) for _ in range(n)]
+        what = f"case {case}: hq{hq} Ls{Ls} Lr{Lr} K{K} Lo{Lo} w{w} L{lengths}"
+        layer, seqs = _compress_and_check(wl, lengths, 1000 * case)
+        slots = torch.arange(n, dtype=torch.int32, device="cuda")
+        for st in range(int(rng.integers(1, 12))):
+            d = synth.make_decode_inputs(wl, n, case, st)
+            out = layer.decode(d["q"].cuda(), d["k_new"].cuda(), None, slots)
+            for i in range(n):
+                ref = orc.decode_step(seqs[i], synth.to_f64(d["q"][i]), synth.to_f64(d["k_new"][i]), None)
+                H.check_output(out[i], ref, wl, f"{what} step {st} seq {i}")
+        _finish(layer, seqs, wl)
