@@ -93,3 +93,34 @@ def test_random_latent_configurations():
                 ref = orc.decode_step(seqs[i], synth.to_f64(d["q"][i]), synth.to_f64(d["k_new"][i]), None)
                 H.check_output(out[i], ref, wl, f"{what} step {st} seq {i}")
         _finish(layer, seqs, wl)
+
+
+def test_random_compress_configurations():
+    """Prompts of a few thousand tokens through each score kernel family (128-wide tcgen05, wide tcgen05 at
+    other head and group sizes, latent layout), both pooling modes, several pooling widths and budgets."""
+    rng = np.random.default_rng(1)
+    for case in range(18):
+        kind = case % 3
+        if kind == 0:
+            hkv, g, d = int(rng.choice([1, 2])), int(rng.choice([2, 4])), 128
+            Lo = int(rng.choice([32, 64])) if g == 4 else int(rng.choice([64, 128]))
+        elif kind == 1:
+            hkv, g = int(rng.choice([1, 2])), int(rng.choice([1, 3, 5, 8]))
+            Lo, d = int(rng.choice([8, 16, 48])), int(rng.choice([64, 128, 256]))
+        else:
+            hkv, g, Lo, d = 1, int(rng.choice([64, 128])), int(rng.choice([4, 16])), 576
+        Ls, Lr = int(rng.integers(0, 8)), int(rng.integers(max(Lo, 8), 600))
+        K, w = int(rng.choice([0, 64, 500, 2048])), int(rng.choice([1, 3, 7, 13]))
+        mode = str(rng.choice(["avg", "max"]))
+        L = int(rng.integers(Ls + Lr + 1, 20000))
+        if kind == 2:
+            wl = synth.Workload("rnd", g, 1, 576, 512, "bf16", Ls, Lr, K, Lo, w, batch=1, prompt_len=(L, L),
+                                decode_steps=1, salience="planted", n_planted=16, v_aliases_k=True,
+                                softmax_scale=2.0 ** -0.5, pool_mode=mode)
+        else:
+            wl = synth.Workload("rnd", g * hkv, hkv, d, d, "bf16", Ls, Lr, K, Lo, w, batch=1, prompt_len=(L, L),
+                                decode_steps=1, salience=str(rng.choice(["zipf", "planted"])), n_planted=16,
+                                pool_mode=mode)
+        layer, seqs = _compress_and_check(wl, [L], 77 * case + 1)
+        assert layer.status() == 0, f"case {case}"
+        H.check_cache_image(layer, seqs[0], 0, wl)
