@@ -103,3 +103,34 @@ def test_workspace_queries_and_argument_errors_without_gpu():
     assert cc(one, None, one, 2, one, one, two, two, one, None, None) == -4  # missing new values
     assert cc(one, one, one, -3, one, one, two, two, one, None, None) == -1
     assert cc(one, one, one, 0, one, one, two, two, one, None, None) == 0    # nothing to do
+
+
+def test_header_is_plain_c99(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 on its own, and a C caller must be able to
+    link against the library and use the host-only entry points."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "use_header.c"
+    src.write_text(
+        '#include "snapstream.h"\n'
+        "#include <stdio.h>\n"
+        "int main(void) {\n"
+        "  snap_config_t cfg = {32, 8, 128, 128, 0, SNAP_BF16, 4, 1024, 4096, 64, 7, SNAP_POOL_AVG, 0.088388f, 32};\n"
+        "  snap_layout_t lay;\n"
+        "  int rc = snap_cache_layout(&cfg, &lay);\n"
+        '  printf("%d %d %d %d %d %s\\n", rc, lay.slots, lay.sink_off, lay.ring_off, lay.topk_off, snap_status_string(-3));\n'
+        "  cfg.l_obs = 0;\n"
+        "  return snap_cache_layout(&cfg, &lay) == SNAP_ERR_INVALID_ARG ? 0 : 1;\n"
+        "}\n")
+    obj = tmp_path / "use_header.o"
+    subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(root, "include"),
+                    "-c", str(src), "-o", str(obj)], check=True)
+    libdir = os.path.join(root, "paper_2511_03092_b200")
+    exe = tmp_path / "use_header"
+    subprocess.run([gcc, str(obj), "-L", libdir, "-lsnapstream", "-Wl,-rpath," + libdir, "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    assert out[:5] == ["0", "5124", "0", "4", "1028"]
