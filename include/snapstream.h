@@ -13,6 +13,10 @@
  *   snap_decode_attn    Section 3.3: (optional Eq. 3 scatter, then) attention of one query token
  *                       per sequence over the valid cache slots
  *
+ * and, around it: snap_decode_attn_multi (several new tokens per sequence and step),
+ * snap_decode_attn_static (the decode step without a caller-provided scratch buffer) and
+ * snap_append_kv_concat (the slice-and-concatenate update of Section 3.2.1, as a baseline).
+ *
  * Conventions
  *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are plain
  *     host memory.  Every device buffer must be 16-byte aligned.
