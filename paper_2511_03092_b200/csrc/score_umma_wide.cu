@@ -11,10 +11,11 @@
 // accumulator buffers let the next tile's MMAs overlap the epilogue of the current one.
 //   pass 1  M = 128 query rows, N = 256 candidates; thread = query row; the two epilogue groups
 //           take 128 candidates each and their (reference max, sum) pairs are merged at the end.
-//   pass 2  M = 128 candidates, N = 128 query rows; thread = candidate; each group sums
-//           exp2(s_ij - m_i - log2 l_i) over 64 rows (constants in registers); the per-row-block
-//           partial column sums go to scratch and a small kernel adds the row blocks in a fixed
-//           order (deterministic, no atomics).
+//   pass 2  the same MMAs (an N = 128 instruction would occupy the tensor pipe almost as long for half
+//           the work); thread = query row scales its row by exp2(-(m_i + log2 l_i)) and the 128 rows
+//           are summed per candidate with a transposing shuffle reduction and one shared-memory
+//           step; the per-row-block partial column sums go to scratch and a small kernel adds the
+//           row blocks in a fixed order (deterministic, no atomics).
 // Every mbarrier wait is bounded; a wait that runs out raises SNAP_DEV_WAIT_TIMEOUT.
 #include <cstdlib>
 
@@ -42,7 +43,7 @@ template <int PASS>
 __global__ void __launch_bounds__(NTHREADS, 1)
 score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tmap_q,
                        const __grid_constant__ CUtensorMap tmap_k) {
-  constexpr int TNP = PASS == 1 ? 256 : 128;                  // candidates per tile
+  constexpr int TNP = 256;                                    // candidates per tile
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int NH = a.NH, NS = a.NS;
@@ -50,7 +51,8 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
   unsigned char* Ks = Qs + NH * QH_B;                         // [NS][up to 256 rows][128 B]
   float* mu_s = reinterpret_cast<float*>(Ks + NS * STAGE_B);  // [128] pass 2: m_i + log2 l_i of this row block
   float2* xch = reinterpret_cast<float2*>(mu_s + 128);        // [128] exchange between the epilogue groups
-  uint64_t* bars = reinterpret_cast<uint64_t*>(xch + 128);    // full[NS] empty[NS] tfull[2] tempty[2] qfull
+  float* red = reinterpret_cast<float*>(xch + 128);           // [2 tile parities][2 groups][4 warps][128] pass-2 column partials
+  uint64_t* bars = reinterpret_cast<uint64_t*>(red + 2 * 2 * 4 * 128);   // full[NS] empty[NS] tfull[2] tempty[2] qfull
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NS + 5);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -119,7 +121,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0 && nt > 0) {
-      const uint32_t idesc = PASS == 1 ? idesc_bf16(128, 256) : idesc_bf16(128, 128);
+      const uint32_t idesc = idesc_bf16(128, 256);
       bool ok = mbar_wait(qfull_bar, 0u, abort_flag);
       for (int it = 0; it < nt && ok; ++it) {
         const int b = it & 1;
@@ -132,10 +134,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
           const uint32_t kst = smem_u32(Ks) + s * STAGE_B, qst = smem_u32(Qs) + h * QH_B;
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
-            if (PASS == 1)
-              mma_bf16(tmem_base + b * 256, smem_desc(qst + ks * 32), smem_desc(kst + ks * 32), idesc, (h | ks) != 0);
-            else
-              mma_bf16(tmem_base + b * 256, smem_desc(kst + ks * 32), smem_desc(qst + ks * 32), idesc, (h | ks) != 0);
+            mma_bf16(tmem_base + b * 256, smem_desc(qst + ks * 32), smem_desc(kst + ks * 32), idesc, (h | ks) != 0);
           }
           mma_commit(empty_bar(s));                            // slab may be refilled once these MMAs have read it
         }
@@ -147,11 +146,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
     // ---------------- epilogue warps ----------------
     const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
     bool ok = true;
-    float mu[64];
-    if (PASS == 2) {
-#pragma unroll
-      for (int i = 0; i < 64; ++i) mu[i] = -mu_s[64 * eg + i];
-    }
+    const float neg_mu = PASS == 2 ? -mu_s[lrow] : 0.f;        // pass 2: this thread's row offset (-inf for a padding row)
     for (int it = 0; it < nt; ++it) {
       const int b = it & 1;
       const bool landed = mbar_wait(tfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag);
@@ -211,39 +206,62 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
         }
         l_sum += sum;
       } else {
-        const uint32_t col0 = lane_addr + b * 256 + eg * 64;
-        const int cand = (t0 + it) * TNP + lrow;
-        float s = 0.f;
+        // thread = query row; this group's 128 candidates of the tile.  The weights exp2(s - m_i - log2 l_i)
+        // are summed over the 128 rows of the block: a transposing shuffle reduction inside each warp (every
+        // step halves the values a lane holds), then over the group's four warps through shared memory.
+        const uint32_t col0 = lane_addr + b * 256 + eg * 128;
+        const int cand0 = (t0 + it) * TNP + eg * 128;
+        float v[128];
         if (landed) {
-          float s4[4] = {0.f, 0.f, 0.f, 0.f};
           tmem_ld16_issue(col0, ra);
 #pragma unroll
-          for (int c = 0; c < 4; c += 2) {
+          for (int c = 0; c < 8; c += 2) {
             tmem_ld16_wait(ra);
             tmem_ld16_issue(col0 + 16 * (c + 1), rb16);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, mu[16 * c + i]));
+            for (int i = 0; i < 16; ++i) v[16 * c + i] = fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, neg_mu));
             tmem_ld16_wait(rb16);
-            if (c + 2 < 4) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
+            if (c + 2 < 8) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(rb16[i]), a.scale_log2, mu[16 * (c + 1) + i]));
+            for (int i = 0; i < 16; ++i) v[16 * (c + 1) + i] = fast_exp2(fmaf(__uint_as_float(rb16[i]), a.scale_log2, neg_mu));
           }
-          s = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 128; ++i) v[i] = 0.f;
         }
-        float* xs = reinterpret_cast<float*>(xch) + b * 128;
-        if (eg == 1) xs[lrow] = s;
-        unsigned stop;                                         // barrier over the 8 epilogue warps + agreement on giving up
+        fence_before();                                        // the accumulator buffer is free again
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(b));
+#pragma unroll
+        for (int bit = 16, width = 64; bit >= 1; bit >>= 1, width >>= 1) {
+          const bool upper = (lane & bit) != 0;
+#pragma unroll
+          for (int e = 0; e < width; ++e) {
+            const float send = upper ? v[e] : v[e + width];
+            const float keep = upper ? v[e + width] : v[e];
+            v[e] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
+          }
+        }
+        // the lane now holds the sums over its warp's 32 rows of four consecutive candidates
+        const int colbase = ((lane >> 4) & 1) * 64 + ((lane >> 3) & 1) * 32 + ((lane >> 2) & 1) * 16 + ((lane >> 1) & 1) * 8 +
+                            (lane & 1) * 4;
+        float* rg = red + ((it & 1) * 2 + eg) * 4 * 128;       // double-buffered by tile parity: one barrier per tile
+        *reinterpret_cast<float4*>(rg + (warp & 3) * 128 + colbase) = make_float4(v[0], v[1], v[2], v[3]);
+        unsigned stop;                                         // barrier over the group's 4 warps + agreement on giving up
         asm volatile(
             "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
-            "bar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(stop) : "r"((unsigned)(!landed || *abort_flag)) : "memory");
-        if (eg == 0 && !stop && cand < Le)
-          a.cpart[((long long)z * a.RB + rb) * a.buf.c_stride + cand] = s + xs[lrow];
+            "bar.red.or.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(stop) : "r"((unsigned)(!landed || *abort_flag)), "r"(1 + eg) : "memory");
+        if (!stop && cand0 + lrow < Le)
+          a.cpart[((long long)z * a.RB + rb) * a.buf.c_stride + cand0 + lrow] =
+              (rg[lrow] + rg[128 + lrow]) + (rg[256 + lrow] + rg[384 + lrow]);
         if (stop) { *abort_flag = 1; ok = false; }
       }
-      fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(b));
+      if (PASS == 1) {
+        fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(b));
+      }
       if (!ok) break;
     }
     if (!ok) *abort_flag = 1;
@@ -276,7 +294,8 @@ __global__ void score_rowblock_reduce_kernel(const float* __restrict__ cpart, fl
 }
 
 size_t wide_smem_bytes(int NH, int NS) {
-  return (size_t)NH * QH_B + NS * STAGE_B + 128 * sizeof(float) + 128 * sizeof(float2) + (2 * NS + 5) * 8 + 16 + 1024;
+  return (size_t)NH * QH_B + NS * STAGE_B + 128 * sizeof(float) + 128 * sizeof(float2) + 2 * 2 * 4 * 128 * sizeof(float) +
+         (2 * NS + 5) * 8 + 16 + 1024;
 }
 
 // SNAP_WIDE_STAGES caps the ring depth (tuning aid).
@@ -322,7 +341,7 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.b = b; a.buf = buf; a.cpart = cpart; a.status = status;
 
-  CUtensorMap tq, tk1, tk2;
+  CUtensorMap tq, tk1;
   const cuuint32_t estr2[2] = {1, 1}, estr3[3] = {1, 1, 1};
   {
     const cuuint64_t dims[2] = {(cuuint64_t)s.d_qk, (cuuint64_t)(b.first_seq + b.n) * s.Hq * s.Lo};
@@ -338,13 +357,11 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   const long long head_stride = src.k_head_stride >= s.d_qk ? src.k_head_stride : s.d_qk;
   const cuuint64_t kdims[3] = {(cuuint64_t)s.d_qk, (cuuint64_t)s.Hkv, (cuuint64_t)tokens};
   const cuuint64_t kstrides[2] = {(cuuint64_t)head_stride * 2, (cuuint64_t)src.k_tok_stride * 2};
-  for (int pass = 1; pass <= 2; ++pass) {
-    const cuuint32_t box[3] = {64, 1, (cuuint32_t)(pass == 1 ? 256 : 128)};
-    if (enc(pass == 1 ? &tk1 : &tk2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(src.k), kdims, kstrides,
-            box, estr3, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaErrorInvalidValue;
-  }
+  const cuuint32_t kbox[3] = {64, 1, 256};                     // one 64-dim slab of a 256-candidate tile
+  if (enc(&tk1, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(src.k), kdims, kstrides, kbox, estr3,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
   const size_t smem = wide_smem_bytes(a.NH, a.NS);
   static SmemLimit limit1 = {}, limit2 = {};
   if (cudaError_t e = ensure_dyn_smem(score_umma_wide_kernel<1>, smem, limit1)) return e;
@@ -358,7 +375,7 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   count_launch();
   cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
   if (e != cudaSuccess) return e;
-  score_umma_wide_kernel<2><<<grid, NTHREADS, smem, st>>>(a, tq, tk2);
+  score_umma_wide_kernel<2><<<grid, NTHREADS, smem, st>>>(a, tq, tk1);
   count_launch();
   score_rowblock_reduce_kernel<<<dim3((max_le + 255) / 256, nz), 256, 0, st>>>(cpart, buf.C, a.RB, buf.c_stride, b,
                                                                             s.Hkv, s.Ls, s.Lr);
