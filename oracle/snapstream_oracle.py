@@ -37,7 +37,9 @@ Parity pins (tests/test_oracle_*.py): Fig. 4's worked ring example, Eq. 3 agains
 the closed-form slot map, the appendix's valid_topk expression, the
 hyper-parameter table totals, sum_j C = Lo*g, the weighted pooled-sum identity,
 the all-equal tie pattern, brute-force top-k, the single-row softmax special case
-against scipy, dense-attention equalities, permutation invariance.
+against scipy, dense-attention equalities, permutation invariance; prefill attention
+against torch's double-precision causal routine, the running-mean closed form and
+causality; the Eq. 4 normalisers against scipy's logsumexp and by rebuilding Eq. 1.
 Parity unpinned by the paper (fixed only by the readings above): which softmax
 domain, pooling domain, GQA reduction order and ring-fill convention the
 authors' own implementation uses.
@@ -359,3 +361,47 @@ def expected_cache_position_order(seq: OracleSequence):
                 Kc[kvh, s] = seq.k_hist[p][kvh]
                 Vc[kvh, s] = seq.v_hist[p][kvh]
     return Kc, (None if cfg.v_aliases_k else Vc), pos_map
+
+
+# ----------------------------------------------------------------------------
+# Prefill attention that also yields Eq. 4's normalisers (the step Section 3.2.2
+# leaves to future optimisation: the scores' denominators are by-products of the
+# prompt's own causal attention pass).
+# ----------------------------------------------------------------------------
+
+def prefill_attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, cfg: OracleConfig) -> np.ndarray:
+    """Causal attention of a whole prompt, plain definition: query position t of head h
+    attends over key positions 0..t of KV head h // g.
+
+    q: [L, Hq, d_qk], k: [L, Hkv, d_qk], v: [L, Hkv, d_v]  ->  float64 [L, Hq, d_v].
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    L = q.shape[0]
+    out = np.zeros((L, cfg.n_q_heads, v.shape[2]), dtype=np.float64)
+    for h in range(cfg.n_q_heads):
+        kvh = h // cfg.group
+        for t in range(L):
+            out[t, h] = attention_over(q[t, h], k[: t + 1, kvh], v[: t + 1, kvh], cfg.softmax_scale)
+    return out
+
+
+def candidate_log2_normalisers(q_obs: np.ndarray, k: np.ndarray, cfg: OracleConfig) -> np.ndarray:
+    """mu[h, i] = log2 sum_{j in [Ls, L-Lr)} exp(scale * q_obs[h, i] . k_j): the denominator of
+    Eq. 4 for window row i of head h, as a base-2 logarithm, so that the Eq. 4 weight of
+    candidate j is 2 ** (log2(e) * scale * q.k_j - mu).  -> float64 [Hq, Lo]; -inf where the
+    prompt has no candidate."""
+    q_obs = np.asarray(q_obs, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    L = k.shape[0]
+    lo, hi = cfg.l_sink, L - cfg.l_recent
+    mu = np.full((cfg.n_q_heads, cfg.l_obs), -np.inf, dtype=np.float64)
+    if hi <= lo:
+        return mu
+    for h in range(cfg.n_q_heads):
+        kvh = h // cfg.group
+        S = cfg.softmax_scale * (q_obs[h] @ k[lo:hi, kvh].T)           # [Lo, Le]
+        m = S.max(axis=1)
+        mu[h] = (m + np.log(np.exp(S - m[:, None]).sum(axis=1))) / np.log(2.0)
+    return mu

@@ -446,3 +446,53 @@ def test_position_order_image_equals_repeated_array_concatenation():
             assert sorted(pm[kvh].tolist()) == sorted(pr[kvh].tolist())
         if (seq.n_tokens - Ls) % Lr == 0:
             np.testing.assert_array_equal(Kr, Kp)
+
+
+# ------------------------------------------------------------------ prefill attention + Eq. 4 normalisers
+
+def test_prefill_attention_matches_the_library_causal_routine_and_closed_forms():
+    import torch
+    cfg = _cfg()
+    rng = np.random.default_rng(71)
+    L = 37
+    q = rng.standard_normal((L, cfg.n_q_heads, cfg.d_qk))
+    k = rng.standard_normal((L, cfg.n_kv_heads, cfg.d_qk))
+    v = rng.standard_normal((L, cfg.n_kv_heads, cfg.d_v))
+    out = orc.prefill_attention(q, k, v, cfg)
+    # library routine: torch's fused causal attention in double precision, heads expanded
+    tq = torch.from_numpy(q).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(k).permute(1, 0, 2).repeat_interleave(cfg.group, dim=0)[None]
+    tv = torch.from_numpy(v).permute(1, 0, 2).repeat_interleave(cfg.group, dim=0)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True, scale=cfg.softmax_scale)
+    np.testing.assert_allclose(out, ref[0].permute(1, 0, 2).numpy(), rtol=1e-12, atol=1e-13)
+    # the first token sees only itself
+    for h in range(cfg.n_q_heads):
+        np.testing.assert_allclose(out[0, h], v[0, h // cfg.group], rtol=0, atol=1e-15)
+    # equal keys: uniform weights, the output is the running mean of the values
+    k_same = np.broadcast_to(k[:1], k.shape)
+    out_same = orc.prefill_attention(q, k_same, v, cfg)
+    running = np.cumsum(v, axis=0) / np.arange(1, L + 1)[:, None, None]
+    for h in range(cfg.n_q_heads):
+        np.testing.assert_allclose(out_same[:, h], running[:, h // cfg.group], rtol=1e-12, atol=1e-13)
+    # a future token cannot change an earlier row
+    k2, v2 = k.copy(), v.copy()
+    k2[20:] += 3.0
+    v2[20:] -= 5.0
+    np.testing.assert_array_equal(orc.prefill_attention(q, k2, v2, cfg)[:20], out[:20])
+
+
+def test_candidate_normalisers_are_the_library_logsumexp_and_rebuild_eq1():
+    cfg = _cfg()
+    L = 61
+    q, k, _ = _rand_prompt(cfg, L, seed=72, sharp=2.0)
+    mu = orc.candidate_log2_normalisers(q, k, cfg)
+    lo, hi = cfg.l_sink, L - cfg.l_recent
+    C = np.zeros((cfg.n_kv_heads, hi - lo))
+    for h in range(cfg.n_q_heads):
+        S = cfg.softmax_scale * np.einsum("id,jd->ij", q[h], k[lo:hi, h // cfg.group])
+        np.testing.assert_allclose(mu[h], scipy.special.logsumexp(S, axis=1) / math.log(2.0), rtol=1e-13)
+        C[h // cfg.group] += np.exp2(S * math.log2(math.e) - mu[h][:, None]).sum(axis=0)
+    # weights rebuilt from the normalisers are Eq. 4's, so their window sum is Eq. 1
+    np.testing.assert_allclose(C, orc.observation_scores(q, k, cfg), rtol=1e-11)
+    # a prompt that fits the budget has no candidate
+    assert np.all(np.isneginf(orc.candidate_log2_normalisers(q, k[: cfg.l_sink + cfg.l_recent], cfg)))
