@@ -14,8 +14,10 @@
  *                       per sequence over the valid cache slots
  *
  * and, around it: snap_decode_attn_multi (several new tokens per sequence and step),
- * snap_decode_attn_static (the decode step without a caller-provided scratch buffer) and
- * snap_append_kv_concat (the slice-and-concatenate update of Section 3.2.1, as a baseline).
+ * snap_decode_attn_static (the decode step without a caller-provided scratch buffer),
+ * snap_append_kv_concat (the slice-and-concatenate update of Section 3.2.1, as a baseline),
+ * and snap_prefill_attn + snap_compress_with_row_stats (the prompt's causal attention emitting
+ * the normalisers of Eq. 4, and the compression that consumes them).
  *
  * Conventions
  *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are plain
@@ -131,6 +133,52 @@ int64_t snap_decode_workspace_bytes(const snap_config_t* cfg, int32_t n_active);
  */
 int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout,
                   const void* q_obs_dev,
+                  const void* k_dev, int64_t k_token_stride, int64_t k_head_stride,
+                  const void* v_dev, int64_t v_token_stride, int64_t v_head_stride,
+                  const int32_t* cu_seqlens_host, const int32_t* slot_ids_host, int32_t n_seq,
+                  void* k_cache_dev, void* v_cache_dev,
+                  int32_t* seq_len_dev, int32_t* valid_topk_dev,
+                  int32_t* topk_idx_dev,
+                  void* workspace_dev, size_t workspace_bytes,
+                  uint32_t* status_dev, void* cuda_stream);
+
+/*
+ * Causal attention of n_seq whole prompts that also yields the denominators of Eq. 4
+ * (Section 3.2.2 names the score recomputation as the step left to optimise: the normalisers
+ * of the observation window's scores are by-products of the prompt's own attention pass).
+ *
+ *   q_dev     [T][Hq][d_qk] dense, token-major and ragged like k_dev (T = cu[n_seq]); the
+ *             queries after positional encoding
+ *   k_dev, v_dev and their strides: as in snap_compress
+ *   out_dev   [T][Hq][d_v] dense: row t of head h is softmax(scale * q_t . K[0..t]^T) V[0..t]
+ *             over the keys of KV head h / (Hq/Hkv) of the same prompt
+ *   row_mu_dev  NULL, or [n_seq][Hq][Lo] float: for the prompt's last Lo positions (entry i is
+ *             position L - Lo + i; entries of positions below 0 are left untouched)
+ *               log2( sum over candidates j in [Ls, L - Lr) of exp(scale * q . k_j) ),
+ *             -inf when the prompt has no candidate.  This is what snap_compress_with_row_stats
+ *             takes in place of its own first pass over the keys.
+ * Built for bf16 layers with d_qk = d_v = 128 and separate V (SNAP_ERR_UNSUPPORTED otherwise).
+ * Needs no workspace.  Only the model-shape fields, l_sink, l_recent, l_obs and softmax_scale
+ * of cfg are used.
+ */
+int snap_prefill_attn(const snap_config_t* cfg, const void* q_dev,
+                      const void* k_dev, int64_t k_token_stride, int64_t k_head_stride,
+                      const void* v_dev, int64_t v_token_stride, int64_t v_head_stride,
+                      const int32_t* cu_seqlens_host, int32_t n_seq,
+                      void* out_dev, float* row_mu_dev,
+                      uint32_t* status_dev, void* cuda_stream);
+
+/*
+ * snap_compress with the Eq. 4 normalisers supplied by the caller (row_mu_dev as written by
+ * snap_prefill_attn; NULL = compute them here, which is snap_compress): the score kernel then
+ * makes one pass over the candidate keys instead of two.  Same arguments, results, workspace
+ * and errors as snap_compress otherwise.  Consumed by the tensor-core score kernels (bf16,
+ * d_qk a multiple of 64 up to 576); SNAP_ERR_UNSUPPORTED for other layers when a prompt has to
+ * be scored.  The selection can differ from snap_compress's only where two pooled scores are
+ * equal to within single-precision rounding.
+ */
+int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* layout,
+                  const void* q_obs_dev, const float* row_mu_dev,
                   const void* k_dev, int64_t k_token_stride, int64_t k_head_stride,
                   const void* v_dev, int64_t v_token_stride, int64_t v_head_stride,
                   const int32_t* cu_seqlens_host, const int32_t* slot_ids_host, int32_t n_seq,

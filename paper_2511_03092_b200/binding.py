@@ -66,6 +66,11 @@ def lib() -> C.CDLL:
     L.snap_compress.restype = C.c_int
     L.snap_compress.argtypes = [pcfg, play, vp, vp, i64, i64, vp, i64, i64, C.POINTER(i32), C.POINTER(i32), i32,
                                 vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    L.snap_compress_with_row_stats.restype = C.c_int
+    L.snap_compress_with_row_stats.argtypes = [pcfg, play, vp, vp, vp, i64, i64, vp, i64, i64, C.POINTER(i32),
+                                               C.POINTER(i32), i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    L.snap_prefill_attn.restype = C.c_int
+    L.snap_prefill_attn.argtypes = [pcfg, vp, vp, i64, i64, vp, i64, i64, C.POINTER(i32), i32, vp, vp, vp, vp]
     L.snap_append_kv.restype = C.c_int
     L.snap_append_kv.argtypes = [pcfg, play, vp, vp, vp, i32, vp, vp, vp, vp, vp]
     L.snap_append_kv_concat.restype = C.c_int
@@ -85,7 +90,7 @@ def lib() -> C.CDLL:
 EXPORTS = ("snap_cache_layout", "snap_compress_workspace_bytes", "snap_decode_workspace_bytes",
            "snap_compress", "snap_append_kv", "snap_append_kv_concat", "snap_decode_attn",
            "snap_decode_multi_workspace_bytes", "snap_decode_attn_multi", "snap_decode_attn_static", "snap_status_string",
-           "snap_kernel_launch_count")
+           "snap_kernel_launch_count", "snap_prefill_attn", "snap_compress_with_row_stats")
 
 
 def status_string(code: int) -> str:
@@ -163,6 +168,32 @@ def snap_compress(cfg: SnapConfig, layout: SnapLayout, q_obs, k, v, cu_seqlens: 
                                vs[0], vs[1], cu, sl, len(slot_ids), _ptr(k_cache), _ptr(v_cache),
                                _ptr(seq_len), _ptr(valid_topk), _ptr(topk_idx), _ptr(workspace), ws_bytes,
                                _ptr(status), _stream(stream)), "snap_compress")
+
+
+def snap_compress_with_row_stats(cfg: SnapConfig, layout: SnapLayout, q_obs, row_mu, k, v, cu_seqlens: Sequence[int],
+                                 slot_ids: Sequence[int], k_cache, v_cache, seq_len, valid_topk, topk_idx=None,
+                                 workspace=None, status=None, stream=None) -> None:
+    """snap_compress with the Eq. 4 normalisers (row_mu: [n_seq, Hq, Lo] float32, as written by
+    snap_prefill_attn) supplied instead of computed."""
+    vs = (v.stride(0), v.stride(1)) if v is not None else (0, 0)
+    cu = _i32_array(cu_seqlens)
+    sl = _i32_array(slot_ids)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().snap_compress_with_row_stats(C.byref(cfg), C.byref(layout), _ptr(q_obs), _ptr(row_mu), _ptr(k),
+                                              k.stride(0), k.stride(1), _ptr(v), vs[0], vs[1], cu, sl, len(slot_ids),
+                                              _ptr(k_cache), _ptr(v_cache), _ptr(seq_len), _ptr(valid_topk),
+                                              _ptr(topk_idx), _ptr(workspace), ws_bytes, _ptr(status),
+                                              _stream(stream)), "snap_compress_with_row_stats")
+
+
+def snap_prefill_attn(cfg: SnapConfig, q, k, v, cu_seqlens: Sequence[int], out, row_mu=None, status=None,
+                      stream=None) -> None:
+    """Causal attention of whole prompts.  q: [T, Hq, d] dense; k, v: [T, Hkv, d] (dense last dim);
+    out: [T, Hq, d_v]; row_mu: None or [n_seq, Hq, Lo] float32 receiving the Eq. 4 normalisers."""
+    cu = _i32_array(cu_seqlens)
+    _check(lib().snap_prefill_attn(C.byref(cfg), _ptr(q), _ptr(k), k.stride(0), k.stride(1), _ptr(v), v.stride(0),
+                                   v.stride(1), cu, len(cu_seqlens) - 1, _ptr(out), _ptr(row_mu), _ptr(status),
+                                   _stream(stream)), "snap_prefill_attn")
 
 
 def snap_append_kv(cfg: SnapConfig, layout: SnapLayout, k_new, v_new, slot_ids_dev, n_active: int, k_cache,

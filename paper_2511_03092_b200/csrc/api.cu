@@ -248,6 +248,55 @@ int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout, const v
                   void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
                   int32_t* valid_topk_dev, int32_t* topk_idx_dev, void* workspace_dev,
                   size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
+  return snap_compress_with_row_stats(cfg, layout, q_obs_dev, nullptr, k_dev, k_token_stride, k_head_stride, v_dev,
+                                      v_token_stride, v_head_stride, cu_seqlens_host, slot_ids_host, n_seq, k_cache_dev,
+                                      v_cache_dev, seq_len_dev, valid_topk_dev, topk_idx_dev, workspace_dev,
+                                      workspace_bytes, status_dev, cuda_stream);
+}
+
+int snap_prefill_attn(const snap_config_t* cfg, const void* q_dev,
+                      const void* k_dev, int64_t k_token_stride, int64_t k_head_stride,
+                      const void* v_dev, int64_t v_token_stride, int64_t v_head_stride,
+                      const int32_t* cu_seqlens_host, int32_t n_seq, void* out_dev, float* row_mu_dev,
+                      uint32_t* status_dev, void* cuda_stream) {
+  int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  rc = check_cu(cu_seqlens_host, n_seq);
+  if (rc != SNAP_OK) return rc;
+  const Shape s = make_shape(cfg);
+  if (!prefill_attn_supported(cfg->dtype, s)) return SNAP_ERR_UNSUPPORTED;
+  if (n_seq == 0 || cu_seqlens_host[n_seq] == cu_seqlens_host[0]) return SNAP_OK;
+  if (!q_dev || !k_dev || !v_dev || !out_dev) return SNAP_ERR_NULL_POINTER;
+  if ((k_token_stride * 2) % 16 || (k_head_stride * 2) % 16 || k_token_stride < s.d_qk || (v_token_stride * 2) % 16 ||
+      (v_head_stride * 2) % 16 || v_token_stride < s.d_v)
+    return SNAP_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVSource src;
+  src.k = k_dev; src.v = v_dev;
+  src.k_tok_stride = k_token_stride; src.k_head_stride = k_head_stride;
+  src.v_tok_stride = v_token_stride; src.v_head_stride = v_head_stride;
+  for (int first = 0; first < n_seq; first += kMaxBatchSeqs) {
+    const int n = n_seq - first < kMaxBatchSeqs ? n_seq - first : kMaxBatchSeqs;
+    SeqBatch b;
+    std::memset(&b, 0, sizeof(b));
+    b.n = n; b.first_seq = first;
+    for (int i = 0; i < n; ++i) {
+      b.tok_off[i] = cu_seqlens_host[first + i];
+      b.len[i] = cu_seqlens_host[first + i + 1] - cu_seqlens_host[first + i];
+    }
+    if (launch_prefill_attn(s, b, q_dev, src, out_dev, row_mu_dev, status_dev, st) != cudaSuccess) return SNAP_ERR_CUDA;
+  }
+  return SNAP_OK;
+}
+
+int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_obs_dev,
+                                 const float* row_mu_dev,
+                                 const void* k_dev, int64_t k_token_stride, int64_t k_head_stride,
+                                 const void* v_dev, int64_t v_token_stride, int64_t v_head_stride,
+                                 const int32_t* cu_seqlens_host, const int32_t* slot_ids_host, int32_t n_seq,
+                                 void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
+                                 int32_t* valid_topk_dev, int32_t* topk_idx_dev, void* workspace_dev,
+                                 size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
   int rc = validate(cfg);
   if (rc != SNAP_OK) return rc;
   if (!layout || !slot_ids_host) return SNAP_ERR_NULL_POINTER;
@@ -279,6 +328,8 @@ int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout, const v
     if (s.K > 0 && L - s.Ls - s.Lr > s.K) any_scored = true;
   }
   if (any_scored && !q_obs_dev) return SNAP_ERR_NULL_POINTER;
+  // normalisers from outside are consumed by the tcgen05 score kernels only
+  if (any_scored && row_mu_dev && !use_umma(cfg->dtype, s) && !use_umma_wide(cfg->dtype, s)) return SNAP_ERR_UNSUPPORTED;
   if ((any_scored || !topk_idx_dev) && s.K > 0) {
     if (!workspace_dev) return SNAP_ERR_NULL_POINTER;
     if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
@@ -317,6 +368,7 @@ int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout, const v
       buf.C = reinterpret_cast<float*>(chunk_ws + p.c_off);
       buf.P = reinterpret_cast<float*>(chunk_ws + p.p_off);
       buf.c_stride = p.c_stride; buf.nsplit = p.nsplit;
+      buf.ext_mu = row_mu_dev;
       const cudaError_t e = use_umma(cfg->dtype, s)  ? launch_score_umma(s, b, q_obs_dev, src, buf, status_dev, st)
                             : use_umma_wide(cfg->dtype, s)
                                 ? launch_score_umma_wide(s, b, q_obs_dev, src, buf,

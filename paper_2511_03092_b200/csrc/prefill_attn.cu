@@ -1,0 +1,401 @@
+// Causal prefill attention on tcgen05 that also emits the normalisers of Eq. 4 for the
+// observation window (Section 3.2.2 leaves the score recomputation as a step to optimise: the
+// denominators of the scores are by-products of the prompt's own attention pass, so the first of
+// the two passes of the score kernel can be dropped when the prompt's attention ran here).
+//
+// One CTA computes 128 query rows of one head against key tiles 0 .. its own (128 keys each):
+//   S = Q K^T      M = 128 rows, N = 128 keys, both operands K-major in shared memory
+//   O += P V       A = P from tensor memory (bf16 pairs written over the tile's own logits),
+//                  B = the V tile as loaded (MN-major)
+// Tensor memory: S0 128 | S1 128 | O 128 columns; the next tile's logits are computed while the
+// softmax warps work on this one.  K and V tiles stream through a ring of four 32 KB stages in
+// the order the MMAs consume them: K(0), K(1), V(0), K(2), V(1), ...
+//   warp 0      TMA producer
+//   warp 1      MMA issuer (whole warp converged, instructions predicated on one lane)
+//   warps 2-5   thread = query row: online softmax in the log2 domain with a lazily refreshed
+//               reference (O is rescaled in tensor memory only when a logit exceeds it by 8)
+// Rows of the last Lo positions also accumulate the same exponentials over the eviction
+// candidates [Ls, L - Lr) alone; reference + log2 of that sum is what Eq. 4 divides by.
+// Every mbarrier wait is bounded; one that runs out raises SNAP_DEV_WAIT_TIMEOUT.
+#include "snap_internal.cuh"
+#include "umma_helpers.cuh"
+
+namespace snap {
+namespace {
+
+using namespace umma;
+
+constexpr int D = 128, BM = 128, BN = 128, NSTG = 4, NTH = 192;
+constexpr int SLAB_B = 128 * 128, TILE_B = 2 * SLAB_B;           // a tile = two 64-dim slabs of 128 rows x 128 B
+constexpr uint32_t COL_S = 0, COL_O = 256;
+
+struct PArgs {
+  SeqBatch b;
+  int Hq, g, Ls, Lr, Lo;
+  float scale_log2;
+  __nv_bfloat16* out;                          // [tokens][Hq][D]
+  float* mu;                                   // NULL or [prompts][Hq][Lo]
+  uint32_t* status;
+};
+
+__host__ __device__ constexpr uint32_t idesc_f16(int M, int N, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
+}
+// MN-major operand, 128-byte swizzle: 64 contiguous elements per row of the contraction dim,
+// 8-row groups 1024 bytes apart, the next 64 elements `lbo_bytes` further on.
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t saddr, uint32_t lbo_bytes) {
+  return (uint64_t)((saddr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+         ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void mma_ss_pred(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc,
+                                            uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void mma_ts_pred(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc,
+                                            uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void commit_pred(uint32_t bar, uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ bool wait_warp(uint32_t bar, unsigned parity, volatile int* abort_flag) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+}
+
+__global__ void __launch_bounds__(NTH, 1)
+prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                    const __grid_constant__ CUtensorMap tmap_v) {
+  const int seq = blockIdx.z, head = blockIdx.y;
+  const int L = a.b.len[seq];
+  const int n_qt = (L + BM - 1) / BM;
+  if ((int)blockIdx.x >= n_qt) return;                         // the grid is sized for the longest prompt
+  const int qt = n_qt - 1 - (int)blockIdx.x;                   // longest rows first
+  const int q0 = qt * BM, nt = qt + 1;
+  const int tok0 = a.b.tok_off[seq], kvh = head / a.g;
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* Qs = smem;                                    // [2 slabs][128 rows][128 B]
+  unsigned char* Rs = Qs + TILE_B;                             // [NSTG][32 KB] ring
+  uint64_t* bars = reinterpret_cast<uint64_t*>(Rs + NSTG * TILE_B);
+  // full[NSTG] empty[NSTG] s_full[2] p_ready[2] pv_done[2] q_full
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTG + 7);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8 * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8 * (NSTG + s); };
+  auto sfull_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + b); };
+  auto pready_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 2 + b); };
+  auto pvdone_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 4 + b); };
+  const uint32_t qfull_bar = bar0 + 8 * (2 * NSTG + 6);
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < NSTG; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(sfull_bar(b), 1); mbar_init(pready_bar(b), 4); mbar_init(pvdone_bar(b), 1); }
+    mbar_init(qfull_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      mbar_expect_tx(qfull_bar, (unsigned)TILE_B);
+      for (int h = 0; h < 2; ++h) tma_load_3d(smem_u32(Qs) + h * SLAB_B, &tmap_q, h * 64, head, tok0 + q0, qfull_bar);
+      int q = 0;                                               // stages issued so far
+      bool ok = true;
+      auto load_tile = [&](const CUtensorMap* map, int it) {
+        const int s = q % NSTG;
+        if (!mbar_wait(empty_bar(s), ((unsigned)(q / NSTG) & 1u) ^ 1u, abort_flag)) { *abort_flag = 1; ok = false; return; }
+        mbar_expect_tx(full_bar(s), (unsigned)TILE_B);
+        for (int h = 0; h < 2; ++h)
+          tma_load_3d(smem_u32(Rs) + s * TILE_B + h * SLAB_B, map, h * 64, kvh, tok0 + it * BN, full_bar(s));
+        ++q;
+      };
+      load_tile(&tmap_k, 0);
+      for (int it = 0; it < nt && ok; ++it) {
+        if (it + 1 < nt) load_tile(&tmap_k, it + 1);
+        if (ok) load_tile(&tmap_v, it);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    const uint32_t leader = lane == 0;
+    const uint32_t idesc_s = idesc_f16(BM, BN, false), idesc_pv = idesc_f16(BM, D, true);
+    const uint64_t qd0 = smem_desc(smem_u32(Qs));
+    int q = 0;                                                 // stages consumed so far
+    bool ok = wait_warp(qfull_bar, 0u, abort_flag);
+    fence_after();
+    auto issue_s = [&](int it) -> bool {                      // S[it & 1] = Q K(it)^T
+      const int s = q % NSTG;
+      if (!wait_warp(full_bar(s), (unsigned)(q / NSTG) & 1u, abort_flag)) return false;
+      fence_after();
+      const uint32_t sd = tmem_base + COL_S + (it & 1) * BN;
+      const uint64_t kd0 = smem_desc(smem_u32(Rs) + s * TILE_B);
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          mma_ss_pred(sd, qd0 + (uint64_t)((h * SLAB_B) >> 4) + (uint64_t)(ks * 2),
+                      kd0 + (uint64_t)((h * SLAB_B) >> 4) + (uint64_t)(ks * 2), idesc_s, (h | ks) != 0, leader);
+      commit_pred(empty_bar(s), leader);
+      commit_pred(sfull_bar(it & 1), leader);
+      ++q;
+      return true;
+    };
+    if (ok) ok = issue_s(0);
+    for (int it = 0; it < nt && ok; ++it) {
+      const int b = it & 1;
+      if (it + 1 < nt) { ok = issue_s(it + 1); if (!ok) break; }
+      ok = wait_warp(pready_bar(b), (unsigned)(it / 2) & 1u, abort_flag);
+      if (!ok) break;
+      const int s = q % NSTG;
+      ok = wait_warp(full_bar(s), (unsigned)(q / NSTG) & 1u, abort_flag);
+      if (!ok) break;
+      fence_after();
+      const uint32_t vst = smem_u32(Rs) + s * TILE_B;
+      const int tile_nrows = L - it * BN;
+      if (tile_nrows < BN) {
+        // rows past the prompt's end hold another prompt's tokens or nothing at all, and a zero
+        // probability does not silence a NaN in V: clear them before the tensor core reads
+        for (int e = lane; e < (BN - tile_nrows) * 16; e += 32) {
+          const int r = tile_nrows + e / 16, j = (e / 8) % 2, ch = e % 8;
+          *reinterpret_cast<uint4*>(Rs + s * TILE_B + j * SLAB_B + r * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+      }
+      const uint32_t pa = tmem_base + COL_S + b * BN;         // P(it) lies over the first 64 columns of S(it)
+#pragma unroll
+      for (int ks = 0; ks < BN / 16; ++ks)                    // O += P(it) V(it), 16 keys per instruction
+        mma_ts_pred(tmem_base + COL_O, pa + 8 * ks, smem_desc_mn(vst + ks * 16 * 128, SLAB_B), idesc_pv, (it | ks) != 0, leader);
+      commit_pred(empty_bar(s), leader);
+      commit_pred(pvdone_bar(b), leader);
+      ++q;
+    }
+    if (!ok && lane == 0) *abort_flag = 1;
+  } else {
+    // ---------------- softmax warps: thread = query row ----------------
+    const int lrow = 32 * (warp & 3) + lane;                   // TMEM lane
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+    const int row = q0 + lrow;                                 // position within the prompt
+    // does this warp hold rows of the observation window?  (warp-uniform)
+    const int wrow0 = q0 + 32 * (warp & 3);
+    const bool warp_window = a.mu != nullptr && wrow0 + 31 >= L - a.Lo && wrow0 < L;
+    const int cand_lo = a.Ls, cand_n = L - a.Lr - a.Ls;        // candidates [cand_lo, cand_lo + cand_n)
+    float m_ref = -INFINITY, l_sum = 0.f, l_cand = 0.f;
+    bool ok = true;
+    for (int it = 0; it < nt; ++it) {
+      const int b = it & 1;
+      if (!wait_warp(sfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag)) { ok = false; break; }
+      fence_after();
+      const uint32_t s_addr = lane_addr + COL_S + b * BN;
+      float v[BN];
+      float mx = -INFINITY;
+      if (it == nt - 1) {
+        // the tile on the diagonal: key j of the tile is visible to row lrow iff j <= lrow
+#pragma unroll
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r0[16], r1[16];
+          tmem_ld16_issue(s_addr + 32 * c, r0);
+          tmem_ld16_issue(s_addr + 32 * c + 16, r1);
+          tmem_ld16_wait(r0);
+          tmem_ld16_wait(r1);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            v[32 * c + j] = 32 * c + j <= lrow ? __uint_as_float(r0[j]) * a.scale_log2 : -INFINITY;
+            v[32 * c + 16 + j] = 32 * c + 16 + j <= lrow ? __uint_as_float(r1[j]) * a.scale_log2 : -INFINITY;
+            mx = fmaxf(mx, fmaxf(v[32 * c + j], v[32 * c + 16 + j]));
+          }
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r0[16], r1[16];
+          tmem_ld16_issue(s_addr + 32 * c, r0);
+          tmem_ld16_issue(s_addr + 32 * c + 16, r1);
+          tmem_ld16_wait(r0);
+          tmem_ld16_wait(r1);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            v[32 * c + j] = __uint_as_float(r0[j]) * a.scale_log2;
+            v[32 * c + 16 + j] = __uint_as_float(r1[j]) * a.scale_log2;
+            mx = fmaxf(mx, fmaxf(v[32 * c + j], v[32 * c + 16 + j]));
+          }
+        }
+      }
+      // Lazy reference: refreshed (and O rescaled) only when some row of the warp sees a logit 8
+      // above its reference; the tensor-memory accesses are warp-collective, so the warp votes.
+      if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+        const float m_new = fmaxf(m_ref, mx);
+        const float alpha = m_ref == -INFINITY ? 0.f : exp2f(m_ref - m_new);
+        if (it > 0) {
+          if (!wait_warp(pvdone_bar((it - 1) & 1), (unsigned)((it - 1) / 2) & 1u, abort_flag)) { ok = false; break; }
+          fence_after();
+#pragma unroll 1
+          for (int c = 0; c < D / 16; ++c) {
+            uint32_t o[16];
+            tmem_ld16_issue(lane_addr + COL_O + 16 * c, o);
+            tmem_ld16_wait(o);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st16(lane_addr + COL_O + 16 * c, o);
+          }
+          tmem_st_wait();
+        }
+        l_sum *= alpha;
+        l_cand *= alpha;
+        m_ref = m_new;
+      }
+      const float mr = m_ref == -INFINITY ? 0.f : m_ref;
+      float ls0 = 0.f, ls1 = 0.f;
+      // this tile's overlap with the candidate range, as tile columns [clo, clo + cn)
+      const int clo = cand_lo - it * BN;
+      const unsigned cn = warp_window && cand_n > 0 ? (unsigned)cand_n : 0u;
+      // the logits of this tile are all in registers, so the probabilities may overwrite them
+#pragma unroll
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t pk[16];
+        float pc = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float p0 = fast_exp2(v[32 * c + 2 * j] - mr), p1 = fast_exp2(v[32 * c + 2 * j + 1] - mr);
+          ls0 += p0;
+          ls1 += p1;
+          if (warp_window) {
+            pc += (unsigned)(32 * c + 2 * j - clo) < cn ? p0 : 0.f;
+            pc += (unsigned)(32 * c + 2 * j + 1 - clo) < cn ? p1 : 0.f;
+          }
+          pk[j] = pack_bf16(p0, p1);
+        }
+        l_cand += pc;
+        tmem_st16(s_addr + 16 * c, pk);
+      }
+      l_sum += ls0 + ls1;
+      tmem_st_wait();
+      fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pready_bar(b));
+    }
+    if (!ok) *abort_flag = 1;
+    // ---------------- normalise and store ----------------
+    if (ok) ok = wait_warp(pvdone_bar((nt - 1) & 1), (unsigned)((nt - 1) / 2) & 1u, abort_flag);
+    if (!ok) *abort_flag = 1;
+    fence_after();
+    if (__all_sync(0xffffffffu, ok)) {
+      const float inv = 1.f / l_sum;
+      __nv_bfloat16* orow = a.out + ((long long)(tok0 + row) * a.Hq + head) * D;
+#pragma unroll 1
+      for (int c = 0; c < D / 16; ++c) {
+        uint32_t o[16];
+        tmem_ld16_issue(lane_addr + COL_O + 16 * c, o);
+        tmem_ld16_wait(o);
+        if (row < L) {
+          uint4 w0, w1;
+          w0.x = pack_bf16(__uint_as_float(o[0]) * inv, __uint_as_float(o[1]) * inv);
+          w0.y = pack_bf16(__uint_as_float(o[2]) * inv, __uint_as_float(o[3]) * inv);
+          w0.z = pack_bf16(__uint_as_float(o[4]) * inv, __uint_as_float(o[5]) * inv);
+          w0.w = pack_bf16(__uint_as_float(o[6]) * inv, __uint_as_float(o[7]) * inv);
+          w1.x = pack_bf16(__uint_as_float(o[8]) * inv, __uint_as_float(o[9]) * inv);
+          w1.y = pack_bf16(__uint_as_float(o[10]) * inv, __uint_as_float(o[11]) * inv);
+          w1.z = pack_bf16(__uint_as_float(o[12]) * inv, __uint_as_float(o[13]) * inv);
+          w1.w = pack_bf16(__uint_as_float(o[14]) * inv, __uint_as_float(o[15]) * inv);
+          reinterpret_cast<uint4*>(orow + 16 * c)[0] = w0;
+          reinterpret_cast<uint4*>(orow + 16 * c)[1] = w1;
+        }
+      }
+      const int w = row - (L - a.Lo);
+      if (warp_window && row < L && w >= 0)
+        a.mu[((long long)(a.b.first_seq + seq) * a.Hq + head) * a.Lo + w] = l_cand > 0.f ? m_ref + log2f(l_cand) : -INFINITY;
+    }
+  }
+
+  fence_before();
+  __syncthreads();
+  fence_after();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
+}
+
+size_t prefill_smem_bytes() { return (size_t)TILE_B + NSTG * TILE_B + (2 * NSTG + 7) * 8 + 16 + 1024; }
+
+}  // namespace
+
+bool prefill_attn_supported(int dtype, const Shape& s) {
+  return dtype == SNAP_BF16 && !s.v_aliases_k && s.d_qk == D && s.d_v == D && umma::encode_tiled_fn() != nullptr;
+}
+
+cudaError_t launch_prefill_attn(const Shape& s, const SeqBatch& b, const void* q, const KVSource& src, void* out,
+                                float* mu, uint32_t* status, cudaStream_t st) {
+  long long tokens = 0;
+  int max_len = 0;
+  for (int i = 0; i < b.n; ++i) {
+    tokens = tokens > (long long)b.tok_off[i] + b.len[i] ? tokens : (long long)b.tok_off[i] + b.len[i];
+    max_len = max_len > b.len[i] ? max_len : b.len[i];
+  }
+  if (b.n == 0 || max_len == 0) return cudaSuccess;
+  umma::EncodeTiledFn enc = umma::encode_tiled_fn();
+  if (!enc) return cudaErrorNotSupported;
+  CUtensorMap tq, tk, tv;
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const cuuint32_t box[3] = {64, 1, (cuuint32_t)BM};
+  auto encode = [&](CUtensorMap* m, const void* base, int heads, long long head_stride, long long tok_stride) {
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)heads, (cuuint64_t)tokens};
+    const cuuint64_t strides[2] = {(cuuint64_t)(head_stride >= D ? head_stride : D) * 2, (cuuint64_t)tok_stride * 2};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  };
+  if (!encode(&tq, q, s.Hq, D, (long long)s.Hq * D) || !encode(&tk, src.k, s.Hkv, src.k_head_stride, src.k_tok_stride) ||
+      !encode(&tv, src.v, s.Hkv, src.v_head_stride, src.v_tok_stride))
+    return cudaErrorInvalidValue;
+  PArgs a;
+  a.b = b;
+  a.Hq = s.Hq; a.g = s.g; a.Ls = s.Ls; a.Lr = s.Lr; a.Lo = s.Lo;
+  a.scale_log2 = s.scale * 1.4426950408889634f;
+  a.out = static_cast<__nv_bfloat16*>(out);
+  a.mu = mu;
+  a.status = status;
+  const size_t smem = prefill_smem_bytes();
+  static SmemLimit limit = {};
+  if (cudaError_t e = ensure_dyn_smem(prefill_attn_kernel, smem, limit)) return e;
+  prefill_attn_kernel<<<dim3((max_len + BM - 1) / BM, s.Hq, b.n), NTH, smem, st>>>(a, tq, tk, tv);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace snap

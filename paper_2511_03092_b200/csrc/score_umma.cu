@@ -201,9 +201,15 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   pdl_wait();                                                 // everything above overlaps the previous kernel's tail
   float* mu_s = reinterpret_cast<float*>(stats_s);            // pass 2: m_i + log2(l_i) per query row
   if (PASS == 2) {
+    // the g * Lo rows of a KV head are consecutive in [prompt][Hq][Lo] order
+    const float* ext = a.buf.ext_mu ? a.buf.ext_mu + ((long long)(a.b.first_seq + seq) * a.Hq + kvh * a.g) * a.Lo : nullptr;
     for (int i = tid; i < R; i += NTHREADS) {
-      const float2 st = a.buf.stats[(long long)z * R + i];
-      mu_s[i] = st.x - log2f(st.y);
+      if (ext) {
+        mu_s[i] = ext[i];
+      } else {
+        const float2 st = a.buf.stats[(long long)z * R + i];
+        mu_s[i] = st.x - log2f(st.y);
+      }
     }
   }
   if (warp == 0) {                                            // tensor memory: 512 columns (2 x 256)
@@ -499,10 +505,12 @@ cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_o
   if (cudaError_t e = ensure_dyn_smem(score_umma_kernel<2>, kSmemBytes, limit2)) return e;
   const int nz = b.n_scored * s.Hkv;
   dim3 grid(buf.nsplit, nz);
-  if (launch_pdl(score_umma_kernel<1>, grid, dim3(NTHREADS), kSmemBytes, st, a, tq, tk) != cudaSuccess) return cudaGetLastError();
-  count_launch();
-  cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
-  if (e != cudaSuccess) return e;
+  if (!buf.ext_mu) {                                          // Eq. 4's normalisers: pass 1, unless the caller has them
+    if (launch_pdl(score_umma_kernel<1>, grid, dim3(NTHREADS), kSmemBytes, st, a, tq, tk) != cudaSuccess) return cudaGetLastError();
+    count_launch();
+    cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
+    if (e != cudaSuccess) return e;
+  }
   if (launch_pdl(score_umma_kernel<2>, grid, dim3(NTHREADS), kSmemBytes, st, a, tq, tk) != cudaSuccess) return cudaGetLastError();
   count_launch();
   return cudaGetLastError();

@@ -85,8 +85,12 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
     const int row = rb * 128 + tid;
     float mu = INFINITY;
     if (row < a.R) {
-      const float2 st = a.buf.stats[(long long)z * a.R + row];
-      mu = st.x - log2f(st.y);
+      if (a.buf.ext_mu) {                                      // [prompt][Hq][Lo]: a KV head's rows are consecutive
+        mu = a.buf.ext_mu[((long long)(a.b.first_seq + seq) * a.Hq + kvh * a.g) * a.Lo + row];
+      } else {
+        const float2 st = a.buf.stats[(long long)z * a.R + row];
+        mu = st.x - log2f(st.y);
+      }
     }
     mu_s[tid] = mu;
   }
@@ -371,10 +375,12 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   for (int i = 0; i < b.n; ++i)
     if (b.score_idx[i] >= 0) max_le = max_le > b.len[i] - s.Ls - s.Lr ? max_le : b.len[i] - s.Ls - s.Lr;
   dim3 grid(buf.nsplit, a.RB, nz);
-  score_umma_wide_kernel<1><<<grid, NTHREADS, smem, st>>>(a, tq, tk1);
-  count_launch();
-  cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
-  if (e != cudaSuccess) return e;
+  if (!buf.ext_mu) {                                          // Eq. 4's normalisers: pass 1, unless the caller has them
+    score_umma_wide_kernel<1><<<grid, NTHREADS, smem, st>>>(a, tq, tk1);
+    count_launch();
+    cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
+    if (e != cudaSuccess) return e;
+  }
   score_umma_wide_kernel<2><<<grid, NTHREADS, smem, st>>>(a, tq, tk1);
   count_launch();
   score_rowblock_reduce_kernel<<<dim3((max_le + 255) / 256, nz), 256, 0, st>>>(cpart, buf.C, a.RB, buf.c_stride, b,

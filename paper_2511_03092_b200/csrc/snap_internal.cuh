@@ -43,6 +43,8 @@ struct ScoreBuffers {
   float* P;             // [n_scored*Hkv][c_stride]   pooled scores
   int c_stride;         // floats per (prompt, kv head) row of C and P
   int nsplit;
+  const float* ext_mu;  // NULL, or [prompts][Hq][Lo] log2 normalisers of Eq. 4 computed elsewhere
+                        // (the prefill attention kernel): pass 1 and the combine step are skipped
 };
 
 extern unsigned long long g_launches;
@@ -103,6 +105,10 @@ int score_umma_wide_row_blocks(const Shape& s);
 int score_umma_wide_nsplit(const Shape& s, int n_scored, int max_le, int sm_count);
 cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
                                    const ScoreBuffers& buf, float* cpart, uint32_t* status, cudaStream_t st);
+// causal prefill attention on tcgen05 that also emits Eq. 4's normalisers (bf16, 128-wide heads)
+bool prefill_attn_supported(int dtype, const Shape& s);
+cudaError_t launch_prefill_attn(const Shape& s, const SeqBatch& b, const void* q, const KVSource& src, void* out,
+                                float* mu, uint32_t* status, cudaStream_t st);
 cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffers& buf,
                              int* idx_out, uint32_t* status, cudaStream_t st);
 cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KVSource& src,

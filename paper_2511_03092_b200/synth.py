@@ -156,6 +156,19 @@ def make_decode_inputs(wl: Workload, n: int, seed: int, step: int, device="cpu")
             "v_new": v}
 
 
+def make_prompt_queries(wl: Workload, prompt: dict, seed: int, device="cpu") -> torch.Tensor:
+    """Queries of every prompt position, [L, Hq, d_qk], for the prefill attention pass: random
+    rows whose last Lo positions are the prompt's observation queries."""
+    dev = torch.device(device)
+    L = prompt["k"].shape[0]
+    g = _gen(seed * 7 + 13, dev)
+    q = torch.randn(L, wl.n_q_heads, wl.d_qk, generator=g, device=dev).to(wl.torch_dtype)
+    n = min(L, wl.l_obs)
+    if n > 0:
+        q[L - n:] = prompt["q_obs"][:, wl.l_obs - n:].transpose(0, 1).to(dev)
+    return q.contiguous()
+
+
 def draw_prompt_lengths(wl: Workload, n: int, seed: int) -> List[int]:
     lo, hi = wl.prompt_len
     rng = np.random.default_rng(seed + 104729)
