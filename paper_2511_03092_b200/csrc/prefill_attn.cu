@@ -17,6 +17,8 @@
 // Rows of the last Lo positions also accumulate the same exponentials over the eviction
 // candidates [Ls, L - Lr) alone; reference + log2 of that sum is what Eq. 4 divides by.
 // Every mbarrier wait is bounded; one that runs out raises SNAP_DEV_WAIT_TIMEOUT.
+#include <cstdlib>
+
 #include "snap_internal.cuh"
 #include "umma_helpers.cuh"
 
@@ -25,7 +27,7 @@ namespace {
 
 using namespace umma;
 
-constexpr int D = 128, BM = 128, BN = 128, NSTG = 4, NTH = 192;
+constexpr int D = 128, BM = 128, BN = 128, NSTG = 4;
 constexpr int SLAB_B = 128 * 128, TILE_B = 2 * SLAB_B;           // a tile = two 64-dim slabs of 128 rows x 128 B
 constexpr uint32_t COL_S = 0, COL_O = 256;
 
@@ -85,21 +87,27 @@ __device__ __forceinline__ bool wait_warp(uint32_t bar, unsigned parity, volatil
   return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
 }
 
-__global__ void __launch_bounds__(NTH, 1)
+// NQ = 1: one head per CTA, S double-buffered (the next tile's logits are computed while the
+// softmax warps work on this one).  NQ = 2: two query heads of one KV head per CTA, each with
+// its own softmax warpgroup, S and O; they share every K and V tile, which halves the traffic
+// from L2 (what bounds the one-head kernel), and while one head's warps work the tensor core
+// serves the other head.
+template <int NQ>
+__global__ void __launch_bounds__(64 + 128 * NQ, 1)
 prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v) {
-  const int seq = blockIdx.z, head = blockIdx.y;
+  const int seq = blockIdx.z, head0 = blockIdx.y * NQ;
   const int L = a.b.len[seq];
   const int n_qt = (L + BM - 1) / BM;
   if ((int)blockIdx.x >= n_qt) return;                         // the grid is sized for the longest prompt
   const int qt = n_qt - 1 - (int)blockIdx.x;                   // longest rows first
   const int q0 = qt * BM, nt = qt + 1;
-  const int tok0 = a.b.tok_off[seq], kvh = head / a.g;
+  const int tok0 = a.b.tok_off[seq], kvh = head0 / a.g;
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char* Qs = smem;                                    // [2 slabs][128 rows][128 B]
-  unsigned char* Rs = Qs + TILE_B;                             // [NSTG][32 KB] ring
+  unsigned char* Qs = smem;                                    // [NQ heads][2 slabs][128 rows][128 B]
+  unsigned char* Rs = Qs + NQ * TILE_B;                        // [NSTG][32 KB] ring
   uint64_t* bars = reinterpret_cast<uint64_t*>(Rs + NSTG * TILE_B);
   // full[NSTG] empty[NSTG] s_full[2] p_ready[2] pv_done[2] q_full
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTG + 7);
@@ -113,6 +121,10 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
   auto pready_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 2 + b); };
   auto pvdone_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 4 + b); };
   const uint32_t qfull_bar = bar0 + 8 * (2 * NSTG + 6);
+  // S / P buffer, its barriers and their phase for tile `it` of head x:
+  //   NQ = 1: two buffers used alternately by the one head; NQ = 2: one buffer per head
+  auto buf_of = [&](int x, int it) { return NQ == 1 ? (it & 1) : x; };
+  auto phase_of = [&](int it) { return NQ == 1 ? ((unsigned)(it / 2) & 1u) : ((unsigned)it & 1u); };
 
   if (tid == 0) {
     *abort_flag = 0;
@@ -133,8 +145,10 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      mbar_expect_tx(qfull_bar, (unsigned)TILE_B);
-      for (int h = 0; h < 2; ++h) tma_load_3d(smem_u32(Qs) + h * SLAB_B, &tmap_q, h * 64, head, tok0 + q0, qfull_bar);
+      mbar_expect_tx(qfull_bar, (unsigned)(NQ * TILE_B));
+      for (int x = 0; x < NQ; ++x)
+        for (int h = 0; h < 2; ++h)
+          tma_load_3d(smem_u32(Qs) + x * TILE_B + h * SLAB_B, &tmap_q, h * 64, head0 + x, tok0 + q0, qfull_bar);
       int q = 0;                                               // stages issued so far
       bool ok = true;
       auto load_tile = [&](const CUtensorMap* map, int it) {
@@ -145,10 +159,17 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
           tma_load_3d(smem_u32(Rs) + s * TILE_B + h * SLAB_B, map, h * 64, kvh, tok0 + it * BN, full_bar(s));
         ++q;
       };
+      // in the order the MMA warp consumes: NQ = 1: K(0), K(1), V(0), K(2), V(1), ...
+      //                                     NQ = 2: K(0), V(0), K(1), V(1), ...
       load_tile(&tmap_k, 0);
       for (int it = 0; it < nt && ok; ++it) {
-        if (it + 1 < nt) load_tile(&tmap_k, it + 1);
-        if (ok) load_tile(&tmap_v, it);
+        if (NQ == 1) {
+          if (it + 1 < nt) load_tile(&tmap_k, it + 1);
+          if (ok) load_tile(&tmap_v, it);
+        } else {
+          load_tile(&tmap_v, it);
+          if (ok && it + 1 < nt) load_tile(&tmap_k, it + 1);
+        }
       }
     }
   } else if (warp == 1) {
@@ -159,34 +180,35 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
     int q = 0;                                                 // stages consumed so far
     bool ok = wait_warp(qfull_bar, 0u, abort_flag);
     fence_after();
-    auto issue_s = [&](int it) -> bool {                      // S[it & 1] = Q K(it)^T
-      const int s = q % NSTG;
-      if (!wait_warp(full_bar(s), (unsigned)(q / NSTG) & 1u, abort_flag)) return false;
+    auto wait_stage = [&]() -> bool {
+      const bool r = wait_warp(full_bar(q % NSTG), (unsigned)(q / NSTG) & 1u, abort_flag);
       fence_after();
-      const uint32_t sd = tmem_base + COL_S + (it & 1) * BN;
-      const uint64_t kd0 = smem_desc(smem_u32(Rs) + s * TILE_B);
+      return r;
+    };
+    auto issue_s = [&](int x, int it, int s) {                // S of head x = Q_x K(it)^T, K in stage s
+      const uint32_t sd = tmem_base + COL_S + buf_of(x, it) * BN;
+      const uint64_t kd0 = smem_desc(smem_u32(Rs) + s * TILE_B), qdx = qd0 + (uint64_t)((x * TILE_B) >> 4);
 #pragma unroll
       for (int h = 0; h < 2; ++h)
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          mma_ss_pred(sd, qd0 + (uint64_t)((h * SLAB_B) >> 4) + (uint64_t)(ks * 2),
+          mma_ss_pred(sd, qdx + (uint64_t)((h * SLAB_B) >> 4) + (uint64_t)(ks * 2),
                       kd0 + (uint64_t)((h * SLAB_B) >> 4) + (uint64_t)(ks * 2), idesc_s, (h | ks) != 0, leader);
-      commit_pred(empty_bar(s), leader);
-      commit_pred(sfull_bar(it & 1), leader);
-      ++q;
-      return true;
+      commit_pred(sfull_bar(buf_of(x, it)), leader);
     };
-    if (ok) ok = issue_s(0);
-    for (int it = 0; it < nt && ok; ++it) {
-      const int b = it & 1;
-      if (it + 1 < nt) { ok = issue_s(it + 1); if (!ok) break; }
-      ok = wait_warp(pready_bar(b), (unsigned)(it / 2) & 1u, abort_flag);
-      if (!ok) break;
-      const int s = q % NSTG;
-      ok = wait_warp(full_bar(s), (unsigned)(q / NSTG) & 1u, abort_flag);
-      if (!ok) break;
+    auto issue_pv = [&](int x, int it, int s) -> bool {       // O_x += P_x(it) V(it), V in stage s
+      if (!wait_warp(pready_bar(buf_of(x, it)), phase_of(it), abort_flag)) return false;
       fence_after();
       const uint32_t vst = smem_u32(Rs) + s * TILE_B;
+      const uint32_t pa = tmem_base + COL_S + buf_of(x, it) * BN;   // P lies over the first 64 columns of its S
+#pragma unroll
+      for (int ks = 0; ks < BN / 16; ++ks)                    // 16 keys per instruction
+        mma_ts_pred(tmem_base + COL_O + x * D, pa + 8 * ks, smem_desc_mn(vst + ks * 16 * 128, SLAB_B), idesc_pv,
+                    (it | ks) != 0, leader);
+      commit_pred(pvdone_bar(buf_of(x, it)), leader);
+      return true;
+    };
+    auto clear_ragged_v = [&](int it, int s) {
       const int tile_nrows = L - it * BN;
       if (tile_nrows < BN) {
         // rows past the prompt's end hold another prompt's tokens or nothing at all, and a zero
@@ -198,32 +220,78 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
       }
-      const uint32_t pa = tmem_base + COL_S + b * BN;         // P(it) lies over the first 64 columns of S(it)
-#pragma unroll
-      for (int ks = 0; ks < BN / 16; ++ks)                    // O += P(it) V(it), 16 keys per instruction
-        mma_ts_pred(tmem_base + COL_O, pa + 8 * ks, smem_desc_mn(vst + ks * 16 * 128, SLAB_B), idesc_pv, (it | ks) != 0, leader);
-      commit_pred(empty_bar(s), leader);
-      commit_pred(pvdone_bar(b), leader);
+    };
+    if (ok) ok = wait_stage();
+    if (ok) {
+      for (int x = 0; x < NQ; ++x) issue_s(x, 0, q % NSTG);
+      commit_pred(empty_bar(q % NSTG), leader);
       ++q;
+    }
+    for (int it = 0; it < nt && ok; ++it) {
+      if (NQ == 1) {
+        if (it + 1 < nt) {
+          ok = wait_stage();
+          if (!ok) break;
+          issue_s(0, it + 1, q % NSTG);
+          commit_pred(empty_bar(q % NSTG), leader);
+          ++q;
+        }
+        ok = wait_stage();
+        if (!ok) break;
+        clear_ragged_v(it, q % NSTG);
+        ok = issue_pv(0, it, q % NSTG);
+        if (!ok) break;
+        commit_pred(empty_bar(q % NSTG), leader);
+        ++q;
+      } else {
+        // a head's next logits go where its probabilities are, so they follow its P V; the other
+        // head's instructions fill the time its softmax warps need
+        ok = wait_stage();
+        if (!ok) break;
+        const int sv = q % NSTG;
+        ++q;
+        clear_ragged_v(it, sv);
+        const bool more = it + 1 < nt;
+        int sk = 0;
+        ok = issue_pv(0, it, sv);
+        if (!ok) break;
+        if (more) {
+          ok = wait_stage();
+          if (!ok) break;
+          sk = q % NSTG;
+          ++q;
+          issue_s(0, it + 1, sk);
+        }
+        ok = issue_pv(1, it, sv);
+        if (!ok) break;
+        commit_pred(empty_bar(sv), leader);
+        if (more) {
+          issue_s(1, it + 1, sk);
+          commit_pred(empty_bar(sk), leader);
+        }
+      }
     }
     if (!ok && lane == 0) *abort_flag = 1;
   } else {
-    // ---------------- softmax warps: thread = query row ----------------
+    // ---------------- softmax warps: thread = query row, one warpgroup per head ----------------
+    const int x = (warp - 2) >> 2, head = head0 + x;
     const int lrow = 32 * (warp & 3) + lane;                   // TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+    const uint32_t o_addr = lane_addr + COL_O + x * D;
     const int row = q0 + lrow;                                 // position within the prompt
     // does this warp hold rows of the observation window?  (warp-uniform)
     const int wrow0 = q0 + 32 * (warp & 3);
     const bool warp_window = a.mu != nullptr && wrow0 + 31 >= L - a.Lo && wrow0 < L;
     const int cand_lo = a.Ls, cand_n = L - a.Lr - a.Ls;        // candidates [cand_lo, cand_lo + cand_n)
+    const float sc = a.scale_log2;                             // > 0: the largest raw logit is the largest scaled one
     float m_ref = -INFINITY, l_sum = 0.f, l_cand = 0.f;
     bool ok = true;
     for (int it = 0; it < nt; ++it) {
-      const int b = it & 1;
-      if (!wait_warp(sfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag)) { ok = false; break; }
+      const int b = buf_of(x, it);
+      if (!wait_warp(sfull_bar(b), phase_of(it), abort_flag)) { ok = false; break; }
       fence_after();
       const uint32_t s_addr = lane_addr + COL_S + b * BN;
-      float v[BN];
+      float v[BN];                                             // raw logits
       float mx = -INFINITY;
       if (it == nt - 1) {
         // the tile on the diagonal: key j of the tile is visible to row lrow iff j <= lrow
@@ -236,8 +304,8 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
           tmem_ld16_wait(r1);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            v[32 * c + j] = 32 * c + j <= lrow ? __uint_as_float(r0[j]) * a.scale_log2 : -INFINITY;
-            v[32 * c + 16 + j] = 32 * c + 16 + j <= lrow ? __uint_as_float(r1[j]) * a.scale_log2 : -INFINITY;
+            v[32 * c + j] = 32 * c + j <= lrow ? __uint_as_float(r0[j]) : -INFINITY;
+            v[32 * c + 16 + j] = 32 * c + 16 + j <= lrow ? __uint_as_float(r1[j]) : -INFINITY;
             mx = fmaxf(mx, fmaxf(v[32 * c + j], v[32 * c + 16 + j]));
           }
         }
@@ -251,28 +319,29 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
           tmem_ld16_wait(r1);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            v[32 * c + j] = __uint_as_float(r0[j]) * a.scale_log2;
-            v[32 * c + 16 + j] = __uint_as_float(r1[j]) * a.scale_log2;
+            v[32 * c + j] = __uint_as_float(r0[j]);
+            v[32 * c + 16 + j] = __uint_as_float(r1[j]);
             mx = fmaxf(mx, fmaxf(v[32 * c + j], v[32 * c + 16 + j]));
           }
         }
       }
+      mx *= sc;
       // Lazy reference: refreshed (and O rescaled) only when some row of the warp sees a logit 8
       // above its reference; the tensor-memory accesses are warp-collective, so the warp votes.
       if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
         const float m_new = fmaxf(m_ref, mx);
         const float alpha = m_ref == -INFINITY ? 0.f : exp2f(m_ref - m_new);
         if (it > 0) {
-          if (!wait_warp(pvdone_bar((it - 1) & 1), (unsigned)((it - 1) / 2) & 1u, abort_flag)) { ok = false; break; }
+          if (!wait_warp(pvdone_bar(buf_of(x, it - 1)), phase_of(it - 1), abort_flag)) { ok = false; break; }
           fence_after();
 #pragma unroll 1
           for (int c = 0; c < D / 16; ++c) {
             uint32_t o[16];
-            tmem_ld16_issue(lane_addr + COL_O + 16 * c, o);
+            tmem_ld16_issue(o_addr + 16 * c, o);
             tmem_ld16_wait(o);
 #pragma unroll
             for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st16(lane_addr + COL_O + 16 * c, o);
+            tmem_st16(o_addr + 16 * c, o);
           }
           tmem_st_wait();
         }
@@ -280,7 +349,7 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
         l_cand *= alpha;
         m_ref = m_new;
       }
-      const float mr = m_ref == -INFINITY ? 0.f : m_ref;
+      const float nmr = m_ref == -INFINITY ? 0.f : -m_ref;
       float ls0 = 0.f, ls1 = 0.f;
       // this tile's overlap with the candidate range, as tile columns [clo, clo + cn)
       const int clo = cand_lo - it * BN;
@@ -292,7 +361,7 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
         float pc = 0.f;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const float p0 = fast_exp2(v[32 * c + 2 * j] - mr), p1 = fast_exp2(v[32 * c + 2 * j + 1] - mr);
+          const float p0 = fast_exp2(fmaf(v[32 * c + 2 * j], sc, nmr)), p1 = fast_exp2(fmaf(v[32 * c + 2 * j + 1], sc, nmr));
           ls0 += p0;
           ls1 += p1;
           if (warp_window) {
@@ -312,7 +381,7 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
     }
     if (!ok) *abort_flag = 1;
     // ---------------- normalise and store ----------------
-    if (ok) ok = wait_warp(pvdone_bar((nt - 1) & 1), (unsigned)((nt - 1) / 2) & 1u, abort_flag);
+    if (ok) ok = wait_warp(pvdone_bar(buf_of(x, nt - 1)), phase_of(nt - 1), abort_flag);
     if (!ok) *abort_flag = 1;
     fence_after();
     if (__all_sync(0xffffffffu, ok)) {
@@ -321,7 +390,7 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
 #pragma unroll 1
       for (int c = 0; c < D / 16; ++c) {
         uint32_t o[16];
-        tmem_ld16_issue(lane_addr + COL_O + 16 * c, o);
+        tmem_ld16_issue(o_addr + 16 * c, o);
         tmem_ld16_wait(o);
         if (row < L) {
           uint4 w0, w1;
@@ -351,7 +420,7 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
   if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
 }
 
-size_t prefill_smem_bytes() { return (size_t)TILE_B + NSTG * TILE_B + (2 * NSTG + 7) * 8 + 16 + 1024; }
+size_t prefill_smem_bytes(int nq) { return (size_t)nq * TILE_B + NSTG * TILE_B + (2 * NSTG + 7) * 8 + 16 + 1024; }
 
 }  // namespace
 
@@ -390,10 +459,19 @@ cudaError_t launch_prefill_attn(const Shape& s, const SeqBatch& b, const void* q
   a.out = static_cast<__nv_bfloat16*>(out);
   a.mu = mu;
   a.status = status;
-  const size_t smem = prefill_smem_bytes();
-  static SmemLimit limit = {};
-  if (cudaError_t e = ensure_dyn_smem(prefill_attn_kernel, smem, limit)) return e;
-  prefill_attn_kernel<<<dim3((max_len + BM - 1) / BM, s.Hq, b.n), NTH, smem, st>>>(a, tq, tk, tv);
+  // pairs of heads that share a KV head when the group allows (SNAP_PREFILL_HEADS=1 forces single heads)
+  const char* env = getenv("SNAP_PREFILL_HEADS");
+  const int nq = s.g % 2 == 0 && !(env && env[0] == '1') ? 2 : 1;
+  const size_t smem = prefill_smem_bytes(nq);
+  static SmemLimit limit1 = {}, limit2 = {};
+  const dim3 grid((max_len + BM - 1) / BM, s.Hq / nq, b.n);
+  if (nq == 2) {
+    if (cudaError_t e = ensure_dyn_smem(prefill_attn_kernel<2>, smem, limit2)) return e;
+    prefill_attn_kernel<2><<<grid, 64 + 128 * 2, smem, st>>>(a, tq, tk, tv);
+  } else {
+    if (cudaError_t e = ensure_dyn_smem(prefill_attn_kernel<1>, smem, limit1)) return e;
+    prefill_attn_kernel<1><<<grid, 64 + 128, smem, st>>>(a, tq, tk, tv);
+  }
   count_launch();
   return cudaGetLastError();
 }

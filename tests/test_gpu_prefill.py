@@ -17,6 +17,8 @@ MU_ATOL = 1e-3      # log2 units: fp32 accumulation of bf16 products and the har
 WL64 = synth.Workload("prefill_g4", 8, 2, 128, 128, "bf16", 4, 48, 96, 16, 7, batch=1,
                       prompt_len=(700, 700), decode_steps=1, salience="zipf")
 WL128 = WL64.scaled(name="prefill_g8", n_q_heads=16, n_kv_heads=2)
+WL_MHA = WL64.scaled(name="prefill_g1", n_q_heads=4, n_kv_heads=4)       # odd group: one head per CTA
+WL_G3 = WL64.scaled(name="prefill_g3", n_q_heads=6, n_kv_heads=2)
 
 
 def _prefill(wl, lengths, seed, want_mu=True):
@@ -57,11 +59,16 @@ def _check_prefill(wl, lengths, seed):
     return layer, prompts, cu, mu
 
 
-@pytest.mark.parametrize("wl", [WL64, WL128], ids=lambda w: w.name)
+@pytest.mark.parametrize("wl", [WL64, WL128, WL_MHA, WL_G3], ids=lambda w: w.name)
 def test_prefill_attention_and_normalisers_match_oracle(wl):
     # one row, shorter than the window, around one tile, several tiles with ragged tails, the
     # window straddling a tile boundary (L = 520: rows 504..519), neighbours in one ragged batch
     _check_prefill(wl, [1, 5, 127, 128, 129, 300, 520, 700], seed=310)
+
+
+def test_single_head_kernel_stays_selectable_for_even_groups(monkeypatch):
+    monkeypatch.setenv("SNAP_PREFILL_HEADS", "1")
+    _check_prefill(WL64, [129, 700], seed=315)
 
 
 def test_prefill_handles_empty_prompts_and_no_normaliser_buffer():
