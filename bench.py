@@ -442,6 +442,36 @@ def extras(hp, wl, dev):
     out["multi_token_decode_ms"] = statistics.median(times[2:])
     out["multi_token_tokens_per_s"] = wl.batch * q_len / (out["multi_token_decode_ms"] * 1e-3)
     out["multi_token_status"] = int(c.status.item())
+    # (5) the prompt's causal attention emitting the Eq. 4 normalisers, and the compression that takes
+    #     them instead of making its own first pass over the keys (one 128k-token prompt, one layer)
+    p = synth.make_prompt(wl, L, SEED + 99, dev)
+    qf = synth.make_prompt_queries(wl, p, SEED + 99, dev)
+    attn = torch.empty(L, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device=dev)
+    mu = torch.empty(1, wl.n_q_heads, wl.l_obs, dtype=torch.float32, device=dev)
+    times = []
+    for r in range(3):
+        a, b = ev(), ev()
+        a.record()
+        B.snap_prefill_attn(hp.cfg, qf, p["k"], p["v"], [0, L], attn, mu, c.status)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    out["prefill_attn_ms_per_128k_prompt"] = min(times[1:])
+    out["prefill_attn_tflops_causal"] = 2.0 * L * L * wl.d_qk * wl.n_q_heads / (out["prefill_attn_ms_per_128k_prompt"] * 1e-3) / 1e12
+    cws = torch.empty(B.snap_compress_workspace_bytes(hp.cfg, [0, L]), dtype=torch.uint8, device=dev)
+    times = []
+    for r in range(7):
+        a, b = ev(), ev()
+        a.record()
+        B.snap_compress_with_row_stats(hp.cfg, hp.layout, p["q_obs"][None], mu, p["k"], p["v"], [0, L], [0], c.k_cache,
+                                       c.v_cache, c.seq_len, c.valid_topk, None, cws, c.status)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b) * 1e3)
+    out["compress_us_per_128k_prefill_with_row_stats"] = statistics.median(times[2:])
+    out["prefill_status"] = int(c.status.item())
+    hp.compress_prompt(hp.pool[hp.resident[0]], 0)          # restore slot 0
+    del p, qf, attn, cws
     out["concat_update_bytes"] = 2 * wl.batch * wl.n_kv_heads * hp.layout.slots * (wl.d_qk + wl.d_v) * 2
     out["ring_append_bytes"] = 2 * wl.batch * wl.n_kv_heads * (wl.d_qk + wl.d_v) * 2
     return out
@@ -541,7 +571,9 @@ def run_case(args):
     """Small single-kernel-family cases for profiler captures (bounded device memory):
     `decode`   32 sequences with 8192-token prompts compressed, then a few decode steps
                (672 MB of cache read per step, ~1.5 GB resident);
-    `compress` one prompt of --case-len tokens compressed a few times."""
+    `compress` one prompt of --case-len tokens compressed a few times;
+    `prefill`  the same, then the prompt's causal attention (emitting the Eq. 4 normalisers) and the
+               compression that consumes them."""
     from paper_2511_03092_b200 import binding as B
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
@@ -601,6 +633,35 @@ def run_case(args):
         flops = 2 * 2.0 * wl.n_q_heads * wl.l_obs * (L - wl.l_sink - wl.l_recent) * wl.d_qk
         print(json.dumps({"case": "compress", "prompt_tokens": L, "us_per_prompt": ms * 1e3,
                           "score_TFLOPs": flops / ms / 1e9, "status": int(hp.cache.status.item())}))
+        if args.case == "prefill":
+            qf = synth.make_prompt_queries(wl, p, SEED, dev)
+            attn = torch.empty(L, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device=dev)
+            mu = torch.empty(1, wl.n_q_heads, wl.l_obs, dtype=torch.float32, device=dev)
+            run = lambda: B.snap_prefill_attn(hp.cfg, qf, p["k"], p["v"], [0, L], attn, mu, hp.cache.status)
+            for s in range(args.warmup):
+                run()
+            torch.cuda.synchronize()
+            t0.record()
+            for s in range(args.steps):
+                run()
+            t1.record()
+            torch.cuda.synchronize()
+            ms = t0.elapsed_time(t1) / args.steps
+            run2 = lambda: B.snap_compress_with_row_stats(hp.cfg, hp.layout, p["q_obs"][None], mu, p["k"], p["v"], [0, L],
+                                                          [0], hp.cache.k_cache, hp.cache.v_cache, hp.cache.seq_len,
+                                                          hp.cache.valid_topk, None, hp.ws, hp.cache.status)
+            for s in range(args.warmup):
+                run2()
+            torch.cuda.synchronize()
+            t0.record()
+            for s in range(args.steps):
+                run2()
+            t1.record()
+            torch.cuda.synchronize()
+            print(json.dumps({"case": "prefill", "prompt_tokens": L, "ms_per_prompt": ms,
+                              "causal_TFLOPs": 2.0 * L * L * wl.d_qk * wl.n_q_heads / ms / 1e9,
+                              "compress_with_row_stats_us": t0.elapsed_time(t1) / args.steps * 1e3,
+                              "status": int(hp.cache.status.item())}))
 
 
 def run_config(args):
@@ -694,7 +755,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the 128k-compress and full-KV side measurements")
-    ap.add_argument("--case", choices=["decode", "compress"], default=None,
+    ap.add_argument("--case", choices=["decode", "compress", "prefill"], default=None,
                     help="small single-kernel-family case for profiler captures")
     ap.add_argument("--case-len", type=int, default=131072)
     ap.add_argument("--workload", type=int, choices=[0, 1, 3, 4], default=None,

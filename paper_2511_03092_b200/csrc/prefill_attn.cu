@@ -83,6 +83,24 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+typedef unsigned long long u64;
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+  u64 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ float lo2(u64 a) { return __uint_as_float((uint32_t)a); }
+__device__ __forceinline__ float hi2(u64 a) { return __uint_as_float((uint32_t)(a >> 32)); }
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+  u64 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ bool wait_warp(uint32_t bar, unsigned parity, volatile int* abort_flag) {
   return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
 }
@@ -109,8 +127,8 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
   unsigned char* Qs = smem;                                    // [NQ heads][2 slabs][128 rows][128 B]
   unsigned char* Rs = Qs + NQ * TILE_B;                        // [NSTG][32 KB] ring
   uint64_t* bars = reinterpret_cast<uint64_t*>(Rs + NSTG * TILE_B);
-  // full[NSTG] empty[NSTG] s_full[2] p_ready[2] pv_done[2] q_full
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTG + 7);
+  // full[NSTG] empty[NSTG] s_full[2] p_ready[2][2 halves of the keys] pv_done[2] q_full
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTG + 9);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -118,9 +136,9 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
   auto full_bar = [&](int s) { return bar0 + 8 * s; };
   auto empty_bar = [&](int s) { return bar0 + 8 * (NSTG + s); };
   auto sfull_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + b); };
-  auto pready_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 2 + b); };
-  auto pvdone_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 4 + b); };
-  const uint32_t qfull_bar = bar0 + 8 * (2 * NSTG + 6);
+  auto pready_bar = [&](int b, int half) { return bar0 + 8 * (2 * NSTG + 2 + 2 * b + half); };
+  auto pvdone_bar = [&](int b) { return bar0 + 8 * (2 * NSTG + 6 + b); };
+  const uint32_t qfull_bar = bar0 + 8 * (2 * NSTG + 8);
   // S / P buffer, its barriers and their phase for tile `it` of head x:
   //   NQ = 1: two buffers used alternately by the one head; NQ = 2: one buffer per head
   auto buf_of = [&](int x, int it) { return NQ == 1 ? (it & 1) : x; };
@@ -129,7 +147,9 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
   if (tid == 0) {
     *abort_flag = 0;
     for (int s = 0; s < NSTG; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(sfull_bar(b), 1); mbar_init(pready_bar(b), 4); mbar_init(pvdone_bar(b), 1); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(sfull_bar(b), 1); mbar_init(pready_bar(b, 0), 4); mbar_init(pready_bar(b, 1), 4); mbar_init(pvdone_bar(b), 1);
+    }
     mbar_init(qfull_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -197,14 +217,17 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
       commit_pred(sfull_bar(buf_of(x, it)), leader);
     };
     auto issue_pv = [&](int x, int it, int s) -> bool {       // O_x += P_x(it) V(it), V in stage s
-      if (!wait_warp(pready_bar(buf_of(x, it)), phase_of(it), abort_flag)) return false;
-      fence_after();
       const uint32_t vst = smem_u32(Rs) + s * TILE_B;
       const uint32_t pa = tmem_base + COL_S + buf_of(x, it) * BN;   // P lies over the first 64 columns of its S
 #pragma unroll
-      for (int ks = 0; ks < BN / 16; ++ks)                    // 16 keys per instruction
-        mma_ts_pred(tmem_base + COL_O + x * D, pa + 8 * ks, smem_desc_mn(vst + ks * 16 * 128, SLAB_B), idesc_pv,
-                    (it | ks) != 0, leader);
+      for (int half = 0; half < 2; ++half) {                  // the first 64 keys go while the rest are exponentiated
+        if (!wait_warp(pready_bar(buf_of(x, it), half), phase_of(it), abort_flag)) return false;
+        fence_after();
+#pragma unroll
+        for (int ks = 4 * half; ks < 4 * half + 4; ++ks)      // 16 keys per instruction
+          mma_ts_pred(tmem_base + COL_O + x * D, pa + 8 * ks, smem_desc_mn(vst + ks * 16 * 128, SLAB_B), idesc_pv,
+                      (it | ks) != 0, leader);
+      }
       commit_pred(pvdone_bar(buf_of(x, it)), leader);
       return true;
     };
@@ -292,39 +315,30 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
       fence_after();
       const uint32_t s_addr = lane_addr + COL_S + b * BN;
       float v[BN];                                             // raw logits
-      float mx = -INFINITY;
+      {
+        // all eight loads in flight before the one wait: the tensor-memory latency is paid once per tile
+        uint32_t r[8][16];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) tmem_ld16_issue(s_addr + 16 * c, r[c]);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) tmem_ld16_wait(r[c]);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[16 * c + j] = __uint_as_float(r[c][j]);
+      }
       if (it == nt - 1) {
         // the tile on the diagonal: key j of the tile is visible to row lrow iff j <= lrow
 #pragma unroll
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r0[16], r1[16];
-          tmem_ld16_issue(s_addr + 32 * c, r0);
-          tmem_ld16_issue(s_addr + 32 * c + 16, r1);
-          tmem_ld16_wait(r0);
-          tmem_ld16_wait(r1);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            v[32 * c + j] = 32 * c + j <= lrow ? __uint_as_float(r0[j]) : -INFINITY;
-            v[32 * c + 16 + j] = 32 * c + 16 + j <= lrow ? __uint_as_float(r1[j]) : -INFINITY;
-            mx = fmaxf(mx, fmaxf(v[32 * c + j], v[32 * c + 16 + j]));
-          }
-        }
-      } else {
-#pragma unroll
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t r0[16], r1[16];
-          tmem_ld16_issue(s_addr + 32 * c, r0);
-          tmem_ld16_issue(s_addr + 32 * c + 16, r1);
-          tmem_ld16_wait(r0);
-          tmem_ld16_wait(r1);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            v[32 * c + j] = __uint_as_float(r0[j]);
-            v[32 * c + 16 + j] = __uint_as_float(r1[j]);
-            mx = fmaxf(mx, fmaxf(v[32 * c + j], v[32 * c + 16 + j]));
-          }
-        }
+        for (int j = 0; j < BN; ++j) v[j] = j <= lrow ? v[j] : -INFINITY;
       }
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < BN; j += 4) {
+        mx0 = fmaxf(mx0, fmaxf(v[j], v[j + 1]));
+        mx1 = fmaxf(mx1, fmaxf(v[j + 2], v[j + 3]));
+      }
+      float mx = fmaxf(mx0, mx1);
       mx *= sc;
       // Lazy reference: refreshed (and O rescaled) only when some row of the warp sees a logit 8
       // above its reference; the tensor-memory accesses are warp-collective, so the warp votes.
@@ -355,29 +369,45 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
       const int clo = cand_lo - it * BN;
       const unsigned cn = warp_window && cand_n > 0 ? (unsigned)cand_n : 0u;
       // the logits of this tile are all in registers, so the probabilities may overwrite them
+      u64 ls2 = pack2(0.f, 0.f);
+      const u64 sc2 = pack2(sc, sc), nmr2 = pack2(nmr, nmr);
 #pragma unroll
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t pk[16];
-        float pc = 0.f;
+        if (!warp_window) {
+          // two-wide multiply-adds and sums: the arithmetic around the exponentials takes half the issue slots
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float p0 = fast_exp2(fmaf(v[32 * c + 2 * j], sc, nmr)), p1 = fast_exp2(fmaf(v[32 * c + 2 * j + 1], sc, nmr));
-          ls0 += p0;
-          ls1 += p1;
-          if (warp_window) {
+          for (int j = 0; j < 16; ++j) {
+            const u64 x2 = fma2(pack2(v[32 * c + 2 * j], v[32 * c + 2 * j + 1]), sc2, nmr2);
+            const float p0 = fast_exp2(lo2(x2)), p1 = fast_exp2(hi2(x2));
+            ls2 = add2(ls2, pack2(p0, p1));
+            pk[j] = pack_bf16(p0, p1);
+          }
+        } else {
+          // rows of the observation window also sum over the candidate columns alone
+          float pc = 0.f;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float p0 = fast_exp2(fmaf(v[32 * c + 2 * j], sc, nmr)), p1 = fast_exp2(fmaf(v[32 * c + 2 * j + 1], sc, nmr));
+            ls0 += p0;
+            ls1 += p1;
             pc += (unsigned)(32 * c + 2 * j - clo) < cn ? p0 : 0.f;
             pc += (unsigned)(32 * c + 2 * j + 1 - clo) < cn ? p1 : 0.f;
+            pk[j] = pack_bf16(p0, p1);
           }
-          pk[j] = pack_bf16(p0, p1);
+          l_cand += pc;
         }
-        l_cand += pc;
         tmem_st16(s_addr + 16 * c, pk);
+        if (c & 1) {                                           // a half of the keys is complete
+          tmem_st_wait();
+          fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(pready_bar(b, c >> 1));
+        }
       }
+      ls0 += lo2(ls2);
+      ls1 += hi2(ls2);
       l_sum += ls0 + ls1;
-      tmem_st_wait();
-      fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(pready_bar(b));
     }
     if (!ok) *abort_flag = 1;
     // ---------------- normalise and store ----------------
@@ -420,7 +450,7 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
   if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
 }
 
-size_t prefill_smem_bytes(int nq) { return (size_t)nq * TILE_B + NSTG * TILE_B + (2 * NSTG + 7) * 8 + 16 + 1024; }
+size_t prefill_smem_bytes(int nq) { return (size_t)nq * TILE_B + NSTG * TILE_B + (2 * NSTG + 9) * 8 + 16 + 1024; }
 
 }  // namespace
 
