@@ -146,6 +146,35 @@ __device__ __forceinline__ float fast_exp2(float x) {     // one MUFU op, relati
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Two-wide packed fp32 arithmetic: the multiply-add in front of an exponential and the addition
+// behind it cost half an issue slot per element.
+typedef unsigned long long u64;
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+  u64 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ float lo2(u64 a) { return __uint_as_float((uint32_t)a); }
+__device__ __forceinline__ float hi2(u64 a) { return __uint_as_float((uint32_t)(a >> 32)); }
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+  u64 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// acc (two pairs, alternated) += exp2(r[i] * scale + off) over 2 n raw logits, off the same for all
+template <int N2>
+__device__ __forceinline__ void exp_sum_const(const uint32_t* r, u64 sc2, u64 off2, u64 (&acc)[2]) {
+#pragma unroll
+  for (int i = 0; i < N2; ++i) {
+    const u64 x = fma2(pack2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, off2);
+    acc[i & 1] = add2(acc[i & 1], pack2(fast_exp2(lo2(x)), fast_exp2(hi2(x))));
+  }
+}
 __device__ __forceinline__ void merge_ml(float& m, float& l, float m2, float l2) {
   const float mn = fmaxf(m, m2);
   const float f1 = m == -INFINITY ? 0.f : exp2f(m - mn), f2 = m2 == -INFINITY ? 0.f : exp2f(m2 - mn);
@@ -282,10 +311,11 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
     // pass 2: minus the log-sum-exp (log2 domain) of each query row this group sums over, in
     // registers, so that the inner loop is fma -> exp2 -> add with no memory operand
     const int nc2 = R / 64;                                   // 32-column chunks per group: 2 or 4
-    float mu[128];
+    u64 mu2[64];                                              // pairs of adjacent columns' constants
     if (PASS == 2) {
 #pragma unroll
-      for (int i = 0; i < 128; ++i) mu[i] = i < 32 * nc2 ? -mu_s[32 * nc2 * eg + i] : 0.f;
+      for (int i = 0; i < 64; ++i)
+        mu2[i] = 2 * i < 32 * nc2 ? pack2(-mu_s[32 * nc2 * eg + 2 * i], -mu_s[32 * nc2 * eg + 2 * i + 1]) : pack2(0.f, 0.f);
     }
     for (int it = both ? 0 : eg; it < nt; it += both ? 1 : 2) {
       const int b = it & 1;
@@ -306,25 +336,21 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
           // software pipeline: the next 32 columns are in flight while these are exponentiated;
           // four partial sums break the dependency chain of the additions
           uint32_t ra[32], rb[32];
-          float s4[4] = {0.f, 0.f, 0.f, 0.f};
-          const float nm = -m_ref;
+          u64 acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+          const u64 sc2 = pack2(a.scale_log2, a.scale_log2), nm2 = pack2(-m_ref, -m_ref);
           tmem_ld32_issue(col0, ra);
           tmem_ld_wait(ra);
           tmem_ld32_issue(col0 + 32, rb);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, nm));
+          exp_sum_const<16>(ra, sc2, nm2, acc);
           tmem_ld_wait(rb);
           tmem_ld32_issue(col0 + 64, ra);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(rb[i]), a.scale_log2, nm));
+          exp_sum_const<16>(rb, sc2, nm2, acc);
           tmem_ld_wait(ra);
           tmem_ld32_issue(col0 + 96, rb);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, nm));
+          exp_sum_const<16>(ra, sc2, nm2, acc);
           tmem_ld_wait(rb);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) s4[i & 3] += fast_exp2(fmaf(__uint_as_float(rb[i]), a.scale_log2, nm));
-          sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+          exp_sum_const<16>(rb, sc2, nm2, acc);
+          sum = (lo2(acc[0]) + hi2(acc[0])) + (lo2(acc[1]) + hi2(acc[1]));
         } else {
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
@@ -370,7 +396,8 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
           // software pipeline over 16-column chunks (two small register buffers leave room for the
           // 128 row constants); four partial sums break the dependency chain of the additions
           uint32_t ra[16], rb[16];
-          float s4[4] = {0.f, 0.f, 0.f, 0.f};
+          u64 acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+          const u64 sc2 = pack2(a.scale_log2, a.scale_log2);
           const int nch = 2 * nc2;                             // 16-column chunks: 4 or 8
           tmem_ld16_issue(col0, ra);
 #pragma unroll
@@ -379,16 +406,20 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
               tmem_ld16_wait(ra);
               tmem_ld16_issue(col0 + 16 * (c + 1), rb);
 #pragma unroll
-              for (int i = 0; i < 16; ++i)
-                s4[i & 3] += fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, mu[16 * c + i]));
+              for (int i = 0; i < 8; ++i) {
+                const u64 x = fma2(pack2(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1])), sc2, mu2[8 * c + i]);
+                acc[i & 1] = add2(acc[i & 1], pack2(fast_exp2(lo2(x)), fast_exp2(hi2(x))));
+              }
               tmem_ld16_wait(rb);
               if (c + 2 < nch) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
 #pragma unroll
-              for (int i = 0; i < 16; ++i)
-                s4[i & 3] += fast_exp2(fmaf(__uint_as_float(rb[i]), a.scale_log2, mu[16 * (c + 1) + i]));
+              for (int i = 0; i < 8; ++i) {
+                const u64 x = fma2(pack2(__uint_as_float(rb[2 * i]), __uint_as_float(rb[2 * i + 1])), sc2, mu2[8 * (c + 1) + i]);
+                acc[i & 1] = add2(acc[i & 1], pack2(fast_exp2(lo2(x)), fast_exp2(hi2(x))));
+              }
             }
           }
-          s = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+          s = (lo2(acc[0]) + hi2(acc[0])) + (lo2(acc[1]) + hi2(acc[1]));
         }
         float* xs = reinterpret_cast<float*>(xch) + b * 128;
         if (eg == 1) xs[lrow] = s;
