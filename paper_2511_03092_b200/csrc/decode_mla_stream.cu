@@ -5,7 +5,7 @@
 // produces, so this kernel is built around wide instructions: S = Q K^T in 128-row tiles
 // (N = 128) and O += P V over 256 value dims at a time (N = 256).  The 128 x 576 query block
 // stays in shared memory (nine 64-dim slabs, 128-byte swizzle) as the A operand of S; what is
-// left of shared memory is a ring of four 16 KB stages through which the cache rows stream
+// left of shared memory is a ring of five 16 KB stages through which the cache rows stream
 // twice: as key slabs (128 rows x 64 dims, K-major B operand of S) and, once the tile's
 // probabilities exist, as value chunks (32 rows x 256 dims, MN-major B operand of P V).  The
 // second pass costs 0.44 of the first in L2 traffic and buys a tile four times as wide as one
@@ -30,7 +30,7 @@ namespace {
 
 using namespace umma;
 
-constexpr int DQK = 576, DV = 512, HBLK = 128, TR = 128, NSTG = 4, NTH = 192, DVH = 256, NHALF = DV / DVH;
+constexpr int DQK = 576, DV = 512, HBLK = 128, TR = 128, NSTG = 5, NTH = 192, DVH = 256, NHALF = DV / DVH;
 constexpr int NSLAB = DQK / 64, QSLAB_B = HBLK * 128, STAGE_B = 16384;   // key slab = 128 rows x 128 B = one stage
 constexpr int VROWS = 32, VSUB_B = VROWS * 128, NVCH = TR / VROWS;       // value chunk = 4 sub-slabs of 32 rows x 64 dims
 constexpr int PSM = DV + 2;
@@ -280,22 +280,30 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
       const uint32_t s_addr = lane_addr + COL_S + b * TR;
       const TileRows tr = tile_rows(g0 + it, nA, n_low, Lsr, n_top);
       const int nrows = tr.row_end - tr.row0;                  // >= 1; columns at or past it are masked
-      float v[TR];
-      float mx = -INFINITY;
+      float v[TR];                                             // raw logits
+      {
+        // all eight loads in flight before the one wait: the tensor-memory latency is paid once per tile
+        uint32_t r[8][16];
 #pragma unroll
-      for (int c = 0; c < TR / 32; ++c) {
-        uint32_t r0[16], r1[16];
-        tmem_ld16_issue(s_addr + 32 * c, r0);
-        tmem_ld16_issue(s_addr + 32 * c + 16, r1);
-        tmem_ld16_wait(r0);
-        tmem_ld16_wait(r1);
+        for (int c = 0; c < 8; ++c) tmem_ld16_issue(s_addr + 16 * c, r[c]);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          v[32 * c + j] = 32 * c + j < nrows ? __uint_as_float(r0[j]) * a.scale_log2 : -INFINITY;
-          v[32 * c + 16 + j] = 32 * c + 16 + j < nrows ? __uint_as_float(r1[j]) * a.scale_log2 : -INFINITY;
-          mx = fmaxf(mx, fmaxf(v[32 * c + j], v[32 * c + 16 + j]));
-        }
+        for (int c = 0; c < 8; ++c) tmem_ld16_wait(r[c]);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[16 * c + j] = __uint_as_float(r[c][j]);
       }
+      if (nrows < TR) {                                        // ragged tile: columns at or past nrows are masked
+#pragma unroll
+        for (int j = 0; j < TR; ++j) v[j] = j < nrows ? v[j] : -INFINITY;
+      }
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < TR; j += 4) {
+        mx0 = fmaxf(mx0, fmaxf(v[j], v[j + 1]));
+        mx1 = fmaxf(mx1, fmaxf(v[j + 2], v[j + 3]));
+      }
+      const float mx = fmaxf(mx0, mx1) * a.scale_log2;         // scale > 0: the largest raw logit is the largest scaled one
       // Lazy reference: refreshed (and O rescaled) only when some head of the warp sees a logit 8
       // above its reference; the tensor-memory accesses are warp-collective, so the warp votes.
       if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
@@ -318,22 +326,24 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
         l_sum *= alpha;
         m_ref = m_new;
       }
-      const float mr = m_ref == -INFINITY ? 0.f : m_ref;
-      float ls0 = 0.f, ls1 = 0.f;
-      // the logits of this tile are all in registers, so the probabilities may overwrite them
+      const float nmr = m_ref == -INFINITY ? 0.f : -m_ref;
+      // the logits of this tile are all in registers, so the probabilities may overwrite them;
+      // two-wide packed multiply-adds and sums around the exponentials
+      const u64 sc2 = pack2(a.scale_log2, a.scale_log2), nmr2 = pack2(nmr, nmr);
+      u64 ls2 = pack2(0.f, 0.f);
 #pragma unroll
       for (int c = 0; c < TR / 32; ++c) {
         uint32_t pk[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const float p0 = fast_exp2(v[32 * c + 2 * j] - mr), p1 = fast_exp2(v[32 * c + 2 * j + 1] - mr);
-          ls0 += p0;
-          ls1 += p1;
+          const u64 x2 = fma2(pack2(v[32 * c + 2 * j], v[32 * c + 2 * j + 1]), sc2, nmr2);
+          const float p0 = fast_exp2(lo2(x2)), p1 = fast_exp2(hi2(x2));
+          ls2 = add2(ls2, pack2(p0, p1));
           pk[j] = pack_bf16(p0, p1);
         }
         tmem_st16(s_addr + 16 * c, pk);
       }
-      l_sum += ls0 + ls1;
+      l_sum += lo2(ls2) + hi2(ls2);
       tmem_st_wait();
       fence_before();
       __syncwarp();

@@ -192,8 +192,33 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
           }
           return (s4[0] + s4[1]) + (s4[2] + s4[3]);
         };
+        // the common case (a tile wholly inside the candidates, reference up to date) with two-wide
+        // packed arithmetic: half an issue slot per element for the multiply-add and for the sum
+        auto sweep_full = [&](float ref) -> float {
+          u64 acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+          const u64 sc2 = pack2(a.scale_log2, a.scale_log2), nr2 = pack2(-ref, -ref);
+          tmem_ld16_issue(col0, ra);
+#pragma unroll
+          for (int c = 0; c < 8; c += 2) {
+            tmem_ld16_wait(ra);
+            tmem_ld16_issue(col0 + 16 * (c + 1), rb16);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const u64 x = fma2(pack2(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1])), sc2, nr2);
+              acc[i & 1] = add2(acc[i & 1], pack2(fast_exp2(lo2(x)), fast_exp2(hi2(x))));
+            }
+            tmem_ld16_wait(rb16);
+            if (c + 2 < 8) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const u64 x = fma2(pack2(__uint_as_float(rb16[2 * i]), __uint_as_float(rb16[2 * i + 1])), sc2, nr2);
+              acc[i & 1] = add2(acc[i & 1], pack2(fast_exp2(lo2(x)), fast_exp2(hi2(x))));
+            }
+          }
+          return (lo2(acc[0]) + hi2(acc[0])) + (lo2(acc[1]) + hi2(acc[1]));
+        };
         float dummy = 0.f;
-        float sum = sweep(m_ref, false, dummy);
+        float sum = full_tile ? sweep_full(m_ref) : sweep(m_ref, false, dummy);
         // a logit far above the reference (or the first tile): refresh it; the TMEM loads are
         // warp-collective, so the whole warp takes the branch if any row needs it
         if (__any_sync(0xffffffffu, !(sum < 65536.f))) {
@@ -216,6 +241,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
         const uint32_t col0 = lane_addr + b * 256 + eg * 128;
         const int cand0 = (t0 + it) * TNP + eg * 128;
         float v[128];
+        const u64 sc2 = pack2(a.scale_log2, a.scale_log2), nmu2 = pack2(neg_mu, neg_mu);
         if (landed) {
           tmem_ld16_issue(col0, ra);
 #pragma unroll
@@ -223,11 +249,19 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
             tmem_ld16_wait(ra);
             tmem_ld16_issue(col0 + 16 * (c + 1), rb16);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v[16 * c + i] = fast_exp2(fmaf(__uint_as_float(ra[i]), a.scale_log2, neg_mu));
+            for (int i = 0; i < 8; ++i) {
+              const u64 x = fma2(pack2(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1])), sc2, nmu2);
+              v[16 * c + 2 * i] = fast_exp2(lo2(x));
+              v[16 * c + 2 * i + 1] = fast_exp2(hi2(x));
+            }
             tmem_ld16_wait(rb16);
             if (c + 2 < 8) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v[16 * (c + 1) + i] = fast_exp2(fmaf(__uint_as_float(rb16[i]), a.scale_log2, neg_mu));
+            for (int i = 0; i < 8; ++i) {
+              const u64 x = fma2(pack2(__uint_as_float(rb16[2 * i]), __uint_as_float(rb16[2 * i + 1])), sc2, nmu2);
+              v[16 * (c + 1) + 2 * i] = fast_exp2(lo2(x));
+              v[16 * (c + 1) + 2 * i + 1] = fast_exp2(hi2(x));
+            }
           }
         } else {
 #pragma unroll

@@ -125,6 +125,32 @@ def test_compress_with_prefill_normalisers_matches_oracle(wl):
     assert with_stats < B.snap_kernel_launch_count() - launches
 
 
+def test_more_prompts_than_one_launch_takes():
+    """Prompts are launched in groups of 64: the normalisers of a later group land in its own rows."""
+    wl = WL64
+    lengths = [int(x) for x in np.random.default_rng(350).integers(1, 260, size=70)]
+    lengths[66] = 400                                  # a scored prompt in the second group
+    _check_prefill(wl, lengths, seed=351)
+
+
+def test_prefill_reads_strided_keys_and_values():
+    """K and V as slices of one fused [T, 2 * Hkv, d] buffer (token and head strides differ from dense)."""
+    wl = WL64
+    lengths = [300, 131]
+    layer, prompts, qs, cu, (q, k, v), out, mu = _prefill(wl, lengths, seed=360)
+    fused = torch.full((cu[-1], 2 * wl.n_kv_heads + 1, wl.d_qk), float("nan"), dtype=torch.bfloat16, device="cuda")
+    fused[:, 0:wl.n_kv_heads] = k
+    fused[:, wl.n_kv_heads + 1:] = v
+    kv, vv = fused[:, 0:wl.n_kv_heads], fused[:, wl.n_kv_heads + 1:]
+    assert not kv.is_contiguous() and kv.stride(0) == (2 * wl.n_kv_heads + 1) * wl.d_qk
+    out2 = torch.empty_like(out)
+    mu2 = torch.full_like(mu, float("nan"))
+    B.snap_prefill_attn(layer.cfg, q, kv, vv, cu, out2, mu2, layer.cache.status)
+    assert layer.status() == 0
+    assert torch.equal(out2, out)
+    assert torch.equal(mu2, mu)
+
+
 def test_prefill_rejects_what_it_cannot_do():
     wl = synth.Workload("mla", 16, 1, 96, 64, "bf16", 3, 40, 64, 8, 5, batch=1, prompt_len=(100, 100),
                         decode_steps=1, salience="none", v_aliases_k=True)
