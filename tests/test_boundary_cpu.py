@@ -105,6 +105,32 @@ def test_workspace_queries_and_argument_errors_without_gpu():
     assert cc(one, one, one, 0, one, one, two, two, one, None, None) == 0    # nothing to do
 
 
+def test_prefill_entry_points_validate_before_touching_memory():
+    cfg = _cfg()
+    lay = B.snap_cache_layout(cfg)
+    lib = B.lib()
+    one = C.c_void_p(256)   # never dereferenced: validation fails first
+    cu_bad = (C.c_int32 * 3)(0, 10, 5)
+    cu = (C.c_int32 * 2)(0, 9000)
+    pre = lambda c, cup, n: lib.snap_prefill_attn(c, one, one, 1024, 128, one, 1024, 128, cup, n, one, None, None, None)
+    assert pre(None, cu, 1) == -4                                            # no config
+    assert pre(C.byref(cfg), cu_bad, 2) == -1                                # decreasing offsets
+    assert pre(C.byref(cfg), None, 1) == -4
+    assert pre(C.byref(_cfg(softmax_scale=-1.0)), cu, 1) == -1
+    latent = _cfg(n_q_heads=128, n_kv_heads=1, d_qk=576, d_v=512, v_aliases_k=True, l_recent=2048, topk=8192, l_obs=32)
+    assert pre(C.byref(latent), cu, 1) == -2                                 # no prefill kernel for the latent layout
+    assert pre(C.byref(_cfg(dtype=B.SNAP_F32)), cu, 1) == -2
+    # the compress variant shares snap_compress's validation
+    ok_slot = (C.c_int32 * 1)(0)
+    bad_slot = (C.c_int32 * 1)(7)
+    crs = lambda slots, ws_bytes, kts=1024, mu=one: lib.snap_compress_with_row_stats(
+        C.byref(cfg), C.byref(lay), one, mu, one, kts, 128, one, 1024, 128, cu, slots, 1, one, one, one, one, None, one,
+        ws_bytes, None, None)
+    assert crs(bad_slot, 1 << 40) == -1
+    assert crs(ok_slot, 1 << 40, kts=1023) == -1
+    assert crs(ok_slot, 16, mu=None) == -3                                   # without normalisers it is snap_compress
+
+
 def test_header_is_plain_c99(tmp_path):
     """The boundary is a C ABI: the header must compile as C99 on its own, and a C caller must be able to
     link against the library and use the host-only entry points."""
