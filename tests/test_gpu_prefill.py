@@ -19,6 +19,8 @@ WL64 = synth.Workload("prefill_g4", 8, 2, 128, 128, "bf16", 4, 48, 96, 16, 7, ba
 WL128 = WL64.scaled(name="prefill_g8", n_q_heads=16, n_kv_heads=2)
 WL_MHA = WL64.scaled(name="prefill_g1", n_q_heads=4, n_kv_heads=4)       # odd group: one head per CTA
 WL_G3 = WL64.scaled(name="prefill_g3", n_q_heads=6, n_kv_heads=2)
+# an observation window longer than a 128-row tile: its rows sit in two or three CTAs
+WL_LONGWIN = WL64.scaled(name="prefill_lo160", n_q_heads=4, n_kv_heads=2, l_sink=3, l_recent=200, topk=64, l_obs=160)
 
 
 def _prefill(wl, lengths, seed, want_mu=True):
@@ -59,7 +61,7 @@ def _check_prefill(wl, lengths, seed):
     return layer, prompts, cu, mu
 
 
-@pytest.mark.parametrize("wl", [WL64, WL128, WL_MHA, WL_G3], ids=lambda w: w.name)
+@pytest.mark.parametrize("wl", [WL64, WL128, WL_MHA, WL_G3, WL_LONGWIN], ids=lambda w: w.name)
 def test_prefill_attention_and_normalisers_match_oracle(wl):
     # one row, shorter than the window, around one tile, several tiles with ragged tails, the
     # window straddling a tile boundary (L = 520: rows 504..519), neighbours in one ragged batch
@@ -94,7 +96,7 @@ def test_prefill_isolates_prompts_from_nan_neighbours():
     assert torch.equal(out2[:cu[1]], out[:cu[1]])
 
 
-@pytest.mark.parametrize("wl", [WL64, WL128], ids=lambda w: w.name)
+@pytest.mark.parametrize("wl", [WL64, WL128, WL_LONGWIN], ids=lambda w: w.name)
 def test_compress_with_prefill_normalisers_matches_oracle(wl):
     lengths = [700, 100, 149, 1300]          # scored, unscored (fits the budget), just scored, many tiles
     layer, prompts, cu, mu = _check_prefill(wl, lengths, seed=340)
