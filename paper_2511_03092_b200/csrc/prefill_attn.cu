@@ -3,17 +3,19 @@
 // denominators of the scores are by-products of the prompt's own attention pass, so the first of
 // the two passes of the score kernel can be dropped when the prompt's attention ran here).
 //
-// One CTA computes 128 query rows of one head against key tiles 0 .. its own (128 keys each):
+// A CTA computes 128 query rows of one head, or of two heads that share a KV head, against key
+// tiles 0 .. its own (128 keys each):
 //   S = Q K^T      M = 128 rows, N = 128 keys, both operands K-major in shared memory
 //   O += P V       A = P from tensor memory (bf16 pairs written over the tile's own logits),
 //                  B = the V tile as loaded (MN-major)
-// Tensor memory: S0 128 | S1 128 | O 128 columns; the next tile's logits are computed while the
-// softmax warps work on this one.  K and V tiles stream through a ring of four 32 KB stages in
-// the order the MMAs consume them: K(0), K(1), V(0), K(2), V(1), ...
+// K and V tiles stream through a ring of four 32 KB stages in the order the MMAs consume them.
 //   warp 0      TMA producer
 //   warp 1      MMA issuer (whole warp converged, instructions predicated on one lane)
-//   warps 2-5   thread = query row: online softmax in the log2 domain with a lazily refreshed
-//               reference (O is rescaled in tensor memory only when a logit exceeds it by 8)
+//   warps 2-5 (and 6-9 for the second head)
+//               thread = query row: online softmax in the log2 domain with a lazily refreshed
+//               reference (O is rescaled in tensor memory only when a logit exceeds it by 8);
+//               the arithmetic around the exponentials is packed two-wide, and P is handed to
+//               the MMA warp in two halves of 64 keys
 // Rows of the last Lo positions also accumulate the same exponentials over the eviction
 // candidates [Ls, L - Lr) alone; reference + log2 of that sum is what Eq. 4 divides by.
 // Every mbarrier wait is bounded; one that runs out raises SNAP_DEV_WAIT_TIMEOUT.
@@ -87,11 +89,12 @@ __device__ __forceinline__ bool wait_warp(uint32_t bar, unsigned parity, volatil
   return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
 }
 
-// NQ = 1: one head per CTA, S double-buffered (the next tile's logits are computed while the
-// softmax warps work on this one).  NQ = 2: two query heads of one KV head per CTA, each with
-// its own softmax warpgroup, S and O; they share every K and V tile, which halves the traffic
-// from L2 (what bounds the one-head kernel), and while one head's warps work the tensor core
-// serves the other head.
+// NQ = 1: one head per CTA; tensor memory S0 128 | S1 128 | O 128 columns, S double-buffered
+// (the next tile's logits are computed while the softmax warps work on this one).
+// NQ = 2: two query heads of one KV head per CTA, each with its own softmax warpgroup, S and O
+// (4 x 128 columns: tensor memory is full).  They share every K and V tile, which halves the
+// traffic from L2, and while one head's warps work the tensor core serves the other head: a
+// head's next S follows its P V (its logits are overwritten by its probabilities).
 template <int NQ>
 __global__ void __launch_bounds__(64 + 128 * NQ, 1)
 prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
