@@ -161,7 +161,7 @@ int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout,
  * Needs no workspace.  cfg is validated as a whole (as by snap_cache_layout); the kernel uses its
  * model-shape fields, l_sink, l_recent, l_obs and softmax_scale.  Errors: SNAP_ERR_NULL_POINTER,
  * SNAP_ERR_INVALID_ARG (cfg, offsets that decrease, strides that are not multiples of 16 bytes),
- * SNAP_ERR_UNSUPPORTED, SNAP_ERR_CUDA; nothing is launched when an error is returned.
+ * SNAP_ERR_UNSUPPORTED: nothing was launched; SNAP_ERR_CUDA: a launch failed.
  */
 int snap_prefill_attn(const snap_config_t* cfg, const void* q_dev,
                       const void* k_dev, int64_t k_token_stride, int64_t k_head_stride,
