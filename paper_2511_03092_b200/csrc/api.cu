@@ -449,13 +449,33 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
   return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
 }
 
-// Several query tokens per sequence in one step: only the tensor-core kernel for 128-wide bf16
-// heads takes them (the tokens' heads share the N side of its MMAs, so q_len * group <= 8).
-static int multi_supported(const snap_config_t* cfg, const Shape& s, int q_len) {
-  if (q_len < 1 || q_len > s.Lr) return SNAP_ERR_INVALID_ARG;
-  if (!decode_use_gqa_mma(cfg->dtype, s) || q_len * s.g > 8)
-    return SNAP_ERR_UNSUPPORTED;
-  return SNAP_OK;
+// Several query tokens per sequence in one step.  The tensor-core kernel for bf16 heads serves
+// them in one pass over the cache (the tokens' heads share the N side of its MMAs, so
+// q_len * group <= 8); every other shape is served as the definition reads: q_len single steps,
+// each token's rows staged densely in the workspace by strided device-to-device copies.
+static int multi_check(const Shape& s, int q_len) {
+  return q_len < 1 || q_len > s.Lr ? SNAP_ERR_INVALID_ARG : SNAP_OK;
+}
+static bool multi_one_pass(const snap_config_t* cfg, const Shape& s, int q_len) {
+  return decode_use_gqa_mma(cfg->dtype, s) && q_len * s.g <= 8;
+}
+
+// Dense staging of one token's rows for the step-wise path: q, k_new, v_new, out.
+struct StepStage { size_t q_row, k_row, v_row, o_row, q_off, k_off, v_off, o_off, bytes; };
+static StepStage step_stage(const snap_config_t* cfg, const Shape& s, int n_active) {
+  StepStage t;
+  const size_t eb = (size_t)elt_bytes(cfg->dtype), n = (size_t)(n_active > 0 ? n_active : 0);
+  t.q_row = (size_t)s.Hq * s.d_qk * eb;
+  t.k_row = (size_t)s.Hkv * s.d_qk * eb;
+  t.v_row = s.v_aliases_k ? 0 : (size_t)s.Hkv * s.d_v * eb;
+  t.o_row = (size_t)s.Hq * s.d_v * eb;
+  size_t off = 0;
+  t.q_off = off; off += align_up(n * t.q_row);
+  t.k_off = off; off += align_up(n * t.k_row);
+  t.v_off = off; off += align_up(n * t.v_row);
+  t.o_off = off; off += align_up(n * t.o_row);
+  t.bytes = off;
+  return t;
 }
 
 int64_t snap_decode_multi_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t q_len) {
@@ -463,10 +483,15 @@ int64_t snap_decode_multi_workspace_bytes(const snap_config_t* cfg, int32_t n_ac
   if (rc != SNAP_OK) return rc;
   if (n_active < 0) return SNAP_ERR_INVALID_ARG;
   const Shape s = make_shape(cfg);
-  const int ms = multi_supported(cfg, s, q_len);
-  if (ms != SNAP_OK) return ms;
-  const int nsplit = decode_gqa_mma_nsplit(s, n_active > 0 ? n_active : 1, sm_count());
-  return (int64_t)(decode_gqa_mma_partial_floats(s, n_active * q_len, nsplit) * sizeof(float) + 256);
+  const int mc = multi_check(s, q_len);
+  if (mc != SNAP_OK) return mc;
+  if (multi_one_pass(cfg, s, q_len)) {
+    const int nsplit = decode_gqa_mma_nsplit(s, n_active > 0 ? n_active : 1, sm_count());
+    return (int64_t)(decode_gqa_mma_partial_floats(s, n_active * q_len, nsplit) * sizeof(float) + 256);
+  }
+  const int64_t single = snap_decode_workspace_bytes(cfg, n_active);
+  if (single < 0) return single;
+  return (int64_t)step_stage(cfg, s, n_active).bytes + single;
 }
 
 int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,
@@ -479,22 +504,49 @@ int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout
   if (!layout) return SNAP_ERR_NULL_POINTER;
   if (n_active < 0) return SNAP_ERR_INVALID_ARG;
   const Shape s = make_shape(cfg);
-  const int ms = multi_supported(cfg, s, q_len);
-  if (ms != SNAP_OK) return ms;
+  const int mc = multi_check(s, q_len);
+  if (mc != SNAP_OK) return mc;
   if (n_active == 0) return SNAP_OK;
-  if (!q_dev || !k_new_dev || !v_new_dev || !slot_ids_dev || !k_cache_dev || !v_cache_dev || !seq_len_dev ||
-      !valid_topk_dev || !out_dev || !workspace_dev)
+  if (!q_dev || !k_new_dev || !slot_ids_dev || !k_cache_dev || !seq_len_dev || !valid_topk_dev || !out_dev ||
+      !workspace_dev)
     return SNAP_ERR_NULL_POINTER;
+  if (!s.v_aliases_k && (!v_new_dev || !v_cache_dev)) return SNAP_ERR_NULL_POINTER;
   if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
   const int64_t need = snap_decode_multi_workspace_bytes(cfg, n_active, q_len);
   if (need < 0) return (int)need;
   if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
-  const int nsplit = decode_gqa_mma_nsplit(s, n_active, sm_count());
-  const cudaError_t e = launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
-                                              v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
-                                              static_cast<float*>(workspace_dev), nsplit, status_dev,
-                                              static_cast<cudaStream_t>(cuda_stream), q_len);
-  return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (multi_one_pass(cfg, s, q_len)) {
+    const int nsplit = decode_gqa_mma_nsplit(s, n_active, sm_count());
+    const cudaError_t e = launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
+                                                v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
+                                                static_cast<float*>(workspace_dev), nsplit, status_dev, st, q_len);
+    return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+  }
+  // q_len single steps: token u of every sequence is gathered into dense rows, attended, and its
+  // output scattered back
+  const StepStage t = step_stage(cfg, s, n_active);
+  char* ws = static_cast<char*>(workspace_dev);
+  char* single_ws = ws + t.bytes;
+  const size_t single_bytes = workspace_bytes - t.bytes;
+  auto gather = [&](char* dst, const void* src, size_t row, int u) {
+    return row == 0 ? cudaSuccess
+                    : cudaMemcpy2DAsync(dst, row, static_cast<const char*>(src) + (size_t)u * row, (size_t)q_len * row, row,
+                                        (size_t)n_active, cudaMemcpyDeviceToDevice, st);
+  };
+  for (int u = 0; u < q_len; ++u) {
+    if (gather(ws + t.q_off, q_dev, t.q_row, u) != cudaSuccess || gather(ws + t.k_off, k_new_dev, t.k_row, u) != cudaSuccess ||
+        gather(ws + t.v_off, v_new_dev, t.v_row, u) != cudaSuccess)
+      return SNAP_ERR_CUDA;
+    const int r = snap_decode_attn(cfg, layout, ws + t.q_off, ws + t.k_off, s.v_aliases_k ? nullptr : ws + t.v_off,
+                                   slot_ids_dev, n_active, k_cache_dev, v_cache_dev, seq_len_dev, valid_topk_dev,
+                                   ws + t.o_off, single_ws, single_bytes, status_dev, cuda_stream);
+    if (r != SNAP_OK) return r;
+    if (cudaMemcpy2DAsync(static_cast<char*>(out_dev) + (size_t)u * t.o_row, (size_t)q_len * t.o_row, ws + t.o_off, t.o_row,
+                          t.o_row, (size_t)n_active, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return SNAP_ERR_CUDA;
+  }
+  return SNAP_OK;
 }
 
 }  // extern "C"

@@ -391,14 +391,14 @@ def _run_multi(wl, lengths, q_len, steps, seed):
         ds = [synth.make_decode_inputs(wl, n, seed, step * q_len + u) for u in range(q_len)]
         q = torch.stack([d["q"] for d in ds], dim=1).contiguous().cuda()            # [n][q_len][Hq][d]
         kn = torch.stack([d["k_new"] for d in ds], dim=1).contiguous().cuda()
-        vn = torch.stack([d["v_new"] for d in ds], dim=1).contiguous().cuda()
+        vn = None if wl.v_aliases_k else torch.stack([d["v_new"] for d in ds], dim=1).contiguous().cuda()
         out = torch.empty(n, q_len, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device="cuda")
         B.snap_decode_attn_multi(layer.cfg, layer.layout, q, kn, vn, slots_dev, n, q_len, c.k_cache, c.v_cache,
                                  c.seq_len, c.valid_topk, out, ws, c.status)
         for i in range(n):
             for u in range(q_len):
                 ref = orc.decode_step(seqs[i], synth.to_f64(ds[u]["q"][i]), synth.to_f64(ds[u]["k_new"][i]),
-                                      synth.to_f64(ds[u]["v_new"][i]))
+                                      None if wl.v_aliases_k else synth.to_f64(ds[u]["v_new"][i]))
                 H.check_output(out[i, u], ref, wl, f"step {step} seq {i} token {u}")
     assert layer.status() == 0
     for i in range(n):
@@ -416,19 +416,22 @@ def test_multi_token_decode_steps(hq, hkv, q_len):
     _run_multi(wl, [1, 3, 45, 50, 51, 52, 300, wl.prompt_len[0]], q_len, steps=max(4, 60 // q_len), seed=83)
 
 
-def test_multi_token_decode_rejects_what_it_cannot_do():
-    wl = SMALL_BF16                                   # 4 heads per KV head
+@pytest.mark.parametrize("wl,q_len", [(SMALL_BF16, 3), (SMALL_F32, 2), (SMALL_MLA, 3), (LATENT_128, 2)],
+                         ids=["bf16_g4x3", "f32_g4x2", "latent_x3", "latent_128_heads_x2"])
+def test_multi_token_decode_on_shapes_served_step_by_step(wl, q_len):
+    """Shapes the one-pass kernel does not take (more than 8 query rows per KV head, fp32, the latent
+    layout) go through q_len single steps inside the library: same definition, same results."""
+    _run_multi(wl, [1, 3, 45, 50, 51, 52, 300, wl.prompt_len[0]], q_len, steps=6, seed=87)
+
+
+def test_multi_token_decode_rejects_invalid_token_counts():
+    wl = SMALL_BF16
     layer = H.GpuLayer(wl, 1)
-    with pytest.raises(B.SnapError) as e:
-        B.snap_decode_multi_workspace_bytes(layer.cfg, 1, 3)          # 3 tokens x 4 heads > 8 columns
-    assert e.value.code == -2
-    with pytest.raises(B.SnapError) as e:
-        B.snap_decode_multi_workspace_bytes(layer.cfg, 1, 0)
-    assert e.value.code == -1
-    f32 = H.GpuLayer(SMALL_F32, 1)
-    with pytest.raises(B.SnapError) as e:
-        B.snap_decode_multi_workspace_bytes(f32.cfg, 1, 2)            # no fp32 kernel for it
-    assert e.value.code == -2
+    for q_len in (0, wl.l_recent + 1):                # at least one token, at most a window's worth
+        with pytest.raises(B.SnapError) as e:
+            B.snap_decode_multi_workspace_bytes(layer.cfg, 1, q_len)
+        assert e.value.code == -1
+    assert B.snap_decode_multi_workspace_bytes(layer.cfg, 4, 3) > B.snap_decode_workspace_bytes(layer.cfg, 4)
 
 
 @pytest.mark.parametrize("wl", [SMALL_BF16, LATENT_128, SMALL_F32], ids=lambda w: w.name)
