@@ -157,11 +157,13 @@ int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout,
  *               log2( sum over candidates j in [Ls, L - Lr) of exp(scale * q . k_j) ),
  *             -inf when the prompt has no candidate.  This is what snap_compress_with_row_stats
  *             takes in place of its own first pass over the keys.
- * Built for bf16 layers with d_qk = d_v = 128 and separate V (SNAP_ERR_UNSUPPORTED otherwise).
- * Needs no workspace.  cfg is validated as a whole (as by snap_cache_layout); the kernel uses its
+ * bf16 layers with d_qk = d_v = 128 and a separate V run on the tensor cores; every other layer
+ * (fp32, other head sizes, the latent layout, where v_dev is ignored) runs on a portable kernel
+ * that is there for coverage, not for speed.
+ * Needs no workspace.  cfg is validated as a whole (as by snap_cache_layout); the kernels use its
  * model-shape fields, l_sink, l_recent, l_obs and softmax_scale.  Errors: SNAP_ERR_NULL_POINTER,
- * SNAP_ERR_INVALID_ARG (cfg, offsets that decrease, strides that are not multiples of 16 bytes),
- * SNAP_ERR_UNSUPPORTED: nothing was launched; SNAP_ERR_CUDA: a launch failed.
+ * SNAP_ERR_INVALID_ARG (cfg, offsets that decrease, strides that are not multiples of 16 bytes):
+ * nothing was launched; SNAP_ERR_CUDA: a launch failed.
  */
 int snap_prefill_attn(const snap_config_t* cfg, const void* q_dev,
                       const void* k_dev, int64_t k_token_stride, int64_t k_head_stride,
@@ -174,10 +176,9 @@ int snap_prefill_attn(const snap_config_t* cfg, const void* q_dev,
  * snap_compress with the Eq. 4 normalisers supplied by the caller (row_mu_dev as written by
  * snap_prefill_attn; NULL = compute them here, which is snap_compress): the score kernel then
  * makes one pass over the candidate keys instead of two.  Same arguments, results, workspace
- * and errors as snap_compress otherwise.  Consumed by the tensor-core score kernels (bf16,
- * d_qk a multiple of 64 up to 576); SNAP_ERR_UNSUPPORTED for other layers when a prompt has to
- * be scored.  The selection can differ from snap_compress's only where two pooled scores are
- * equal to within single-precision rounding.
+ * and errors as snap_compress otherwise; every score kernel takes them.  The selection can
+ * differ from snap_compress's only where two pooled scores are equal to within single-precision
+ * rounding.
  */
 int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* layout,
                   const void* q_obs_dev, const float* row_mu_dev,

@@ -188,12 +188,14 @@ def snap_compress_with_row_stats(cfg: SnapConfig, layout: SnapLayout, q_obs, row
 
 def snap_prefill_attn(cfg: SnapConfig, q, k, v, cu_seqlens: Sequence[int], out, row_mu=None, status=None,
                       stream=None) -> None:
-    """Causal attention of whole prompts.  q: [T, Hq, d] dense; k, v: [T, Hkv, d] (dense last dim);
+    """Causal attention of whole prompts.  q: [T, Hq, d] dense; k, v: [T, Hkv, d] (dense last dim; v None for
+    the latent layout);
     out: [T, Hq, d_v]; row_mu: None or [n_seq, Hq, Lo] float32 receiving the Eq. 4 normalisers."""
     cu = _i32_array(cu_seqlens)
-    _check(lib().snap_prefill_attn(C.byref(cfg), _ptr(q), _ptr(k), k.stride(0), k.stride(1), _ptr(v), v.stride(0),
-                                   v.stride(1), cu, len(cu_seqlens) - 1, _ptr(out), _ptr(row_mu), _ptr(status),
-                                   _stream(stream)), "snap_prefill_attn")
+    vs = (v.stride(0), v.stride(1)) if v is not None else (0, 0)
+    _check(lib().snap_prefill_attn(C.byref(cfg), _ptr(q), _ptr(k), k.stride(0), k.stride(1), _ptr(v), vs[0], vs[1], cu,
+                                   len(cu_seqlens) - 1, _ptr(out), _ptr(row_mu), _ptr(status), _stream(stream)),
+           "snap_prefill_attn")
 
 
 def snap_append_kv(cfg: SnapConfig, layout: SnapLayout, k_new, v_new, slot_ids_dev, n_active: int, k_cache,

@@ -264,12 +264,15 @@ int snap_prefill_attn(const snap_config_t* cfg, const void* q_dev,
   rc = check_cu(cu_seqlens_host, n_seq);
   if (rc != SNAP_OK) return rc;
   const Shape s = make_shape(cfg);
-  if (!prefill_attn_supported(cfg->dtype, s)) return SNAP_ERR_UNSUPPORTED;
   if (n_seq == 0 || cu_seqlens_host[n_seq] == cu_seqlens_host[0]) return SNAP_OK;
-  if (!q_dev || !k_dev || !v_dev || !out_dev) return SNAP_ERR_NULL_POINTER;
-  if ((k_token_stride * 2) % 16 || (k_head_stride * 2) % 16 || k_token_stride < s.d_qk || (v_token_stride * 2) % 16 ||
-      (v_head_stride * 2) % 16 || v_token_stride < s.d_v)
+  if (!q_dev || !k_dev || !out_dev || (!cfg->v_aliases_k && !v_dev)) return SNAP_ERR_NULL_POINTER;
+  const int eb = elt_bytes(cfg->dtype);
+  if ((k_token_stride * eb) % 16 || (k_head_stride * eb) % 16 || k_token_stride < s.d_qk) return SNAP_ERR_INVALID_ARG;
+  if (!cfg->v_aliases_k && ((v_token_stride * eb) % 16 || (v_head_stride * eb) % 16 || v_token_stride < s.d_v))
     return SNAP_ERR_INVALID_ARG;
+  // SNAP_PREFILL_PATH=simt forces the portable kernel (testing aid)
+  const char* env = getenv("SNAP_PREFILL_PATH");
+  const bool tensor_path = prefill_attn_supported(cfg->dtype, s) && !(env && !strcmp(env, "simt"));
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   KVSource src;
   src.k = k_dev; src.v = v_dev;
@@ -284,7 +287,9 @@ int snap_prefill_attn(const snap_config_t* cfg, const void* q_dev,
       b.tok_off[i] = cu_seqlens_host[first + i];
       b.len[i] = cu_seqlens_host[first + i + 1] - cu_seqlens_host[first + i];
     }
-    if (launch_prefill_attn(s, b, q_dev, src, out_dev, row_mu_dev, status_dev, st) != cudaSuccess) return SNAP_ERR_CUDA;
+    const cudaError_t e = tensor_path ? launch_prefill_attn(s, b, q_dev, src, out_dev, row_mu_dev, status_dev, st)
+                                      : launch_prefill_generic(cfg->dtype, s, b, q_dev, src, out_dev, row_mu_dev, st);
+    if (e != cudaSuccess) return SNAP_ERR_CUDA;
   }
   return SNAP_OK;
 }
@@ -328,8 +333,6 @@ int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* 
     if (s.K > 0 && L - s.Ls - s.Lr > s.K) any_scored = true;
   }
   if (any_scored && !q_obs_dev) return SNAP_ERR_NULL_POINTER;
-  // normalisers from outside are consumed by the tcgen05 score kernels only
-  if (any_scored && row_mu_dev && !use_umma(cfg->dtype, s) && !use_umma_wide(cfg->dtype, s)) return SNAP_ERR_UNSUPPORTED;
   if ((any_scored || !topk_idx_dev) && s.K > 0) {
     if (!workspace_dev) return SNAP_ERR_NULL_POINTER;
     if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;

@@ -101,7 +101,11 @@ __global__ void __launch_bounds__(256, 2) score_mma_kernel(const MmaArgs a) {
     const int row = 32 * w + 8 * (c >> 1) + 2 * (lane & 3) + (c & 1);
     if (PASS == 1) { cm[c] = -INFINITY; cl[c] = 0.f; }
     else {
-      const float2 st = row < R ? a.buf.stats[(long long)z * R + row] : make_float2(0.f, 0.f);
+      float2 st = make_float2(0.f, 0.f);
+      if (row < R)
+        st = a.buf.ext_mu   // log2 normaliser from outside: (m, 1/l) = (mu, 1)
+                 ? make_float2(a.buf.ext_mu[((long long)(a.b.first_seq + seq) * a.Hq + (long long)kvh * a.g) * a.Lo + row], 1.f)
+                 : a.buf.stats[(long long)z * R + row];
       cm[c] = st.x; cl[c] = st.y;
     }
   }
@@ -318,9 +322,11 @@ cudaError_t launch_score_mma(const Shape& s, const SeqBatch& b, const void* q_ob
   if (cudaError_t e = ensure_dyn_smem(score_mma_kernel<2>, 110 * 1024, limit2)) return e;
   const int nz = b.n_scored * s.Hkv;
   dim3 grid(buf.nsplit, nz);
-  score_mma_kernel<1><<<grid, 32 * nrw, smem, st>>>(a);
-  count_launch();
-  if (launch_score_combine_log2(buf, nz, a.R, st) != cudaSuccess) return cudaGetLastError();
+  if (!buf.ext_mu) {                                          // Eq. 4's normalisers, unless the caller has them
+    score_mma_kernel<1><<<grid, 32 * nrw, smem, st>>>(a);
+    count_launch();
+    if (launch_score_combine_log2(buf, nz, a.R, st) != cudaSuccess) return cudaGetLastError();
+  }
   score_mma_kernel<2><<<grid, 32 * nrw, smem, st>>>(a);
   count_launch();
   return cudaGetLastError();

@@ -167,7 +167,11 @@ __global__ void __launch_bounds__(NT) score_colsum_kernel(const ScoreArgs a) {
   for (int row0 = 0; row0 < R; row0 += BM) {
     if (threadIdx.x < BM) {
       const int row = row0 + threadIdx.x;
-      st[threadIdx.x] = row < R ? a.buf.stats[(long long)z * R + row] : make_float2(0.f, 0.f);
+      if (row >= R) st[threadIdx.x] = make_float2(0.f, 0.f);
+      else if (a.buf.ext_mu)                                   // log2 normaliser from outside: (m, 1/l) = (mu ln 2, 1)
+        st[threadIdx.x] = make_float2(
+            a.buf.ext_mu[((long long)(a.b.first_seq + seq) * a.Hq + (long long)kvh * a.g) * a.Lo + row] * 0.6931471805599453f, 1.f);
+      else st[threadIdx.x] = a.buf.stats[(long long)z * R + row];
     }
     tile_scores<T>(qbase, kbase, a.k_tok_stride, a.d, R, Le, row0, cand0, acc, As, Bs);
 #pragma unroll
@@ -195,11 +199,13 @@ template <typename T>
 cudaError_t launch_t(const ScoreArgs& a, int max_le, cudaStream_t st) {
   const int R = a.g * a.Lo;
   const int nz = a.b.n_scored * a.Hkv;
-  dim3 g1(a.buf.nsplit, (R + BM - 1) / BM, nz);
-  score_stats_kernel<T><<<g1, NT, 0, st>>>(a);
-  count_launch();
-  score_combine_kernel<<<nz, 256, 0, st>>>(a.buf.part_stats, a.buf.stats, a.buf.nsplit, R);
-  count_launch();
+  if (!a.buf.ext_mu) {                                        // Eq. 4's normalisers, unless the caller has them
+    dim3 g1(a.buf.nsplit, (R + BM - 1) / BM, nz);
+    score_stats_kernel<T><<<g1, NT, 0, st>>>(a);
+    count_launch();
+    score_combine_kernel<<<nz, 256, 0, st>>>(a.buf.part_stats, a.buf.stats, a.buf.nsplit, R);
+    count_launch();
+  }
   dim3 g2((max_le + BN - 1) / BN, 1, nz);
   score_colsum_kernel<T><<<g2, NT, 0, st>>>(a);
   count_launch();

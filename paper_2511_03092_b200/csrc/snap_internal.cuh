@@ -109,6 +109,9 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
 bool prefill_attn_supported(int dtype, const Shape& s);
 cudaError_t launch_prefill_attn(const Shape& s, const SeqBatch& b, const void* q, const KVSource& src, void* out,
                                 float* mu, uint32_t* status, cudaStream_t st);
+// portable version (any element type and head sizes, the latent layout included)
+cudaError_t launch_prefill_generic(int dtype, const Shape& s, const SeqBatch& b, const void* q, const KVSource& src,
+                                   void* out, float* mu, cudaStream_t st);
 cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffers& buf,
                              int* idx_out, uint32_t* status, cudaStream_t st);
 cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KVSource& src,

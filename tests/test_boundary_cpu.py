@@ -117,9 +117,10 @@ def test_prefill_entry_points_validate_before_touching_memory():
     assert pre(C.byref(cfg), cu_bad, 2) == -1                                # decreasing offsets
     assert pre(C.byref(cfg), None, 1) == -4
     assert pre(C.byref(_cfg(softmax_scale=-1.0)), cu, 1) == -1
-    latent = _cfg(n_q_heads=128, n_kv_heads=1, d_qk=576, d_v=512, v_aliases_k=True, l_recent=2048, topk=8192, l_obs=32)
-    assert pre(C.byref(latent), cu, 1) == -2                                 # no prefill kernel for the latent layout
-    assert pre(C.byref(_cfg(dtype=B.SNAP_F32)), cu, 1) == -2
+    assert lib.snap_prefill_attn(C.byref(cfg), one, one, 1023, 128, one, 1024, 128, cu, 1, one, None, None, None) == -1
+    assert lib.snap_prefill_attn(C.byref(cfg), one, one, 1024, 128, None, 1024, 128, cu, 1, one, None, None, None) == -4
+    empty = (C.c_int32 * 3)(0, 0, 0)
+    assert pre(C.byref(cfg), empty, 2) == 0                                  # nothing to do
     # the compress variant shares snap_compress's validation
     ok_slot = (C.c_int32 * 1)(0)
     bad_slot = (C.c_int32 * 1)(7)

@@ -153,22 +153,79 @@ def test_prefill_reads_strided_keys_and_values():
     assert torch.equal(mu2, mu)
 
 
-def test_prefill_rejects_what_it_cannot_do():
-    wl = synth.Workload("mla", 16, 1, 96, 64, "bf16", 3, 40, 64, 8, 5, batch=1, prompt_len=(100, 100),
-                        decode_steps=1, salience="none", v_aliases_k=True)
-    cfg = H.snap_config(wl, 1)
-    t = torch.zeros(4, 16, 96, dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(B.SnapError) as e:
-        B.snap_prefill_attn(cfg, t, t[:, :1], t[:, :1], [0, 4], t, None)
-    assert e.value.code == -2
-    f32 = WL64.scaled(dtype="f32")
-    lay = H.GpuLayer(f32, 1)
-    x = torch.zeros(200, 8, 128, device="cuda")
-    kv = torch.zeros(200, 2, 128, device="cuda")
-    mu = torch.zeros(1, 8, 16, device="cuda")
-    ws = torch.empty(B.snap_compress_workspace_bytes(lay.cfg, [0, 200]), dtype=torch.uint8, device="cuda")
-    c = lay.cache
-    with pytest.raises(B.SnapError) as e:
-        B.snap_compress_with_row_stats(lay.cfg, lay.layout, x[:16].reshape(1, 8, 16, 128), mu, kv, kv, [0, 200], [0],
-                                       c.k_cache, c.v_cache, c.seq_len, c.valid_topk, None, ws, c.status)
-    assert e.value.code == -2
+WL_F32 = WL64.scaled(name="prefill_f32", dtype="f32", salience="planted", n_planted=12)
+WL_D64 = WL64.scaled(name="prefill_d64", d_qk=64, d_v=64)
+WL_LATENT = synth.Workload("prefill_latent", 16, 1, 96, 64, "bf16", 3, 40, 64, 8, 5, batch=1, prompt_len=(500, 500),
+                           decode_steps=1, salience="planted", n_planted=8, v_aliases_k=True,
+                           softmax_scale=2.0 ** -0.5)
+
+
+def _prefill_any(wl, lengths, seed):
+    """Like _prefill, for layouts without a separate V as well."""
+    n = len(lengths)
+    prompts = [synth.make_prompt(wl, L, seed + i) for i, L in enumerate(lengths)]
+    qs = [synth.make_prompt_queries(wl, p, seed + i) for i, p in enumerate(prompts)]
+    cu = [0]
+    for L in lengths:
+        cu.append(cu[-1] + L)
+    layer = H.GpuLayer(wl, max_seqs=n + 1)
+    q = torch.cat(qs).cuda()
+    k = torch.cat([p["k"] for p in prompts]).cuda()
+    v = None if wl.v_aliases_k else torch.cat([p["v"] for p in prompts]).cuda()
+    out = torch.full((cu[-1], wl.n_q_heads, wl.d_v), float("nan"), dtype=wl.torch_dtype, device="cuda")
+    mu = torch.full((n, wl.n_q_heads, wl.l_obs), float("nan"), dtype=torch.float32, device="cuda")
+    B.snap_prefill_attn(layer.cfg, q, k, v, cu, out, mu, layer.cache.status)
+    assert layer.status() == 0
+    return layer, prompts, qs, cu, (k, v), out, mu
+
+
+@pytest.mark.parametrize("wl", [WL_F32, WL_D64, WL_LATENT], ids=lambda w: w.name)
+def test_portable_prefill_kernel_and_every_score_path_take_the_normalisers(wl):
+    """fp32, 64-wide heads and the latent layout: the portable prefill kernel, then compression with its
+    normalisers through the SIMT, mma.sync-free and wide tcgen05 score paths these shapes select."""
+    lengths = [1, 5, 33, 150, 420]
+    layer, prompts, qs, cu, (k, v), out, mu = _prefill_any(wl, lengths, seed=370)
+    ocfg = H.oracle_config(wl)
+    mu_host = mu.cpu().numpy().astype(np.float64)
+    for i, (p, q, L) in enumerate(zip(prompts, qs, lengths)):
+        kk = synth.to_f64(p["k"])
+        vv = kk[:, :, :wl.d_v] if wl.v_aliases_k else synth.to_f64(p["v"])
+        ref = orc.prefill_attention(synth.to_f64(q), kk, vv, ocfg)
+        H.check_output(out[cu[i]:cu[i + 1]], ref, wl, f"prompt {i} (L={L})")
+        n = min(L, wl.l_obs)
+        want = orc.candidate_log2_normalisers(synth.to_f64(p["q_obs"]), kk, ocfg)[:, wl.l_obs - n:]
+        got = mu_host[i][:, wl.l_obs - n:]
+        if np.isneginf(want).all():
+            assert np.isneginf(got).all()
+        else:
+            np.testing.assert_allclose(got, want, rtol=0, atol=MU_ATOL, err_msg=f"prompt {i} (L={L})")
+    n = len(lengths)
+    slots = list(range(n))
+    q_obs = torch.stack([p["q_obs"] for p in prompts]).cuda()
+    ws = torch.empty(B.snap_compress_workspace_bytes(layer.cfg, cu), dtype=torch.uint8, device="cuda")
+    idx = torch.full((n, wl.n_kv_heads, wl.topk), -7, dtype=torch.int32, device="cuda")
+    c = layer.cache
+    B.snap_compress_with_row_stats(layer.cfg, layer.layout, q_obs, mu, k, v, cu, slots, c.k_cache, c.v_cache, c.seq_len,
+                                   c.valid_topk, idx, ws, c.status)
+    assert layer.status() == 0
+    idx = idx.cpu().numpy()
+    for i, p in enumerate(prompts):
+        seq = H.oracle_compress(wl, p)
+        H.check_selection(idx[i], seq, wl)
+        seq.topk_pos = [idx[i][h][idx[i][h] >= 0].astype(np.int64) for h in range(wl.n_kv_heads)]
+        H.check_cache_image(layer, seq, slots[i], wl)
+
+
+def test_normalisers_through_the_mma_sync_score_path(monkeypatch):
+    monkeypatch.setenv("SNAP_SCORE_PATH", "mma")
+    test_compress_with_prefill_normalisers_matches_oracle(WL128)
+
+
+def test_portable_prefill_kernel_matches_the_tensor_core_one(monkeypatch):
+    wl = WL64
+    lengths = [129, 300]
+    _, _, _, cu, _, out_t, mu_t = _prefill(wl, lengths, seed=380)
+    monkeypatch.setenv("SNAP_PREFILL_PATH", "simt")
+    _, _, _, _, _, out_s, mu_s = _prefill(wl, lengths, seed=380)
+    assert (out_t.float() - out_s.float()).abs().max().item() <= 2e-2
+    assert (mu_t - mu_s).abs().max().item() <= 2 * MU_ATOL
