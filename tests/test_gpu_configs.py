@@ -107,3 +107,39 @@ def test_config4_one_sequence_layer_unit():
     wl = synth.CONFIGS[4]
     swaps = _run(wl, [131072], seed=500, steps=4)
     assert swaps <= 2
+
+
+def test_config1_prompt_attention_hands_its_normalisers_to_the_compression():
+    """Llama-shaped bf16 layer, prompt 32768, the launch shape bench.py's prefill extra uses: the
+    prompt's causal attention checked on sampled (position, head) pairs the oracle computes one by
+    one, every normaliser of the observation window, and the selection made from them."""
+    from paper_2511_03092_b200 import binding as B
+    wl = synth.CONFIGS[1]
+    L = 32768
+    p = synth.make_prompt(wl, L, 200)
+    q = synth.make_prompt_queries(wl, p, 200)
+    layer = H.GpuLayer(wl, max_seqs=1)
+    qd, kd, vd = q.cuda(), p["k"].cuda(), p["v"].cuda()
+    out = torch.empty(L, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device="cuda")
+    mu = torch.full((1, wl.n_q_heads, wl.l_obs), float("nan"), dtype=torch.float32, device="cuda")
+    c = layer.cache
+    B.snap_prefill_attn(layer.cfg, qd, kd, vd, [0, L], out, mu, c.status)
+    assert layer.status() == 0
+    ocfg = H.oracle_config(wl)
+    k64, v64 = synth.to_f64(p["k"]), synth.to_f64(p["v"])
+    rng = np.random.default_rng(201)
+    rows = [0, 1, 127, 128, 129, 4095, 4096, L - wl.l_obs - 1, L - wl.l_obs, L - 1] + [int(x) for x in rng.integers(0, L, 6)]
+    for t in rows:
+        for h in (0, int(rng.integers(0, wl.n_q_heads)), wl.n_q_heads - 1):
+            kvh = h // (wl.n_q_heads // wl.n_kv_heads)
+            ref = orc.attention_over(synth.to_f64(q[t, h]), k64[: t + 1, kvh], v64[: t + 1, kvh], ocfg.softmax_scale)
+            H.check_output(out[t, h], ref, wl, f"position {t} head {h}")
+    want = orc.candidate_log2_normalisers(synth.to_f64(p["q_obs"]), k64, ocfg)
+    np.testing.assert_allclose(mu[0].cpu().numpy().astype(np.float64), want, rtol=0, atol=1e-3)
+    ws = torch.empty(B.snap_compress_workspace_bytes(layer.cfg, [0, L]), dtype=torch.uint8, device="cuda")
+    idx = torch.full((1, wl.n_kv_heads, wl.topk), -7, dtype=torch.int32, device="cuda")
+    B.snap_compress_with_row_stats(layer.cfg, layer.layout, p["q_obs"][None].cuda(), mu, kd, vd, [0, L], [0], c.k_cache,
+                                   c.v_cache, c.seq_len, c.valid_topk, idx, ws, c.status)
+    assert layer.status() == 0
+    seq = H.oracle_compress(wl, p)
+    H.check_selection(idx.cpu().numpy()[0], seq, wl)
