@@ -1,6 +1,7 @@
 """Seeded random small configurations through the C ABI against the oracle: head size, group size,
 sink / window / budget sizes, pooling width, ragged prompt lengths, one or several tokens per step,
-and the latent layout with 64, 128 and 256 heads.  Every case checks the selected indices, every
+the latent layout with 64, 128 and 256 heads, and the prompt attention that feeds the compression
+its normalisers.  Every case checks the selected indices, every
 decode output, the sequence lengths and the final cache image."""
 import numpy as np
 import pytest
@@ -124,3 +125,57 @@ def test_random_compress_configurations():
         layer, seqs = _compress_and_check(wl, [L], 77 * case + 1)
         assert layer.status() == 0, f"case {case}"
         H.check_cache_image(layer, seqs[0], 0, wl)
+
+
+@pytest.mark.parametrize("seed", [11, 12])
+def test_random_prefill_configurations(seed):
+    """Prompt attention, its Eq. 4 normalisers, and the compression that takes them: random head size (the
+    tensor-core kernel for 128, the portable one otherwise), group size, hyper-parameters and ragged batches."""
+    rng = np.random.default_rng(seed)
+    for case in range(14):
+        d = int(rng.choice([128, 128, 128, 64, 256]))
+        hkv = int(rng.choice([1, 2, 4]))
+        g = int(rng.integers(1, 9))
+        Ls, Lr, K = int(rng.integers(0, 6)), int(rng.integers(1, 70)), int(rng.choice([5, 16, 33, 64]))
+        Lo, w = int(rng.integers(1, min(Lr, 40) + 1)), int(rng.choice([1, 3, 7]))
+        wl = synth.Workload("rnd", g * hkv, hkv, d, d, "bf16", Ls, Lr, K, Lo, w, batch=1, prompt_len=(100, 100),
+                            decode_steps=1, salience="zipf")
+        n = int(rng.integers(1, 5))
+        lengths = [int(rng.integers(1, 420)) for _ in range(n)]
+        what = f"case {case}: d{d} hkv{hkv} g{g} Ls{Ls} Lr{Lr} K{K} Lo{Lo} w{w} L{lengths}"
+        prompts = [synth.make_prompt(wl, L, 1000 * case + seed + i) for i, L in enumerate(lengths)]
+        qs = [synth.make_prompt_queries(wl, p, 1000 * case + seed + i) for i, p in enumerate(prompts)]
+        cu = [0]
+        for L in lengths:
+            cu.append(cu[-1] + L)
+        layer = H.GpuLayer(wl, n)
+        q = torch.cat(qs).cuda()
+        k = torch.cat([p["k"] for p in prompts]).cuda()
+        v = torch.cat([p["v"] for p in prompts]).cuda()
+        out = torch.full((cu[-1], wl.n_q_heads, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+        mu = torch.full((n, wl.n_q_heads, Lo), float("nan"), dtype=torch.float32, device="cuda")
+        c = layer.cache
+        B.snap_prefill_attn(layer.cfg, q, k, v, cu, out, mu, c.status)
+        ocfg = H.oracle_config(wl)
+        mu_host = mu.cpu().numpy().astype(np.float64)
+        for i, (p, qq, L) in enumerate(zip(prompts, qs, lengths)):
+            ref = orc.prefill_attention(synth.to_f64(qq), synth.to_f64(p["k"]), synth.to_f64(p["v"]), ocfg)
+            H.check_output(out[cu[i]:cu[i + 1]], ref, wl, f"{what} prompt {i}")
+            m = min(L, Lo)
+            want = orc.candidate_log2_normalisers(synth.to_f64(p["q_obs"]), synth.to_f64(p["k"]), ocfg)[:, Lo - m:]
+            got = mu_host[i][:, Lo - m:]
+            if np.isneginf(want).all():
+                assert np.isneginf(got).all(), what
+            else:
+                np.testing.assert_allclose(got, want, rtol=0, atol=1e-3, err_msg=what)
+        ws = torch.empty(B.snap_compress_workspace_bytes(layer.cfg, cu), dtype=torch.uint8, device="cuda")
+        idx = torch.full((n, hkv, K), -7, dtype=torch.int32, device="cuda")
+        B.snap_compress_with_row_stats(layer.cfg, layer.layout, torch.stack([p["q_obs"] for p in prompts]).cuda(), mu, k, v,
+                                       cu, list(range(n)), c.k_cache, c.v_cache, c.seq_len, c.valid_topk, idx, ws, c.status)
+        assert layer.status() == 0, what
+        idx = idx.cpu().numpy()
+        for i, p in enumerate(prompts):
+            seq = H.oracle_compress(wl, p)
+            H.check_selection(idx[i], seq, wl)
+            seq.topk_pos = [idx[i][h][idx[i][h] >= 0].astype(np.int64) for h in range(hkv)]
+            H.check_cache_image(layer, seq, i, wl)
