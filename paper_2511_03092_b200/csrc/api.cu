@@ -86,7 +86,7 @@ bool use_mma(int dtype, const Shape& s) {
 
 // Scratch regions of one chunk of prompts (offsets relative to the chunk area).
 struct ChunkPlan {
-  int n_scored, max_le, nsplit, c_stride;
+  int n_scored, min_le, max_le, nsplit, c_stride;
   size_t part_off, stats_off, c_off, p_off, cpart_off, bytes;
 };
 
@@ -96,7 +96,11 @@ ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, in
   for (int i = 0; i < n; ++i) {
     const int L = cu[first + i + 1] - cu[first + i];
     const int Le = L - s.Ls - s.Lr;
-    if (s.K > 0 && Le > s.K) { ++p.n_scored; p.max_le = Le > p.max_le ? Le : p.max_le; }
+    if (s.K > 0 && Le > s.K) {
+      p.min_le = p.n_scored == 0 || Le < p.min_le ? Le : p.min_le;
+      p.max_le = Le > p.max_le ? Le : p.max_le;
+      ++p.n_scored;
+    }
   }
   if (p.n_scored == 0) return p;
   const int R = s.g * s.Lo;
@@ -107,7 +111,7 @@ ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, in
   if (nsplit > tiles) nsplit = tiles;
   if (nsplit > 64) nsplit = 64;
   if (nsplit < 1) nsplit = 1;
-  if (use_umma(dtype, s)) p.nsplit = score_umma_nsplit(s, p.n_scored, p.max_le, sm_count());
+  if (use_umma(dtype, s)) p.nsplit = score_umma_nsplit(s, p.n_scored, p.min_le, p.max_le, sm_count());
   else if (use_umma_wide(dtype, s)) p.nsplit = score_umma_wide_nsplit(s, p.n_scored, p.max_le, sm_count());
   else if (use_mma(dtype, s)) p.nsplit = score_mma_nsplit(s, p.n_scored, p.max_le, sm_count());
   else p.nsplit = (int)nsplit;

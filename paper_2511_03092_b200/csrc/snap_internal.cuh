@@ -96,7 +96,7 @@ cudaError_t launch_score_mma(const Shape& s, const SeqBatch& b, const void* q_ob
 cudaError_t launch_score_combine_log2(const ScoreBuffers& buf, int nz, int R, cudaStream_t st);
 // tcgen05 / TMEM / TMA version (bf16, 128-wide heads, g*Lo = 128 or 256)
 bool score_umma_supported(int dtype, const Shape& s);
-int score_umma_nsplit(const Shape& s, int n_scored, int max_le, int sm_count);
+int score_umma_nsplit(const Shape& s, int n_scored, int min_le, int max_le, int sm_count);
 cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
                               const ScoreBuffers& buf, uint32_t* status, cudaStream_t st);
 // tcgen05 version for wide rows / many window rows (d_qk up to 576, g*Lo a multiple of 128)
