@@ -361,6 +361,10 @@ int score_umma_wide_row_blocks(const Shape& s) { return (s.g * s.Lo + 127) / 128
 int score_umma_wide_nsplit(const Shape& s, int n_scored, int max_le, int sm_count) {
   const int tiles = (max_le + 255) / 256;
   const long long base = (long long)n_scored * s.Hkv * score_umma_wide_row_blocks(s);
+  if (const char* env = getenv("SNAP_SCORE_NSPLIT")) {          // tuning aid
+    const int v = atoi(env);
+    if (v >= 1) return v < tiles ? (v < 512 ? v : 512) : tiles;
+  }
   long long ns = (2LL * sm_count + base / 2) / base;
   if (ns > tiles) ns = tiles;
   if (ns > 512) ns = 512;
