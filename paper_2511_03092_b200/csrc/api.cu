@@ -86,20 +86,20 @@ bool use_mma(int dtype, const Shape& s) {
 
 // Scratch regions of one chunk of prompts (offsets relative to the chunk area).
 struct ChunkPlan {
-  int n_scored, min_le, max_le, nsplit, c_stride;
+  int n_scored, max_le, nsplit, chunk_tiles, c_stride;
   size_t part_off, stats_off, c_off, p_off, cpart_off, bytes;
 };
 
 ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, int n) {
   ChunkPlan p;
   std::memset(&p, 0, sizeof(p));
+  int le[kMaxBatchSeqs];                                        // candidates of each scored prompt
   for (int i = 0; i < n; ++i) {
     const int L = cu[first + i + 1] - cu[first + i];
     const int Le = L - s.Ls - s.Lr;
     if (s.K > 0 && Le > s.K) {
-      p.min_le = p.n_scored == 0 || Le < p.min_le ? Le : p.min_le;
+      le[p.n_scored++] = Le;
       p.max_le = Le > p.max_le ? Le : p.max_le;
-      ++p.n_scored;
     }
   }
   if (p.n_scored == 0) return p;
@@ -111,7 +111,7 @@ ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, in
   if (nsplit > tiles) nsplit = tiles;
   if (nsplit > 64) nsplit = 64;
   if (nsplit < 1) nsplit = 1;
-  if (use_umma(dtype, s)) p.nsplit = score_umma_nsplit(s, p.n_scored, p.min_le, p.max_le, sm_count());
+  if (use_umma(dtype, s)) p.nsplit = score_umma_nsplit(s, le, p.n_scored, sm_count(), &p.chunk_tiles);
   else if (use_umma_wide(dtype, s)) p.nsplit = score_umma_wide_nsplit(s, p.n_scored, p.max_le, sm_count());
   else if (use_mma(dtype, s)) p.nsplit = score_mma_nsplit(s, p.n_scored, p.max_le, sm_count());
   else p.nsplit = (int)nsplit;
@@ -374,7 +374,7 @@ int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* 
       buf.stats = reinterpret_cast<float2*>(chunk_ws + p.stats_off);
       buf.C = reinterpret_cast<float*>(chunk_ws + p.c_off);
       buf.P = reinterpret_cast<float*>(chunk_ws + p.p_off);
-      buf.c_stride = p.c_stride; buf.nsplit = p.nsplit;
+      buf.c_stride = p.c_stride; buf.nsplit = p.nsplit; buf.chunk_tiles = p.chunk_tiles;
       buf.ext_mu = row_mu_dev;
       const cudaError_t e = use_umma(cfg->dtype, s)  ? launch_score_umma(s, b, q_obs_dev, src, buf, status_dev, st)
                             : use_umma_wide(cfg->dtype, s)

@@ -208,8 +208,9 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   const int seq = a.b.seq_of_score[si];
   const int Le = a.b.len[seq] - a.Ls - a.Lr;
   const int ntiles = (Le + TN - 1) / TN;
-  const int t0 = (int)((long long)ntiles * blockIdx.x / a.buf.nsplit);
-  const int t1 = (int)((long long)ntiles * (blockIdx.x + 1) / a.buf.nsplit);
+  // equal chunks of candidate tiles for every prompt of the launch: a shorter prompt uses fewer of the splits
+  const int t0 = min(ntiles, (int)blockIdx.x * a.buf.chunk_tiles);
+  const int t1 = min(ntiles, t0 + a.buf.chunk_tiles);
   const int nt = t1 - t0;
   // Both epilogue groups work on every tile -- pass 1 with two row blocks (one block each) and
   // pass 2 (half of the query-row columns each) -- or they alternate tiles (pass 1, one row block).
@@ -489,24 +490,39 @@ bool score_umma_supported(int dtype, const Shape& s) {
   return dtype == SNAP_BF16 && s.d_qk == D && (R == 128 || R == 256) && encode_fn() != nullptr;
 }
 
-// Candidate splits per (prompt, KV head).  Prompts of about one length (a single prompt above all):
-// one CTA per SM, each as long as possible -- a CTA's set-up (query block, tensor memory,
-// barriers) is paid once per SM (measured: 171 -> 157 us for a 77k-token prompt, 242 -> 234 us at
-// 128k, against two CTAs per SM in sequence).  Ragged batches: two CTAs per SM in sequence, so that
-// the short prompts' short CTAs even out.
-int score_umma_nsplit(const Shape& s, int n_scored, int min_le, int max_le, int sm_count) {
-  const int tiles = (max_le + TN - 1) / TN;
-  const long long base = (long long)n_scored * s.Hkv;
-  if (const char* env = getenv("SNAP_SCORE_NSPLIT")) {          // tuning aid
+// Candidate splits.  Every CTA takes the same number of candidate tiles (the chunk), whatever the
+// prompt it works on, and the chunk is the smallest for which the CTAs of the launch fit whole
+// waves of one CTA per SM -- one wave unless there are more (prompt, KV head) pairs than SMs.
+// Long CTAs pay their set-up (query block, tensor memory, barriers) once per SM (measured: 171 ->
+// 157 us for a 77k-token prompt, 242 -> 234 us at 128k, against two CTAs per SM in sequence), and
+// equal ones leave no tail in a ragged batch.  Returns the splits of the longest prompt (the grid's x
+// extent and the stride of the per-split statistics) and the chunk.
+int score_umma_nsplit(const Shape& s, const int* le, int n_scored, int sm_count, int* chunk_tiles) {
+  int max_tiles = 1;
+  for (int i = 0; i < n_scored; ++i) max_tiles = max_tiles > (le[i] + TN - 1) / TN ? max_tiles : (le[i] + TN - 1) / TN;
+  auto ctas = [&](int c) {
+    long long n = 0;
+    for (int i = 0; i < n_scored; ++i) n += ((le[i] + TN - 1) / TN + c - 1) / c;
+    return n * s.Hkv;
+  };
+  int c = max_tiles;
+  if (const char* env = getenv("SNAP_SCORE_NSPLIT")) {          // tuning aid: splits of the longest prompt
     const int v = atoi(env);
-    if (v >= 1) return v < tiles ? (v < 512 ? v : 512) : tiles;
+    if (v >= 1) c = (max_tiles + v - 1) / v;
+  } else {
+    const long long nz = (long long)n_scored * s.Hkv;
+    const long long target = (nz + sm_count - 1) / sm_count * sm_count;
+    int lo = 1, hi = max_tiles;                                 // smallest chunk whose CTAs fit the target
+    while (lo < hi) {
+      const int mid = (lo + hi) / 2;
+      if (ctas(mid) <= target) hi = mid; else lo = mid + 1;
+    }
+    c = lo;
   }
-  const bool even = 4LL * min_le >= 3LL * max_le && base <= sm_count;
-  long long ns = even ? sm_count / base : (2LL * sm_count + base / 2) / base;
-  if (ns > tiles) ns = tiles;
-  if (ns > 512) ns = 512;
-  if (ns < 1) ns = 1;
-  return (int)ns;
+  if ((max_tiles + c - 1) / c > 512) c = (max_tiles + 511) / 512;
+  if (c < 1) c = 1;
+  *chunk_tiles = c;
+  return (max_tiles + c - 1) / c;
 }
 
 cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,

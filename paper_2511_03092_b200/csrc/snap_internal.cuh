@@ -43,6 +43,7 @@ struct ScoreBuffers {
   float* P;             // [n_scored*Hkv][c_stride]   pooled scores
   int c_stride;         // floats per (prompt, kv head) row of C and P
   int nsplit;
+  int chunk_tiles;      // 128-wide tcgen05 score kernel: candidate tiles per CTA (split x covers tiles [x c, x c + c))
   const float* ext_mu;  // NULL, or [prompts][Hq][Lo] log2 normalisers of Eq. 4 computed elsewhere
                         // (the prefill attention kernel): pass 1 and the combine step are skipped
 };
@@ -96,7 +97,7 @@ cudaError_t launch_score_mma(const Shape& s, const SeqBatch& b, const void* q_ob
 cudaError_t launch_score_combine_log2(const ScoreBuffers& buf, int nz, int R, cudaStream_t st);
 // tcgen05 / TMEM / TMA version (bf16, 128-wide heads, g*Lo = 128 or 256)
 bool score_umma_supported(int dtype, const Shape& s);
-int score_umma_nsplit(const Shape& s, int n_scored, int min_le, int max_le, int sm_count);
+int score_umma_nsplit(const Shape& s, const int* le, int n_scored, int sm_count, int* chunk_tiles);
 cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
                               const ScoreBuffers& buf, uint32_t* status, cudaStream_t st);
 // tcgen05 version for wide rows / many window rows (d_qk up to 576, g*Lo a multiple of 128)
