@@ -23,15 +23,17 @@
 #include <cstdlib>
 
 #include "snap_internal.cuh"
+#include "umma_helpers.cuh"
 
 namespace snap {
 namespace {
+
+using namespace umma;
 
 constexpr int D = 128, TN = 128, NS = 4;
 constexpr int HALF_B = TN * 128;             // one K half of a 128-row tile: 128 rows x 128 bytes
 constexpr int STAGE_B = 2 * HALF_B;          // 32 KB
 constexpr int NTHREADS = 320;                // 10 warps
-constexpr unsigned kWaitLimit = 1u << 21;
 
 struct UmmaArgs {
   int Hq, Hkv, g, Lo, Ls, Lr, R;
@@ -41,133 +43,6 @@ struct UmmaArgs {
   uint32_t* status;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity) {
-  unsigned ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait; also gives up as soon as another role has raised the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, unsigned parity, volatile int* abort_flag) {
-  for (unsigned it = 0; it < kWaitLimit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 1023u) == 1023u && *abort_flag) return false;
-  }
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
-}
-// K-major operand, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
-  return (uint64_t)((saddr >> 4) & 0x3fffu) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-// Split form for software pipelining: issue the load, and wait later.  The wait lists the
-// registers as in/out operands so that no use of them can be scheduled above it.
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-               :: "memory");
-}
-__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_ld16_wait(uint32_t (&r)[16]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
-               :: "memory");
-}
-__device__ __forceinline__ float fast_exp2(float x) {     // one MUFU op, relative error ~2^-22
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// Two-wide packed fp32 arithmetic: the multiply-add in front of an exponential and the addition
-// behind it cost half an issue slot per element.
-typedef unsigned long long u64;
-__device__ __forceinline__ u64 pack2(float lo, float hi) {
-  u64 r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ float lo2(u64 a) { return __uint_as_float((uint32_t)a); }
-__device__ __forceinline__ float hi2(u64 a) { return __uint_as_float((uint32_t)(a >> 32)); }
-__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ u64 add2(u64 a, u64 b) {
-  u64 d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
 // acc (two pairs, alternated) += exp2(r[i] * scale + off) over 2 n raw logits, off the same for all
 template <int N2>
 __device__ __forceinline__ void exp_sum_const(const uint32_t* r, u64 sc2, u64 off2, u64 (&acc)[2]) {
@@ -177,18 +52,6 @@ __device__ __forceinline__ void exp_sum_const(const uint32_t* r, u64 sc2, u64 of
     acc[i & 1] = add2(acc[i & 1], pack2(fast_exp2(lo2(x)), fast_exp2(hi2(x))));
   }
 }
-__device__ __forceinline__ void merge_ml(float& m, float& l, float m2, float l2) {
-  const float mn = fmaxf(m, m2);
-  const float f1 = m == -INFINITY ? 0.f : exp2f(m - mn), f2 = m2 == -INFINITY ? 0.f : exp2f(m2 - mn);
-  l = l * f1 + l2 * f2;
-  m = mn;
-}
-
-// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major
-__host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
 template <int PASS>
 __global__ void __launch_bounds__(NTHREADS, 1)
 score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k) {
@@ -278,7 +141,7 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0 && nt > 0) {
-      const uint32_t idesc = PASS == 1 ? make_idesc(128, 128) : make_idesc(128, R);
+      const uint32_t idesc = PASS == 1 ? idesc_bf16(128, 128) : idesc_bf16(128, R);
       bool ok = mbar_wait(qfull_bar, 0u, abort_flag);
       for (int it = 0; it < nt && ok; ++it) {
         const int s = it % NS, b = it & 1;
@@ -291,17 +154,17 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
           for (int mb = 0; mb < MB; ++mb)
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks)
-              umma_bf16(tmem_base + b * 256 + mb * 128,
-                        umma_desc(qst + (ks >> 2) * (R * 128) + mb * HALF_B + (ks & 3) * 32),
-                        umma_desc(kst + (ks >> 2) * HALF_B + (ks & 3) * 32), idesc, ks > 0);
+              mma_bf16(tmem_base + b * 256 + mb * 128,
+                        smem_desc(qst + (ks >> 2) * (R * 128) + mb * HALF_B + (ks & 3) * 32),
+                        smem_desc(kst + (ks >> 2) * HALF_B + (ks & 3) * 32), idesc, ks > 0);
         } else {
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
-            umma_bf16(tmem_base + b * 256, umma_desc(kst + (ks >> 2) * HALF_B + (ks & 3) * 32),
-                      umma_desc(qst + (ks >> 2) * (R * 128) + (ks & 3) * 32), idesc, ks > 0);
+            mma_bf16(tmem_base + b * 256, smem_desc(kst + (ks >> 2) * HALF_B + (ks & 3) * 32),
+                      smem_desc(qst + (ks >> 2) * (R * 128) + (ks & 3) * 32), idesc, ks > 0);
         }
-        umma_commit(empty_bar(s));        // the stage may be refilled once these MMAs have read it
-        umma_commit(tfull_bar(b));        // the accumulator buffer is complete
+        mma_commit(empty_bar(s));        // the stage may be refilled once these MMAs have read it
+        mma_commit(tfull_bar(b));        // the accumulator buffer is complete
       }
       if (!ok) *abort_flag = 1;
     }
@@ -464,22 +327,6 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
 constexpr size_t kSmemBytes = 256 * 256 + NS * STAGE_B + 256 * sizeof(float2) + 128 * sizeof(float2) +
                               (2 * NS + 5) * 8 + 16 + 1024;
 
@@ -487,7 +334,7 @@ constexpr size_t kSmemBytes = 256 * 256 + NS * STAGE_B + 256 * sizeof(float2) + 
 
 bool score_umma_supported(int dtype, const Shape& s) {
   const int R = s.g * s.Lo;
-  return dtype == SNAP_BF16 && s.d_qk == D && (R == 128 || R == 256) && encode_fn() != nullptr;
+  return dtype == SNAP_BF16 && s.d_qk == D && (R == 128 || R == 256) && encode_tiled_fn() != nullptr;
 }
 
 // Candidate splits.  Every CTA takes the same number of candidate tiles (the chunk), whatever the
@@ -528,7 +375,7 @@ int score_umma_nsplit(const Shape& s, const int* le, int n_scored, int sm_count,
 cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
                               const ScoreBuffers& buf, uint32_t* status, cudaStream_t st) {
   if (b.n_scored == 0) return cudaSuccess;
-  EncodeTiledFn enc = encode_fn();
+  EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
   UmmaArgs a;
   a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Lo = s.Lo; a.Ls = s.Ls; a.Lr = s.Lr; a.R = s.g * s.Lo;
