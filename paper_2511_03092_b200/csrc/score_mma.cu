@@ -16,10 +16,13 @@
 //
 // mma.sync.m16n8k16 (bf16 in, fp32 accumulate) is the instruction used here; statistics are in
 // the log2 domain (logits are multiplied by scale * log2 e once).
+#include "mma_helpers.cuh"
 #include "snap_internal.cuh"
 
 namespace snap {
 namespace {
+
+using namespace mmasync;
 
 constexpr int D = 128, TN = 64, ROW_B = D * 2, KT_B = TN * ROW_B;
 
@@ -31,27 +34,6 @@ struct MmaArgs {
   SeqBatch b;
   ScoreBuffers buf;
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, unsigned src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 
 // rows x 256 bytes, 16-byte chunk c of row r stored at chunk c ^ (r & 7)
 __device__ __forceinline__ uint32_t swz(int row, int chunk) { return row * ROW_B + ((chunk ^ (row & 7)) << 4); }
