@@ -143,3 +143,17 @@ def test_config1_prompt_attention_hands_its_normalisers_to_the_compression():
     assert layer.status() == 0
     seq = H.oracle_compress(wl, p)
     H.check_selection(idx.cpu().numpy()[0], seq, wl)
+
+
+@pytest.mark.parametrize("row", ["llama", "deepseek"])
+def test_paper_hyperparameter_rows(row):
+    """The two rows of the appendix table "SnapStream Hyperparameters" (sink, top-K, recent, observation
+    window, pooling kernel) on their own attention shapes, with prompts just long enough to need scoring."""
+    if row == "llama":        # sink 768, top-K 6400, recent 1024 (8192 slots), window 32, kernel 13
+        wl = synth.CONFIGS[1].scaled(name="paper_llama", l_sink=768, topk=6400, l_recent=1024, l_obs=32, pool_kernel=13)
+        lengths, steps = [20000, 9000], 4
+    else:                     # sink 512, top-K 512, recent 31744 (32768 slots), latent attention
+        wl = synth.CONFIGS[3].scaled(name="paper_deepseek", l_sink=512, topk=512, l_recent=31744, l_obs=32, pool_kernel=13)
+        lengths, steps = [36000], 3
+    assert wl.slots in (8192, 32768)
+    _run(wl, lengths, seed=500, steps=steps)
