@@ -46,6 +46,16 @@ DECODE_RING = 8            # distinct pre-generated decode inputs cycled through
 DECODE_TRAFFIC_BYTES = 672.03e6 + 8.11e6
 
 
+def _bf16_peak():
+    """Measured dense bf16 TFLOP/s of this machine's B200s (sustained figure), None if not recorded."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            d = json.load(f)
+        return float(d.get("bf16_tflops_sustained") or d.get("bf16_tflops"))
+    except Exception:
+        return None
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -737,6 +747,9 @@ def run_config(args):
     rows = min(L + 1, wl.slots)
     step_bytes = n_layers * nseq * wl.n_kv_heads * rows * (wl.d_qk + (0 if wl.v_aliases_k else wl.d_v)) * eb
     peak, _ = _peaks()
+    # arithmetic of a step: q.K^T and p.V over the valid rows for every query head
+    step_flops = 2.0 * n_layers * nseq * wl.n_q_heads * rows * (wl.d_qk + wl.d_v)
+    bf16_peak = _bf16_peak()
     print(json.dumps({
         "workload": wl.name, "n_layers": n_layers, "sequences": nseq, "prompt_tokens": L, "cache_slots": wl.slots,
         "compress_us_per_prompt_layer_median": statistics.median(comp_us),
@@ -744,6 +757,8 @@ def run_config(args):
         "decode_us_per_step_cuda_graph": ms_graph * 1e3,
         "decode_tokens_per_s": nseq / (ms * 1e-3), "decode_bytes_per_step": step_bytes,
         "decode_GBps": step_bytes / (ms * 1e-3) / 1e9, "decode_frac_of_measured_hbm": step_bytes / (ms * 1e-3) / 1e9 / peak,
+        "decode_TFLOPs": step_flops / (ms * 1e-3) / 1e12,
+        "decode_frac_of_measured_bf16": None if bf16_peak is None else step_flops / (ms * 1e-3) / 1e12 / bf16_peak,
         "status": int(cache.status.item())}), flush=True)
 
 
