@@ -30,7 +30,8 @@ namespace {
 
 using namespace umma;
 
-constexpr int D = 128, TN = 128, NS = 4;
+constexpr int D = 128, TN = 128;
+constexpr int kStagesPass1 = 4, kStagesPass2 = 3;          // pass 2 gives one stage up for its extra operand slabs
 constexpr int HALF_B = TN * 128;             // one K half of a 128-row tile: 128 rows x 128 bytes
 constexpr int STAGE_B = 2 * HALF_B;          // 32 KB
 constexpr int NTHREADS = 320;                // 10 warps
@@ -58,9 +59,14 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int R = a.R, MB = R / 128;
+  constexpr int NS = PASS == 1 ? kStagesPass1 : kStagesPass2;
   unsigned char* Qs = smem;                                   // [2 halves][R][128 B]
   unsigned char* Ks = Qs + R * 256;                           // [NS][2 halves][128][128 B]
-  float2* stats_s = reinterpret_cast<float2*>(Ks + NS * STAGE_B);   // [R]  (pass 2: m_i, 1/l_i)
+  // pass 2: one more 16-wide step of the contraction, whose operands are constants of the launch
+  unsigned char* tail = Ks + NS * STAGE_B;
+  unsigned char* Qx = tail;                                   // [256][128 B]  row i: -mu_i / scale as three bf16 pieces
+  unsigned char* Kx = Qx + 256 * 128;                         // [128][128 B]  ones against those pieces
+  float2* stats_s = reinterpret_cast<float2*>(PASS == 2 ? Kx + HALF_B : tail);   // [R] floats: mu_i (pass 2)
   float2* xch = stats_s + 256;                                // [128] pass-1 exchange between epilogue groups
   uint64_t* bars = reinterpret_cast<uint64_t*>(xch + 128);    // full[NS] empty[NS] tfull[2] tempty[2] qfull
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NS + 5);
@@ -75,9 +81,9 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   const int t0 = min(ntiles, (int)blockIdx.x * a.buf.chunk_tiles);
   const int t1 = min(ntiles, t0 + a.buf.chunk_tiles);
   const int nt = t1 - t0;
-  // Both epilogue groups work on every tile -- pass 1 with two row blocks (one block each) and
-  // pass 2 (half of the query-row columns each) -- or they alternate tiles (pass 1, one row block).
-  const bool both = PASS == 2 || MB == 2;
+  // Pass 1 with two row blocks: both epilogue groups work on every tile, one block each.  Otherwise
+  // (pass 1 with one row block, pass 2) the groups alternate tiles.
+  const bool both = PASS == 1 && MB == 2;
 
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8 * s; };
@@ -106,6 +112,36 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
         mu_s[i] = st.x - log2f(st.y);
       }
     }
+    __syncthreads();
+    // Fold the normalisers into the contraction: one more 16-wide step whose B rows hold
+    // -mu_i / scale split into three bf16 pieces (their sum is exact to 2^-24) and whose A rows hold
+    // ones, so that the accumulator is q_i . k_j - mu_i / scale and the epilogue is exp2(scale * acc)
+    // with no per-row constant.  Rows of 128 bytes, 128-byte swizzle, only chunks 0 and 1 are read.
+    const float inv_scale = 1.f / a.scale_log2;
+    for (int i = tid; i < 256 + 128; i += NTHREADS) {
+      uint4 c0 = make_uint4(0u, 0u, 0u, 0u);
+      unsigned char* rowp;
+      if (i < 256) {
+        rowp = Qx + i * 128;
+        if (i < R) {
+          const float c = -mu_s[i] * inv_scale;
+          const __nv_bfloat16 hi = __float2bfloat16_rn(c);
+          const float r1 = c - __bfloat162float(hi);
+          const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+          c0.x = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16);
+          c0.y = (uint32_t)__bfloat16_as_ushort(lo);
+        }
+      } else {
+        rowp = Kx + (i - 256) * 128;
+        c0.x = 0x3f803f80u;                                    // bf16 1.0, 1.0
+        c0.y = 0x00003f80u;                                    // bf16 1.0, 0
+      }
+      const int sw = (i < 256 ? i : i - 256) & 7;
+      *reinterpret_cast<uint4*>(rowp + ((0 ^ sw) << 4)) = c0;
+      *reinterpret_cast<uint4*>(rowp + ((1 ^ sw) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 0) {                                            // tensor memory: 512 columns (2 x 256)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
@@ -162,6 +198,7 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
           for (int ks = 0; ks < D / 16; ++ks)
             mma_bf16(tmem_base + b * 256, smem_desc(kst + (ks >> 2) * HALF_B + (ks & 3) * 32),
                       smem_desc(qst + (ks >> 2) * (R * 128) + (ks & 3) * 32), idesc, ks > 0);
+          mma_bf16(tmem_base + b * 256, smem_desc(smem_u32(Kx)), smem_desc(smem_u32(Qx)), idesc, 1);   // - mu_i / scale
         }
         mma_commit(empty_bar(s));        // the stage may be refilled once these MMAs have read it
         mma_commit(tfull_bar(b));        // the accumulator buffer is complete
@@ -174,22 +211,13 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
     const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
     const int mb = both ? eg : 0;
     bool ok = true;
-    // pass 2: minus the log-sum-exp (log2 domain) of each query row this group sums over, in
-    // registers, so that the inner loop is fma -> exp2 -> add with no memory operand
-    const int nc2 = R / 64;                                   // 32-column chunks per group: 2 or 4
-    u64 mu2[64];                                              // pairs of adjacent columns' constants
-    if (PASS == 2) {
-#pragma unroll
-      for (int i = 0; i < 64; ++i)
-        mu2[i] = 2 * i < 32 * nc2 ? pack2(-mu_s[32 * nc2 * eg + 2 * i], -mu_s[32 * nc2 * eg + 2 * i + 1]) : pack2(0.f, 0.f);
-    }
     for (int it = both ? 0 : eg; it < nt; it += both ? 1 : 2) {
       const int b = it & 1;
       const bool landed = mbar_wait(tfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag);
       if (!landed) {
         *abort_flag = 1;
         ok = false;
-        if (PASS == 1) break;            // pass 2 leaves through the group barrier below
+        break;
       }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int cand0 = (t0 + it) * TN;
@@ -255,49 +283,28 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
         }
         l_sum += sum;
       } else {
-        // this group's half of the query-row columns; group 1 hands its partial sum to group 0
-        const uint32_t col0 = lane_addr + b * 256 + 32 * (eg * nc2);
-        float s = 0.f;
-        if (landed) {
-          // software pipeline over 16-column chunks (two small register buffers leave room for the
-          // 128 row constants); four partial sums break the dependency chain of the additions
-          uint32_t ra[16], rb[16];
-          u64 acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
-          const u64 sc2 = pack2(a.scale_log2, a.scale_log2);
-          const int nch = 2 * nc2;                             // 16-column chunks: 4 or 8
-          tmem_ld16_issue(col0, ra);
+        // thread = candidate: the accumulator row already holds q_i . k_j - mu_i / scale for every
+        // query row i of the KV head, so the Eq. 1 score is the plain sum of exp2(scale * acc) over the
+        // R columns -- no constants, no exchange with the other group (the groups alternate tiles)
+        const uint32_t col0 = lane_addr + b * 256;
+        uint32_t ra[32], rb[32];
+        u64 acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+        const u64 sc2 = pack2(a.scale_log2, a.scale_log2), zero2 = pack2(0.f, 0.f);
+        const int nch = R / 32;                                // 32-column chunks: 4 or 8
+        tmem_ld32_issue(col0, ra);
 #pragma unroll
-          for (int c = 0; c < 8; c += 2) {
-            if (c < nch) {
-              tmem_ld16_wait(ra);
-              tmem_ld16_issue(col0 + 16 * (c + 1), rb);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const u64 x = fma2(pack2(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1])), sc2, mu2[8 * c + i]);
-                acc[i & 1] = add2(acc[i & 1], pack2(fast_exp2(lo2(x)), fast_exp2(hi2(x))));
-              }
-              tmem_ld16_wait(rb);
-              if (c + 2 < nch) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const u64 x = fma2(pack2(__uint_as_float(rb[2 * i]), __uint_as_float(rb[2 * i + 1])), sc2, mu2[8 * (c + 1) + i]);
-                acc[i & 1] = add2(acc[i & 1], pack2(fast_exp2(lo2(x)), fast_exp2(hi2(x))));
-              }
-            }
+        for (int c = 0; c < 8; c += 2) {
+          if (c < nch) {
+            tmem_ld_wait(ra);
+            tmem_ld32_issue(col0 + 32 * (c + 1), rb);
+            exp_sum_const<16>(ra, sc2, zero2, acc);
+            tmem_ld_wait(rb);
+            if (c + 2 < nch) tmem_ld32_issue(col0 + 32 * (c + 2), ra);
+            exp_sum_const<16>(rb, sc2, zero2, acc);
           }
-          s = (lo2(acc[0]) + hi2(acc[0])) + (lo2(acc[1]) + hi2(acc[1]));
         }
-        float* xs = reinterpret_cast<float*>(xch) + b * 128;
-        if (eg == 1) xs[lrow] = s;
-        // barrier over the 8 epilogue warps that also agrees on whether anyone has given up
-        unsigned stop;
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
-            "bar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(stop) : "r"((unsigned)(!landed || *abort_flag)) : "memory");
-        if (eg == 0 && !stop && cand0 + lrow < Le)
-          a.buf.C[(long long)z * a.buf.c_stride + cand0 + lrow] = s + xs[lrow];
-        if (stop) { *abort_flag = 1; ok = false; }
+        if (cand0 + lrow < Le)
+          a.buf.C[(long long)z * a.buf.c_stride + cand0 + lrow] = (lo2(acc[0]) + hi2(acc[0])) + (lo2(acc[1]) + hi2(acc[1]));
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -327,8 +334,10 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
 }
 
-constexpr size_t kSmemBytes = 256 * 256 + NS * STAGE_B + 256 * sizeof(float2) + 128 * sizeof(float2) +
-                              (2 * NS + 5) * 8 + 16 + 1024;
+constexpr size_t smem_bytes(int pass) {
+  return 256 * 256 + (pass == 1 ? kStagesPass1 * STAGE_B : kStagesPass2 * STAGE_B + 256 * 128 + HALF_B) +
+         256 * sizeof(float2) + 128 * sizeof(float2) + (2 * kStagesPass1 + 5) * 8 + 16 + 1024;
+}
 
 }  // namespace
 
@@ -406,17 +415,17 @@ cudaError_t launch_score_umma(const Shape& s, const SeqBatch& b, const void* q_o
       return cudaErrorInvalidValue;
   }
   static SmemLimit limit1 = {}, limit2 = {};
-  if (cudaError_t e = ensure_dyn_smem(score_umma_kernel<1>, kSmemBytes, limit1)) return e;
-  if (cudaError_t e = ensure_dyn_smem(score_umma_kernel<2>, kSmemBytes, limit2)) return e;
+  if (cudaError_t e = ensure_dyn_smem(score_umma_kernel<1>, smem_bytes(1), limit1)) return e;
+  if (cudaError_t e = ensure_dyn_smem(score_umma_kernel<2>, smem_bytes(2), limit2)) return e;
   const int nz = b.n_scored * s.Hkv;
   dim3 grid(buf.nsplit, nz);
   if (!buf.ext_mu) {                                          // Eq. 4's normalisers: pass 1, unless the caller has them
-    if (launch_pdl(score_umma_kernel<1>, grid, dim3(NTHREADS), kSmemBytes, st, a, tq, tk) != cudaSuccess) return cudaGetLastError();
+    if (launch_pdl(score_umma_kernel<1>, grid, dim3(NTHREADS), smem_bytes(1), st, a, tq, tk) != cudaSuccess) return cudaGetLastError();
     count_launch();
     cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
     if (e != cudaSuccess) return e;
   }
-  if (launch_pdl(score_umma_kernel<2>, grid, dim3(NTHREADS), kSmemBytes, st, a, tq, tk) != cudaSuccess) return cudaGetLastError();
+  if (launch_pdl(score_umma_kernel<2>, grid, dim3(NTHREADS), smem_bytes(2), st, a, tq, tk) != cudaSuccess) return cudaGetLastError();
   count_launch();
   return cudaGetLastError();
 }
