@@ -68,8 +68,8 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   unsigned char* Kx = Qx + 256 * 128;                         // [128][128 B]  ones against those pieces
   float2* stats_s = reinterpret_cast<float2*>(PASS == 2 ? Kx + HALF_B : tail);   // [R] floats: mu_i (pass 2)
   float2* xch = stats_s + 256;                                // [128] pass-1 exchange between epilogue groups
-  uint64_t* bars = reinterpret_cast<uint64_t*>(xch + 128);    // full[NS] empty[NS] tfull[2] tempty[2] qfull
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NS + 5);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(xch + 128);    // full[NS] empty[NS] tfull[2] tempty[2] qfull xfull[2] xempty[2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NS + 9);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -81,9 +81,10 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   const int t0 = min(ntiles, (int)blockIdx.x * a.buf.chunk_tiles);
   const int t1 = min(ntiles, t0 + a.buf.chunk_tiles);
   const int nt = t1 - t0;
-  // Pass 1 with two row blocks: both epilogue groups work on every tile, one block each.  Otherwise
-  // (pass 1 with one row block, pass 2) the groups alternate tiles.
-  const bool both = PASS == 1 && MB == 2;
+  // Both epilogue groups work on every tile -- pass 1 with two row blocks (one block each) and pass 2
+  // (half of the accumulator columns each) -- so that a tile's buffer is free again after half the
+  // time and the next MMA never waits for it; pass 1 with one row block alternates tiles instead.
+  const bool both = PASS == 2 || MB == 2;
 
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8 * s; };
@@ -91,12 +92,15 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   auto tfull_bar = [&](int b) { return bar0 + 8 * (2 * NS + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8 * (2 * NS + 2 + b); };
   const uint32_t qfull_bar = bar0 + 8 * (2 * NS + 4);
+  auto xfull_bar = [&](int b) { return bar0 + 8 * (2 * NS + 5 + b); };    // pass 2: group 1's partial sums are in xch
+  auto xempty_bar = [&](int b) { return bar0 + 8 * (2 * NS + 7 + b); };   //         ... and have been taken
 
   if (tid == 0) {
     *abort_flag = 0;
     for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), both ? 8 : 4); }
     mbar_init(qfull_bar, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(xfull_bar(b), 4); mbar_init(xempty_bar(b), 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   pdl_wait();                                                 // everything above overlaps the previous kernel's tail
@@ -221,6 +225,7 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
       }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int cand0 = (t0 + it) * TN;
+      float part = 0.f;                                        // pass 2: this group's half of the candidate's sum
       if (PASS == 1) {
         const uint32_t col0 = lane_addr + b * 256 + mb * 128;
         const bool full_tile = cand0 + TN <= Le;
@@ -285,15 +290,16 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
       } else {
         // thread = candidate: the accumulator row already holds q_i . k_j - mu_i / scale for every
         // query row i of the KV head, so the Eq. 1 score is the plain sum of exp2(scale * acc) over the
-        // R columns -- no constants, no exchange with the other group (the groups alternate tiles)
-        const uint32_t col0 = lane_addr + b * 256;
+        // R columns -- no constants.  This group sums its half of the columns; group 1 hands its
+        // partial to group 0 through shared memory (below, after the buffer has been released).
+        const uint32_t col0 = lane_addr + b * 256 + eg * (R / 2);
         uint32_t ra[32], rb[32];
         u64 acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
         const u64 sc2 = pack2(a.scale_log2, a.scale_log2), zero2 = pack2(0.f, 0.f);
-        const int nch = R / 32;                                // 32-column chunks: 4 or 8
+        const int nch = R / 64;                                // 32-column chunks of this half: 2 or 4
         tmem_ld32_issue(col0, ra);
 #pragma unroll
-        for (int c = 0; c < 8; c += 2) {
+        for (int c = 0; c < 4; c += 2) {
           if (c < nch) {
             tmem_ld_wait(ra);
             tmem_ld32_issue(col0 + 32 * (c + 1), rb);
@@ -303,12 +309,27 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
             exp_sum_const<16>(rb, sc2, zero2, acc);
           }
         }
-        if (cand0 + lrow < Le)
-          a.buf.C[(long long)z * a.buf.c_stride + cand0 + lrow] = (lo2(acc[0]) + hi2(acc[0])) + (lo2(acc[1]) + hi2(acc[1]));
+        part = (lo2(acc[0]) + hi2(acc[0])) + (lo2(acc[1]) + hi2(acc[1]));
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(b));
+      if (PASS == 2) {
+        // the two halves of a candidate's sum meet in shared memory (one slot per tile parity)
+        float* xs = reinterpret_cast<float*>(xch) + b * 128;
+        const unsigned ph = (unsigned)(it / 2) & 1u;
+        if (eg == 1) {
+          if (!mbar_wait(xempty_bar(b), ph ^ 1u, abort_flag)) { *abort_flag = 1; ok = false; break; }
+          xs[lrow] = part;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(xfull_bar(b));
+        } else {
+          if (!mbar_wait(xfull_bar(b), ph, abort_flag)) { *abort_flag = 1; ok = false; break; }
+          if (cand0 + lrow < Le) a.buf.C[(long long)z * a.buf.c_stride + cand0 + lrow] = part + xs[lrow];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(xempty_bar(b));
+        }
+      }
       if (!ok) break;
     }
     if (!ok) *abort_flag = 1;
@@ -336,7 +357,7 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
 
 constexpr size_t smem_bytes(int pass) {
   return 256 * 256 + (pass == 1 ? kStagesPass1 * STAGE_B : kStagesPass2 * STAGE_B + 256 * 128 + HALF_B) +
-         256 * sizeof(float2) + 128 * sizeof(float2) + (2 * kStagesPass1 + 5) * 8 + 16 + 1024;
+         256 * sizeof(float2) + 128 * sizeof(float2) + (2 * kStagesPass1 + 9) * 8 + 16 + 1024;
 }
 
 }  // namespace
