@@ -64,7 +64,7 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
   unsigned char* Ks = Qs + R * 256;                           // [NS][2 halves][128][128 B]
   // pass 2: one more 16-wide step of the contraction, whose operands are constants of the launch
   unsigned char* tail = Ks + NS * STAGE_B;
-  unsigned char* Qx = tail;                                   // [256][128 B]  row i: -mu_i / scale as three bf16 pieces
+  unsigned char* Qx = tail;                                   // [256][128 B]  row i: -mu_i / scale as four bf16 pieces
   unsigned char* Kx = Qx + 256 * 128;                         // [128][128 B]  ones against those pieces
   float2* stats_s = reinterpret_cast<float2*>(PASS == 2 ? Kx + HALF_B : tail);   // [R] floats: mu_i (pass 2)
   float2* xch = stats_s + 256;                                // [128] pass-1 exchange between epilogue groups
@@ -118,7 +118,7 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
     }
     __syncthreads();
     // Fold the normalisers into the contraction: one more 16-wide step whose B rows hold
-    // -mu_i / scale split into three bf16 pieces (their sum is exact to 2^-24) and whose A rows hold
+    // -mu_i / scale split into four bf16 pieces (their sum is the fp32 value exactly) and whose A rows hold
     // ones, so that the accumulator is q_i . k_j - mu_i / scale and the epilogue is exp2(scale * acc)
     // with no per-row constant.  Rows of 128 bytes, 128-byte swizzle, only chunks 0 and 1 are read.
     const float inv_scale = 1.f / a.scale_log2;
@@ -132,14 +132,16 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
           const __nv_bfloat16 hi = __float2bfloat16_rn(c);
           const float r1 = c - __bfloat162float(hi);
           const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-          const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+          const float r2 = r1 - __bfloat162float(mid);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(r2);
+          const __nv_bfloat16 lo2 = __float2bfloat16_rn(r2 - __bfloat162float(lo));   // zero unless c needs all 24 bits
           c0.x = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16);
-          c0.y = (uint32_t)__bfloat16_as_ushort(lo);
+          c0.y = (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(lo2) << 16);
         }
       } else {
         rowp = Kx + (i - 256) * 128;
         c0.x = 0x3f803f80u;                                    // bf16 1.0, 1.0
-        c0.y = 0x00003f80u;                                    // bf16 1.0, 0
+        c0.y = 0x3f803f80u;                                    // bf16 1.0, 1.0
       }
       const int sw = (i < 256 ? i : i - 256) & 7;
       *reinterpret_cast<uint4*>(rowp + ((0 ^ sw) << 4)) = c0;
