@@ -69,6 +69,26 @@ def test_sharp_softmax_outputs(wl):
     _run_compress_and_decode(wl, [wl.prompt_len[0], 260], seed=5, steps=4, sharp=4.0)
 
 
+@pytest.mark.parametrize("hq,l_obs,sharp", [(16, 32, 4.0), (32, 32, 8.0), (16, 16, 6.0)],
+                         ids=["rows128_x4", "rows256_x8", "rows64_x6"])
+def test_scores_with_large_logits(hq, l_obs, sharp):
+    """Observation queries scaled up: logits of +-30 and more, normalisers far from zero.  The second score
+    pass carries the normalisers inside the contraction, so their magnitude must not cost precision."""
+    wl = SMALL_BF16.scaled(n_q_heads=hq, n_kv_heads=4, l_obs=l_obs, l_recent=48)
+    lengths = [700, 1500, 149]
+    layer = H.GpuLayer(wl, max_seqs=len(lengths))
+    prompts = [synth.make_prompt(wl, L, 91 + i) for i, L in enumerate(lengths)]
+    for p in prompts:
+        p["q_obs"] = (p["q_obs"].float() * sharp).to(wl.torch_dtype)
+    idx = layer.compress(prompts, list(range(len(lengths))))
+    assert layer.status() == 0
+    for i, p in enumerate(prompts):
+        seq = H.oracle_compress(wl, p)
+        H.check_selection(idx[i], seq, wl)
+        seq.topk_pos = [idx[i][h][idx[i][h] >= 0].astype(np.int64) for h in range(wl.n_kv_heads)]
+        H.check_cache_image(layer, seq, i, wl)
+
+
 def test_ring_wraps_many_times():
     wl = SMALL_BF16.scaled(l_recent=9, l_obs=4, topk=20, l_sink=2)
     _run_compress_and_decode(wl, [5, 11, 40, 300], seed=3, steps=40, check_ring_every=5)
