@@ -3,8 +3,8 @@
 // Covers bf16 layers with 128-wide heads and 128 or 256 window rows per KV head (g * Lo).
 //
 // One CTA per SM, warp specialised, persistent over a run of 128-candidate tiles:
-//   warp 0   TMA producer: the query block once, then key tiles into a 4-stage ring
-//            (cp.async.bulk.tensor, 128-byte swizzle, two 64-element K halves per tile)
+//   warp 0   TMA producer: the query block once, then key tiles into a ring of four stages (three
+//            in pass 2) (cp.async.bulk.tensor, 128-byte swizzle, two 64-element K halves per tile)
 //   warp 1   MMA issuer: one elected thread issues tcgen05.mma (M128, K16 steps) from shared
 //            memory descriptors into one of two TMEM accumulator buffers and commits to mbarriers
 //   warps 2-9  epilogue: read the accumulators with tcgen05.ld (thread = TMEM lane) while the
@@ -13,8 +13,10 @@
 // Pass 1 puts the query rows on M (two 128-row blocks share each key tile; N = 128 candidates),
 // so a thread owns one query row and keeps that row's running (reference max, sum of exp2) with
 // no cross-thread traffic.  Pass 2 puts the candidates on M (N = all query rows), so a thread
-// owns one candidate; the two epilogue groups each sum exp2(s_ij - m_i) / l_i over half of the
-// rows, group 1 hands its partial to group 0 through shared memory, and group 0 stores C[j].
+// owns one candidate, and carries the normalisers in the contraction: one more 16-wide step adds
+// -mu_i / scale (mu_i = m_i + log2 l_i, split into bf16 pieces against ones) to column i, so the
+// epilogue is a plain sum of exp2(scale * acc).  The two epilogue groups each sum half of the
+// columns, group 1 hands its partial to group 0 through shared memory, and group 0 stores C[j].
 // The reference max of pass 1 is refreshed lazily (only when a tile's partial sum shows a logit
 // far above it).  Statistics are in the log2 domain.  Every mbarrier wait is bounded; a wait
 // that runs out raises SNAP_DEV_WAIT_TIMEOUT and the CTA drains and frees its tensor memory.
