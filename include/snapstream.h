@@ -22,9 +22,15 @@
  * Conventions
  *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are plain
  *     host memory.  Every device buffer must be 16-byte aligned.
- *   - The caller owns every buffer.  The library allocates nothing and keeps no per-call
- *     state; all work is enqueued on the CUDA stream given and the calls return without
- *     synchronising.
+ *   - The caller owns every buffer.  The library allocates no device memory; all work is
+ *     enqueued on the CUDA stream given and the calls return without synchronising.
+ *   - What the library keeps between calls, all of it on the host: per device, the SM count and
+ *     which kernels already had their shared-memory limit raised (so the first call of each
+ *     entry point on a device must come before any stream capture); per host thread, the
+ *     tensor maps of the last few cache buffers the decode kernel was given, keyed on their
+ *     addresses and shape; per process, a launch counter and the testing options of
+ *     snap_debug_set_option.  Nothing of one call's data outlives the call, except in the fixed
+ *     scratch array of snap_decode_attn_static, which says so below.
  *   - Token positions are 0-indexed.  Ls = l_sink, Lr = l_recent, K = topk, Lsr = Ls + Lr,
  *     Sc = Ls + Lr + K, g = n_q_heads / n_kv_heads.
  *   - Element type: all of q, k, v, caches and out share cfg->dtype.
@@ -262,8 +268,10 @@ int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout
  * that treats late allocations as failures.
  *
  *   - Every GPU that loads this library holds the array from load until process exit.
- *   - If n_active * n_q_heads * splits * (d_v + 2) floats exceed the array (splits is the
- *     library's choice for that batch size, at most 64), the call returns
+ *   - The step runs the same kernels with the same split count as snap_decode_attn (the latent
+ *     layout included) and needs snap_decode_workspace_bytes(cfg, n_active) - 256 bytes of the
+ *     array: n_active * n_q_heads * splits * (d_v + 2) floats, splits being the library's choice
+ *     for that batch size.  If that exceeds the array the call returns
  *     SNAP_ERR_STATIC_SCRATCH_EXCEEDED and launches nothing; use snap_decode_attn instead.
  *     The 32-sequence, 32-head, d_v = 128 batch of a Llama-3.1-8B layer needs about 4.3 MB.
  *   - All calls share the one array and it keeps the previous call's contents.  Nothing has to
@@ -300,6 +308,28 @@ int snap_append_kv_concat(const snap_config_t* cfg, const snap_layout_t* layout,
                           const void* k_cache_in_dev, const void* v_cache_in_dev,
                           void* k_cache_out_dev, void* v_cache_out_dev,
                           int32_t* seq_len_dev, uint32_t* status_dev, void* cuda_stream);
+
+/*
+ * Testing and tuning aids (the paper has no counterpart).  Each option is one non-negative
+ * integer, process-wide, 0 by default = the library's own choice; changing one while calls are
+ * in flight on other threads is not synchronised.  Every kernel choice yields the same results
+ * within the tolerances of the tests; the options exist so that the slower kernels and other
+ * split counts can be tested and timed.  At the first use of any option each is seeded once
+ * from its environment variable (named on the right); the environment is not read again.
+ * Returns the option's previous value, or SNAP_ERR_INVALID_ARG.
+ */
+#define SNAP_OPT_SCORE_KERNEL 0          /* 1: mma.sync score kernel, 2: SIMT       SNAP_SCORE_PATH=mma|simt */
+#define SNAP_OPT_DECODE_GQA_KERNEL 1     /* 1: packed-FP32 GQA decode kernel        SNAP_DECODE_GQA=simt     */
+#define SNAP_OPT_DECODE_LATENT_KERNEL 2  /* 1: mma.sync latent decode kernel        SNAP_DECODE_MLA=mma      */
+#define SNAP_OPT_DECODE_NSPLIT 3         /* n: splits per (sequence, KV head)       SNAP_DECODE_NSPLIT=n     */
+#define SNAP_OPT_SCORE_NSPLIT 4          /* n: candidate splits of the longest prompt  SNAP_SCORE_NSPLIT=n   */
+#define SNAP_OPT_WIDE_STAGES 5           /* n: ring depth of the wide score kernel  SNAP_WIDE_STAGES=n       */
+#define SNAP_OPT_PREFILL_KERNEL 6        /* 1: portable prefill attention kernel    SNAP_PREFILL_PATH=simt   */
+#define SNAP_OPT_PREFILL_SINGLE_HEADS 7  /* 1: one head per CTA in prefill attention  SNAP_PREFILL_HEADS=1   */
+#define SNAP_OPT_REFINE_OFF 8            /* 1: skip the double-precision re-scoring near the top-K
+                                               threshold (single-precision order)  SNAP_REFINE=0            */
+#define SNAP_OPT_COUNT 9
+int snap_debug_set_option(int option, int value);
 
 /* Text for a snap_status value (static storage). */
 const char* snap_status_string(int status);

@@ -83,6 +83,8 @@ def lib() -> C.CDLL:
     L.snap_decode_attn_multi.argtypes = [pcfg, play, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
     L.snap_decode_attn_static.restype = C.c_int
     L.snap_decode_attn_static.argtypes = [pcfg, play, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
+    L.snap_debug_set_option.restype = C.c_int
+    L.snap_debug_set_option.argtypes = [C.c_int, C.c_int]
     _lib = L
     return L
 
@@ -90,7 +92,12 @@ def lib() -> C.CDLL:
 EXPORTS = ("snap_cache_layout", "snap_compress_workspace_bytes", "snap_decode_workspace_bytes",
            "snap_compress", "snap_append_kv", "snap_append_kv_concat", "snap_decode_attn",
            "snap_decode_multi_workspace_bytes", "snap_decode_attn_multi", "snap_decode_attn_static", "snap_status_string",
-           "snap_kernel_launch_count", "snap_prefill_attn", "snap_compress_with_row_stats")
+           "snap_kernel_launch_count", "snap_prefill_attn", "snap_compress_with_row_stats", "snap_debug_set_option")
+
+# testing / tuning options of snap_debug_set_option
+(SNAP_OPT_SCORE_KERNEL, SNAP_OPT_DECODE_GQA_KERNEL, SNAP_OPT_DECODE_LATENT_KERNEL, SNAP_OPT_DECODE_NSPLIT,
+ SNAP_OPT_SCORE_NSPLIT, SNAP_OPT_WIDE_STAGES, SNAP_OPT_PREFILL_KERNEL, SNAP_OPT_PREFILL_SINGLE_HEADS,
+ SNAP_OPT_REFINE_OFF) = range(9)
 
 
 def status_string(code: int) -> str:
@@ -124,6 +131,14 @@ def make_config(*, n_q_heads, n_kv_heads, d_qk, d_v, dtype, l_sink, l_recent, to
         pool_mode = {"avg": SNAP_POOL_AVG, "max": SNAP_POOL_MAX}[pool_mode]
     return SnapConfig(n_q_heads, n_kv_heads, d_qk, d_v, int(bool(v_aliases_k)), dtype, l_sink, l_recent, topk,
                       l_obs, pool_kernel, pool_mode, float(softmax_scale), max_seqs)
+
+
+def snap_debug_set_option(option: int, value: int) -> int:
+    """Set a process-wide testing / tuning option; returns its previous value."""
+    old = lib().snap_debug_set_option(int(option), int(value))
+    if old < 0:
+        raise SnapError(int(old), "snap_debug_set_option")
+    return int(old)
 
 
 def snap_kernel_launch_count() -> int:

@@ -1,9 +1,10 @@
 // Host side of the C ABI: argument validation, slot arithmetic, scratch planning and the
-// launch sequences.  No allocation, no synchronisation, no state besides the launch counter
-// and a cached SM count.
+// launch sequences.  No allocation, no synchronisation.  State kept between calls: the launch
+// counter, a per-device SM count, and the process-wide testing options below.
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "snap_internal.cuh"
@@ -12,11 +13,35 @@ namespace snap {
 
 unsigned long long g_launches = 0;
 
+// Testing and tuning options: one integer each, process-wide, set through snap_debug_set_option.
+// Each starts from its environment variable, which is read once, at the first use of any option.
+namespace {
+int g_opt[SNAP_OPT_COUNT] = {};
+std::once_flag g_opt_once;
+
+void seed_options() {
+  auto env_int = [](const char* name) { const char* e = getenv(name); const int v = e ? atoi(e) : 0; return v > 0 ? v : 0; };
+  if (const char* e = getenv("SNAP_SCORE_PATH")) g_opt[SNAP_OPT_SCORE_KERNEL] = !strcmp(e, "mma") ? 1 : !strcmp(e, "simt") ? 2 : 0;
+  if (const char* e = getenv("SNAP_DECODE_GQA")) g_opt[SNAP_OPT_DECODE_GQA_KERNEL] = e[0] == 's';
+  if (const char* e = getenv("SNAP_DECODE_MLA")) g_opt[SNAP_OPT_DECODE_LATENT_KERNEL] = e[0] == 'm';
+  if (const char* e = getenv("SNAP_PREFILL_PATH")) g_opt[SNAP_OPT_PREFILL_KERNEL] = !strcmp(e, "simt");
+  if (const char* e = getenv("SNAP_PREFILL_HEADS")) g_opt[SNAP_OPT_PREFILL_SINGLE_HEADS] = e[0] == '1';
+  if (const char* e = getenv("SNAP_REFINE")) g_opt[SNAP_OPT_REFINE_OFF] = e[0] == '0';
+  g_opt[SNAP_OPT_DECODE_NSPLIT] = env_int("SNAP_DECODE_NSPLIT");
+  g_opt[SNAP_OPT_SCORE_NSPLIT] = env_int("SNAP_SCORE_NSPLIT");
+  g_opt[SNAP_OPT_WIDE_STAGES] = env_int("SNAP_WIDE_STAGES");
+}
+}  // namespace
+
+int option(int which) {
+  std::call_once(g_opt_once, seed_options);
+  return which >= 0 && which < SNAP_OPT_COUNT ? g_opt[which] : 0;
+}
+
 // 128-wide bf16 heads decode on the tensor-core kernel (faster than the packed-FP32 kernel at every
-// group size); SNAP_DECODE_GQA=simt keeps the packed-FP32 kernel (testing aid).
+// group size); option SNAP_OPT_DECODE_GQA_KERNEL = 1 keeps the packed-FP32 kernel (testing aid).
 bool decode_use_gqa_mma(int dtype, const Shape& s) {
-  const char* env = getenv("SNAP_DECODE_GQA");
-  if (env && env[0] == 's') return false;
+  if (option(SNAP_OPT_DECODE_GQA_KERNEL) == 1) return false;
   return decode_gqa_mma_supported(dtype, s);
 }
 
@@ -67,20 +92,18 @@ Shape make_shape(const snap_config_t* c) {
 
 size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
-// SNAP_SCORE_PATH=mma|simt forces a slower score kernel (testing aid); default: the best one.
+// Option SNAP_OPT_SCORE_KERNEL = 1 (mma.sync) or 2 (SIMT) forces a slower score kernel (testing
+// aid); default: the best one.
 bool use_umma(int dtype, const Shape& s) {
-  const char* env = getenv("SNAP_SCORE_PATH");
-  if (env && (!strcmp(env, "mma") || !strcmp(env, "simt"))) return false;
+  if (option(SNAP_OPT_SCORE_KERNEL) != 0) return false;
   return score_umma_supported(dtype, s);
 }
 bool use_umma_wide(int dtype, const Shape& s) {
-  const char* env = getenv("SNAP_SCORE_PATH");
-  if (env && (!strcmp(env, "mma") || !strcmp(env, "simt"))) return false;
+  if (option(SNAP_OPT_SCORE_KERNEL) != 0) return false;
   return !score_umma_supported(dtype, s) && score_umma_wide_supported(dtype, s);
 }
 bool use_mma(int dtype, const Shape& s) {
-  const char* env = getenv("SNAP_SCORE_PATH");
-  if (env && !strcmp(env, "simt")) return false;
+  if (option(SNAP_OPT_SCORE_KERNEL) == 2) return false;
   return score_mma_supported(dtype, s);
 }
 
@@ -141,10 +164,9 @@ struct DecodePlan { bool gqa, gqa_mma, mla, mla_stream; int nsplit; size_t float
 bool use_gqa_mma(int dtype, const Shape& s) { return decode_use_gqa_mma(dtype, s); }
 
 // Kernel for the latent layout: the streamed tcgen05 kernel when the head count allows (multiples
-// of 128), else the mma.sync kernel; SNAP_DECODE_MLA=mma forces the latter (testing aid).
+// of 128), else the mma.sync kernel; option SNAP_OPT_DECODE_LATENT_KERNEL = 1 forces the latter.
 bool use_mla_stream(int dtype, const Shape& s) {
-  const char* env = getenv("SNAP_DECODE_MLA");
-  if (env && env[0] == 'm') return false;
+  if (option(SNAP_OPT_DECODE_LATENT_KERNEL) == 1) return false;
   return decode_mla_stream_supported(dtype, s);
 }
 
@@ -179,6 +201,50 @@ size_t idx_bytes(const Shape& s, int n_seq) {
 }
 
 }  // namespace
+
+// One decode step with its partial results in `scratch`: the body of snap_decode_attn, shared with
+// snap_decode_attn_static so that both choose the same kernel and split count.  `slack_bytes` is
+// the margin the size query adds for the caller's own alignment; `too_small` is the status
+// returned when the partial results do not fit.
+int decode_step_with_scratch(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,
+                             const void* k_new_dev, const void* v_new_dev, const int32_t* slot_ids_dev,
+                             int32_t n_active, void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
+                             const int32_t* valid_topk_dev, void* out_dev, float* scratch, size_t scratch_bytes,
+                             size_t slack_bytes, int too_small, uint32_t* status_dev, void* cuda_stream) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (!layout) return SNAP_ERR_NULL_POINTER;
+  if (n_active < 0) return SNAP_ERR_INVALID_ARG;
+  if (n_active == 0) return SNAP_OK;
+  if (!q_dev || !slot_ids_dev || !k_cache_dev || !seq_len_dev || !valid_topk_dev || !out_dev || !scratch)
+    return SNAP_ERR_NULL_POINTER;
+  if (!cfg->v_aliases_k && !v_cache_dev) return SNAP_ERR_NULL_POINTER;
+  if (k_new_dev && !cfg->v_aliases_k && !v_new_dev) return SNAP_ERR_NULL_POINTER;
+  const Shape s = make_shape(cfg);
+  if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
+  const DecodePlan p = plan_decode(cfg->dtype, s, n_active);
+  if (scratch_bytes < p.floats * sizeof(float) + slack_bytes) return too_small;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e;
+  if (p.mla_stream)
+    e = launch_decode_mla_stream(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev,
+                                 valid_topk_dev, out_dev, scratch, p.nsplit, status_dev, st);
+  else if (p.mla)
+    e = launch_decode_mla(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev,
+                          valid_topk_dev, out_dev, scratch, p.nsplit, status_dev, st);
+  else if (p.gqa && p.gqa_mma)
+    e = launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
+                              v_cache_dev, seq_len_dev, valid_topk_dev, out_dev, scratch, p.nsplit, status_dev, st);
+  else if (p.gqa)
+    e = launch_decode_gqa(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
+                          v_cache_dev, seq_len_dev, valid_topk_dev, out_dev, scratch, p.nsplit, status_dev, st);
+  else
+    e = launch_decode_generic(cfg->dtype, s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active,
+                              k_cache_dev, v_cache_dev, seq_len_dev, valid_topk_dev, out_dev, scratch, p.nsplit,
+                              status_dev, st);
+  return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+}
+
 }  // namespace snap
 
 using namespace snap;
@@ -199,6 +265,13 @@ const char* snap_status_string(int status) {
 }
 
 int64_t snap_kernel_launch_count(void) { return (int64_t)g_launches; }
+
+int snap_debug_set_option(int opt, int value) {
+  if (opt < 0 || opt >= SNAP_OPT_COUNT || value < 0) return SNAP_ERR_INVALID_ARG;
+  const int old = option(opt);
+  g_opt[opt] = value;
+  return old;
+}
 
 int snap_cache_layout(const snap_config_t* cfg, snap_layout_t* out) {
   if (!cfg || !out) return SNAP_ERR_NULL_POINTER;
@@ -274,9 +347,8 @@ int snap_prefill_attn(const snap_config_t* cfg, const void* q_dev,
   if ((k_token_stride * eb) % 16 || (k_head_stride * eb) % 16 || k_token_stride < s.d_qk) return SNAP_ERR_INVALID_ARG;
   if (!cfg->v_aliases_k && ((v_token_stride * eb) % 16 || (v_head_stride * eb) % 16 || v_token_stride < s.d_v))
     return SNAP_ERR_INVALID_ARG;
-  // SNAP_PREFILL_PATH=simt forces the portable kernel (testing aid)
-  const char* env = getenv("SNAP_PREFILL_PATH");
-  const bool tensor_path = prefill_attn_supported(cfg->dtype, s) && !(env && !strcmp(env, "simt"));
+  // option SNAP_OPT_PREFILL_KERNEL = 1 forces the portable kernel (testing aid)
+  const bool tensor_path = prefill_attn_supported(cfg->dtype, s) && option(SNAP_OPT_PREFILL_KERNEL) != 1;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   KVSource src;
   src.k = k_dev; src.v = v_dev;
@@ -417,43 +489,9 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
                      int32_t n_active, void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
                      const int32_t* valid_topk_dev, void* out_dev, void* workspace_dev,
                      size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
-  const int rc = validate(cfg);
-  if (rc != SNAP_OK) return rc;
-  if (!layout) return SNAP_ERR_NULL_POINTER;
-  if (n_active < 0) return SNAP_ERR_INVALID_ARG;
-  if (n_active == 0) return SNAP_OK;
-  if (!q_dev || !slot_ids_dev || !k_cache_dev || !seq_len_dev || !valid_topk_dev || !out_dev ||
-      !workspace_dev)
-    return SNAP_ERR_NULL_POINTER;
-  if (!cfg->v_aliases_k && !v_cache_dev) return SNAP_ERR_NULL_POINTER;
-  if (k_new_dev && !cfg->v_aliases_k && !v_new_dev) return SNAP_ERR_NULL_POINTER;
-  const Shape s = make_shape(cfg);
-  if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
-  const int64_t need = snap_decode_workspace_bytes(cfg, n_active);
-  if (need < 0) return (int)need;
-  if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
-  const DecodePlan p = plan_decode(cfg->dtype, s, n_active);
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  cudaError_t e;
-  if (p.mla_stream)
-    e = launch_decode_mla_stream(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev,
-                                 valid_topk_dev, out_dev, static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
-  else if (p.mla)
-    e = launch_decode_mla(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev,
-                          valid_topk_dev, out_dev, static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
-  else if (p.gqa && p.gqa_mma)
-    e = launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
-                              v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
-                              static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
-  else if (p.gqa)
-    e = launch_decode_gqa(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
-                          v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
-                          static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
-  else
-    e = launch_decode_generic(cfg->dtype, s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active,
-                              k_cache_dev, v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
-                              static_cast<float*>(workspace_dev), p.nsplit, status_dev, st);
-  return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+  return decode_step_with_scratch(cfg, layout, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
+                                  v_cache_dev, seq_len_dev, valid_topk_dev, out_dev, static_cast<float*>(workspace_dev),
+                                  workspace_bytes, 256, SNAP_ERR_WORKSPACE_TOO_SMALL, status_dev, cuda_stream);
 }
 
 // Several query tokens per sequence in one step.  The tensor-core kernel for bf16 heads serves

@@ -484,13 +484,10 @@ bool decode_gqa_supported(int dtype, const Shape& s) {
 // batches -- more splits only lengthen the merge -- and three splits are best once the batch
 // alone fills the GPU (they even out the tail).  A split keeps at least two 64-row blocks and,
 // for very long caches, at most about 48.
-// SNAP_DECODE_NSPLIT overrides the choice (tuning aid).
+// Option SNAP_OPT_DECODE_NSPLIT overrides the choice (tuning aid).
 int decode_gqa_nsplit_for(const Shape& s, int n_active, int sm_count, int ctas_per_sm) {
   const int tiles = (s.Sc + 63) / 64;
-  if (const char* env = getenv("SNAP_DECODE_NSPLIT")) {
-    const int v = atoi(env);
-    if (v >= 1) return v < tiles ? v : tiles;
-  }
+  if (const int v = option(SNAP_OPT_DECODE_NSPLIT)) return v < tiles ? v : tiles;
   const long long base = (long long)(n_active > 0 ? n_active : 1) * s.Hkv;
   long long ns = (7LL * sm_count / 4 + base / 2) / base;
   if (ns < 3) ns = 3;

@@ -427,9 +427,8 @@ cudaError_t launch_prefill_attn(const Shape& s, const SeqBatch& b, const void* q
   a.out = static_cast<__nv_bfloat16*>(out);
   a.mu = mu;
   a.status = status;
-  // pairs of heads that share a KV head when the group allows (SNAP_PREFILL_HEADS=1 forces single heads)
-  const char* env = getenv("SNAP_PREFILL_HEADS");
-  const int nq = s.g % 2 == 0 && !(env && env[0] == '1') ? 2 : 1;
+  // pairs of heads that share a KV head when the group allows (option SNAP_OPT_PREFILL_SINGLE_HEADS forces single heads)
+  const int nq = s.g % 2 == 0 && option(SNAP_OPT_PREFILL_SINGLE_HEADS) != 1 ? 2 : 1;
   const size_t smem = prefill_smem_bytes(nq);
   static SmemLimit limit1 = {}, limit2 = {};
   const dim3 grid((max_len + BM - 1) / BM, s.Hq / nq, b.n);

@@ -387,9 +387,8 @@ int score_umma_nsplit(const Shape& s, const int* le, int n_scored, int sm_count,
     return n * s.Hkv;
   };
   int c = max_tiles;
-  if (const char* env = getenv("SNAP_SCORE_NSPLIT")) {          // tuning aid: splits of the longest prompt
-    const int v = atoi(env);
-    if (v >= 1) c = (max_tiles + v - 1) / v;
+  if (const int v = option(SNAP_OPT_SCORE_NSPLIT)) {            // tuning aid: splits of the longest prompt
+    c = (max_tiles + v - 1) / v;
   } else {
     const long long nz = (long long)n_scored * s.Hkv;
     const long long target = (nz + sm_count - 1) / sm_count * sm_count;

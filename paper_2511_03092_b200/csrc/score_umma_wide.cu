@@ -336,13 +336,11 @@ size_t wide_smem_bytes(int NH, int NS) {
          (2 * NS + 5) * 8 + 16 + 1024;
 }
 
-// SNAP_WIDE_STAGES caps the ring depth (tuning aid).
+// Option SNAP_OPT_WIDE_STAGES caps the ring depth (tuning aid).
 int wide_stages(int NH) {
   int ns = MAXNS;
-  if (const char* env = getenv("SNAP_WIDE_STAGES")) {
-    const int v = atoi(env);
+  if (const int v = option(SNAP_OPT_WIDE_STAGES))
     if (v >= 2 && v < ns) ns = v;
-  }
   while (ns > 2 && wide_smem_bytes(NH, ns) > 227u * 1024u) --ns;
   return ns;
 }
@@ -361,10 +359,8 @@ int score_umma_wide_row_blocks(const Shape& s) { return (s.g * s.Lo + 127) / 128
 int score_umma_wide_nsplit(const Shape& s, int n_scored, int max_le, int sm_count) {
   const int tiles = (max_le + 255) / 256;
   const long long base = (long long)n_scored * s.Hkv * score_umma_wide_row_blocks(s);
-  if (const char* env = getenv("SNAP_SCORE_NSPLIT")) {          // tuning aid
-    const int v = atoi(env);
-    if (v >= 1) return v < tiles ? (v < 512 ? v : 512) : tiles;
-  }
+  if (const int v = option(SNAP_OPT_SCORE_NSPLIT))              // tuning aid
+    return v < tiles ? (v < 512 ? v : 512) : tiles;
   long long ns = (2LL * sm_count + base / 2) / base;
   if (ns > tiles) ns = tiles;
   if (ns > 512) ns = 512;

@@ -51,6 +51,16 @@ struct ScoreBuffers {
 extern unsigned long long g_launches;
 inline void count_launch() { ++g_launches; }
 
+// Current value of a process-wide testing / tuning option (SNAP_OPT_* of snapstream.h).
+int option(int which);
+
+// Body of snap_decode_attn with the scratch passed as a plain pointer (api.cu).
+int decode_step_with_scratch(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,
+                             const void* k_new_dev, const void* v_new_dev, const int32_t* slot_ids_dev,
+                             int32_t n_active, void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
+                             const int32_t* valid_topk_dev, void* out_dev, float* scratch, size_t scratch_bytes,
+                             size_t slack_bytes, int too_small, uint32_t* status_dev, void* cuda_stream);
+
 // A kernel's dynamic shared-memory limit is a per-device attribute: raise it once on every
 // device the library is used on.  `done` is the caller's per-kernel record (static storage).
 constexpr int kMaxDevices = 64;

@@ -24,3 +24,17 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture
+def snap_option():
+    """Set process-wide testing options of the library for one test; restored afterwards."""
+    from paper_2511_03092_b200 import binding as B
+    changed = []
+
+    def set_option(option, value):
+        changed.append((option, B.snap_debug_set_option(option, value)))
+
+    yield set_option
+    for option, old in reversed(changed):
+        B.snap_debug_set_option(option, old)

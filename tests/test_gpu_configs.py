@@ -101,6 +101,54 @@ def test_config3_latent_sample():
     _run(wl, [16384], seed=400, steps=3)
 
 
+def test_config3_full_size_unit():
+    """Config 3 at its real size: eight 131072-token latent prompts (Ls 4, Lr 2048, K 8192, Lo 32,
+    w 7, 128 heads over one 576-wide row) compressed by one call into a batch-8 layer, then decoded
+    together, so that the wide score kernel runs its full split count and 32 row blocks, the
+    selection sees 129020 candidates at K = 8192 and the latent decode kernel its 10244-slot,
+    batch-8 grid and split rule.  The oracle follows one of the eight sequences (units are
+    independent); the others only have to leave the status word clean and their cache sections in
+    place.  Oracle wall time: about 11 s for the compression of the followed prompt (8 host cores)
+    and 0.3 s per decode step."""
+    wl = synth.CONFIGS[3]
+    n, L, followed = wl.batch, 131072, 5
+    assert (n, wl.topk, wl.l_recent, wl.l_obs, wl.pool_kernel, wl.slots) == (8, 8192, 2048, 32, 7, 10244)
+    layer = H.GpuLayer(wl, max_seqs=n)
+    prompts = [synth.make_prompt(wl, L, 400 + 13 * i) for i in range(n)]
+    idx = layer.compress(prompts, list(range(n)))
+    assert layer.status() == 0
+    seq = H.oracle_compress(wl, prompts[followed])
+    swaps = H.check_selection(idx[followed], seq, wl)
+    assert swaps <= 2
+    seq.topk_pos = [idx[followed][0].astype(np.int64)]
+    H.check_cache_image(layer, seq, followed, wl)
+    for i in range(n):                                      # every planted heavy hitter is kept (sanity, all prompts)
+        assert np.isin(prompts[i]["planted"][0], idx[i][0]).all()
+        assert (np.diff(idx[i][0]) > 0).all() and idx[i][0][0] >= wl.l_sink and idx[i][0][-1] < L - wl.l_recent
+    assert [int(x) for x in layer.cache.seq_len.cpu()] == [L] * n
+    assert [int(x) for x in layer.cache.valid_topk.cpu()] == [wl.topk] * n
+    slots_dev = torch.arange(n, dtype=torch.int32, device="cuda")
+    for step in range(3):
+        d = synth.make_decode_inputs(wl, n, 400, step)
+        out = layer.decode(d["q"].cuda(), d["k_new"].cuda(), None, slots_dev)
+        ref = orc.decode_step(seq, synth.to_f64(d["q"][followed]), synth.to_f64(d["k_new"][followed]), None)
+        H.check_output(out[followed], ref, wl, f"step {step}")
+        assert torch.isfinite(out.float()).all()
+    H.check_cache_image(layer, seq, followed, wl)
+    assert layer.status() == 0
+    assert [int(x) for x in layer.cache.seq_len.cpu()] == [L + 3] * n
+
+
+def test_config2_ragged_batch_with_a_128k_prompt():
+    """Config 2's compress call as bench.py issues it: one call over a ragged batch that holds a
+    prompt near the 131072-token end of the range next to short ones (the candidate splits of the
+    score kernel are cut to the batch as a whole).  Every sequence is followed by the oracle
+    (about 4 s for the long prompt's compression)."""
+    wl = synth.CONFIGS[2]
+    swaps = _run(wl, [9000, 126000 + 77, 30011, 8192], seed=700, steps=3)
+    assert swaps <= 2
+
+
 def test_config4_one_sequence_layer_unit():
     """One (sequence, layer) unit of the 32-layer, 128k-prompt configuration: units are independent,
     so parity on a unit at full prompt length covers the kernels in the launch shape bench.py uses."""

@@ -218,9 +218,9 @@ def test_group_sizes(hq, hkv):
 
 
 @pytest.mark.parametrize("hq,hkv", [(4, 4), (16, 4), (20, 4), (32, 4)], ids=["g1", "g4", "g5", "g8"])
-def test_packed_fp32_decode_kernel_stays_selectable(hq, hkv, monkeypatch):
+def test_packed_fp32_decode_kernel_stays_selectable(hq, hkv, snap_option):
     """The packed-FP32 decode kernel (the default before the tensor-core one) on the same cases."""
-    monkeypatch.setenv("SNAP_DECODE_GQA", "simt")
+    snap_option(B.SNAP_OPT_DECODE_GQA_KERNEL, 1)
     wl = SMALL_BF16.scaled(n_q_heads=hq, n_kv_heads=hkv)
     _run_compress_and_decode(wl, [wl.prompt_len[0], 50, 3], seed=13, steps=5)
     _run_compress_and_decode(wl, [300], seed=17, steps=2 * wl.l_recent + 5, check_ring_every=16)
@@ -273,10 +273,10 @@ def test_latent_attention_kernel_shapes(hq):
     _run_compress_and_decode(wl, [500, 70], seed=31, steps=45, sharp=3.0, check_ring_every=9)
 
 
-def test_latent_attention_mma_sync_decode_kernel_with_128_heads(monkeypatch):
+def test_latent_attention_mma_sync_decode_kernel_with_128_heads(snap_option):
     """The mma.sync decode kernel for the latent layout stays selectable at 128 heads, where the
     tcgen05 kernel is the default: same cases."""
-    monkeypatch.setenv("SNAP_DECODE_MLA", "mma")
+    snap_option(B.SNAP_OPT_DECODE_LATENT_KERNEL, 1)
     wl = synth.Workload("mla_small", 128, 1, 576, 512, "bf16", 3, 40, 64, 8, 5, batch=1,
                         prompt_len=(500, 500), decode_steps=6, salience="planted", n_planted=8,
                         v_aliases_k=True, softmax_scale=2.0 ** -0.5)

@@ -68,8 +68,8 @@ def test_prefill_attention_and_normalisers_match_oracle(wl):
     _check_prefill(wl, [1, 5, 127, 128, 129, 300, 520, 700], seed=310)
 
 
-def test_single_head_kernel_stays_selectable_for_even_groups(monkeypatch):
-    monkeypatch.setenv("SNAP_PREFILL_HEADS", "1")
+def test_single_head_kernel_stays_selectable_for_even_groups(snap_option):
+    snap_option(B.SNAP_OPT_PREFILL_SINGLE_HEADS, 1)
     _check_prefill(WL64, [129, 700], seed=315)
 
 
@@ -216,16 +216,16 @@ def test_portable_prefill_kernel_and_every_score_path_take_the_normalisers(wl):
         H.check_cache_image(layer, seq, slots[i], wl)
 
 
-def test_normalisers_through_the_mma_sync_score_path(monkeypatch):
-    monkeypatch.setenv("SNAP_SCORE_PATH", "mma")
+def test_normalisers_through_the_mma_sync_score_path(snap_option):
+    snap_option(B.SNAP_OPT_SCORE_KERNEL, 1)
     test_compress_with_prefill_normalisers_matches_oracle(WL128)
 
 
-def test_portable_prefill_kernel_matches_the_tensor_core_one(monkeypatch):
+def test_portable_prefill_kernel_matches_the_tensor_core_one(snap_option):
     wl = WL64
     lengths = [129, 300]
     _, _, _, cu, _, out_t, mu_t = _prefill(wl, lengths, seed=380)
-    monkeypatch.setenv("SNAP_PREFILL_PATH", "simt")
+    snap_option(B.SNAP_OPT_PREFILL_KERNEL, 1)
     _, _, _, _, _, out_s, mu_s = _prefill(wl, lengths, seed=380)
     assert (out_t.float() - out_s.float()).abs().max().item() <= 2e-2
     assert (mu_t - mu_s).abs().max().item() <= 2 * MU_ATOL
