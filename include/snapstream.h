@@ -68,8 +68,12 @@ typedef enum snap_status {
 /* bits of *status_dev */
 #define SNAP_DEV_BAD_SLOT 1u        /* a slot id was outside [0, max_seqs): that sequence was skipped */
 #define SNAP_DEV_WAIT_TIMEOUT 2u    /* a bounded wait on an async copy gave up: results invalid */
-#define SNAP_DEV_BAND_OVERFLOW 4u   /* more near-threshold candidates than the refinement can hold:
-                                       the single-precision order was kept for that head */
+#define SNAP_DEV_BAND_OVERFLOW 4u   /* snap_compress: a KV head had more candidates within the re-scoring
+                                       band of its top-K threshold than the band buffer holds (512, or
+                                       256 for layers with more than 2^18 query elements per KV head);
+                                       that head keeps its single-precision order.  The results are
+                                       valid; exactly tied scores, which go to the lower position in
+                                       either precision, are the usual cause */
 
 /* One attention layer's shape and SnapStream hyper-parameters (appendix table
  * "SnapStream Hyperparameters": sink, top-K, recent, observation window, pooling kernel). */
@@ -136,6 +140,14 @@ int64_t snap_decode_workspace_bytes(const snap_config_t* cfg, int32_t n_active);
  *               ascending, -1 after the valid ones.
  *   A prompt with L <= Lsr + K is not scored: all its candidates are kept.  Otherwise the K
  *   largest pooled scores win, ties to the lower position.
+ *   Precision of the selection: scores are computed in single precision (the part of their error
+ *   that can reorder two pooled scores was measured at 1e-7 relative, 2.2e-7 at most, on 32k-
+ *   to 128k-token prompts); every candidate whose pooled score lies within 1e-4 relative of the
+ *   K-th largest (2e-5 for layers with more than 2^18 query elements per KV head, such as the
+ *   latent layout) is then scored again in double precision from q_obs and k, with the
+ *   normalisers of Eq. 4 from the single-precision pass, and the order inside that band decides
+ *   (measured order error 2e-9, 1.3e-8 at most).  Pooling kernels wider than 33 are not
+ *   re-scored.  SNAP_DEV_BAND_OVERFLOW reports a band that did not fit its buffer.
  */
 int snap_compress(const snap_config_t* cfg, const snap_layout_t* layout,
                   const void* q_obs_dev,

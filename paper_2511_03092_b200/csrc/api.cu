@@ -111,7 +111,25 @@ bool use_mma(int dtype, const Shape& s) {
 struct ChunkPlan {
   int n_scored, max_le, nsplit, chunk_tiles, c_stride;
   size_t part_off, stats_off, c_off, p_off, cpart_off, bytes;
+  // double-precision refinement of the selection near the threshold (cap == 0: none)
+  int ref_cap, ref_chunks;
+  float ref_rel;
+  size_t ref_band_off, ref_part_off, ref_mu_off, ref_head_off;
 };
+
+// Band of the refinement: wide (1e-4 relative, up to 512 members) where re-scoring a member is cheap,
+// narrower (2e-5, up to 256 members) where one member costs millions of multiply-adds (the latent
+// shape: 4096 window rows x 576 dims).  Both are far above the single-precision error of a pooled
+// score (measured: 2e-8 .. 6e-7 relative on the benchmark shapes).  Pooling kernels wider than 33
+// are not refined.
+void plan_refine(const Shape& s, ChunkPlan& p) {
+  p.ref_cap = 0;
+  if (option(SNAP_OPT_REFINE_OFF) == 1 || s.w > 33 || p.n_scored == 0) return;
+  const long long member_cost = (long long)s.g * s.Lo * s.d_qk;
+  p.ref_cap = member_cost <= (1LL << 18) ? 512 : 256;
+  p.ref_rel = member_cost <= (1LL << 18) ? 1e-4f : 2e-5f;
+  p.ref_chunks = refine_row_chunks(s);
+}
 
 ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, int n) {
   ChunkPlan p;
@@ -147,6 +165,13 @@ ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, in
   p.p_off = off;     off += align_up(nz * p.c_stride * sizeof(float));
   p.cpart_off = off;
   if (use_umma_wide(dtype, s)) off += align_up(nz * score_umma_wide_row_blocks(s) * p.c_stride * sizeof(float));
+  plan_refine(s, p);
+  if (p.ref_cap > 0) {
+    p.ref_band_off = off; off += align_up(nz * p.ref_cap * sizeof(BandEntry));
+    p.ref_part_off = off; off += align_up(nz * p.ref_cap * p.ref_chunks * s.w * sizeof(double));
+    p.ref_mu_off = off;   off += align_up(nz * R * sizeof(double));
+    p.ref_head_off = off; off += align_up(nz * sizeof(RefineHead));
+  }
   p.bytes = off;
   return p;
 }
@@ -448,6 +473,14 @@ int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* 
       buf.P = reinterpret_cast<float*>(chunk_ws + p.p_off);
       buf.c_stride = p.c_stride; buf.nsplit = p.nsplit; buf.chunk_tiles = p.chunk_tiles;
       buf.ext_mu = row_mu_dev;
+      if (p.ref_cap > 0) {
+        buf.ref.head = reinterpret_cast<RefineHead*>(chunk_ws + p.ref_head_off);
+        buf.ref.band = reinterpret_cast<BandEntry*>(chunk_ws + p.ref_band_off);
+        buf.ref.part = reinterpret_cast<double*>(chunk_ws + p.ref_part_off);
+        buf.ref.mu64 = row_mu_dev ? nullptr : reinterpret_cast<double*>(chunk_ws + p.ref_mu_off);
+        buf.ref.cap = p.ref_cap; buf.ref.chunks = p.ref_chunks; buf.ref.rel = p.ref_rel;
+        buf.ref.stats_natural = !use_umma(cfg->dtype, s) && !use_umma_wide(cfg->dtype, s) && !use_mma(cfg->dtype, s);
+      }
       const cudaError_t e = use_umma(cfg->dtype, s)  ? launch_score_umma(s, b, q_obs_dev, src, buf, status_dev, st)
                             : use_umma_wide(cfg->dtype, s)
                                 ? launch_score_umma_wide(s, b, q_obs_dev, src, buf,
@@ -459,6 +492,9 @@ int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* 
     if (launch_pool_topk(s, b, buf, idx, status_dev, st) != cudaSuccess) return SNAP_ERR_CUDA;
     if (launch_gather(cfg->dtype, s, b, src, idx, k_cache_dev, v_cache_dev, seq_len_dev,
                       valid_topk_dev, status_dev, st) != cudaSuccess)
+      return SNAP_ERR_CUDA;
+    if (launch_topk_refine(cfg->dtype, s, b, q_obs_dev, src, buf, idx, k_cache_dev, v_cache_dev, status_dev, sm_count(),
+                           st) != cudaSuccess)
       return SNAP_ERR_CUDA;
   }
   return SNAP_OK;

@@ -72,6 +72,9 @@ __device__ __forceinline__ void copy_rows(const char* __restrict__ src_base, lon
 
 __global__ void __launch_bounds__(NT) gather_kernel(const GatherArgs a) {
   pdl_wait();
+  // the refinement of the selection (launched next) may start now: it reads only what the selection
+  // kernel wrote, and waits for this grid itself before it corrects anything
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int seq = blockIdx.z, kvh = blockIdx.y;
   const int L = a.b.len[seq], slot = a.b.slot[seq];
   if (slot < 0 || slot >= a.max_seqs) {

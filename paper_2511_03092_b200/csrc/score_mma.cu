@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(256, 2) score_mma_kernel(const MmaArgs a) {
 
 // Merge the per-split statistics (log2 domain): m = max_s m_s, l = sum_s l_s 2^(m_s - m); keep (m, 1/l).
 __global__ void score_mma_combine_kernel(const float2* __restrict__ part, float2* __restrict__ stats,
-                                         int nsplit, int R) {
+                                         double* __restrict__ mu64, int nsplit, int R) {
   // one warp per query row, lanes over the splits
   pdl_wait();
   const long long z = blockIdx.y;
@@ -259,14 +259,17 @@ __global__ void score_mma_combine_kernel(const float2* __restrict__ part, float2
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-  if (lane == 0) stats[z * R + row] = make_float2(m, (float)(1.0 / l));
+  if (lane == 0) {
+    stats[z * R + row] = make_float2(m, (float)(1.0 / l));
+    if (mu64) mu64[z * R + row] = (double)m + log2(l);       // the same normaliser, unrounded, for the refinement
+  }
 }
 
 }  // namespace
 
 cudaError_t launch_score_combine_log2(const ScoreBuffers& buf, int nz, int R, cudaStream_t st) {
   const cudaError_t e = launch_pdl(score_mma_combine_kernel, dim3((R + 7) / 8, nz), dim3(256), 0, st,
-                                   static_cast<const float2*>(buf.part_stats), buf.stats, buf.nsplit, R);
+                                   static_cast<const float2*>(buf.part_stats), buf.stats, buf.ref.mu64, buf.nsplit, R);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }

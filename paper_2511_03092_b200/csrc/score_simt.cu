@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(NT) score_stats_kernel(const ScoreArgs a) {
 
 // Merge the per-split statistics: m = max_s m_s, l = sum_s l_s exp(m_s - m), kept as (m, 1/l).
 __global__ void score_combine_kernel(const float2* __restrict__ part, float2* __restrict__ stats,
-                                     int nsplit, int R) {
+                                     double* __restrict__ mu64, int nsplit, int R) {
   const long long z = blockIdx.x;
   for (int row = threadIdx.x; row < R; row += blockDim.x) {
     float m = -INFINITY;
@@ -141,6 +141,7 @@ __global__ void score_combine_kernel(const float2* __restrict__ part, float2* __
       if (p.y > 0.f) l += (double)p.y * exp((double)p.x - (double)m);
     }
     stats[z * R + row] = make_float2(m, (float)(1.0 / l));
+    if (mu64) mu64[z * R + row] = ((double)m + log(l)) * 1.4426950408889634074;   // log2 domain, unrounded
   }
 }
 
@@ -203,7 +204,7 @@ cudaError_t launch_t(const ScoreArgs& a, int max_le, cudaStream_t st) {
     dim3 g1(a.buf.nsplit, (R + BM - 1) / BM, nz);
     score_stats_kernel<T><<<g1, NT, 0, st>>>(a);
     count_launch();
-    score_combine_kernel<<<nz, 256, 0, st>>>(a.buf.part_stats, a.buf.stats, a.buf.nsplit, R);
+    score_combine_kernel<<<nz, 256, 0, st>>>(a.buf.part_stats, a.buf.stats, a.buf.ref.mu64, a.buf.nsplit, R);
     count_launch();
   }
   dim3 g2((max_le + BN - 1) / BN, 1, nz);

@@ -36,6 +36,30 @@ struct KVSource {
   long long k_tok_stride, k_head_stride, v_tok_stride, v_head_stride;   // elements
 };
 
+// Double-precision re-scoring of the candidates near the top-K threshold (topk_refine.cu).
+// The selection kernel lists every candidate whose single-precision pooled score lies within
+// `rel` (relative) of the K-th largest -- the band -- and counts the candidates above the band;
+// the refinement kernel recomputes the band members' pooled scores in double and corrects the
+// emitted index list where the order inside the band differs.
+struct RefineHead {       // one per (scored prompt, KV head); zeroed by the selection kernel
+  int n_band;             // band members found (may exceed cap: then nothing is refined)
+  int n_sure;             // candidates above the band: selected whatever the band's order
+  int done;               // refinement CTAs of this head that have finished
+  int changed;            // out: index pairs exchanged by the refinement
+  float max_dev;          // out: largest |single / double - 1| over the band's pooled scores
+  int pad[3];
+};
+struct BandEntry { int idx_flag; float p32; };   // candidate index | (selected in single precision) << 31
+struct RefineBuffers {
+  RefineHead* head;       // [nz]; NULL = no refinement
+  BandEntry* band;        // [nz][cap]
+  double* part;           // [nz][cap][chunks][w] column sums of Eq. 1 per block of 256 window rows
+  double* mu64;           // [nz][R] Eq. 4 normalisers (log2 domain) as the statistics merge computed them
+  int cap, chunks;
+  float rel;
+  int stats_natural;      // 1: `stats` holds (m, 1/l) of natural-base exponentials (SIMT path)
+};
+
 struct ScoreBuffers {
   float2* part_stats;   // [n_scored*Hkv][nsplit][R]  (running max, sum of exp) per candidate split
   float2* stats;        // [n_scored*Hkv][R]          (row max m_i, 1 / l_i)
@@ -46,6 +70,7 @@ struct ScoreBuffers {
   int chunk_tiles;      // 128-wide tcgen05 score kernel: candidate tiles per CTA (split x covers tiles [x c, x c + c))
   const float* ext_mu;  // NULL, or [prompts][Hq][Lo] log2 normalisers of Eq. 4 computed elsewhere
                         // (the prefill attention kernel): pass 1 and the combine step are skipped
+  RefineBuffers ref;
 };
 
 extern unsigned long long g_launches;
@@ -125,6 +150,11 @@ cudaError_t launch_prefill_generic(int dtype, const Shape& s, const SeqBatch& b,
                                    void* out, float* mu, cudaStream_t st);
 cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffers& buf,
                              int* idx_out, uint32_t* status, cudaStream_t st);
+// double-precision re-scoring of the near-threshold band; corrects idx_out and the cache rows (runs after the gather)
+int refine_row_chunks(const Shape& s);
+cudaError_t launch_topk_refine(int dtype, const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
+                               const ScoreBuffers& buf, int* idx_out, void* k_cache, void* v_cache, uint32_t* status,
+                               int sm_count, cudaStream_t st);
 cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KVSource& src,
                           const int* idx, void* k_cache, void* v_cache, int* seq_len,
                           int* valid_topk, uint32_t* status, cudaStream_t st);

@@ -19,6 +19,11 @@
 // thread order is index order one block scan places the whole slice.  The streaming one keeps
 // pooled scores in scratch and handles any length.
 // Prompts with at most K candidates keep them all and are not scored.
+//
+// For the double-precision refinement (topk_refine.cu) the emission step also records the band:
+// every candidate whose pooled score lies within a relative distance of the threshold, with a
+// flag saying whether the single-precision order selected it, and the number of candidates
+// above the band.
 #include <cooperative_groups.h>
 
 #include "snap_internal.cuh"
@@ -50,6 +55,49 @@ struct TopkShared {
 __device__ __forceinline__ unsigned key_of(float x) {
   const unsigned u = __float_as_uint(x);
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float value_of(unsigned key) {
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
+// The band around the threshold key and where its members are recorded.
+struct Band {
+  RefineHead* head;
+  BandEntry* entries;
+  int cap;
+  unsigned lo, hi;
+};
+__device__ __forceinline__ Band make_band(const TopkArgs& a, long long z, unsigned tau) {
+  Band bd;
+  bd.head = a.buf.ref.head ? a.buf.ref.head + z : nullptr;
+  bd.entries = a.buf.ref.head ? a.buf.ref.band + z * a.buf.ref.cap : nullptr;
+  bd.cap = a.buf.ref.cap;
+  const float t = value_of(tau), dt = fabsf(t) * a.buf.ref.rel;
+  bd.lo = key_of(t - dt);
+  bd.hi = key_of(t + dt);
+  return bd;
+}
+__device__ __forceinline__ void band_record(const Band& bd, unsigned key, int j, bool selected) {
+  if (key < bd.lo || key > bd.hi) return;
+  const int slot = atomicAdd(&bd.head->n_band, 1);
+  if (slot < bd.cap) {
+    BandEntry e;
+    e.idx_flag = j | (selected ? (int)0x80000000u : 0);
+    e.p32 = value_of(key);
+    bd.entries[slot] = e;
+  }
+}
+// Adds this thread's count of candidates above the band to the head's total (one atomic per warp).
+__device__ __forceinline__ void band_count_sure(const Band& bd, int n) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+  if ((threadIdx.x & 31) == 0 && n > 0) atomicAdd(&bd.head->n_sure, n);
+}
+__device__ __forceinline__ void band_reset(const TopkArgs& a, long long z, int rank) {
+  if (a.buf.ref.head && rank == 0 && threadIdx.x == 0) {
+    RefineHead h = {};
+    a.buf.ref.head[z] = h;       // ordered before every use by the cluster barriers of the select
+  }
 }
 
 // Exclusive prefix sum of one int per thread over the whole CTA (thread order), plus the total.
@@ -213,7 +261,9 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_regs_
   const int tid = threadIdx.x, wid = tid >> 5;
   if (trivial_case(a, seq, Le, rank, out)) return;
 
-  const float* __restrict__ C = a.buf.C + ((long long)a.b.score_idx[seq] * a.Hkv + kvh) * a.buf.c_stride;
+  const long long z = (long long)a.b.score_idx[seq] * a.Hkv + kvh;
+  band_reset(a, z, rank);
+  const float* __restrict__ C = a.buf.C + z * a.buf.c_stride;
   const int j0 = (int)((long long)Le * rank / CL), j1 = (int)((long long)Le * (rank + 1) / CL);
   const int base = j0 + tid * MAXE;                  // first candidate of this thread
   const int nmine = max(0, min(MAXE, j1 - base));
@@ -275,17 +325,21 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_regs_
   cluster_offsets(cluster, sh, rank, need_eq, run_eq, run_out);
   int eq_left = min(max(need_eq - (run_eq + eq_before), 0), eq_t);
   int pos = run_out + block_exscan(gt_t + eq_left, sh.warp_tot, tot_sel);
+  const Band bd = make_band(a, z, tau);
+  int sure = 0;
 #pragma unroll
   for (int k = 0; k < MAXE; ++k) {
     if (k < nmine) {
-      if (keys[k] > tau) {
-        out[pos++] = a.Ls + base + k;
-      } else if (keys[k] == tau && eq_left > 0) {
-        out[pos++] = a.Ls + base + k;
-        --eq_left;
+      bool sel = keys[k] > tau;
+      if (keys[k] == tau && eq_left > 0) { sel = true; --eq_left; }
+      if (sel) out[pos++] = a.Ls + base + k;
+      if (bd.head) {
+        band_record(bd, keys[k], base + k, sel);
+        sure += keys[k] > bd.hi;
       }
     }
   }
+  if (bd.head) band_count_sure(bd, sure);
 }
 
 // ---- streaming kernel: any length and pooling width; pooled scores live in scratch ----
@@ -300,7 +354,9 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_strea
   const int tid = threadIdx.x, wid = tid >> 5;
   if (trivial_case(a, seq, Le, rank, out)) return;
 
-  const long long zoff = ((long long)a.b.score_idx[seq] * a.Hkv + kvh) * a.buf.c_stride;
+  const long long z = (long long)a.b.score_idx[seq] * a.Hkv + kvh;
+  band_reset(a, z, rank);
+  const long long zoff = z * a.buf.c_stride;
   const float* __restrict__ C = a.buf.C + zoff;
   float* __restrict__ P = a.buf.P + zoff;
   const int j0 = (int)((long long)Le * rank / CL), j1 = (int)((long long)Le * (rank + 1) / CL);
@@ -351,6 +407,8 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_strea
   int run_eq, run_out;
   cluster_offsets(cluster, sh, rank, need_eq, run_eq, run_out);
 
+  const Band bd = make_band(a, z, tau);
+  int sure = 0;
   for (int tb = j0; tb < j1; tb += NT) {             // ordered emission, 1024 candidates at a time
     const int j = tb + tid;
     const unsigned key = j < j1 ? key_of(P[j]) : 0u;
@@ -361,9 +419,14 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_strea
     const bool sel = gt || (eq && run_eq + rank_eq < need_eq);
     const int rank_sel = block_exscan(sel, sh.warp_tot, ts);
     if (sel) out[run_out + rank_sel] = a.Ls + j;
+    if (bd.head && j < j1) {
+      band_record(bd, key, j, sel);
+      sure += key > bd.hi;
+    }
     run_eq += te;
     run_out += ts;
   }
+  if (bd.head) band_count_sure(bd, sure);
 }
 
 }  // namespace
