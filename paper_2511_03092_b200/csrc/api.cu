@@ -114,7 +114,7 @@ struct ChunkPlan {
   // double-precision refinement of the selection near the threshold (cap == 0: none)
   int ref_cap, ref_chunks;
   float ref_rel;
-  size_t ref_band_off, ref_part_off, ref_mu_off, ref_head_off;
+  size_t ref_band_off, ref_part_off, ref_mu_off, ref_lists_off, ref_head_off;
 };
 
 // Band of the refinement: wide (1e-4 relative, up to 512 members) where re-scoring a member is cheap,
@@ -170,6 +170,7 @@ ChunkPlan plan_chunk(int dtype, const Shape& s, const int32_t* cu, int first, in
     p.ref_band_off = off; off += align_up(nz * p.ref_cap * sizeof(BandEntry));
     p.ref_part_off = off; off += align_up(nz * p.ref_cap * p.ref_chunks * s.w * sizeof(double));
     p.ref_mu_off = off;   off += align_up(nz * R * sizeof(double));
+    p.ref_lists_off = off; off += align_up(nz * 2 * p.ref_cap * sizeof(int));
     p.ref_head_off = off; off += align_up(nz * sizeof(RefineHead));
   }
   p.bytes = off;
@@ -478,6 +479,7 @@ int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* 
         buf.ref.band = reinterpret_cast<BandEntry*>(chunk_ws + p.ref_band_off);
         buf.ref.part = reinterpret_cast<double*>(chunk_ws + p.ref_part_off);
         buf.ref.mu64 = row_mu_dev ? nullptr : reinterpret_cast<double*>(chunk_ws + p.ref_mu_off);
+        buf.ref.lists = reinterpret_cast<int*>(chunk_ws + p.ref_lists_off);
         buf.ref.cap = p.ref_cap; buf.ref.chunks = p.ref_chunks; buf.ref.rel = p.ref_rel;
         buf.ref.stats_natural = !use_umma(cfg->dtype, s) && !use_umma_wide(cfg->dtype, s) && !use_mma(cfg->dtype, s);
       }
@@ -490,11 +492,10 @@ int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* 
       if (e != cudaSuccess) return SNAP_ERR_CUDA;
     }
     if (launch_pool_topk(s, b, buf, idx, status_dev, st) != cudaSuccess) return SNAP_ERR_CUDA;
-    if (launch_gather(cfg->dtype, s, b, src, idx, k_cache_dev, v_cache_dev, seq_len_dev,
-                      valid_topk_dev, status_dev, st) != cudaSuccess)
+    if (launch_topk_refine(cfg->dtype, s, b, q_obs_dev, src, buf, status_dev, sm_count(), st) != cudaSuccess)
       return SNAP_ERR_CUDA;
-    if (launch_topk_refine(cfg->dtype, s, b, q_obs_dev, src, buf, idx, k_cache_dev, v_cache_dev, status_dev, sm_count(),
-                           st) != cudaSuccess)
+    if (launch_gather(cfg->dtype, s, b, src, idx, k_cache_dev, v_cache_dev, seq_len_dev,
+                      valid_topk_dev, status_dev, st, &buf) != cudaSuccess)
       return SNAP_ERR_CUDA;
   }
   return SNAP_OK;

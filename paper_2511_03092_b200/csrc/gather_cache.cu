@@ -8,6 +8,8 @@
 //   s >= Lsr                -> idx[s - Lsr] for the first valid_topk entries
 // and rows with no source are zero-filled, so a slot is fully rewritten by one launch.
 // Rows move as 16-byte vectors; a row's vectors are read and written by adjacent threads.
+#include <cstring>
+
 #include "snap_internal.cuh"
 
 namespace snap {
@@ -23,9 +25,12 @@ struct GatherArgs {
   int k_row_b, v_row_b;
   int Hkv, Ls, Lr, K, Sc, max_seqs;
   SeqBatch b;
-  const int* idx;
+  int* idx;
   int* seq_len; int* valid_topk;
   uint32_t* status;
+  // the verdict of the double-precision re-scoring of the selection (head == NULL: there was none)
+  RefineBuffers ref;
+  float* P; int c_stride;                              // pooled-score scratch, free by now: holds the old index list
 };
 
 __device__ __forceinline__ int source_position(int s, int L, int Ls, int Lr, int vt,
@@ -70,15 +75,64 @@ __device__ __forceinline__ void copy_rows(const char* __restrict__ src_base, lon
   }
 }
 
-__global__ void __launch_bounds__(NT) gather_kernel(const GatherArgs a) {
-  pdl_wait();
-  // the refinement of the selection (launched next) may start now: it reads only what the selection
-  // kernel wrote, and waits for this grid itself before it corrects anything
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+// The re-scoring found that n positions leave the selection of a (prompt, KV head) and n others
+// enter it.  Run by the last CTA of the head, after every CTA of the head has finished copying:
+// rewrite the ascending index list and copy again the cache rows of the ranks whose position changed.
+struct CorrectionArgs {
+  const int* leaving; const int* entering;   // candidate indices (position - Ls), n of each
+  int* out; int* old;                        // the head's index list, and scratch for its previous content
+  const char* ksrc; const char* vsrc; char* kdst; char* vdst;   // this head's prompt rows and cache rows (v: NULL if aliased)
+  long long k_tok_b, v_tok_b;
+  int k_row_b, v_row_b, n, K, Ls, Lsr;
+};
+__device__ __noinline__ void apply_selection_correction(const CorrectionArgs c) {
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  for (int i = tid; i < c.K; i += NT) c.old[i] = c.out[i];
+  __syncthreads();
+  auto shift_of = [&](int j) {                               // entering below j minus leaving below j
+    int sft = 0;
+    for (int u = 0; u < c.n; ++u) sft += (c.entering[u] < j) - (c.leaving[u] < j);
+    return sft;
+  };
+  for (int i = tid; i < c.K; i += NT) {
+    const int j = c.old[i] - c.Ls;
+    bool leaves = false;
+    for (int u = 0; u < c.n; ++u) leaves |= c.leaving[u] == j;
+    if (!leaves) c.out[i + shift_of(j)] = c.old[i];
+  }
+  for (int u = tid; u < c.n; u += NT) {
+    const int j = c.entering[u], pos_abs = c.Ls + j;
+    int lo = 0, hi = c.K;                                    // entries of the old list below this one
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (c.old[mid] < pos_abs) lo = mid + 1; else hi = mid;
+    }
+    c.out[lo + shift_of(j)] = pos_abs;
+  }
+  __syncthreads();
+  for (int i = wid; i < c.K; i += NT / 32) {                 // a warp per changed row
+    const int pos = c.out[i];
+    if (pos == c.old[i]) continue;
+    const uint4* s4 = reinterpret_cast<const uint4*>(c.ksrc + (long long)pos * c.k_tok_b);
+    uint4* d4 = reinterpret_cast<uint4*>(c.kdst + (long long)(c.Lsr + i) * c.k_row_b);
+    for (int v = lane; v < c.k_row_b / 16; v += 32) d4[v] = s4[v];
+    if (c.vdst) {
+      s4 = reinterpret_cast<const uint4*>(c.vsrc + (long long)pos * c.v_tok_b);
+      d4 = reinterpret_cast<uint4*>(c.vdst + (long long)(c.Lsr + i) * c.v_row_b);
+      for (int v = lane; v < c.v_row_b / 16; v += 32) d4[v] = s4[v];
+    }
+  }
+}
+
+__global__ void __launch_bounds__(NT, 6) gather_kernel(const GatherArgs a) {
+  // With a re-scoring kernel in front, this grid was released by that kernel after its own wait:
+  // the selection kernel's index list is complete, and the re-scoring's verdict is read at the end.
+  if (!a.ref.head) pdl_wait();
   const int seq = blockIdx.z, kvh = blockIdx.y;
   const int L = a.b.len[seq], slot = a.b.slot[seq];
   if (slot < 0 || slot >= a.max_seqs) {
     if (threadIdx.x == 0 && a.status) atomicOr(a.status, SNAP_DEV_BAD_SLOT);
+    if (a.ref.head) pdl_wait();                              // this grid must not finish before the one in front of it
     return;
   }
   const int Lsr = a.Ls + a.Lr;
@@ -96,6 +150,35 @@ __global__ void __launch_bounds__(NT) gather_kernel(const GatherArgs a) {
   if (blockIdx.x == 0 && kvh == 0 && threadIdx.x == 0) {
     a.seq_len[slot] = L;
     a.valid_topk[slot] = vt;
+  }
+  if (!a.ref.head) return;
+  pdl_wait();                                                // the re-scoring kernel has finished
+  const int si = a.b.score_idx[seq];
+  if (si < 0) return;
+  const long long z = (long long)si * a.Hkv + kvh;
+  RefineHead* head = a.ref.head + z;
+  const int n = head->changed;
+  if (n <= 0) return;                                        // the single-precision order stands (the usual case)
+  __shared__ int last_s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    last_s = atomicAdd(&head->gather_done, 1) == (int)gridDim.x - 1;
+    __threadfence();
+  }
+  __syncthreads();
+  if (last_s) {
+    CorrectionArgs c;
+    c.leaving = a.ref.lists + z * 2 * a.ref.cap; c.entering = c.leaving + a.ref.cap;
+    c.out = a.idx + ((long long)(a.b.first_seq + seq) * a.Hkv + kvh) * a.K;
+    c.old = reinterpret_cast<int*>(a.P + z * a.c_stride);
+    c.ksrc = a.k + tok0 * a.k_tok_b + kvh * a.k_head_b;
+    c.kdst = a.kc + slot * a.kc_seq_b + kvh * a.kc_head_b;
+    c.vsrc = a.vc ? a.v + tok0 * a.v_tok_b + kvh * a.v_head_b : nullptr;
+    c.vdst = a.vc ? a.vc + slot * a.vc_seq_b + kvh * a.vc_head_b : nullptr;
+    c.k_tok_b = a.k_tok_b; c.v_tok_b = a.v_tok_b; c.k_row_b = a.k_row_b; c.v_row_b = a.v_row_b;
+    c.n = n; c.K = a.K; c.Ls = a.Ls; c.Lsr = Lsr;
+    apply_selection_correction(c);
   }
 }
 
@@ -137,8 +220,8 @@ inline int elt_bytes(int dtype) { return dtype == SNAP_F32 ? 4 : 2; }
 }  // namespace
 
 cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KVSource& src,
-                          const int* idx, void* k_cache, void* v_cache, int* seq_len,
-                          int* valid_topk, uint32_t* status, cudaStream_t st) {
+                          int* idx, void* k_cache, void* v_cache, int* seq_len,
+                          int* valid_topk, uint32_t* status, cudaStream_t st, const ScoreBuffers* buf) {
   if (b.n == 0) return cudaSuccess;
   const int eb = elt_bytes(dtype);
   GatherArgs a;
@@ -153,6 +236,9 @@ cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KV
   a.Hkv = s.Hkv; a.Ls = s.Ls; a.Lr = s.Lr; a.K = s.K; a.Sc = s.Sc; a.max_seqs = s.max_seqs;
   a.b = b; a.idx = s.K > 0 ? idx : nullptr;
   a.seq_len = seq_len; a.valid_topk = valid_topk; a.status = status;
+  std::memset(&a.ref, 0, sizeof(a.ref));
+  a.P = nullptr; a.c_stride = 0;
+  if (buf && buf->ref.head && b.n_scored > 0 && s.K > 0) { a.ref = buf->ref; a.P = buf->P; a.c_stride = buf->c_stride; }
   dim3 grid((s.Sc + ROWS - 1) / ROWS, s.Hkv, b.n);
   const cudaError_t e = launch_pdl(gather_kernel, grid, dim3(NT), 0, st, a);
   count_launch();

@@ -45,9 +45,10 @@ struct RefineHead {       // one per (scored prompt, KV head); zeroed by the sel
   int n_band;             // band members found (may exceed cap: then nothing is refined)
   int n_sure;             // candidates above the band: selected whatever the band's order
   int done;               // refinement CTAs of this head that have finished
-  int changed;            // out: index pairs exchanged by the refinement
+  int changed;            // out: positions that leave the selection (as many enter it)
   float max_dev;          // out: largest |single / double - 1| over the band's pooled scores
-  int pad[3];
+  int gather_done;        // gather CTAs of this head that have finished (counted only when changed > 0)
+  int pad[2];
 };
 struct BandEntry { int idx_flag; float p32; };   // candidate index | (selected in single precision) << 31
 struct RefineBuffers {
@@ -55,6 +56,7 @@ struct RefineBuffers {
   BandEntry* band;        // [nz][cap]
   double* part;           // [nz][cap][chunks][w] column sums of Eq. 1 per block of 256 window rows
   double* mu64;           // [nz][R] Eq. 4 normalisers (log2 domain) as the statistics merge computed them
+  int* lists;             // [nz][2][cap] candidate indices leaving / entering the selection (first `changed` of each)
   int cap, chunks;
   float rel;
   int stats_natural;      // 1: `stats` holds (m, 1/l) of natural-base exponentials (SIMT path)
@@ -150,14 +152,14 @@ cudaError_t launch_prefill_generic(int dtype, const Shape& s, const SeqBatch& b,
                                    void* out, float* mu, cudaStream_t st);
 cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffers& buf,
                              int* idx_out, uint32_t* status, cudaStream_t st);
-// double-precision re-scoring of the near-threshold band; corrects idx_out and the cache rows (runs after the gather)
+// double-precision re-scoring of the near-threshold band (between the selection and the gather, which applies its verdict)
 int refine_row_chunks(const Shape& s);
 cudaError_t launch_topk_refine(int dtype, const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
-                               const ScoreBuffers& buf, int* idx_out, void* k_cache, void* v_cache, uint32_t* status,
-                               int sm_count, cudaStream_t st);
+                               const ScoreBuffers& buf, uint32_t* status, int sm_count, cudaStream_t st);
+// `buf` non-NULL with buf->ref.head set: the refinement kernel was launched just before this one
 cudaError_t launch_gather(int dtype, const Shape& s, const SeqBatch& b, const KVSource& src,
-                          const int* idx, void* k_cache, void* v_cache, int* seq_len,
-                          int* valid_topk, uint32_t* status, cudaStream_t st);
+                          int* idx, void* k_cache, void* v_cache, int* seq_len,
+                          int* valid_topk, uint32_t* status, cudaStream_t st, const ScoreBuffers* buf = nullptr);
 cudaError_t launch_append(int dtype, const Shape& s, const void* k_new, const void* v_new,
                           const int* slot_ids, int n_active, void* k_cache, void* v_cache,
                           int* seq_len, uint32_t* status, cudaStream_t st);

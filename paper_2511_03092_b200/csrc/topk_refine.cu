@@ -15,20 +15,20 @@
 // with mu_i the log2-domain normaliser of Eq. 4 from the first score pass (its value as the
 // statistics merge computed it in double where that is available).  The K - n_sure best band
 // members by (P descending, index ascending) are the selected ones.  Where that differs from
-// the single-precision choice, the emitted ascending index list is rewritten and the cache rows
-// of the ranks that changed are copied again.
+// the single-precision choice, the positions that leave and enter the selection are handed to
+// the gather kernel, which rewrites the index list and copies the affected cache rows again.
 //
-// The kernel runs after the gather kernel, which lets it start early: the re-scoring overlaps
-// the gather, and only a correction (rare) waits for the gather to finish.
+// The kernel runs between the selection and the gather kernel and releases the gather at once
+// (the gather copies with the single-precision list and looks at the verdict when it is done),
+// so the re-scoring overlaps the gather.
 //
 // Work split: one item = one band member x one block of 64 window rows.  The dot products are a
 // small double-precision matrix product -- 64 rows x d columns against the member's w key rows
 // (taps) -- on the FP64 tensor-core instruction mma.m8n8k4: a warp owns 8 rows, the taps are
 // the 8 columns of the product; queries and keys are converted to double on their way into
 // shared memory.  CTAs of a head stride over its items; per-item column sums go to scratch and
-// the last CTA of the head to finish (a counter, no waiting) adds them in a fixed order, ranks
-// the band and applies the correction, so the result does not depend on the order in which
-// CTAs ran.  A band larger than its buffer is left in single-precision order and
+// the last CTA of the head to finish (a counter, no waiting) adds them in a fixed order and
+// ranks the band, so the result does not depend on the order in which CTAs ran.  A band larger than its buffer is left in single-precision order and
 // SNAP_DEV_BAND_OVERFLOW is raised.
 #include "snap_internal.cuh"
 
@@ -38,32 +38,30 @@ namespace {
 constexpr int NT = 256;      // threads per CTA
 constexpr int RB = 64;       // window rows per item (8 per warp)
 constexpr int TG = 8;        // taps per pass = columns of the m8n8k4 product
-constexpr int QTILE_B = 76 * 1024;   // shared memory for the staged query rows
+constexpr int QTILE_B = 76 * 1024;   // shared memory for the staged query rows (two CTAs per SM with the key rows beside it)
 constexpr int MAXCAP = 512;  // band members the ranking step holds in shared memory
 
 struct RefineArgs {
   const void* q;            // [prompts][Hq][Lo][d]
   KVSource src;             // prompt keys / values (strides in elements)
-  int Hq, Hkv, g, Lo, d, d_v, Ls, Lr, K, Sc, w, pool_mode, R, max_seqs, elt;
+  int Hq, Hkv, g, Lo, d, Ls, Lr, K, w, pool_mode, R, elt;
   int dc;                   // query columns staged at a time (a multiple of 16)
   double scale_log2;
   SeqBatch b;
   ScoreBuffers buf;
-  int* idx_out;             // [prompts][Hkv][K]
-  char* kc; char* vc;       // caches (vc NULL when V aliases K)
   uint32_t* status;
 };
 
-// two consecutive elements -> two doubles
+// two consecutive elements -> two floats (exact for both element types)
 template <typename T> struct Pair;
 template <> struct Pair<float> {
   using raw = float2;
-  static __device__ __forceinline__ double2 cvt(float2 v) { return make_double2((double)v.x, (double)v.y); }
+  static __device__ __forceinline__ float2 to_f32(float2 v) { return v; }
 };
 template <> struct Pair<__nv_bfloat16> {
   using raw = uint32_t;
-  static __device__ __forceinline__ double2 cvt(uint32_t v) {
-    return make_double2((double)__uint_as_float(v << 16), (double)__uint_as_float(v & 0xffff0000u));
+  static __device__ __forceinline__ float2 to_f32(uint32_t v) {
+    return make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
   }
 };
 __device__ __forceinline__ double elem_f64(const float* p) { return (double)*p; }
@@ -78,9 +76,9 @@ __device__ __forceinline__ void dmma(double& c0, double& c1, double a, double b)
 
 template <typename T>
 __global__ void __launch_bounds__(NT, 2) topk_refine_kernel(const RefineArgs a) {
-  // No wait here: this grid is released by the gather kernel after that kernel's own wait, so
-  // everything the selection kernel wrote (band, counters, index list) is complete and visible.
-  extern __shared__ __align__(16) double smem_d[];          // [TG][d + 4] key rows as doubles, then [RB] query rows as loaded
+  pdl_wait();                                               // the selection kernel has written band and counters
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the gather may start: it needs nothing from here yet
+  extern __shared__ __align__(16) float smem_f[];           // [TG][d + 4] key rows as floats (exact), then [RB] query rows as loaded
   __shared__ double red[NT / 32][TG];
   __shared__ double p64[MAXCAP];
   __shared__ int jidx[MAXCAP];                              // candidate index of each band member
@@ -101,8 +99,8 @@ __global__ void __launch_bounds__(NT, 2) topk_refine_kernel(const RefineArgs a) 
   const bool overflow = nb_raw > rf.cap || nb_raw > MAXCAP;
   const int nb = overflow ? 0 : nb_raw;
   const int chunks = rf.chunks, r = a.w / 2, d = a.d, KS = d + 4;
-  double* ksd = smem_d;
-  char* qt = reinterpret_cast<char*>(smem_d + TG * KS);
+  float* ksf = smem_f;
+  char* qt = reinterpret_cast<char*>(smem_f + TG * KS);
   const int q_pitch = a.dc * (int)sizeof(T) + 16;             // bytes per staged row: 4 words mod 8, conflict-free fragment loads
   double* part = rf.part + (long long)z * rf.cap * chunks * a.w;
 
@@ -111,8 +109,13 @@ __global__ void __launch_bounds__(NT, 2) topk_refine_kernel(const RefineArgs a) 
                    (long long)kvh * a.src.k_head_stride;
   const int frow = lane >> 2, fk = lane & 3;                 // fragment coordinates of m8n8k4
 
-  for (int item = blockIdx.x; item < nb * chunks; item += gridDim.x) {
-    const int m = item / chunks, c = item % chunks;
+  // A CTA takes a contiguous run of items, ordered row block first: while the row block stays the
+  // same (and a whole row fits the tile) the staged query rows are reused from member to member.
+  const int n_items = nb * chunks, per_cta = (n_items + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int item_end = min(n_items, ((int)blockIdx.x + 1) * per_cta);
+  int staged_chunk = -1;
+  for (int item = blockIdx.x * per_cta; item < item_end; ++item) {
+    const int c = item / nb, m = item - c * nb;
     const int j = band[m].idx_flag & 0x7fffffff;
     const int row0 = c * RB, row = row0 + wid * 8 + frow;    // this item's first window row; this lane's row
     double mu = 0.0;
@@ -144,14 +147,15 @@ __global__ void __launch_bounds__(NT, 2) topk_refine_kernel(const RefineArgs a) 
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u)
-          if (dst[u] >= 0) *reinterpret_cast<double2*>(ksd + dst[u]) = Pair<T>::cvt(v[u]);
+          if (dst[u] >= 0) *reinterpret_cast<float2*>(ksf + dst[u]) = Pair<T>::to_f32(v[u]);
       }
       double c0 = 0.0, c1 = 0.0, e0 = 0.0, e1 = 0.0;         // two accumulation chains
       for (int cb = 0; cb < d; cb += a.dc) {
         if (cb) __syncthreads();
         const int ncol = min(a.dc, d - cb);
         const int vpr = ncol * (int)sizeof(T) / 16;          // 16-byte vectors per row: copied as they are
-        for (int base = 0; base < RB * vpr; base += 4 * NT) {
+        const bool restage = a.dc < d || staged_chunk != c;
+        for (int base = 0; restage && base < RB * vpr; base += 4 * NT) {
           uint4 v[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -166,13 +170,14 @@ __global__ void __launch_bounds__(NT, 2) topk_refine_kernel(const RefineArgs a) 
             if (e < RB * vpr) *reinterpret_cast<uint4*>(qt + rr * q_pitch + vc * 16) = v[u];
           }
         }
+        staged_chunk = c;
         __syncthreads();
         const T* qa = reinterpret_cast<const T*>(qt + (wid * 8 + frow) * q_pitch) + fk;   // A fragment: row = lane / 4, column = lane % 4
-        const double* kb = ksd + frow * KS + cb + fk;                                  // B fragment: tap = lane / 4, column = lane % 4
+        const float* kb = ksf + frow * KS + cb + fk;                                   // B fragment: tap = lane / 4, column = lane % 4
 #pragma unroll 2
         for (int k0 = 0; k0 < ncol; k0 += 8) {               // ncol is a multiple of 16
-          dmma(c0, c1, elem_f64(qa + k0), kb[k0]);
-          dmma(e0, e1, elem_f64(qa + k0 + 4), kb[k0 + 4]);
+          dmma(c0, c1, elem_f64(qa + k0), (double)kb[k0]);
+          dmma(e0, e1, elem_f64(qa + k0 + 4), (double)kb[k0 + 4]);
         }
       }
       c0 += e0; c1 += e1;
@@ -204,14 +209,13 @@ __global__ void __launch_bounds__(NT, 2) topk_refine_kernel(const RefineArgs a) 
     __threadfence();
   }
   __syncthreads();
-  if (!last_s) { pdl_wait(); return; }                       // this grid must not complete before the gather has
+  if (!last_s) return;
   if (overflow) {
     if (tid == 0 && a.status) atomicOr(a.status, SNAP_DEV_BAND_OVERFLOW);
-    pdl_wait();
     return;
   }
   const int n_sel = a.K - head->n_sure;                      // band members that belong to the selection
-  if (nb == 0 || n_sel < 0 || n_sel > nb) { pdl_wait(); return; }   // nothing recorded (or inconsistent): keep the order
+  if (nb == 0 || n_sel < 0 || n_sel > nb) return;            // nothing recorded (or inconsistent): keep the order
   const bool avg = a.pool_mode == SNAP_POOL_AVG;
   float dev = 0.f;
   for (int m = tid; m < nb; m += NT) {
@@ -248,60 +252,18 @@ __global__ void __launch_bounds__(NT, 2) topk_refine_kernel(const RefineArgs a) 
   __syncthreads();
   for (int m = tid; m < nb; m += NT) part[(long long)m * chunks * a.w] = p64[m];   // left in scratch for diagnosis
   const int n_out = n_list[0], n_in = n_list[1];
+  // the verdict for the gather kernel: how many positions change places, and which
+  const bool ok = n_in == n_out;
+  int* glists = rf.lists + (long long)z * 2 * rf.cap;
+  for (int u = tid; u < (ok ? n_in : 0); u += NT) {
+    glists[u] = lists[0][u];
+    glists[rf.cap + u] = lists[1][u];
+  }
   if (tid == 0) {
     float dmax = 0.f;
     for (int w2 = 0; w2 < NT / 32; ++w2) dmax = fmaxf(dmax, dev_s[w2]);
     head->max_dev = dmax;
-    head->changed = n_in;
-  }
-  pdl_wait();                                                // the gather kernel has read the index list and written the cache
-  if (n_in == 0 || n_in != n_out) return;
-
-  // ---- rewrite the ascending index list: drop lists[0], insert lists[1] ----
-  int* out = a.idx_out + ((long long)(a.b.first_seq + seq) * a.Hkv + kvh) * a.K;
-  int* tmp = reinterpret_cast<int*>(a.buf.P + (long long)z * a.buf.c_stride);   // the pooled-score scratch is free by now
-  for (int i = tid; i < a.K; i += NT) tmp[i] = out[i];
-  __syncthreads();
-  auto shift_of = [&](int j) {                               // entering below j minus leaving below j
-    int sft = 0;
-    for (int u = 0; u < n_in; ++u) sft += (lists[1][u] < j) - (lists[0][u] < j);
-    return sft;
-  };
-  for (int i = tid; i < a.K; i += NT) {
-    const int j = tmp[i] - a.Ls;
-    bool leaving = false;
-    for (int u = 0; u < n_out; ++u) leaving |= lists[0][u] == j;
-    if (!leaving) out[i + shift_of(j)] = tmp[i];
-  }
-  for (int u = tid; u < n_in; u += NT) {
-    const int j = lists[1][u], pos_abs = a.Ls + j;
-    int lo = 0, hi = a.K;                                    // entries of the old list below this one
-    while (lo < hi) {
-      const int mid = (lo + hi) >> 1;
-      if (tmp[mid] < pos_abs) lo = mid + 1; else hi = mid;
-    }
-    out[lo + shift_of(j)] = pos_abs;
-  }
-  __syncthreads();
-  // ---- copy again the cache rows of the ranks whose position changed (a warp per row) ----
-  const int slot = a.b.slot[seq];
-  if (slot < 0 || slot >= a.max_seqs) return;                // reported by the gather kernel
-  const long long k_row_b = (long long)d * a.elt, v_row_b = (long long)a.d_v * a.elt;
-  char* kdst = a.kc + ((long long)slot * a.Hkv + kvh) * a.Sc * k_row_b;
-  char* vdst = a.vc ? a.vc + ((long long)slot * a.Hkv + kvh) * a.Sc * v_row_b : nullptr;
-  const char* ksrc = static_cast<const char*>(a.src.k) + ((long long)a.b.tok_off[seq] * a.src.k_tok_stride + (long long)kvh * a.src.k_head_stride) * a.elt;
-  const char* vsrc = a.vc ? static_cast<const char*>(a.src.v) + ((long long)a.b.tok_off[seq] * a.src.v_tok_stride + (long long)kvh * a.src.v_head_stride) * a.elt : nullptr;
-  for (int i = wid; i < a.K; i += NT / 32) {
-    const int pos = out[i];
-    if (pos == tmp[i]) continue;
-    const uint4* s4 = reinterpret_cast<const uint4*>(ksrc + (long long)pos * a.src.k_tok_stride * a.elt);
-    uint4* d4 = reinterpret_cast<uint4*>(kdst + (long long)(a.Ls + a.Lr + i) * k_row_b);
-    for (int v = lane; v < k_row_b / 16; v += 32) d4[v] = s4[v];
-    if (vdst) {
-      s4 = reinterpret_cast<const uint4*>(vsrc + (long long)pos * a.src.v_tok_stride * a.elt);
-      d4 = reinterpret_cast<uint4*>(vdst + (long long)(a.Ls + a.Lr + i) * v_row_b);
-      for (int v = lane; v < v_row_b / 16; v += 32) d4[v] = s4[v];
-    }
+    head->changed = ok ? n_in : 0;
   }
 }
 
@@ -310,25 +272,22 @@ __global__ void __launch_bounds__(NT, 2) topk_refine_kernel(const RefineArgs a) 
 int refine_row_chunks(const Shape& s) { return (s.g * s.Lo + RB - 1) / RB; }
 
 cudaError_t launch_topk_refine(int dtype, const Shape& s, const SeqBatch& b, const void* q_obs, const KVSource& src,
-                               const ScoreBuffers& buf, int* idx_out, void* k_cache, void* v_cache, uint32_t* status,
-                               int sm_count, cudaStream_t st) {
+                               const ScoreBuffers& buf, uint32_t* status, int sm_count, cudaStream_t st) {
   if (!buf.ref.head || b.n_scored == 0 || s.K == 0) return cudaSuccess;
   RefineArgs a;
   a.q = q_obs; a.src = src;
-  a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Lo = s.Lo; a.d = s.d_qk; a.d_v = s.d_v; a.Ls = s.Ls; a.Lr = s.Lr; a.K = s.K;
-  a.Sc = s.Sc; a.w = s.w; a.pool_mode = s.pool_mode; a.R = s.g * s.Lo; a.max_seqs = s.max_seqs;
+  a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Lo = s.Lo; a.d = s.d_qk; a.Ls = s.Ls; a.Lr = s.Lr; a.K = s.K;
+  a.w = s.w; a.pool_mode = s.pool_mode; a.R = s.g * s.Lo;
   a.elt = dtype == SNAP_F32 ? 4 : 2;
   a.scale_log2 = (double)s.scale * 1.4426950408889634074;
-  a.b = b; a.buf = buf; a.idx_out = idx_out; a.status = status;
-  a.kc = static_cast<char*>(k_cache);
-  a.vc = s.v_aliases_k ? nullptr : static_cast<char*>(v_cache);
+  a.b = b; a.buf = buf; a.status = status;
   const int nz = b.n_scored * s.Hkv;
-  int gx = (3 * sm_count + nz - 1) / nz;                     // CTAs per head; they stride over the head's items
+  int gx = (2 * sm_count + nz - 1) / nz;                     // CTAs per head (two per SM in all); each takes a run of the head's items
   gx = gx < 1 ? 1 : gx > 1024 ? 1024 : gx;
   // columns staged at a time: the whole row when 64 rows of it fit the tile, else the largest multiple of 16 that does
   const int max_cols = (QTILE_B / RB - 16) / a.elt / 16 * 16;
   a.dc = s.d_qk < max_cols ? s.d_qk : max_cols;
-  const size_t smem = (size_t)TG * (s.d_qk + 4) * sizeof(double) + (size_t)RB * (a.dc * a.elt + 16);
+  const size_t smem = (size_t)TG * (s.d_qk + 4) * sizeof(float) + (size_t)RB * (a.dc * a.elt + 16);
   static SmemLimit lim_f = {}, lim_b = {};
   cudaError_t e;
   if (dtype == SNAP_F32) {
