@@ -205,3 +205,61 @@ def test_paper_hyperparameter_rows(row):
         lengths, steps = [36000], 3
     assert wl.slots in (8192, 32768)
     _run(wl, lengths, seed=500, steps=steps)
+
+
+def test_head_sharded_compress_reassembles_to_the_full_head_result():
+    """The library's side of a head-sharded deployment (compression with the KV heads spread over
+    ranks, decode with whole sequences per rank): each shard calls snap_compress with its share of
+    the heads -- n_kv_heads and n_q_heads of the shard, q_obs of its query heads, K/V pointers
+    offset to its first head with the strides of the full tensors -- into a cache of its own.
+    Both shards run here on one device, one after the other; their caches, concatenated along the
+    head axis (what the hand-off's all-to-all delivers to a decode rank), must equal byte for byte
+    the cache of one full-head call, the oracle's image, and decode like it."""
+    from paper_2511_03092_b200 import binding as B
+    wl = synth.CONFIGS[1]
+    lengths = [9000, 20000 + 3]
+    n, shards = len(lengths), 2
+    prompts = [synth.make_prompt(wl, L, 900 + i) for i, L in enumerate(lengths)]
+    full = H.GpuLayer(wl, max_seqs=n)
+    idx_full = full.compress(prompts, list(range(n)))
+    assert full.status() == 0
+    hk, g = wl.n_kv_heads // shards, wl.n_q_heads // wl.n_kv_heads
+    wl_shard = wl.scaled(n_kv_heads=hk, n_q_heads=hk * g)
+    cu = [0, lengths[0], lengths[0] + lengths[1]]
+    k_all = torch.cat([p["k"] for p in prompts]).cuda()                     # [T, Hkv, d]: the full tensors
+    v_all = torch.cat([p["v"] for p in prompts]).cuda()
+    q_all = torch.stack([p["q_obs"] for p in prompts]).cuda()               # [n, Hq, Lo, d]
+    parts_k, parts_v, parts_idx = [], [], []
+    for r in range(shards):
+        layer = H.GpuLayer(wl_shard, max_seqs=n)
+        c = layer.cache
+        ws = torch.empty(B.snap_compress_workspace_bytes(layer.cfg, cu), dtype=torch.uint8, device="cuda")
+        idx = torch.full((n, hk, wl.topk), -7, dtype=torch.int32, device="cuda")
+        q_r = q_all[:, r * hk * g:(r + 1) * hk * g].contiguous()
+        k_r, v_r = k_all[:, r * hk:(r + 1) * hk], v_all[:, r * hk:(r + 1) * hk]   # views: offset pointer, full strides
+        assert k_r.stride(0) == wl.n_kv_heads * wl.d_qk and not k_r.is_contiguous()
+        B.snap_compress(layer.cfg, layer.layout, q_r, k_r, v_r, cu, list(range(n)), c.k_cache, c.v_cache, c.seq_len,
+                        c.valid_topk, idx, ws, c.status)
+        assert layer.status() == 0
+        assert torch.equal(c.seq_len, full.cache.seq_len) and torch.equal(c.valid_topk, full.cache.valid_topk)
+        parts_k.append(c.k_cache); parts_v.append(c.v_cache); parts_idx.append(idx)
+    k_cat, v_cat = torch.cat(parts_k, dim=1), torch.cat(parts_v, dim=1)
+    assert torch.equal(k_cat, full.cache.k_cache) and torch.equal(v_cat, full.cache.v_cache)
+    assert np.array_equal(torch.cat(parts_idx, dim=1).cpu().numpy(), idx_full)
+    # the reassembled cache in a decode layer of its own, against the oracle
+    dec = H.GpuLayer(wl, max_seqs=n)
+    dec.cache.k_cache.copy_(k_cat); dec.cache.v_cache.copy_(v_cat)
+    dec.cache.seq_len.copy_(full.cache.seq_len); dec.cache.valid_topk.copy_(full.cache.valid_topk)
+    seqs = [H.oracle_compress(wl, p) for p in prompts]
+    for i, seq in enumerate(seqs):
+        H.check_selection(idx_full[i], seq, wl)
+        seq.topk_pos = [idx_full[i][h].astype(np.int64) for h in range(wl.n_kv_heads)]
+        H.check_cache_image(dec, seq, i, wl)
+    slots_dev = torch.arange(n, dtype=torch.int32, device="cuda")
+    for step in range(2):
+        d = synth.make_decode_inputs(wl, n, 900, step)
+        out = dec.decode(d["q"].cuda(), d["k_new"].cuda(), d["v_new"].cuda(), slots_dev)
+        for i, seq in enumerate(seqs):
+            ref = orc.decode_step(seq, synth.to_f64(d["q"][i]), synth.to_f64(d["k_new"][i]), synth.to_f64(d["v_new"][i]))
+            H.check_output(out[i], ref, wl, f"seq {i} step {step}")
+    assert dec.status() == 0
