@@ -75,6 +75,11 @@ typedef enum snap_status {
                                        valid; exactly tied scores, which go to the lower position in
                                        either precision, are the usual cause */
 
+#define SNAP_DEV_INDEX_CHECK 8u     /* only from the checked build of the library (compiled with
+                                       -DSNAP_DEBUG_BOUNDS): a data-dependent index -- a selected
+                                       position, a ring slot, an output rank, a band entry -- fell
+                                       outside its array; the access was skipped */
+
 /* One attention layer's shape and SnapStream hyper-parameters (appendix table
  * "SnapStream Hyperparameters": sink, top-K, recent, observation window, pooling kernel). */
 typedef struct snap_config {

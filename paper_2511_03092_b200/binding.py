@@ -13,11 +13,13 @@ from typing import Optional, Sequence
 
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsnapstream.so")
+# SNAP_LIBRARY names another build of the library in this directory (the checked build, libsnapstream_dbg.so)
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                         os.path.basename(os.environ.get("SNAP_LIBRARY", "libsnapstream.so")))
 
 SNAP_F32, SNAP_BF16 = 0, 1
 SNAP_POOL_AVG, SNAP_POOL_MAX = 0, 1
-SNAP_DEV_BAD_SLOT, SNAP_DEV_WAIT_TIMEOUT, SNAP_DEV_BAND_OVERFLOW = 1, 2, 4
+SNAP_DEV_BAD_SLOT, SNAP_DEV_WAIT_TIMEOUT, SNAP_DEV_BAND_OVERFLOW, SNAP_DEV_INDEX_CHECK = 1, 2, 4, 8
 
 
 class SnapConfig(C.Structure):

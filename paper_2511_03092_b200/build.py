@@ -1,10 +1,13 @@
 """Build libsnapstream.so (sm_100a only) in-tree with nvcc.
 
-    python -m paper_2511_03092_b200.build [--force] [--verbose]
+    python -m paper_2511_03092_b200.build [--force] [--verbose] [--debug-bounds]
 
 Each csrc/*.cu is compiled to an object under csrc/build/ (in parallel, only when its
 sources are newer) and the objects are linked into paper_2511_03092_b200/libsnapstream.so.
 nvcc cross-compiles, so this works on a machine without a GPU.
+--debug-bounds builds the checked variant instead (-DSNAP_DEBUG_BOUNDS: data-dependent indices are
+tested and a bad one raises a status bit instead of an access; objects under csrc/build_dbg/) as
+libsnapstream_dbg.so; the binding loads it when SNAP_LIBRARY names it.
 """
 from __future__ import annotations
 
@@ -37,8 +40,11 @@ def _newest(paths) -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    obj_dir = OBJ + "_dbg" if debug_bounds else OBJ
+    lib = os.path.join(PKG, "libsnapstream_dbg.so") if debug_bounds else LIB
+    extra = ["-DSNAP_DEBUG_BOUNDS"] if debug_bounds else []
+    os.makedirs(obj_dir, exist_ok=True)
     sources = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     headers = glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
     hdr_time = _newest(headers + [os.path.abspath(__file__)])
@@ -46,12 +52,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
     jobs = []
     objects = []
     for src in sources:
-        obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         objects.append(obj)
         if (not force and os.path.exists(obj)
                 and os.path.getmtime(obj) >= max(os.path.getmtime(src), hdr_time)):
             continue
-        cmd = [nvcc, *ARCH, *COMMON, "-c", src, "-o", obj]
+        cmd = [nvcc, *ARCH, *COMMON, *extra, "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         jobs.append(cmd)
@@ -67,14 +73,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
                     sys.stderr.write(" ".join(cmd) + "\n" + r.stdout + r.stderr)
                 if r.returncode != 0:
                     raise RuntimeError("nvcc failed for " + cmd[-3])
-    if jobs or force or not os.path.exists(LIB) or os.path.getmtime(LIB) < _newest(objects):
-        cmd = [nvcc, *ARCH, "-shared", "-o", LIB, *objects]
+    if jobs or force or not os.path.exists(lib) or os.path.getmtime(lib) < _newest(objects):
+        cmd = [nvcc, *ARCH, "-shared", "-o", lib, *objects]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             sys.stderr.write(r.stdout + r.stderr)
             raise RuntimeError("link failed")
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

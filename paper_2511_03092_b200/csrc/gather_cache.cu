@@ -51,7 +51,7 @@ __device__ __forceinline__ int source_position(int s, int L, int Ls, int Lr, int
 __device__ __forceinline__ void copy_rows(const char* __restrict__ src_base, long long tok_b,
                                           char* __restrict__ dst_base, int row_b, int s0, int Sc,
                                           int L, int Ls, int Lr, int vt,
-                                          const int* __restrict__ idx_row) {
+                                          const int* __restrict__ idx_row, uint32_t* status) {
   const int vecs = row_b / 16, total = ROWS * vecs;
   // four independent 16-byte loads are in flight per thread before anything is stored
   for (int base = threadIdx.x; base < total; base += 4 * NT) {
@@ -66,7 +66,7 @@ __device__ __forceinline__ void copy_rows(const char* __restrict__ src_base, lon
       val[u] = make_uint4(0u, 0u, 0u, 0u);
       if (slot_of[u] >= 0) {
         const int p = source_position(s, L, Ls, Lr, vt, idx_row);
-        if (p >= 0) val[u] = __ldg(reinterpret_cast<const uint4*>(src_base + (long long)p * tok_b) + chunk_of[u]);
+        if (p >= 0 && index_ok(p, L, status)) val[u] = __ldg(reinterpret_cast<const uint4*>(src_base + (long long)p * tok_b) + chunk_of[u]);
       }
     }
 #pragma unroll
@@ -83,7 +83,8 @@ struct CorrectionArgs {
   int* out; int* old;                        // the head's index list, and scratch for its previous content
   const char* ksrc; const char* vsrc; char* kdst; char* vdst;   // this head's prompt rows and cache rows (v: NULL if aliased)
   long long k_tok_b, v_tok_b;
-  int k_row_b, v_row_b, n, K, Ls, Lsr;
+  int k_row_b, v_row_b, n, K, Ls, Lsr, L;
+  uint32_t* status;
 };
 __device__ __noinline__ void apply_selection_correction(const CorrectionArgs c) {
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -98,7 +99,7 @@ __device__ __noinline__ void apply_selection_correction(const CorrectionArgs c) 
     const int j = c.old[i] - c.Ls;
     bool leaves = false;
     for (int u = 0; u < c.n; ++u) leaves |= c.leaving[u] == j;
-    if (!leaves) c.out[i + shift_of(j)] = c.old[i];
+    if (!leaves && index_ok(i + shift_of(j), c.K, c.status)) c.out[i + shift_of(j)] = c.old[i];
   }
   for (int u = tid; u < c.n; u += NT) {
     const int j = c.entering[u], pos_abs = c.Ls + j;
@@ -107,12 +108,12 @@ __device__ __noinline__ void apply_selection_correction(const CorrectionArgs c) 
       const int mid = (lo + hi) >> 1;
       if (c.old[mid] < pos_abs) lo = mid + 1; else hi = mid;
     }
-    c.out[lo + shift_of(j)] = pos_abs;
+    if (index_ok(lo + shift_of(j), c.K, c.status)) c.out[lo + shift_of(j)] = pos_abs;
   }
   __syncthreads();
   for (int i = wid; i < c.K; i += NT / 32) {                 // a warp per changed row
     const int pos = c.out[i];
-    if (pos == c.old[i]) continue;
+    if (pos == c.old[i] || !index_ok(pos, c.L, c.status)) continue;
     const uint4* s4 = reinterpret_cast<const uint4*>(c.ksrc + (long long)pos * c.k_tok_b);
     uint4* d4 = reinterpret_cast<uint4*>(c.kdst + (long long)(c.Lsr + i) * c.k_row_b);
     for (int v = lane; v < c.k_row_b / 16; v += 32) d4[v] = s4[v];
@@ -142,11 +143,11 @@ __global__ void __launch_bounds__(NT, 6) gather_kernel(const GatherArgs a) {
   const long long tok0 = a.b.tok_off[seq];
   copy_rows(a.k + tok0 * a.k_tok_b + kvh * a.k_head_b, a.k_tok_b,
             a.kc + slot * a.kc_seq_b + kvh * a.kc_head_b, a.k_row_b, s0, a.Sc, L, a.Ls, a.Lr, vt,
-            idx_row);
+            idx_row, a.status);
   if (a.vc)
     copy_rows(a.v + tok0 * a.v_tok_b + kvh * a.v_head_b, a.v_tok_b,
               a.vc + slot * a.vc_seq_b + kvh * a.vc_head_b, a.v_row_b, s0, a.Sc, L, a.Ls, a.Lr, vt,
-              idx_row);
+              idx_row, a.status);
   if (blockIdx.x == 0 && kvh == 0 && threadIdx.x == 0) {
     a.seq_len[slot] = L;
     a.valid_topk[slot] = vt;
@@ -177,7 +178,7 @@ __global__ void __launch_bounds__(NT, 6) gather_kernel(const GatherArgs a) {
     c.vsrc = a.vc ? a.v + tok0 * a.v_tok_b + kvh * a.v_head_b : nullptr;
     c.vdst = a.vc ? a.vc + slot * a.vc_seq_b + kvh * a.vc_head_b : nullptr;
     c.k_tok_b = a.k_tok_b; c.v_tok_b = a.v_tok_b; c.k_row_b = a.k_row_b; c.v_row_b = a.v_row_b;
-    c.n = n; c.K = a.K; c.Ls = a.Ls; c.Lsr = Lsr;
+    c.n = n; c.K = a.K; c.Ls = a.Ls; c.Lsr = Lsr; c.L = L; c.status = a.status;
     apply_selection_correction(c);
   }
 }
@@ -186,7 +187,7 @@ struct AppendArgs {
   const char* k_new; const char* v_new;
   char* kc; char* vc;
   long long kc_seq_b, kc_head_b, vc_seq_b, vc_head_b;
-  int k_row_b, v_row_b, Hkv, Ls, Lr, max_seqs, n_active;
+  int k_row_b, v_row_b, Hkv, Ls, Lr, Sc, max_seqs, n_active;
   const int* slot_ids; int* seq_len; uint32_t* status;
 };
 
@@ -201,6 +202,7 @@ __global__ void __launch_bounds__(NT) append_kernel(const AppendArgs a) {
   const int t = a.seq_len[slot];
   __syncthreads();
   const int dst = ring_slot(t, a.Ls, a.Lr);
+  if (!index_ok(dst, a.Sc, a.status) || !index_ok(t, 0x7fffffff, a.status)) return;
   const int kv = a.k_row_b / 16, vv = a.vc ? a.v_row_b / 16 : 0;
   for (int item = threadIdx.x; item < a.Hkv * (kv + vv); item += NT) {
     const int h = item / (kv + vv), c = item % (kv + vv);
@@ -257,7 +259,7 @@ cudaError_t launch_append(int dtype, const Shape& s, const void* k_new, const vo
   a.k_row_b = s.d_qk * eb; a.v_row_b = s.d_v * eb;
   a.kc_head_b = (long long)s.Sc * a.k_row_b; a.kc_seq_b = a.kc_head_b * s.Hkv;
   a.vc_head_b = (long long)s.Sc * a.v_row_b; a.vc_seq_b = a.vc_head_b * s.Hkv;
-  a.Hkv = s.Hkv; a.Ls = s.Ls; a.Lr = s.Lr; a.max_seqs = s.max_seqs; a.n_active = n_active;
+  a.Hkv = s.Hkv; a.Ls = s.Ls; a.Lr = s.Lr; a.Sc = s.Sc; a.max_seqs = s.max_seqs; a.n_active = n_active;
   a.slot_ids = slot_ids; a.seq_len = seq_len; a.status = status;
   append_kernel<<<n_active, NT, 0, st>>>(a);
   count_launch();

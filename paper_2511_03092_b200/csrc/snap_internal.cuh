@@ -210,6 +210,19 @@ cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* 
                                      int n_active, void* k_cache, int* seq_len, const int* valid_topk, void* out,
                                      float* partials, int nsplit, uint32_t* status, cudaStream_t st);
 
+// Checked indexing for the debugging build (-DSNAP_DEBUG_BOUNDS): a data-dependent index that falls
+// outside [0, n) raises SNAP_DEV_INDEX_CHECK in the status word and the access is skipped -- nothing
+// traps.  In the regular build the check compiles to `true`.
+#ifdef SNAP_DEBUG_BOUNDS
+__device__ __forceinline__ bool index_ok(long long i, long long n, uint32_t* status) {
+  if (i >= 0 && i < n) return true;
+  if (status) atomicOr(status, SNAP_DEV_INDEX_CHECK);
+  return false;
+}
+#else
+__device__ __forceinline__ bool index_ok(long long, long long, uint32_t*) { return true; }
+#endif
+
 // --- small device helpers ---
 template <typename T> __device__ __forceinline__ float to_f32(T x);
 template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }

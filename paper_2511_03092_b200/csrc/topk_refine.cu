@@ -117,6 +117,7 @@ __global__ void __launch_bounds__(NT, 2) topk_refine_kernel(const RefineArgs a) 
   for (int item = blockIdx.x * per_cta; item < item_end; ++item) {
     const int c = item / nb, m = item - c * nb;
     const int j = band[m].idx_flag & 0x7fffffff;
+    if (!index_ok(j, Le, a.status)) continue;                // uniform over the CTA
     const int row0 = c * RB, row = row0 + wid * 8 + frow;    // this item's first window row; this lane's row
     double mu = 0.0;
     if (row < a.R) {

@@ -40,6 +40,7 @@ struct TopkArgs {
   SeqBatch b;
   ScoreBuffers buf;
   int* idx_out;      // [n][Hkv][K]
+  uint32_t* status;
 };
 
 struct TopkShared {
@@ -332,7 +333,8 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_regs_
     if (k < nmine) {
       bool sel = keys[k] > tau;
       if (keys[k] == tau && eq_left > 0) { sel = true; --eq_left; }
-      if (sel) out[pos++] = a.Ls + base + k;
+      if (sel && index_ok(pos, a.K, a.status)) out[pos] = a.Ls + base + k;
+      pos += sel;
       if (bd.head) {
         band_record(bd, keys[k], base + k, sel);
         sure += keys[k] > bd.hi;
@@ -418,7 +420,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_strea
     const int rank_eq = block_exscan(eq, sh.warp_tot, te);
     const bool sel = gt || (eq && run_eq + rank_eq < need_eq);
     const int rank_sel = block_exscan(sel, sh.warp_tot, ts);
-    if (sel) out[run_out + rank_sel] = a.Ls + j;
+    if (sel && index_ok(run_out + rank_sel, a.K, a.status)) out[run_out + rank_sel] = a.Ls + j;
     if (bd.head && j < j1) {
       band_record(bd, key, j, sel);
       sure += key > bd.hi;
@@ -433,11 +435,10 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_strea
 
 cudaError_t launch_pool_topk(const Shape& s, const SeqBatch& b, const ScoreBuffers& buf,
                              int* idx_out, uint32_t* status, cudaStream_t st) {
-  (void)status;
   if (s.K == 0 || b.n == 0) return cudaSuccess;
   TopkArgs a;
   a.Hkv = s.Hkv; a.Ls = s.Ls; a.Lr = s.Lr; a.K = s.K; a.w = s.w; a.pool_mode = s.pool_mode;
-  a.b = b; a.buf = buf; a.idx_out = idx_out;
+  a.b = b; a.buf = buf; a.idx_out = idx_out; a.status = status;
   int max_le = 0;
   for (int i = 0; i < b.n; ++i) max_le = max(max_le, b.len[i] - s.Ls - s.Lr);
   dim3 grid(CL, s.Hkv, b.n);
