@@ -325,6 +325,8 @@ __global__ void __launch_bounds__(NT, (G > 4 ? 2 : 3)) decode_gqa_kernel(const F
     __syncwarp();
     if (lane == 0 && n + NSTAGE < T) {
       const int nv = (t_begin + w + (n + NSTAGE) * NWARP) * WT;
+      // generic-proxy reads and patches of this stage come before the bulk copy (async proxy) that refills it
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       issue_tile(stage0 + s * STAGE_B, bar0 + 8 * s, kc, vc, nv, min(v1, nv + WT), n_low, Lsr);
     }
   }

@@ -265,7 +265,12 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     }
     process(sK, sV, ok0, ok1, ok2, ok3);
     __syncwarp();
-    if (lane == 0 && n + NSTAGE < T) issue(n + NSTAGE);
+    if (lane == 0 && n + NSTAGE < T) {
+      // the stage was read, and possibly patched, through the generic proxy; the bulk copy that
+      // refills it goes through the async proxy
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      issue(n + NSTAGE);
+    }
   }
   if (timed_out) {
     if (a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);

@@ -209,30 +209,42 @@ __global__ void __launch_bounds__(NT, 1) decode_mla_kernel(const MlaArgs a) {
   }
 }
 
-// Merge the splits of one (sequence, query head); maxima are in the log2 domain.
+// Merge the splits of one (sequence, query head); maxima are in the log2 domain.  The split
+// weights 2^(m_s - M) / L are computed once per block; a thread then sums two adjacent output
+// dims over the splits with 8-byte loads.
 __global__ void __launch_bounds__(256) decode_mla_merge_kernel(const float* __restrict__ partials,
                                                                __nv_bfloat16* __restrict__ out, int Hq, int nsplit,
                                                                const int* __restrict__ slot_ids, int* seq_len,
                                                                int max_seqs, int bump) {
+  __shared__ float w_s[64];
   const int h = blockIdx.x, i = blockIdx.y;
   const float* p = partials + ((long long)i * Hq + h) * nsplit * PSM;
   // when launched as a programmatic dependent, wait for the split kernel's results (no-op otherwise)
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  float M = -INFINITY;
-  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * PSM]);
-  float L = 0.f;
-  for (int s = 0; s < nsplit; ++s) {
-    const float ms = p[s * PSM];
-    if (ms != -INFINITY) L += p[s * PSM + 1] * exp2f(ms - M);
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    float m0 = lane < nsplit ? p[lane * PSM] : -INFINITY, m1 = lane + 32 < nsplit ? p[(lane + 32) * PSM] : -INFINITY;
+    float M = fmaxf(m0, m1);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    const float e0 = m0 != -INFINITY ? exp2f(m0 - M) : 0.f, e1 = m1 != -INFINITY ? exp2f(m1 - M) : 0.f;
+    float L = (lane < nsplit ? p[lane * PSM + 1] * e0 : 0.f) + (lane + 32 < nsplit ? p[(lane + 32) * PSM + 1] * e1 : 0.f);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    w_s[lane] = e0 * inv;
+    w_s[lane + 32] = e1 * inv;
   }
-  const float inv = L > 0.f ? 1.f / L : 0.f;
-  for (int dim = threadIdx.x; dim < DV; dim += blockDim.x) {
-    float o = 0.f;
+  __syncthreads();
+  for (int dim = 2 * threadIdx.x; dim < DV; dim += 2 * blockDim.x) {
+    float o0 = 0.f, o1 = 0.f;
     for (int s = 0; s < nsplit; ++s) {
-      const float ms = p[s * PSM];
-      if (ms != -INFINITY) o += p[s * PSM + 2 + dim] * exp2f(ms - M);
+      const float w = w_s[s];
+      const float2 v = *reinterpret_cast<const float2*>(p + s * PSM + 2 + dim);   // PSM is even: 8-byte aligned
+      o0 = fmaf(v.x, w, o0);
+      o1 = fmaf(v.y, w, o1);
     }
-    out[((long long)i * Hq + h) * DV + dim] = __float2bfloat16_rn(o * inv);
+    *reinterpret_cast<__nv_bfloat162*>(out + ((long long)i * Hq + h) * DV + dim) = __floats2bfloat162_rn(o0, o1);
   }
   if (bump && h == 0 && threadIdx.x == 0) {
     const int slot = slot_ids[i];

@@ -20,8 +20,11 @@
 //   warps 2-5   thread = head: S from TMEM, online softmax in the log2 domain with a lazily
 //               refreshed reference (O is rescaled in TMEM only when a logit exceeds it by 8),
 //               P back to TMEM.
-// The new token, if any, is appended by a separate launch before this kernel (Eq. 3).  Every
-// mbarrier wait is bounded; one that runs out raises SNAP_DEV_WAIT_TIMEOUT.
+// The new token, if any, is appended here (Eq. 3): the CTAs whose tile range holds its slot
+// patch the row into their staged key slabs and value chunks before the tensor core reads them
+// (nobody else loads that row), one of them stores it to the cache, and the merge kernel
+// advances the length.  Every mbarrier wait is bounded; one that runs out raises
+// SNAP_DEV_WAIT_TIMEOUT.
 #include "snap_internal.cuh"
 #include "umma_helpers.cuh"
 
@@ -37,6 +40,8 @@ constexpr int PSM = DV + 2;
 constexpr uint32_t COL_S = 0, COL_O = 256;                               // tensor memory: S0 128 | S1 128 | O 256
 
 struct SArgs {
+  const __nv_bfloat16* k_new;                  // NULL, or [n_active][576]: the new token's row, appended here (Eq. 3)
+  unsigned char* kc;                           // the cache, for the one global store of that row
   const int* slot_ids; const int* seq_len; const int* valid_topk;
   int Hq, Ls, Lr, Sc, max_seqs, nsplit;
   float scale_log2;
@@ -92,15 +97,17 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
   fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // launched as a programmatic dependent of the append kernel: the set-up above overlaps it; wait
-  // for it before reading lengths or rows
+  // launched as a programmatic dependent of whatever precedes it: the set-up above overlaps that
+  // kernel's tail; wait for it before reading lengths or rows
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int slot = a.slot_ids[i];
   const bool bad = slot < 0 || slot >= a.max_seqs;
   const int Lsr = a.Ls + a.Lr;
-  int n_low = 0, n_top = 0;
+  int n_low = 0, n_top = 0, new_slot = -1;
   if (!bad) {
-    n_low = min(a.seq_len[slot], Lsr);
+    int len = a.seq_len[slot];
+    if (a.k_new) { new_slot = ring_slot(len, a.Ls, a.Lr); ++len; }   // the token being written sees itself
+    n_low = min(len, Lsr);
     n_top = a.valid_topk[slot];
   } else if (tid == 0 && sp == 0 && blockIdx.y == 0 && a.status) {
     atomicOr(a.status, SNAP_DEV_BAD_SLOT);
@@ -109,7 +116,10 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
   const int g0 = (int)((long long)ntiles * sp / a.nsplit);
   const int g1 = (int)((long long)ntiles * (sp + 1) / a.nsplit);
   const int nt = g1 - g0;
-
+  // the new row lies in the low section (sinks or ring): tile new_slot / TR, if this split has it
+  const int it_new = new_slot >= 0 && new_slot / TR >= g0 && new_slot / TR < g1 ? new_slot / TR - g0 : -1;
+  const int r_new = new_slot - (g0 + it_new) * TR;             // its row within that tile
+  const uint4* knew4 = a.k_new ? reinterpret_cast<const uint4*>(a.k_new + (long long)i * DQK) : nullptr;
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -168,6 +178,13 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
           const int s = q % NSTG;
           if (!wait_warp(full_bar(s), (unsigned)(q / NSTG) & 1u, abort_flag)) return false;
           fence_after();
+          if (it == it_new) {
+            // the new token's row: eight 16-byte chunks of this 64-dim slab, at their swizzled places
+            if (lane < 8)
+              *reinterpret_cast<uint4*>(Rs + s * STAGE_B + r_new * 128 + ((lane ^ (r_new & 7)) << 4)) = knew4[h * 8 + lane];
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+          }
           const uint64_t kd = smem_desc(smem_u32(Rs) + s * STAGE_B), qd = qd0 + (uint64_t)((h * QSLAB_B) >> 4);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
@@ -206,6 +223,14 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
           }
+          if (it == it_new && r_new / VROWS == c) {
+            // the new row as a value row: this CTA's 256 dims = 4 sub-slabs x 8 chunks, one per lane
+            const int rr = r_new % VROWS, j = lane >> 3, ch = lane & 7;
+            *reinterpret_cast<uint4*>(Rs + s * STAGE_B + j * VSUB_B + rr * 128 + ((ch ^ (rr & 7)) << 4)) =
+                knew4[(hd * DVH + j * 64) / 8 + ch];
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+          }
 #pragma unroll
           for (int ks = 0; ks < VROWS / 16; ++ks)
             mma_ts_pred(tmem_base + COL_O, pa + 8 * (c * (VROWS / 16) + ks), smem_desc_mn(vst + ks * 16 * 128, VSUB_B),
@@ -220,6 +245,8 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
   } else {
     // ---------------- softmax warps: thread = head ----------------
     const int hrow = 32 * (warp & 3) + lane;                   // TMEM lane = head within the block
+    if (it_new >= 0 && hd == 0 && hb == 0 && hrow < DQK / 8)   // the one store of the new row to the cache
+      reinterpret_cast<uint4*>(a.kc + ((long long)slot * a.Sc + new_slot) * (DQK * 2))[hrow] = knew4[hrow];
     const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
     const int head = hb * HBLK + hrow;
     float m_ref = -INFINITY, l_sum = 0.f;
@@ -346,6 +373,7 @@ bool decode_mla_stream_supported(int dtype, const Shape& s) {
 // fill the SMs once or twice over, with at least two tiles per split.
 int decode_mla_stream_nsplit(const Shape& s, int n_active, int sm_count) {
   const int tiles = (s.Sc + TR - 1) / TR + 1;
+  if (const int v = option(SNAP_OPT_DECODE_NSPLIT)) return v < tiles ? (v < 64 ? v : 64) : tiles;   // tuning aid
   const long long base = (long long)n_active * NHALF * (s.Hq / HBLK);
   int best = 1;
   double best_fill = -1.0;
@@ -369,10 +397,6 @@ cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* 
   if (n_active == 0) return cudaSuccess;
   umma::EncodeTiledFn enc = umma::encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
-  if (k_new) {                                                 // Eq. 3 append (also advances the lengths)
-    cudaError_t e = launch_append(SNAP_BF16, s, k_new, nullptr, slot_ids, n_active, k_cache, nullptr, seq_len, status, st);
-    if (e != cudaSuccess) return e;
-  }
   CUtensorMap tq, tk, tv;
   const cuuint32_t estr2[2] = {1, 1}, estr3[3] = {1, 1, 1};
   {
@@ -393,6 +417,7 @@ cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* 
           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
   SArgs a;
+  a.k_new = static_cast<const __nv_bfloat16*>(k_new); a.kc = static_cast<unsigned char*>(k_cache);
   a.slot_ids = slot_ids; a.seq_len = seq_len; a.valid_topk = valid_topk;
   a.Hq = s.Hq; a.Ls = s.Ls; a.Lr = s.Lr; a.Sc = s.Sc; a.max_seqs = s.max_seqs; a.nsplit = nsplit;
   a.scale_log2 = s.scale * 1.4426950408889634f;
@@ -400,7 +425,7 @@ cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* 
   const size_t smem = stream_smem_bytes();
   static SmemLimit limit = {};
   if (cudaError_t e = ensure_dyn_smem(decode_mla_stream_kernel, smem, limit)) return e;
-  // a programmatic dependent launch: the CTAs may become resident while the append kernel drains
+  // a programmatic dependent launch: the CTAs may become resident while the previous kernel drains
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -414,7 +439,7 @@ cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* 
   cudaError_t e = cudaLaunchKernelEx(&lc, decode_mla_stream_kernel, a, tq, tk, tv);
   count_launch();
   if (e != cudaSuccess) return e;
-  return launch_decode_mla_merge(partials, out, n_active, s.Hq, nsplit, slot_ids, seq_len, s.max_seqs, 0, st, true);
+  return launch_decode_mla_merge(partials, out, n_active, s.Hq, nsplit, slot_ids, seq_len, s.max_seqs, k_new != nullptr, st, true);
 }
 
 }  // namespace snap
