@@ -287,8 +287,8 @@ int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout
  *   - Every GPU that loads this library holds the array from load until process exit.
  *   - The step runs the same kernels with the same split count as snap_decode_attn (the latent
  *     layout included) and needs snap_decode_workspace_bytes(cfg, n_active) - 256 bytes of the
- *     array: n_active * n_q_heads * splits * (d_v + 2) floats, splits being the library's choice
- *     for that batch size.  If that exceeds the array the call returns
+ *     array: n_active * n_q_heads * splits * (d_v + 2) floats (d_v + 4 for the latent layout),
+ *     splits being the library's choice for that batch size.  If that exceeds the array the call returns
  *     SNAP_ERR_STATIC_SCRATCH_EXCEEDED and launches nothing; use snap_decode_attn instead.
  *     The 32-sequence, 32-head, d_v = 128 batch of a Llama-3.1-8B layer needs about 4.3 MB.
  *   - All calls share the one array and it keeps the previous call's contents.  Nothing has to

@@ -25,7 +25,7 @@ constexpr int DQK = 576, DV = 512, HB = 64, TR = 32, NSTG = 3, NT = 256;
 constexpr int ROW_B = DQK * 2;                 // 1152 bytes per cache row
 constexpr int CHUNKS = ROW_B / 16;             // 72 16-byte chunks per row
 constexpr int QS_B = HB * ROW_B, KT_B = TR * ROW_B;
-constexpr int PSM = DV + 2;                    // floats per partial: m, l, acc[DV]
+constexpr int PSM = DV + 4;                    // floats per partial: m, l, two unused, acc[DV] (rows 16-byte aligned)
 
 struct MlaArgs {
   const __nv_bfloat16* q; const __nv_bfloat16* k_new;
@@ -205,14 +205,14 @@ __global__ void __launch_bounds__(NT, 1) decode_mla_kernel(const MlaArgs a) {
     if (dh == 0 && (lane & 3) == 0) { ph[0] = m_run[h]; ph[1] = l_run[h]; }
 #pragma unroll
     for (int j = 0; j < 32; ++j)
-      *reinterpret_cast<float2*>(ph + 2 + dh * 256 + 8 * j + 2 * (lane & 3)) = make_float2(o[j][2 * h], o[j][2 * h + 1]);
+      *reinterpret_cast<float2*>(ph + 4 + dh * 256 + 8 * j + 2 * (lane & 3)) = make_float2(o[j][2 * h], o[j][2 * h + 1]);
   }
 }
 
 // Merge the splits of one (sequence, query head); maxima are in the log2 domain.  The split
-// weights 2^(m_s - M) / L are computed once per block; a thread then sums two adjacent output
-// dims over the splits with 8-byte loads.
-__global__ void __launch_bounds__(256) decode_mla_merge_kernel(const float* __restrict__ partials,
+// weights 2^(m_s - M) / L are computed once per block; a thread then sums four adjacent output
+// dims over the splits with 16-byte loads.
+__global__ void __launch_bounds__(128) decode_mla_merge_kernel(const float* __restrict__ partials,
                                                                __nv_bfloat16* __restrict__ out, int Hq, int nsplit,
                                                                const int* __restrict__ slot_ids, int* seq_len,
                                                                int max_seqs, int bump) {
@@ -236,15 +236,16 @@ __global__ void __launch_bounds__(256) decode_mla_merge_kernel(const float* __re
     w_s[lane + 32] = e1 * inv;
   }
   __syncthreads();
-  for (int dim = 2 * threadIdx.x; dim < DV; dim += 2 * blockDim.x) {
-    float o0 = 0.f, o1 = 0.f;
+  for (int dim = 4 * threadIdx.x; dim < DV; dim += 4 * blockDim.x) {
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < nsplit; ++s) {
       const float w = w_s[s];
-      const float2 v = *reinterpret_cast<const float2*>(p + s * PSM + 2 + dim);   // PSM is even: 8-byte aligned
-      o0 = fmaf(v.x, w, o0);
-      o1 = fmaf(v.y, w, o1);
+      const float4 v = *reinterpret_cast<const float4*>(p + s * PSM + 4 + dim);
+      o.x = fmaf(v.x, w, o.x); o.y = fmaf(v.y, w, o.y); o.z = fmaf(v.z, w, o.z); o.w = fmaf(v.w, w, o.w);
     }
-    *reinterpret_cast<__nv_bfloat162*>(out + ((long long)i * Hq + h) * DV + dim) = __floats2bfloat162_rn(o0, o1);
+    __nv_bfloat162* dst = reinterpret_cast<__nv_bfloat162*>(out + ((long long)i * Hq + h) * DV + dim);
+    dst[0] = __floats2bfloat162_rn(o.x, o.y);
+    dst[1] = __floats2bfloat162_rn(o.z, o.w);
   }
   if (bump && h == 0 && threadIdx.x == 0) {
     const int slot = slot_ids[i];
@@ -262,7 +263,7 @@ cudaError_t launch_decode_mla_merge(const float* partials, void* out, int n_acti
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(Hq, (unsigned)n_active);
-  lc.blockDim = dim3(256);
+  lc.blockDim = dim3(128);
   lc.stream = st;
   lc.attrs = attr;
   lc.numAttrs = programmatic ? 1 : 0;
@@ -311,7 +312,7 @@ cudaError_t launch_decode_mla(const Shape& s, const void* q, const void* k_new, 
   decode_mla_kernel<<<grid, NT, smem, st>>>(a);
   count_launch();
   dim3 mgrid(s.Hq, n_active);
-  decode_mla_merge_kernel<<<mgrid, 256, 0, st>>>(partials, static_cast<__nv_bfloat16*>(out), s.Hq, nsplit,
+  decode_mla_merge_kernel<<<mgrid, 128, 0, st>>>(partials, static_cast<__nv_bfloat16*>(out), s.Hq, nsplit,
                                                  slot_ids, seq_len, s.max_seqs, k_new != nullptr);
   count_launch();
   return cudaGetLastError();

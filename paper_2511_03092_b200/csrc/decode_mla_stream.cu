@@ -36,7 +36,7 @@ using namespace umma;
 constexpr int DQK = 576, DV = 512, HBLK = 128, TR = 128, NSTG = 5, NTH = 192, DVH = 256, NHALF = DV / DVH;
 constexpr int NSLAB = DQK / 64, QSLAB_B = HBLK * 128, STAGE_B = 16384;   // key slab = 128 rows x 128 B = one stage
 constexpr int VROWS = 32, VSUB_B = VROWS * 128, NVCH = TR / VROWS;       // value chunk = 4 sub-slabs of 32 rows x 64 dims
-constexpr int PSM = DV + 2;
+constexpr int PSM = DV + 4;                                              // m, l, two unused, acc[DV]: rows 16-byte aligned
 constexpr uint32_t COL_S = 0, COL_O = 256;                               // tensor memory: S0 128 | S1 128 | O 256
 
 struct SArgs {
@@ -335,19 +335,31 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
     fence_after();
     if (hd == 0) { ph[0] = nt > 0 && ok ? m_ref : -INFINITY; ph[1] = nt > 0 && ok ? l_sum : 0.f; }
     const bool have = __all_sync(0xffffffffu, ok && nt > 0);
+    // O goes out 32 columns at a time through this warp's corner of the (now idle) ring, transposed so that
+    // a store instruction writes four heads' 128-byte runs instead of 32 scattered pieces
+    float* tw = reinterpret_cast<float*>(Rs) + (warp & 3) * (32 * 36);       // [32 heads][36 floats]
+    float* ph_warp = a.partials + (((long long)i * a.Hq + hb * HBLK + 32 * (warp & 3)) * a.nsplit + sp) * PSM;
 #pragma unroll 1
-    for (int c = 0; c < DVH / 16; ++c) {
-      uint32_t o[16];
+    for (int c = 0; c < DVH / 32; ++c) {
+      uint32_t o[32];
       if (have) {
-        tmem_ld16_issue(lane_addr + COL_O + 16 * c, o);
-        tmem_ld16_wait(o);
+        tmem_ld32_issue(lane_addr + COL_O + 32 * c, o);
+        tmem_ld_wait(o);
       } else {
 #pragma unroll
-        for (int e = 0; e < 16; ++e) o[e] = 0u;
+        for (int e = 0; e < 32; ++e) o[e] = 0u;
       }
-      float2* d2 = reinterpret_cast<float2*>(ph + 2 + hd * DVH + 16 * c);   // ph + 2 is 8-byte aligned only
 #pragma unroll
-      for (int e = 0; e < 8; ++e) d2[e] = make_float2(__uint_as_float(o[2 * e]), __uint_as_float(o[2 * e + 1]));
+      for (int e = 0; e < 8; ++e)
+        *reinterpret_cast<uint4*>(tw + lane * 36 + 4 * e) = make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+      __syncwarp();
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int r = 4 * k + (lane >> 3), piece = lane & 7;
+        const uint4 v = *reinterpret_cast<const uint4*>(tw + r * 36 + 4 * piece);
+        *reinterpret_cast<uint4*>(ph_warp + (long long)r * a.nsplit * PSM + 4 + hd * DVH + 32 * c + 4 * piece) = v;
+      }
+      __syncwarp();
     }
   }
 
