@@ -87,7 +87,7 @@ struct CorrectionArgs {
   uint32_t* status;
 };
 __device__ __noinline__ void apply_selection_correction(const CorrectionArgs c) {
-  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int tid = threadIdx.x;
   for (int i = tid; i < c.K; i += NT) c.old[i] = c.out[i];
   __syncthreads();
   auto shift_of = [&](int j) {                               // entering below j minus leaving below j
@@ -111,17 +111,49 @@ __device__ __noinline__ void apply_selection_correction(const CorrectionArgs c) 
     if (index_ok(lo + shift_of(j), c.K, c.status)) c.out[lo + shift_of(j)] = pos_abs;
   }
   __syncthreads();
-  for (int i = wid; i < c.K; i += NT / 32) {                 // a warp per changed row
-    const int pos = c.out[i];
-    if (pos == c.old[i] || !index_ok(pos, c.L, c.status)) continue;
-    const uint4* s4 = reinterpret_cast<const uint4*>(c.ksrc + (long long)pos * c.k_tok_b);
-    uint4* d4 = reinterpret_cast<uint4*>(c.kdst + (long long)(c.Lsr + i) * c.k_row_b);
-    for (int v = lane; v < c.k_row_b / 16; v += 32) d4[v] = s4[v];
-    if (c.vdst) {
-      s4 = reinterpret_cast<const uint4*>(c.vsrc + (long long)pos * c.v_tok_b);
-      d4 = reinterpret_cast<uint4*>(c.vdst + (long long)(c.Lsr + i) * c.v_row_b);
-      for (int v = lane; v < c.v_row_b / 16; v += 32) d4[v] = s4[v];
+  // Copy again the rows of the ranks whose position changed (everything between a leaving and an
+  // entering position moves by one rank).  Ranks are scanned 1024 at a time into a list in shared
+  // memory, then all threads copy the listed rows, 16 bytes per thread and turn.
+  __shared__ int changed[1024], changed_pos[1024];
+  __shared__ int n_changed;
+  const int kv = c.k_row_b / 16, vv = c.vdst ? c.v_row_b / 16 : 0;
+  for (int base = 0; base < c.K; base += 1024) {
+    if (tid == 0) n_changed = 0;
+    __syncthreads();
+    for (int i = base + tid; i < min(base + 1024, c.K); i += NT) {
+      const int pos = c.out[i];
+      if (pos != c.old[i] && index_ok(pos, c.L, c.status)) {
+        const int e = atomicAdd(&n_changed, 1);
+        changed[e] = i;
+        changed_pos[e] = pos;
+      }
     }
+    __syncthreads();
+    const int total = n_changed * (kv + vv);
+    for (int e0 = tid; e0 < total; e0 += 4 * NT) {            // four 16-byte loads in flight per thread
+      uint4 val[4];
+      uint4* dst[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = e0 + u * NT;
+        dst[u] = nullptr;
+        if (e < total) {
+          const int r = e / (kv + vv), v = e % (kv + vv);
+          const long long pos = changed_pos[r], i = changed[r];
+          if (v < kv) {
+            val[u] = reinterpret_cast<const uint4*>(c.ksrc + pos * c.k_tok_b)[v];
+            dst[u] = reinterpret_cast<uint4*>(c.kdst + (c.Lsr + i) * c.k_row_b) + v;
+          } else {
+            val[u] = reinterpret_cast<const uint4*>(c.vsrc + pos * c.v_tok_b)[v - kv];
+            dst[u] = reinterpret_cast<uint4*>(c.vdst + (c.Lsr + i) * c.v_row_b) + (v - kv);
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (dst[u]) *dst[u] = val[u];
+    }
+    __syncthreads();
   }
 }
 
