@@ -256,8 +256,9 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout,
  * 1 <= q_len <= Lr (SNAP_ERR_INVALID_ARG otherwise).  bf16 layers with 64-, 128- or 256-wide heads
  * and q_len * (Hq / Hkv) <= 8 are served in one pass over the cache; every other layer (fp32, the
  * latent layout -- v_new_dev is then ignored --, larger groups) is served as the definition reads,
- * q_len single steps, with each token's rows staged in the workspace: same results, no saving in
- * cache traffic.  Scratch: snap_decode_multi_workspace_bytes(cfg, n_active, q_len).
+ * q_len single steps: same results, no saving in cache traffic.  The tcgen05 latent kernel reads
+ * each token's rows in place; the other kernels have them staged in the workspace first.
+ * Scratch: snap_decode_multi_workspace_bytes(cfg, n_active, q_len).
  */
 int64_t snap_decode_multi_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t q_len);
 int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout,

@@ -605,6 +605,19 @@ int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout
                                                 static_cast<float*>(workspace_dev), nsplit, status_dev, st, q_len);
     return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
   }
+  // the streamed latent kernel reads token u of every sequence in place (strided tensor map, strided rows):
+  // q_len single steps with no staging copies.  (One launch over (sequence, token) was tried: with the 8 sequences
+  // of the latent benchmark shape the grid needs two waves and two tokens took 140 us against 2 x 54.)
+  {
+    const DecodePlan p = plan_decode(cfg->dtype, s, n_active);
+    if (p.mla_stream) {
+      for (int u = 0; u < q_len; ++u)
+        if (launch_decode_mla_stream(s, q_dev, k_new_dev, slot_ids_dev, n_active, k_cache_dev, seq_len_dev, valid_topk_dev,
+                                     out_dev, static_cast<float*>(workspace_dev), p.nsplit, status_dev, st, q_len, u) != cudaSuccess)
+          return SNAP_ERR_CUDA;
+      return SNAP_OK;
+    }
+  }
   // q_len single steps: token u of every sequence is gathered into dense rows, attended, and its
   // output scattered back
   const StepStage t = step_stage(cfg, s, n_active);

@@ -215,7 +215,7 @@ __global__ void __launch_bounds__(NT, 1) decode_mla_kernel(const MlaArgs a) {
 __global__ void __launch_bounds__(128) decode_mla_merge_kernel(const float* __restrict__ partials,
                                                                __nv_bfloat16* __restrict__ out, int Hq, int nsplit,
                                                                const int* __restrict__ slot_ids, int* seq_len,
-                                                               int max_seqs, int bump) {
+                                                               int max_seqs, int bump, int q_len, int u) {
   __shared__ float w_s[64];
   const int h = blockIdx.x, i = blockIdx.y;
   const float* p = partials + ((long long)i * Hq + h) * nsplit * PSM;
@@ -243,7 +243,8 @@ __global__ void __launch_bounds__(128) decode_mla_merge_kernel(const float* __re
       const float4 v = *reinterpret_cast<const float4*>(p + s * PSM + 4 + dim);
       o.x = fmaf(v.x, w, o.x); o.y = fmaf(v.y, w, o.y); o.z = fmaf(v.z, w, o.z); o.w = fmaf(v.w, w, o.w);
     }
-    __nv_bfloat162* dst = reinterpret_cast<__nv_bfloat162*>(out + ((long long)i * Hq + h) * DV + dim);
+    // out is [n_active][q_len][Hq][DV]: this launch serves token u of every sequence
+    __nv_bfloat162* dst = reinterpret_cast<__nv_bfloat162*>(out + (((long long)i * q_len + u) * Hq + h) * DV + dim);
     dst[0] = __floats2bfloat162_rn(o.x, o.y);
     dst[1] = __floats2bfloat162_rn(o.z, o.w);
   }
@@ -257,7 +258,7 @@ __global__ void __launch_bounds__(128) decode_mla_merge_kernel(const float* __re
 
 cudaError_t launch_decode_mla_merge(const float* partials, void* out, int n_active, int Hq, int nsplit,
                                     const int* slot_ids, int* seq_len, int max_seqs, int bump, cudaStream_t st,
-                                    bool programmatic) {
+                                    bool programmatic, int q_len, int u) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -268,7 +269,7 @@ cudaError_t launch_decode_mla_merge(const float* partials, void* out, int n_acti
   lc.attrs = attr;
   lc.numAttrs = programmatic ? 1 : 0;
   cudaError_t e = cudaLaunchKernelEx(&lc, decode_mla_merge_kernel, partials, static_cast<__nv_bfloat16*>(out), Hq, nsplit,
-                                     slot_ids, seq_len, max_seqs, bump);
+                                     slot_ids, seq_len, max_seqs, bump, q_len, u);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -313,7 +314,7 @@ cudaError_t launch_decode_mla(const Shape& s, const void* q, const void* k_new, 
   count_launch();
   dim3 mgrid(s.Hq, n_active);
   decode_mla_merge_kernel<<<mgrid, 128, 0, st>>>(partials, static_cast<__nv_bfloat16*>(out), s.Hq, nsplit,
-                                                 slot_ids, seq_len, s.max_seqs, k_new != nullptr);
+                                                 slot_ids, seq_len, s.max_seqs, k_new != nullptr, 1, 0);
   count_launch();
   return cudaGetLastError();
 }

@@ -44,6 +44,7 @@ struct SArgs {
   unsigned char* kc;                           // the cache, for the one global store of that row
   const int* slot_ids; const int* seq_len; const int* valid_topk;
   int Hq, Ls, Lr, Sc, max_seqs, nsplit;
+  long long knew_seq_stride;                   // elements between two sequences' new rows
   float scale_log2;
   float* partials;                             // [n_active][Hq][nsplit][PSM], maxima in the log2 domain
   uint32_t* status;
@@ -119,14 +120,14 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
   // the new row lies in the low section (sinks or ring): tile new_slot / TR, if this split has it
   const int it_new = new_slot >= 0 && new_slot / TR >= g0 && new_slot / TR < g1 ? new_slot / TR - g0 : -1;
   const int r_new = new_slot - (g0 + it_new) * TR;             // its row within that tile
-  const uint4* knew4 = a.k_new ? reinterpret_cast<const uint4*>(a.k_new + (long long)i * DQK) : nullptr;
+  const uint4* knew4 = a.k_new ? reinterpret_cast<const uint4*>(a.k_new + (long long)i * a.knew_seq_stride) : nullptr;
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0 && nt > 0) {
       mbar_expect_tx(qfull_bar, (unsigned)NSLAB * QSLAB_B);
       for (int h = 0; h < NSLAB; ++h)
-        tma_load_2d(smem_u32(Qs) + h * QSLAB_B, &tmap_q, h * 64, i * a.Hq + hb * HBLK, qfull_bar);
+        tma_load_3d(smem_u32(Qs) + h * QSLAB_B, &tmap_q, h * 64, hb * HBLK, i, qfull_bar);
       int q = 0;                                               // stages issued so far
       bool ok = true;
       auto stage_wait = [&]() -> bool {
@@ -405,17 +406,19 @@ size_t decode_mla_stream_partial_floats(const Shape& s, int n_active, int nsplit
 
 cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* k_new, const int* slot_ids,
                                      int n_active, void* k_cache, int* seq_len, const int* valid_topk, void* out,
-                                     float* partials, int nsplit, uint32_t* status, cudaStream_t st) {
+                                     float* partials, int nsplit, uint32_t* status, cudaStream_t st, int q_len, int u) {
   if (n_active == 0) return cudaSuccess;
   umma::EncodeTiledFn enc = umma::encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
   CUtensorMap tq, tk, tv;
-  const cuuint32_t estr2[2] = {1, 1}, estr3[3] = {1, 1, 1};
+  const cuuint32_t estr3[3] = {1, 1, 1};
   {
-    const cuuint64_t dims[2] = {(cuuint64_t)DQK, (cuuint64_t)n_active * s.Hq};
-    const cuuint64_t strides[1] = {(cuuint64_t)DQK * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)HBLK};
-    if (enc(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(q), dims, strides, box, estr2,
+    // queries [n_active][q_len][Hq][576]: token u of every sequence as a (dim, head, sequence) tensor
+    const cuuint64_t dims[3] = {(cuuint64_t)DQK, (cuuint64_t)s.Hq, (cuuint64_t)n_active};
+    const cuuint64_t strides[2] = {(cuuint64_t)DQK * 2, (cuuint64_t)q_len * s.Hq * DQK * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)HBLK, 1};
+    void* q_u = const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(q) + (long long)u * s.Hq * DQK);
+    if (enc(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, q_u, dims, strides, box, estr3,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorInvalidValue;
@@ -429,7 +432,9 @@ cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* 
           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
   SArgs a;
-  a.k_new = static_cast<const __nv_bfloat16*>(k_new); a.kc = static_cast<unsigned char*>(k_cache);
+  a.k_new = k_new ? static_cast<const __nv_bfloat16*>(k_new) + (long long)u * DQK : nullptr;   // Hkv = 1
+  a.knew_seq_stride = (long long)q_len * DQK;
+  a.kc = static_cast<unsigned char*>(k_cache);
   a.slot_ids = slot_ids; a.seq_len = seq_len; a.valid_topk = valid_topk;
   a.Hq = s.Hq; a.Ls = s.Ls; a.Lr = s.Lr; a.Sc = s.Sc; a.max_seqs = s.max_seqs; a.nsplit = nsplit;
   a.scale_log2 = s.scale * 1.4426950408889634f;
@@ -451,7 +456,8 @@ cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* 
   cudaError_t e = cudaLaunchKernelEx(&lc, decode_mla_stream_kernel, a, tq, tk, tv);
   count_launch();
   if (e != cudaSuccess) return e;
-  return launch_decode_mla_merge(partials, out, n_active, s.Hq, nsplit, slot_ids, seq_len, s.max_seqs, k_new != nullptr, st, true);
+  return launch_decode_mla_merge(partials, out, n_active, s.Hq, nsplit, slot_ids, seq_len, s.max_seqs, k_new != nullptr, st, true,
+                                 q_len, u);
 }
 
 }  // namespace snap

@@ -201,14 +201,15 @@ cudaError_t launch_decode_mla(const Shape& s, const void* q, const void* k_new, 
 
 cudaError_t launch_decode_mla_merge(const float* partials, void* out, int n_active, int Hq, int nsplit,
                                     const int* slot_ids, int* seq_len, int max_seqs, int bump, cudaStream_t st,
-                                    bool programmatic = false);
+                                    bool programmatic = false, int q_len = 1, int u = 0);
 // latent attention on tcgen05, streamed: queries in shared memory, cache rows streamed as key slabs and value chunks
 bool decode_mla_stream_supported(int dtype, const Shape& s);
 int decode_mla_stream_nsplit(const Shape& s, int n_active, int sm_count);
 size_t decode_mla_stream_partial_floats(const Shape& s, int n_active, int nsplit);
+// q_len > 1: q, k_new and out hold q_len tokens per sequence ([n][q_len][...]) and this call serves token u of each
 cudaError_t launch_decode_mla_stream(const Shape& s, const void* q, const void* k_new, const int* slot_ids,
                                      int n_active, void* k_cache, int* seq_len, const int* valid_topk, void* out,
-                                     float* partials, int nsplit, uint32_t* status, cudaStream_t st);
+                                     float* partials, int nsplit, uint32_t* status, cudaStream_t st, int q_len = 1, int u = 0);
 
 // Checked indexing for the debugging build (-DSNAP_DEBUG_BOUNDS): a data-dependent index that falls
 // outside [0, n) raises SNAP_DEV_INDEX_CHECK in the status word and the access is skipped -- nothing
