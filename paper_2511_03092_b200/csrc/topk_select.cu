@@ -51,6 +51,7 @@ struct TopkShared {
   int tot[256];          // cluster-wide histogram of the current pass
   unsigned prefix;
   int remaining;
+  int sure;              // this CTA's candidates above the re-scoring band
 };
 
 __device__ __forceinline__ unsigned key_of(float x) {
@@ -88,11 +89,14 @@ __device__ __forceinline__ void band_record(const Band& bd, unsigned key, int j,
     bd.entries[slot] = e;
   }
 }
-// Adds this thread's count of candidates above the band to the head's total (one atomic per warp).
-__device__ __forceinline__ void band_count_sure(const Band& bd, int n) {
+// Adds this thread's count of candidates above the band to the head's total: summed per warp, then per
+// CTA in shared memory, one global atomic per CTA (hundreds of warps on one address serialise).
+__device__ __forceinline__ void band_count_sure(const Band& bd, int n, int* cta_sum) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
-  if ((threadIdx.x & 31) == 0 && n > 0) atomicAdd(&bd.head->n_sure, n);
+  if ((threadIdx.x & 31) == 0 && n > 0) atomicAdd(cta_sum, n);
+  __syncthreads();
+  if (threadIdx.x == 0 && *cta_sum > 0) atomicAdd(&bd.head->n_sure, *cta_sum);
 }
 __device__ __forceinline__ void band_reset(const TopkArgs& a, long long z, int rank) {
   if (a.buf.ref.head && rank == 0 && threadIdx.x == 0) {
@@ -173,6 +177,7 @@ __device__ __forceinline__ int cluster_common_prefix(cg::cluster_group& cluster,
   if (tid == 0) {
     sh.prefix = nbits >= 32 ? 0u : kmin & ~((1u << nbits) - 1u);
     sh.remaining = K;
+    sh.sure = 0;
   }
   __syncthreads();
   return nbits;
@@ -341,7 +346,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_regs_
       }
     }
   }
-  if (bd.head) band_count_sure(bd, sure);
+  if (bd.head) band_count_sure(bd, sure, &sh.sure);
 }
 
 // ---- streaming kernel: any length and pooling width; pooled scores live in scratch ----
@@ -428,7 +433,7 @@ __global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(NT) pool_topk_strea
     run_eq += te;
     run_out += ts;
   }
-  if (bd.head) band_count_sure(bd, sure);
+  if (bd.head) band_count_sure(bd, sure, &sh.sure);
 }
 
 }  // namespace
