@@ -154,3 +154,14 @@ def test_a_correction_moves_the_index_list_and_the_cache_rows(snap_option):
     print(f"single-precision order differs from the oracle's on {len(differing)} of {len(prompts)} near-tie prompts")
     assert differing, "no prompt exercises the correction: the single-precision order was right everywhere"
     assert _check_exact(wl, prompts, lo, hi) == 0
+    # the same prompts in one ragged call (corrections in prompts other than the first, slots out of order)
+    batch = [p for _, p in differing] + [prompts[0][1]]
+    slots = list(range(len(batch)))[::-1]
+    layer = H.GpuLayer(wl, max_seqs=len(batch))
+    idx = layer.compress(batch, slots)
+    assert layer.status() == 0
+    for i, p in enumerate(batch):
+        seq = H.oracle_compress(wl, p)
+        for h in range(wl.n_kv_heads):
+            np.testing.assert_array_equal(idx[i][h], seq.topk_pos[h])
+        H.check_cache_image(layer, seq, slots[i], wl)
