@@ -161,3 +161,23 @@ def test_header_is_plain_c99(tmp_path):
     subprocess.run([gcc, str(obj), "-L", libdir, "-lsnapstream", "-Wl,-rpath," + libdir, "-o", str(exe)], check=True)
     out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
     assert out[:5] == ["0", "5124", "0", "4", "1028"]
+
+
+def test_debug_options_are_process_wide_integers():
+    """snap_debug_set_option: returns the previous value, rejects unknown options and negative
+    values, and what it sets changes the library's planning (host arithmetic only, no GPU)."""
+    before = B.snap_debug_set_option(B.SNAP_OPT_REFINE_OFF, 1)
+    try:
+        assert B.snap_debug_set_option(B.SNAP_OPT_REFINE_OFF, 1) == 1
+        cfg = _cfg()
+        cu = [0, 40000]
+        without = B.snap_compress_workspace_bytes(cfg, cu)
+        B.snap_debug_set_option(B.SNAP_OPT_REFINE_OFF, 0)
+        with_refine = B.snap_compress_workspace_bytes(cfg, cu)
+        assert with_refine > without                      # band entries, column sums, normalisers, verdict lists
+    finally:
+        B.snap_debug_set_option(B.SNAP_OPT_REFINE_OFF, before)
+    for bad in ((-1, 0), (99, 0), (B.SNAP_OPT_REFINE_OFF, -3)):
+        with pytest.raises(B.SnapError) as e:
+            B.snap_debug_set_option(*bad)
+        assert e.value.code == -1
