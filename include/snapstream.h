@@ -336,7 +336,7 @@ int snap_append_kv_concat(const snap_config_t* cfg, const snap_layout_t* layout,
  * from its environment variable (named on the right); the environment is not read again.
  * Returns the option's previous value, or SNAP_ERR_INVALID_ARG.
  */
-#define SNAP_OPT_SCORE_KERNEL 0          /* 1: mma.sync score kernel, 2: SIMT       SNAP_SCORE_PATH=mma|simt */
+#define SNAP_OPT_SCORE_KERNEL 0          /* 1: mma.sync score kernel, 2: SIMT, 3: tcgen05 without CTA pairs  SNAP_SCORE_PATH=mma|simt|single */
 #define SNAP_OPT_DECODE_GQA_KERNEL 1     /* 1: packed-FP32 GQA decode kernel        SNAP_DECODE_GQA=simt     */
 #define SNAP_OPT_DECODE_LATENT_KERNEL 2  /* 1: mma.sync latent decode kernel        SNAP_DECODE_MLA=mma      */
 #define SNAP_OPT_DECODE_NSPLIT 3         /* n: splits per (sequence, KV head)       SNAP_DECODE_NSPLIT=n     */

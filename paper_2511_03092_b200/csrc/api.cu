@@ -21,7 +21,7 @@ std::once_flag g_opt_once;
 
 void seed_options() {
   auto env_int = [](const char* name) { const char* e = getenv(name); const int v = e ? atoi(e) : 0; return v > 0 ? v : 0; };
-  if (const char* e = getenv("SNAP_SCORE_PATH")) g_opt[SNAP_OPT_SCORE_KERNEL] = !strcmp(e, "mma") ? 1 : !strcmp(e, "simt") ? 2 : 0;
+  if (const char* e = getenv("SNAP_SCORE_PATH")) g_opt[SNAP_OPT_SCORE_KERNEL] = !strcmp(e, "mma") ? 1 : !strcmp(e, "simt") ? 2 : !strcmp(e, "single") ? 3 : 0;
   if (const char* e = getenv("SNAP_DECODE_GQA")) g_opt[SNAP_OPT_DECODE_GQA_KERNEL] = e[0] == 's';
   if (const char* e = getenv("SNAP_DECODE_MLA")) g_opt[SNAP_OPT_DECODE_LATENT_KERNEL] = e[0] == 'm';
   if (const char* e = getenv("SNAP_PREFILL_PATH")) g_opt[SNAP_OPT_PREFILL_KERNEL] = !strcmp(e, "simt");
@@ -92,14 +92,15 @@ Shape make_shape(const snap_config_t* c) {
 
 size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
-// Option SNAP_OPT_SCORE_KERNEL = 1 (mma.sync) or 2 (SIMT) forces a slower score kernel (testing
-// aid); default: the best one.
+// Option SNAP_OPT_SCORE_KERNEL = 1 (mma.sync) or 2 (SIMT) forces a slower score kernel, 3 keeps the
+// tcgen05 kernels but without CTA pairs (testing aids); default: the best one.
+bool forced_legacy_score() { return option(SNAP_OPT_SCORE_KERNEL) == 1 || option(SNAP_OPT_SCORE_KERNEL) == 2; }
 bool use_umma(int dtype, const Shape& s) {
-  if (option(SNAP_OPT_SCORE_KERNEL) != 0) return false;
+  if (forced_legacy_score()) return false;
   return score_umma_supported(dtype, s);
 }
 bool use_umma_wide(int dtype, const Shape& s) {
-  if (option(SNAP_OPT_SCORE_KERNEL) != 0) return false;
+  if (forced_legacy_score()) return false;
   return !score_umma_supported(dtype, s) && score_umma_wide_supported(dtype, s);
 }
 bool use_mma(int dtype, const Shape& s) {

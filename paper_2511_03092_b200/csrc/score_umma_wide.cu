@@ -4,11 +4,17 @@
 // block of window rows is masked).
 //
 // Same roles as the 128-wide kernel (TMA producer warp, single-thread MMA issuer, eight epilogue
-// warps reading TMEM), but the contraction dimension is streamed: grid = (candidate splits,
-// blocks of 128 window rows, prompts).  A CTA keeps its 128-row query block resident in shared
-// memory (one 16 KB swizzled slab per 64 dims) and, for every candidate tile, pulls the keys
-// through a ring of 2 to 6 stages (whatever fits beside the query block) one 64-dim slab at a time, accumulating in tensor memory; two
-// accumulator buffers let the next tile's MMAs overlap the epilogue of the current one.
+// warps reading TMEM), but the contraction dimension is streamed: a CTA keeps its 128-row query
+// block resident in shared memory (one 16 KB swizzled slab per 64 dims) and, for every candidate
+// tile, pulls the keys through a ring of stages (whatever fits beside the query block) one 64-dim
+// slab at a time, accumulating in tensor memory; two accumulator buffers let the next tile's MMAs
+// overlap the epilogue of the current one.
+// With an even number of row blocks two CTAs with adjacent row blocks form a cluster and share every
+// key tile (tcgen05 cta_group::2): each loads half of the tile's rows into its own shared memory,
+// the even CTA issues M = 256 instructions over both, and each CTA finds its 128 rows of the
+// accumulator in its own tensor memory -- half the L2-to-SM traffic per flop, which is what bounds
+// the single-CTA form.  grid = (2 x candidate splits, row blocks / 2, prompts x KV heads) then;
+// otherwise (candidate splits, row blocks, prompts x KV heads).
 //   pass 1  M = 128 query rows, N = 256 candidates; thread = query row; the two epilogue groups
 //           take 128 candidates each and their (reference max, sum) pairs are merged at the end.
 //   pass 2  the same MMAs (an N = 128 instruction would occupy the tensor pipe almost as long for half
@@ -27,7 +33,7 @@ namespace {
 
 using namespace umma;
 
-constexpr int NTHREADS = 320, MAXNS = 6, STAGE_B = 32768, QH_B = 16384, MAXH = 9;
+constexpr int NTHREADS = 320, MAXNS = 6, MAXNS_PAIR = 8, STAGE_B = 32768, QH_B = 16384, MAXH = 9;
 
 struct WideArgs {
   int Hq, Hkv, g, Lo, Ls, Lr, R, NH, RB;
@@ -39,31 +45,40 @@ struct WideArgs {
   uint32_t* status;
 };
 
-template <int PASS>
+// PAIR: two CTAs with adjacent row blocks form a cluster and share every key tile: each loads one
+// half of the tile's rows and the even CTA issues M = 256 instructions over both (cta_group::2).
+template <int PASS, bool PAIR>
 __global__ void __launch_bounds__(NTHREADS, 1)
 score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tmap_q,
                        const __grid_constant__ CUtensorMap tmap_k) {
   constexpr int TNP = 256;                                    // candidates per tile
+  constexpr int STG = PAIR ? STAGE_B / 2 : STAGE_B;           // bytes of a key slab held by this CTA
+  const uint32_t crank = PAIR ? cluster_rank() : 0u;          // 0: issues the pair's MMAs
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int NH = a.NH, NS = a.NS;
   unsigned char* Qs = smem;                                   // [NH][128 rows][128 B]
-  unsigned char* Ks = Qs + NH * QH_B;                         // [NS][up to 256 rows][128 B]
-  float* mu_s = reinterpret_cast<float*>(Ks + NS * STAGE_B);  // [128] pass 2: m_i + log2 l_i of this row block
+  unsigned char* Ks = Qs + NH * QH_B;                         // [NS][256 rows (pair: this CTA's 128)][128 B]
+  float* mu_s = reinterpret_cast<float*>(Ks + NS * STG);      // [128] pass 2: m_i + log2 l_i of this row block
   float2* xch = reinterpret_cast<float2*>(mu_s + 128);        // [128] exchange between the epilogue groups
   float* red = reinterpret_cast<float*>(xch + 128);           // [2 tile parities][2 groups][4 warps][128] pass-2 column partials
-  uint64_t* bars = reinterpret_cast<uint64_t*>(red + 2 * 2 * 4 * 128);   // full[NS] empty[NS] tfull[2] tempty[2] qfull
+  // full[NS] empty[NS] tfull[2] tempty[2] qfull; in a pair the issuing CTA's full and qfull barriers count
+  // the bytes of both CTAs' loads
+  uint64_t* bars = reinterpret_cast<uint64_t*>(red + 2 * 2 * 4 * 128);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NS + 5);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int rb = blockIdx.y, z = blockIdx.z, si = z / a.Hkv, kvh = z % a.Hkv;
+  // a pair is two consecutive CTAs along x: grid = (2 x splits, row blocks / 2, prompts x KV heads) then, so that
+  // CTAs that run at the same time still work on different candidate ranges
+  const int rb = PAIR ? 2 * blockIdx.y + (blockIdx.x & 1) : blockIdx.y, split = PAIR ? blockIdx.x >> 1 : blockIdx.x;
+  const int z = blockIdx.z, si = z / a.Hkv, kvh = z % a.Hkv;
   const int seq = a.b.seq_of_score[si];
   const int Le = a.b.len[seq] - a.Ls - a.Lr;
   const int R = a.R;
   const int ntiles = (Le + TNP - 1) / TNP;
-  const int t0 = (int)((long long)ntiles * blockIdx.x / a.buf.nsplit);
-  const int t1 = (int)((long long)ntiles * (blockIdx.x + 1) / a.buf.nsplit);
+  const int t0 = (int)((long long)ntiles * split / a.buf.nsplit);
+  const int t1 = (int)((long long)ntiles * (split + 1) / a.buf.nsplit);
   const int nt = t1 - t0;
 
   const uint32_t bar0 = smem_u32(bars);
@@ -72,11 +87,12 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
   auto tfull_bar = [&](int b) { return bar0 + 8 * (2 * NS + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8 * (2 * NS + 2 + b); };
   const uint32_t qfull_bar = bar0 + 8 * (2 * NS + 4);
+  auto bwait = [&](uint32_t bar, unsigned parity) { return mbar_wait(bar, parity, abort_flag); };
 
   if (tid == 0) {
     *abort_flag = 0;
     for (int s = 0; s < NS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), PAIR ? 16 : 8); }
     mbar_init(qfull_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -95,11 +111,17 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
     mu_s[tid] = mu;
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {                                                // both CTAs of the pair, same warp, same slot
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   fence_before();
   __syncthreads();
+  if (PAIR) cluster_barrier();                                 // the other CTA's barriers exist before anything arrives on them
   fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int eg = warp >= 2 ? (warp - 2) >> 2 : 0;             // epilogue group
@@ -108,41 +130,77 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
+    // (stage index and phase are carried along: the issuing threads' instruction chains bound these
+    // kernels, so neither loop divides, and the descriptors' constant parts are built once)
     if (lane == 0 && nt > 0) {
       const int row0 = ((a.b.first_seq + seq) * a.Hq + kvh * a.g) * a.Lo + rb * 128;
-      mbar_expect_tx(qfull_bar, (unsigned)NH * QH_B);
-      for (int h = 0; h < NH; ++h) tma_load_2d(smem_u32(Qs) + h * QH_B, &tmap_q, h * 64, row0, qfull_bar);
-      const int tok0 = a.b.tok_off[seq] + a.Ls;
+      int tok = a.b.tok_off[seq] + a.Ls + t0 * TNP + (PAIR ? (int)crank * 128 : 0);
       bool ok = true;
-      for (int it = 0; it < nt && ok; ++it)
+      // in a pair both CTAs' bytes are counted on the issuing CTA's barriers, which that CTA arms for both
+      const uint32_t lead = PAIR ? map_to_rank(bar0, 0) - bar0 : 0u;   // offset to the same barrier in the issuing CTA
+      if (PAIR) {
+        if (crank == 0) mbar_expect_tx(qfull_bar, 2u * (unsigned)NH * QH_B);
+        for (int h = 0; h < NH; ++h) tma_load_2d_pair(smem_u32(Qs) + h * QH_B, &tmap_q, h * 64, row0, qfull_bar + lead);
+      } else {
+        mbar_expect_tx(qfull_bar, (unsigned)NH * QH_B);
+        for (int h = 0; h < NH; ++h) tma_load_2d(smem_u32(Qs) + h * QH_B, &tmap_q, h * 64, row0, qfull_bar);
+      }
+      int s = 0;
+      unsigned ph = 1u;                                        // parity of the "stage is free" phase awaited next
+      uint32_t dst = smem_u32(Ks), fb = full_bar(0);
+      for (int it = 0; it < nt && ok; ++it, tok += TNP)
         for (int h = 0; h < NH; ++h) {
-          const int q = it * NH + h, s = q % NS;
-          if (!mbar_wait(empty_bar(s), ((unsigned)(q / NS) & 1u) ^ 1u, abort_flag)) { *abort_flag = 1; ok = false; break; }
-          mbar_expect_tx(full_bar(s), (unsigned)TNP * 128u);
-          tma_load_3d(smem_u32(Ks) + s * STAGE_B, &tmap_k, h * 64, kvh, tok0 + (t0 + it) * TNP, full_bar(s));
+          if (!bwait(fb + 8 * NS, ph)) { *abort_flag = 1; ok = false; break; }
+          if (PAIR) {
+            if (crank == 0) mbar_expect_tx(fb, 2u * (unsigned)STG);
+            tma_load_3d_pair(dst, &tmap_k, h * 64, kvh, tok, fb + lead);
+          } else {
+            mbar_expect_tx(fb, (unsigned)STG);
+            tma_load_3d(dst, &tmap_k, h * 64, kvh, tok, fb);
+          }
+          if (++s == NS) { s = 0; ph ^= 1u; dst = smem_u32(Ks); fb = full_bar(0); }
+          else { dst += STG; fb += 8; }
         }
+      if (PAIR) {
+        // the issuing CTA's commits arrive on this CTA's barriers asynchronously: take the last ones in
+        // before leaving, so that none lands in a CTA that has exited
+        const int total = nt * NH;
+        for (int q = total > NS ? total - NS : 0; q < total && ok; ++q)
+          ok = bwait(empty_bar(q % NS), (unsigned)(q / NS) & 1u);
+        if (!ok) *abort_flag = 1;
+      }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0 && nt > 0) {
-      const uint32_t idesc = idesc_bf16(128, 256);
+    if (lane == 0 && nt > 0 && crank == 0) {
+      const uint32_t idesc = idesc_bf16(PAIR ? 256 : 128, 256);
+      const uint64_t qdesc0 = smem_desc(smem_u32(Qs)), kdesc0 = smem_desc(smem_u32(Ks));
+      const uint32_t peer = PAIR ? map_to_rank(bar0, 1) - bar0 : 0u;   // offset to the same barrier in the other CTA
       bool ok = mbar_wait(qfull_bar, 0u, abort_flag);
+      int s = 0;
+      unsigned ph = 0u;                                        // parity of the "slab has landed" phase awaited next
+      uint64_t kdesc = kdesc0;
+      uint32_t fb = full_bar(0);
       for (int it = 0; it < nt && ok; ++it) {
         const int b = it & 1;
-        ok = mbar_wait(tempty_bar(b), ((unsigned)(it / 2) & 1u) ^ 1u, abort_flag);
-        for (int h = 0; h < NH && ok; ++h) {
-          const int q = it * NH + h, s = q % NS;
-          ok = mbar_wait(full_bar(s), (unsigned)(q / NS) & 1u, abort_flag);
+        ok = bwait(tempty_bar(b), ((unsigned)(it >> 1) & 1u) ^ 1u);
+        fence_after();
+        uint64_t qdesc = qdesc0;
+        const uint32_t acc = tmem_base + b * 256;
+        for (int h = 0; h < NH && ok; ++h, qdesc += QH_B >> 4) {
+          ok = mbar_wait(fb, ph, abort_flag);
           if (!ok) break;
-          fence_after();
-          const uint32_t kst = smem_u32(Ks) + s * STAGE_B, qst = smem_u32(Qs) + h * QH_B;
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            mma_bf16(tmem_base + b * 256, smem_desc(qst + ks * 32), smem_desc(kst + ks * 32), idesc, (h | ks) != 0);
-          }
-          mma_commit(empty_bar(s));                            // slab may be refilled once these MMAs have read it
+          mma_slab4<PAIR>(acc, qdesc, kdesc, idesc, h != 0);
+          // the slab may be refilled once these MMAs have read it (in both CTAs of a pair)
+          if (PAIR) { mma_commit_pair(fb + 8 * NS); mma_commit_pair(fb + 8 * NS + peer); }
+          else mma_commit(fb + 8 * NS);
+          if (++s == NS) { s = 0; ph ^= 1u; kdesc = kdesc0; fb = full_bar(0); }
+          else { kdesc += STG >> 4; fb += 8; }
         }
-        if (ok) mma_commit(tfull_bar(b));                      // accumulator buffer complete
+        if (ok) {                                              // accumulator buffer complete
+          if (PAIR) { mma_commit_pair(tfull_bar(b)); mma_commit_pair(tfull_bar(b) + peer); }
+          else mma_commit(tfull_bar(b));
+        }
       }
       if (!ok) *abort_flag = 1;
     }
@@ -150,10 +208,14 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
     // ---------------- epilogue warps ----------------
     const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
     bool ok = true;
+    auto release_acc = [&](int b) {                            // the accumulator buffer may be overwritten
+      if (PAIR && crank != 0) mbar_arrive_remote(map_to_rank(tempty_bar(b), 0));
+      else mbar_arrive(tempty_bar(b));
+    };
     const float neg_mu = PASS == 2 ? -mu_s[lrow] : 0.f;        // pass 2: this thread's row offset (-inf for a padding row)
     for (int it = 0; it < nt; ++it) {
       const int b = it & 1;
-      const bool landed = mbar_wait(tfull_bar(b), (unsigned)(it / 2) & 1u, abort_flag);
+      const bool landed = bwait(tfull_bar(b), (unsigned)(it / 2) & 1u);
       if (!landed) {
         *abort_flag = 1;
         ok = false;
@@ -269,7 +331,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
         }
         fence_before();                                        // the accumulator buffer is free again
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(b));
+        if (lane == 0) release_acc(b);
 #pragma unroll
         for (int bit = 16, width = 64; bit >= 1; bit >>= 1, width >>= 1) {
           const bool upper = (lane & bit) != 0;
@@ -298,7 +360,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
       if (PASS == 1) {
         fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(b));
+        if (lane == 0) release_acc(b);
       }
       if (!ok) break;
     }
@@ -312,10 +374,13 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
   if (PASS == 1 && warp >= 2 && eg == 0 && rb * 128 + lrow < R) {   // the two groups took different candidates of each tile
     const float2 o = xch[lrow];
     merge_ml(m_ref, l_sum, o.x, o.y);
-    a.buf.part_stats[((long long)z * a.buf.nsplit + blockIdx.x) * R + rb * 128 + lrow] = make_float2(m_ref, l_sum);
+    a.buf.part_stats[((long long)z * a.buf.nsplit + split) * R + rb * 128 + lrow] = make_float2(m_ref, l_sum);
   }
-  if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  if (PAIR) cluster_barrier();                                 // nobody leaves while the other CTA may still signal it
+  if (warp == 0) {
+    if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
   if (tid == 0 && *abort_flag && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
 }
 
@@ -331,18 +396,39 @@ __global__ void score_rowblock_reduce_kernel(const float* __restrict__ cpart, fl
   C[(long long)z * c_stride + j] = s;
 }
 
-size_t wide_smem_bytes(int NH, int NS) {
-  return (size_t)NH * QH_B + NS * STAGE_B + 128 * sizeof(float) + 128 * sizeof(float2) + 2 * 2 * 4 * 128 * sizeof(float) +
-         (2 * NS + 5) * 8 + 16 + 1024;
+size_t wide_smem_bytes(int NH, int NS, bool pair) {
+  return (size_t)NH * QH_B + NS * (pair ? STAGE_B / 2 : STAGE_B) + 128 * sizeof(float) + 128 * sizeof(float2) +
+         2 * 2 * 4 * 128 * sizeof(float) + (2 * NS + 5) * 8 + 16 + 1024;
 }
 
 // Option SNAP_OPT_WIDE_STAGES caps the ring depth (tuning aid).
-int wide_stages(int NH) {
-  int ns = MAXNS;
+int wide_stages(int NH, bool pair) {
+  int ns = pair ? MAXNS_PAIR : MAXNS;
   if (const int v = option(SNAP_OPT_WIDE_STAGES))
     if (v >= 2 && v < ns) ns = v;
-  while (ns > 2 && wide_smem_bytes(NH, ns) > 227u * 1024u) --ns;
+  while (ns > 2 && wide_smem_bytes(NH, ns, pair) > 227u * 1024u) --ns;
   return ns;
+}
+
+// CTA pairs need an even number of row blocks; option SNAP_OPT_SCORE_KERNEL = 3 keeps single CTAs.
+bool wide_pairs(int RB) { return RB % 2 == 0 && option(SNAP_OPT_SCORE_KERNEL) != 3; }
+
+template <int PASS, bool PAIR>
+cudaError_t launch_wide(dim3 grid, size_t smem, cudaStream_t st, const WideArgs& a, const CUtensorMap& tq, const CUtensorMap& tk) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = grid;
+  lc.blockDim = dim3(NTHREADS);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  count_launch();
+  return cudaLaunchKernelEx(&lc, score_umma_wide_kernel<PASS, PAIR>, a, tq, tk);
 }
 
 }  // namespace
@@ -375,7 +461,9 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   if (!enc) return cudaErrorNotSupported;
   WideArgs a;
   a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Lo = s.Lo; a.Ls = s.Ls; a.Lr = s.Lr; a.R = s.g * s.Lo;
-  a.NH = s.d_qk / 64; a.RB = (a.R + 127) / 128; a.NS = wide_stages(a.NH);
+  a.NH = s.d_qk / 64; a.RB = (a.R + 127) / 128;
+  const bool pair = wide_pairs(a.RB);
+  a.NS = wide_stages(a.NH, pair);
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.b = b; a.buf = buf; a.cpart = cpart; a.status = status;
 
@@ -395,28 +483,33 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   const long long head_stride = src.k_head_stride >= s.d_qk ? src.k_head_stride : s.d_qk;
   const cuuint64_t kdims[3] = {(cuuint64_t)s.d_qk, (cuuint64_t)s.Hkv, (cuuint64_t)tokens};
   const cuuint64_t kstrides[2] = {(cuuint64_t)head_stride * 2, (cuuint64_t)src.k_tok_stride * 2};
-  const cuuint32_t kbox[3] = {64, 1, 256};                     // one 64-dim slab of a 256-candidate tile
+  const cuuint32_t kbox[3] = {64, 1, pair ? 128u : 256u};      // one 64-dim slab of a 256-candidate tile (pair: this CTA's half)
   if (enc(&tk1, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(src.k), kdims, kstrides, kbox, estr3,
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
-  const size_t smem = wide_smem_bytes(a.NH, a.NS);
-  static SmemLimit limit1 = {}, limit2 = {};
-  if (cudaError_t e = ensure_dyn_smem(score_umma_wide_kernel<1>, smem, limit1)) return e;
-  if (cudaError_t e = ensure_dyn_smem(score_umma_wide_kernel<2>, smem, limit2)) return e;
+  const size_t smem = wide_smem_bytes(a.NH, a.NS, pair);
+  static SmemLimit limit1 = {}, limit2 = {}, limit1p = {}, limit2p = {};
+  if (pair) {
+    if (cudaError_t e = ensure_dyn_smem(score_umma_wide_kernel<1, true>, smem, limit1p)) return e;
+    if (cudaError_t e = ensure_dyn_smem(score_umma_wide_kernel<2, true>, smem, limit2p)) return e;
+  } else {
+    if (cudaError_t e = ensure_dyn_smem(score_umma_wide_kernel<1, false>, smem, limit1)) return e;
+    if (cudaError_t e = ensure_dyn_smem(score_umma_wide_kernel<2, false>, smem, limit2)) return e;
+  }
   const int nz = b.n_scored * s.Hkv;
   int max_le = 0;
   for (int i = 0; i < b.n; ++i)
     if (b.score_idx[i] >= 0) max_le = max_le > b.len[i] - s.Ls - s.Lr ? max_le : b.len[i] - s.Ls - s.Lr;
-  dim3 grid(buf.nsplit, a.RB, nz);
+  const dim3 grid = pair ? dim3(2 * buf.nsplit, a.RB / 2, nz) : dim3(buf.nsplit, a.RB, nz);
   if (!buf.ext_mu) {                                          // Eq. 4's normalisers: pass 1, unless the caller has them
-    score_umma_wide_kernel<1><<<grid, NTHREADS, smem, st>>>(a, tq, tk1);
-    count_launch();
-    cudaError_t e = launch_score_combine_log2(buf, nz, a.R, st);
+    cudaError_t e = pair ? launch_wide<1, true>(grid, smem, st, a, tq, tk1) : launch_wide<1, false>(grid, smem, st, a, tq, tk1);
+    if (e != cudaSuccess) return e;
+    e = launch_score_combine_log2(buf, nz, a.R, st);
     if (e != cudaSuccess) return e;
   }
-  score_umma_wide_kernel<2><<<grid, NTHREADS, smem, st>>>(a, tq, tk1);
-  count_launch();
+  if (cudaError_t e = pair ? launch_wide<2, true>(grid, smem, st, a, tq, tk1) : launch_wide<2, false>(grid, smem, st, a, tq, tk1))
+    return e;
   score_rowblock_reduce_kernel<<<dim3((max_le + 255) / 256, nz), 256, 0, st>>>(cpart, buf.C, a.RB, buf.c_stride, b,
                                                                             s.Hkv, s.Ls, s.Lr);
   count_launch();
