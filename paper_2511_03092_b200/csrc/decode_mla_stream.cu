@@ -128,22 +128,26 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
       mbar_expect_tx(qfull_bar, (unsigned)NSLAB * QSLAB_B);
       for (int h = 0; h < NSLAB; ++h)
         tma_load_3d(smem_u32(Qs) + h * QSLAB_B, &tmap_q, h * 64, hb * HBLK, i, qfull_bar);
-      int q = 0;                                               // stages issued so far
+      int s = 0;                                               // stage filled next
+      unsigned ph = 1u;                                        // parity of its "free" phase
+      uint32_t fb = full_bar(0), dst = smem_u32(Rs);
       bool ok = true;
       auto stage_wait = [&]() -> bool {
-        const int s = q % NSTG;
-        if (!mbar_wait(empty_bar(s), ((unsigned)(q / NSTG) & 1u) ^ 1u, abort_flag)) { *abort_flag = 1; return false; }
-        mbar_expect_tx(full_bar(s), (unsigned)STAGE_B);
+        if (!mbar_wait(fb + 8 * NSTG, ph, abort_flag)) { *abort_flag = 1; return false; }
+        mbar_expect_tx(fb, (unsigned)STAGE_B);
         return true;
+      };
+      auto advance = [&]() {
+        if (++s == NSTG) { s = 0; ph ^= 1u; fb = full_bar(0); dst = smem_u32(Rs); }
+        else { fb += 8; dst += STAGE_B; }
       };
       auto load_k = [&](int it) {                              // nine key slabs of tile it
         const TileRows tr = tile_rows(g0 + it, nA, n_low, Lsr, n_top);
         for (int h = 0; h < NSLAB && ok; ++h) {
           ok = stage_wait();
           if (!ok) break;
-          const int s = q % NSTG;
-          tma_load_3d(smem_u32(Rs) + s * STAGE_B, &tmap_k, h * 64, tr.row0, slot, full_bar(s));
-          ++q;
+          tma_load_3d(dst, &tmap_k, h * 64, tr.row0, slot, fb);
+          advance();
         }
       };
       auto load_v = [&](int it) {                              // four value chunks of tile it (this CTA's 256 dims)
@@ -151,10 +155,9 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
         for (int c = 0; c < NVCH && ok; ++c) {
           ok = stage_wait();
           if (!ok) break;
-          const int s = q % NSTG;
           for (int j = 0; j < DVH / 64; ++j)
-            tma_load_3d(smem_u32(Rs) + s * STAGE_B + j * VSUB_B, &tmap_v, hd * DVH + j * 64, tr.row0 + c * VROWS, slot, full_bar(s));
-          ++q;
+            tma_load_3d(dst + j * VSUB_B, &tmap_v, hd * DVH + j * 64, tr.row0 + c * VROWS, slot, fb);
+          advance();
         }
       };
       load_k(0);
@@ -168,17 +171,24 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
     if (nt > 0) {
       const uint32_t leader = lane == 0;
       const uint32_t idesc_s = idesc_f16(128, TR, false), idesc_pv = idesc_f16(128, DVH, true);
-      const uint64_t qd0 = smem_desc(smem_u32(Qs));
-      int q = 0;                                               // stages consumed so far
+      const uint64_t qd0 = smem_desc(smem_u32(Qs)), kd0 = smem_desc(smem_u32(Rs)), vd0 = smem_desc_mn(smem_u32(Rs), VSUB_B);
+      // The stage index, its phase and its barrier are carried along and the descriptors advance by
+      // additions: this warp's instruction chain per stage is what the tensor pipe waits for.
+      int s = 0;                                               // stage consumed next
+      unsigned ph = 0u;                                        // parity of its "landed" phase
+      uint32_t fb = full_bar(0);
+      auto advance = [&]() {
+        if (++s == NSTG) { s = 0; ph ^= 1u; fb = full_bar(0); }
+        else fb += 8;
+      };
       bool ok = wait_warp(qfull_bar, 0u, abort_flag);
       fence_after();
       auto issue_s = [&](int it) -> bool {                    // S[it & 1] = Q K(it)^T, one key slab per stage
         const uint32_t sd = tmem_base + COL_S + (it & 1) * TR;
+        uint64_t qd = qd0;
 #pragma unroll 1
-        for (int h = 0; h < NSLAB; ++h) {
-          const int s = q % NSTG;
-          if (!wait_warp(full_bar(s), (unsigned)(q / NSTG) & 1u, abort_flag)) return false;
-          fence_after();
+        for (int h = 0; h < NSLAB; ++h, qd += QSLAB_B >> 4) {
+          if (!wait_warp(fb, ph, abort_flag)) return false;
           if (it == it_new) {
             // the new token's row: eight 16-byte chunks of this 64-dim slab, at their swizzled places
             if (lane < 8)
@@ -186,12 +196,9 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
           }
-          const uint64_t kd = smem_desc(smem_u32(Rs) + s * STAGE_B), qd = qd0 + (uint64_t)((h * QSLAB_B) >> 4);
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            mma_ss_pred(sd, qd + (uint64_t)(ks * 2), kd + (uint64_t)(ks * 2), idesc_s, (h | ks) != 0, leader);
-          commit_pred(empty_bar(s), leader);
-          ++q;
+          mma_ss_slab4_pred(sd, qd, kd0 + (uint64_t)(s * (STAGE_B >> 4)), idesc_s, h != 0, leader);
+          commit_pred(fb + 8 * NSTG, leader);
+          advance();
         }
         commit_pred(sfull_bar(it & 1), leader);
         return true;
@@ -208,11 +215,8 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
         const int tile_nrows = ptr_.row_end - ptr_.row0;
 #pragma unroll 1
         for (int c = 0; c < NVCH; ++c) {                      // O += P(it) V(it), one 32-row value chunk per stage
-          const int s = q % NSTG;
-          ok = wait_warp(full_bar(s), (unsigned)(q / NSTG) & 1u, abort_flag);
+          ok = wait_warp(fb, ph, abort_flag);
           if (!ok) break;
-          fence_after();
-          const uint32_t vst = smem_u32(Rs) + s * STAGE_B;
           if (tile_nrows < (c + 1) * VROWS) {
             // ragged chunk: rows past the end may hold anything (memory the caller never wrote), and a
             // zero probability does not silence a NaN in V: clear them before the tensor core reads
@@ -232,12 +236,11 @@ decode_mla_stream_kernel(const SArgs a, const __grid_constant__ CUtensorMap tmap
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
           }
-#pragma unroll
-          for (int ks = 0; ks < VROWS / 16; ++ks)
-            mma_ts_pred(tmem_base + COL_O, pa + 8 * (c * (VROWS / 16) + ks), smem_desc_mn(vst + ks * 16 * 128, VSUB_B),
-                        idesc_pv, (it | c | ks) != 0, leader);
-          commit_pred(empty_bar(s), leader);
-          ++q;
+          static_assert(VROWS == 32, "two 16-row steps per value chunk");
+          mma_ts_2_pred(tmem_base + COL_O, pa + 16 * c, vd0 + (uint64_t)(s * (STAGE_B >> 4)), (16 * 128) >> 4, idesc_pv, (it | c) != 0,
+                        leader);
+          commit_pred(fb + 8 * NSTG, leader);
+          advance();
         }
         if (ok) commit_pred(pvdone_bar(b), leader);
       }

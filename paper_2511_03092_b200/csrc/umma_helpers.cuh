@@ -267,6 +267,33 @@ __device__ __forceinline__ void commit_pred(uint32_t bar, uint32_t leader) {
       "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
       ::"r"(bar), "r"(leader) : "memory");
 }
+// Instruction groups for a converged warp whose lane `leader` issues: the four 16-wide steps of a
+// 64-element slab with both operands in shared memory, and two 16-row steps with the A operand in
+// tensor memory (8 columns of bf16 pairs per step) and B advancing by `b_step` (units of 16 bytes).
+// Only the first instruction of a group may start a new accumulation (acc_first = 0).
+__device__ __forceinline__ void mma_ss_slab4_pred(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t acc_first, uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred p, t, q;\n\t.reg .b64 a1, b1, a2, b2, a3, b3;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 t, %3, %3;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+      "add.s64 a1, %1, 2;\n\tadd.s64 b1, %2, 2;\n\tadd.s64 a2, %1, 4;\n\tadd.s64 b2, %2, 4;\n\t"
+      "add.s64 a3, %1, 6;\n\tadd.s64 b3, %2, 6;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %3, t;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %3, t;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %3, t;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc_first), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void mma_ts_2_pred(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t b_step, uint32_t idesc,
+                                              uint32_t acc_first, uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred p, t, q;\n\t.reg .b64 b1, st;\n\t.reg .b32 a1;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 t, %4, %4;\n\tsetp.ne.b32 q, %6, 0;\n\t"
+      "cvt.u64.u32 st, %3;\n\tadd.s64 b1, %2, st;\n\tadd.u32 a1, %1, 8;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %4, p;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a1], b1, %4, t;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(b_step), "r"(idesc), "r"(acc_first), "r"(leader) : "memory");
+}
 // 32 lanes x 16 consecutive columns, registers to tensor memory
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
