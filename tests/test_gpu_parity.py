@@ -308,6 +308,31 @@ def test_late_outlier_logits_latent_shape():
         assert pos in idx[0][0]
 
 
+@pytest.mark.parametrize("hq,hkv,lo,d", [(128, 1, 8, 576), (64, 1, 8, 576), (32, 2, 32, 320), (24, 1, 16, 192)],
+                         ids=["latent_8_row_blocks", "latent_4_row_blocks", "gqa_320_wide_4_row_blocks", "odd_3_row_blocks"])
+def test_wide_score_kernel_with_cta_pairs_and_with_single_ctas(snap_option, hq, hkv, lo, d):
+    """The wide-row score kernel pairs the CTAs of adjacent row blocks when their number is even (each
+    loads half of every key tile, M = 256 instructions over both) and keeps single CTAs when it is
+    odd or when asked to: both forms against the oracle on one ragged call (a partly filled last
+    candidate tile, a prompt shorter than one tile of candidates), and the same selection from both."""
+    latent = d == 576
+    wl = synth.Workload("wide_pairs", hq, hkv, d, 512 if latent else d, "bf16", 3, 40, 96, lo, 5, batch=1,
+                        prompt_len=(3000, 3000), decode_steps=1, salience="planted", n_planted=8,
+                        v_aliases_k=latent, softmax_scale=2.0 ** -0.5 if latent else None)
+    prompts = [synth.make_prompt(wl, L, seed=61 + i) for i, L in enumerate([3000, 1777, 150])]
+    seqs = [H.oracle_compress(wl, p) for p in prompts]
+    picked = []
+    for single in (0, 3):
+        snap_option(B.SNAP_OPT_SCORE_KERNEL, single)
+        layer = H.GpuLayer(wl, max_seqs=3)
+        idx = layer.compress(prompts, [2, 0, 1])
+        assert layer.status() == 0
+        for i, seq in enumerate(seqs):
+            H.check_selection(idx[i], seq, wl)
+        picked.append(idx)
+    assert (picked[0] == picked[1]).all()
+
+
 @pytest.mark.parametrize("wl,lengths", [(SMALL_BF16, [3, 30, 4 + 5 * 48]), (SMALL_MLA, [2, 3 + 2 * 40])])
 def test_concat_update_baseline_matches_oracle(wl, lengths):
     """The slice-and-concatenate update (position-ordered window, new cache every step) gives
