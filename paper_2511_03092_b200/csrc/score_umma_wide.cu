@@ -17,11 +17,14 @@
 // otherwise (candidate splits, row blocks, prompts x KV heads).
 //   pass 1  M = 128 query rows, N = 256 candidates; thread = query row; the two epilogue groups
 //           take 128 candidates each and their (reference max, sum) pairs are merged at the end.
-//   pass 2  the same MMAs (an N = 128 instruction would occupy the tensor pipe almost as long for half
-//           the work); thread = query row scales its row by exp2(-(m_i + log2 l_i)) and the 128 rows
-//           are summed per candidate with a transposing shuffle reduction and one shared-memory
-//           step; the per-row-block partial column sums go to scratch and a small kernel adds the
-//           row blocks in a fixed order (deterministic, no atomics).
+//   pass 2  single CTAs: the same MMAs (an N = 128 instruction would occupy the tensor pipe almost as long
+//           for half the work); thread = query row scales its row by exp2(-(m_i + log2 l_i)) and the 128
+//           rows are summed per candidate with a transposing shuffle reduction and one shared-memory step.
+//           Pairs: the operands are swapped -- M = 256 candidates (each CTA's own 128 of the tile), N = the
+//           256 window rows of the pair's two row blocks -- so thread = candidate sums its own columns
+//           and only the two epilogue groups' halves meet in shared memory.
+//           Either way the per-row-group partial column sums go to scratch and a small kernel adds the
+//           row groups in a fixed order (deterministic, no atomics).
 // Every mbarrier wait is bounded; a wait that runs out raises SNAP_DEV_WAIT_TIMEOUT.
 #include <cstdlib>
 
@@ -37,6 +40,7 @@ constexpr int NTHREADS = 320, MAXNS = 6, MAXNS_PAIR = 8, STAGE_B = 32768, QH_B =
 
 struct WideArgs {
   int Hq, Hkv, g, Lo, Ls, Lr, R, NH, RB;
+  int RBC;               // row groups with a partial column sum each: RB, or RB / 2 when CTAs are paired
   int NS;                // key-slab stages: as many as fit beside the query block (2..MAXNS)
   float scale_log2;
   SeqBatch b;
@@ -96,9 +100,10 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
     mbar_init(qfull_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (PASS == 2 && tid < 128) {
+  if (PASS == 2 && tid < (PAIR ? 256 : 128)) {
     // rows past the group's last one (a partly filled row block) get an infinite offset: weight 0
-    const int row = rb * 128 + tid;
+    // (a pair keeps the offsets of both its row blocks, negated, in the region `red`)
+    const int row = (PAIR ? (rb & ~1) : rb) * 128 + tid;
     float mu = INFINITY;
     if (row < a.R) {
       if (a.buf.ext_mu) {                                      // [prompt][Hq][Lo]: a KV head's rows are consecutive
@@ -108,7 +113,8 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
         mu = st.x - log2f(st.y);
       }
     }
-    mu_s[tid] = mu;
+    if (PAIR) red[tid] = -mu;
+    else mu_s[tid] = mu;
   }
   if (warp == 0) {
     if (PAIR) {                                                // both CTAs of the pair, same warp, same slot
@@ -190,7 +196,8 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
         for (int h = 0; h < NH && ok; ++h, qdesc += QH_B >> 4) {
           ok = mbar_wait(fb, ph, abort_flag);
           if (!ok) break;
-          mma_slab4<PAIR>(acc, qdesc, kdesc, idesc, h != 0);
+          if (PASS == 2 && PAIR) mma_slab4<PAIR>(acc, kdesc, qdesc, idesc, h != 0);   // candidates on M, window rows on N
+          else mma_slab4<PAIR>(acc, qdesc, kdesc, idesc, h != 0);
           // the slab may be refilled once these MMAs have read it (in both CTAs of a pair)
           if (PAIR) { mma_commit_pair(fb + 8 * NS); mma_commit_pair(fb + 8 * NS + peer); }
           else mma_commit(fb + 8 * NS);
@@ -212,7 +219,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
       if (PAIR && crank != 0) mbar_arrive_remote(map_to_rank(tempty_bar(b), 0));
       else mbar_arrive(tempty_bar(b));
     };
-    const float neg_mu = PASS == 2 ? -mu_s[lrow] : 0.f;        // pass 2: this thread's row offset (-inf for a padding row)
+    const float neg_mu = PASS == 2 && !PAIR ? -mu_s[lrow] : 0.f;   // pass 2, single CTAs: this thread's row offset (-inf for a padding row)
     for (int it = 0; it < nt; ++it) {
       const int b = it & 1;
       const bool landed = bwait(tfull_bar(b), (unsigned)(it / 2) & 1u);
@@ -296,6 +303,56 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
           if (mn != -INFINITY) sum = s2;
         }
         l_sum += sum;
+      } else if (PAIR) {
+        // Pair: the operands are swapped, so thread = candidate (this CTA's 128 of the tile's 256) and the columns are
+        // the 256 window rows of the pair's two row blocks, one block per epilogue group.  The weights
+        // exp2(s - m_i - log2 l_i) are summed along the thread's own columns: no exchange between threads, only
+        // the two groups' halves are added through shared memory.
+        const uint32_t col0 = lane_addr + b * 256 + eg * 128;
+        const int cand = (t0 + it) * TNP + (int)crank * 128 + lrow;
+        const float* nmu = red + eg * 128;                       // -(m_i + log2 l_i) of this group's rows
+        const u64 sc2 = pack2(a.scale_log2, a.scale_log2);
+        u64 acc2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+        if (landed) {
+          tmem_ld16_issue(col0, ra);
+#pragma unroll
+          for (int c = 0; c < 8; c += 2) {
+            tmem_ld16_wait(ra);
+            tmem_ld16_issue(col0 + 16 * (c + 1), rb16);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const ulonglong2 m4 = *reinterpret_cast<const ulonglong2*>(nmu + 16 * c + 4 * i);   // the same address in every lane
+              const u64 x0 = fma2(pack2(__uint_as_float(ra[4 * i]), __uint_as_float(ra[4 * i + 1])), sc2, m4.x);
+              const u64 x1 = fma2(pack2(__uint_as_float(ra[4 * i + 2]), __uint_as_float(ra[4 * i + 3])), sc2, m4.y);
+              acc2[0] = add2(acc2[0], pack2(fast_exp2(lo2(x0)), fast_exp2(hi2(x0))));
+              acc2[1] = add2(acc2[1], pack2(fast_exp2(lo2(x1)), fast_exp2(hi2(x1))));
+            }
+            tmem_ld16_wait(rb16);
+            if (c + 2 < 8) tmem_ld16_issue(col0 + 16 * (c + 2), ra);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const ulonglong2 m4 = *reinterpret_cast<const ulonglong2*>(nmu + 16 * (c + 1) + 4 * i);
+              const u64 x0 = fma2(pack2(__uint_as_float(rb16[4 * i]), __uint_as_float(rb16[4 * i + 1])), sc2, m4.x);
+              const u64 x1 = fma2(pack2(__uint_as_float(rb16[4 * i + 2]), __uint_as_float(rb16[4 * i + 3])), sc2, m4.y);
+              acc2[0] = add2(acc2[0], pack2(fast_exp2(lo2(x0)), fast_exp2(hi2(x0))));
+              acc2[1] = add2(acc2[1], pack2(fast_exp2(lo2(x1)), fast_exp2(hi2(x1))));
+            }
+          }
+        }
+        fence_before();                                        // the accumulator buffer is free again
+        __syncwarp();
+        if (lane == 0) release_acc(b);
+        const float sum = (lo2(acc2[0]) + hi2(acc2[0])) + (lo2(acc2[1]) + hi2(acc2[1]));
+        float* gx = reinterpret_cast<float*>(xch) + (it & 1) * 128;   // double-buffered by tile parity: one barrier per tile
+        if (eg == 1) gx[lrow] = sum;
+        unsigned stop;                                         // barrier over both groups + agreement on giving up
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+            "bar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(stop) : "r"((unsigned)(!landed || *abort_flag)) : "memory");
+        if (eg == 0 && !stop && cand < Le)
+          a.cpart[((long long)z * a.RBC + (rb >> 1)) * a.buf.c_stride + cand] = sum + gx[lrow];
+        if (stop) { *abort_flag = 1; ok = false; }
       } else {
         // thread = query row; this group's 128 candidates of the tile.  The weights exp2(s - m_i - log2 l_i)
         // are summed over the 128 rows of the block: a transposing shuffle reduction inside each warp (every
@@ -353,7 +410,7 @@ score_umma_wide_kernel(const WideArgs a, const __grid_constant__ CUtensorMap tma
             "bar.red.or.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(stop) : "r"((unsigned)(!landed || *abort_flag)), "r"(1 + eg) : "memory");
         if (!stop && cand0 + lrow < Le)
-          a.cpart[((long long)z * a.RB + rb) * a.buf.c_stride + cand0 + lrow] =
+          a.cpart[((long long)z * a.RBC + rb) * a.buf.c_stride + cand0 + lrow] =
               (rg[lrow] + rg[128 + lrow]) + (rg[256 + lrow] + rg[384 + lrow]);
         if (stop) { *abort_flag = 1; ok = false; }
       }
@@ -463,6 +520,7 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Lo = s.Lo; a.Ls = s.Ls; a.Lr = s.Lr; a.R = s.g * s.Lo;
   a.NH = s.d_qk / 64; a.RB = (a.R + 127) / 128;
   const bool pair = wide_pairs(a.RB);
+  a.RBC = pair ? a.RB / 2 : a.RB;
   a.NS = wide_stages(a.NH, pair);
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.b = b; a.buf = buf; a.cpart = cpart; a.status = status;
@@ -510,7 +568,7 @@ cudaError_t launch_score_umma_wide(const Shape& s, const SeqBatch& b, const void
   }
   if (cudaError_t e = pair ? launch_wide<2, true>(grid, smem, st, a, tq, tk1) : launch_wide<2, false>(grid, smem, st, a, tq, tk1))
     return e;
-  score_rowblock_reduce_kernel<<<dim3((max_le + 255) / 256, nz), 256, 0, st>>>(cpart, buf.C, a.RB, buf.c_stride, b,
+  score_rowblock_reduce_kernel<<<dim3((max_le + 255) / 256, nz), 256, 0, st>>>(cpart, buf.C, a.RBC, buf.c_stride, b,
                                                                             s.Hkv, s.Ls, s.Lr);
   count_launch();
   return cudaGetLastError();
