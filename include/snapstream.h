@@ -249,15 +249,17 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout,
  * cache).  Defined as q_len steps of
  * snap_decode_attn: token u is appended as in Eq. 3, then query u attends over the cache as it
  * is after tokens 0..u -- a window row that token u evicts is still seen by the queries before
- * u and by none from u on.  One pass over the cache serves all q_len queries.
+ * u and by none from u on.
  *   q_dev     [n_active][q_len][Hq][d_qk]
  *   k_new_dev [n_active][q_len][Hkv][d_qk], v_new_dev [n_active][q_len][Hkv][d_v]   (required)
  *   out_dev   [n_active][q_len][Hq][d_v];  seq_len_dev[slot] += q_len
  * 1 <= q_len <= Lr (SNAP_ERR_INVALID_ARG otherwise).  bf16 layers with 64-, 128- or 256-wide heads
- * and q_len * (Hq / Hkv) <= 8 are served in one pass over the cache; every other layer (fp32, the
- * latent layout -- v_new_dev is then ignored --, larger groups) is served as the definition reads,
- * q_len single steps: same results, no saving in cache traffic.  The tcgen05 latent kernel reads
- * each token's rows in place; the other kernels have them staged in the workspace first.
+ * and up to 8 query heads per KV head take 8 / (Hq / Hkv) tokens per pass over the cache (all
+ * q_len in one pass when q_len * (Hq / Hkv) <= 8, otherwise several passes, each reading its
+ * tokens' rows in place); every other layer (fp32, the latent layout -- v_new_dev is then ignored
+ * --) is served as the definition reads, q_len single steps: same results, no saving in cache
+ * traffic.  The tcgen05 latent kernel reads each token's rows in place; the other single-step
+ * kernels have them staged in the workspace first.
  * Scratch: snap_decode_multi_workspace_bytes(cfg, n_active, q_len).
  */
 int64_t snap_decode_multi_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t q_len);

@@ -539,8 +539,13 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
 static int multi_check(const Shape& s, int q_len) {
   return q_len < 1 || q_len > s.Lr ? SNAP_ERR_INVALID_ARG : SNAP_OK;
 }
-static bool multi_one_pass(const snap_config_t* cfg, const Shape& s, int q_len) {
-  return decode_use_gqa_mma(cfg->dtype, s) && q_len * s.g <= 8;
+// Tokens per launch of the tensor-core grouped-query kernel: its eight MMA columns hold (token, head)
+// pairs, so 8 / g tokens go in one pass and a longer step takes several passes, each reading its
+// tokens' rows in place.  0: the layout is served by other kernels.
+static int multi_tokens_per_pass(const snap_config_t* cfg, const Shape& s, int q_len) {
+  if (!decode_use_gqa_mma(cfg->dtype, s) || s.g > 8) return 0;
+  const int t = 8 / s.g;
+  return t < q_len ? t : q_len;
 }
 
 // Dense staging of one token's rows for the step-wise path: q, k_new, v_new, out.
@@ -568,9 +573,9 @@ int64_t snap_decode_multi_workspace_bytes(const snap_config_t* cfg, int32_t n_ac
   const Shape s = make_shape(cfg);
   const int mc = multi_check(s, q_len);
   if (mc != SNAP_OK) return mc;
-  if (multi_one_pass(cfg, s, q_len)) {
+  if (const int tpp = multi_tokens_per_pass(cfg, s, q_len)) {
     const int nsplit = decode_gqa_mma_nsplit(s, n_active > 0 ? n_active : 1, sm_count());
-    return (int64_t)(decode_gqa_mma_partial_floats(s, n_active * q_len, nsplit) * sizeof(float) + 256);
+    return (int64_t)(decode_gqa_mma_partial_floats(s, n_active * tpp, nsplit) * sizeof(float) + 256);
   }
   const int64_t single = snap_decode_workspace_bytes(cfg, n_active);
   if (single < 0) return single;
@@ -599,12 +604,16 @@ int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout
   if (need < 0) return (int)need;
   if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (multi_one_pass(cfg, s, q_len)) {
+  if (const int tpp = multi_tokens_per_pass(cfg, s, q_len)) {
     const int nsplit = decode_gqa_mma_nsplit(s, n_active, sm_count());
-    const cudaError_t e = launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
-                                                v_cache_dev, seq_len_dev, valid_topk_dev, out_dev,
-                                                static_cast<float*>(workspace_dev), nsplit, status_dev, st, q_len);
-    return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+    for (int u0 = 0; u0 < q_len; u0 += tpp) {
+      const int t = q_len - u0 < tpp ? q_len - u0 : tpp;
+      if (launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev, v_cache_dev, seq_len_dev,
+                                valid_topk_dev, out_dev, static_cast<float*>(workspace_dev), nsplit, status_dev, st, t, q_len,
+                                u0) != cudaSuccess)
+        return SNAP_ERR_CUDA;
+    }
+    return SNAP_OK;
   }
   // the streamed latent kernel reads token u of every sequence in place (strided tensor map, strided rows):
   // q_len single steps with no staging copies.  (One launch over (sequence, token) was tried: with the 8 sequences

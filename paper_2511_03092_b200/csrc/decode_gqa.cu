@@ -395,13 +395,16 @@ __global__ void __launch_bounds__(NT, (G > 4 ? 2 : 3)) decode_gqa_kernel(const F
 }
 
 // Merge the splits of one (sequence, query token, query head); maxima are in the log2 domain.
-// With q_len query tokens per sequence the rows of `partials` and `out` are indexed by
-// sequence * q_len + token, and every token's block advances the sequence length by one.
+// With q_len query tokens per sequence the rows of `partials` are indexed by sequence * q_len +
+// token; the token is token u0 + (its index) of the q_total per sequence in `out`; every token's
+// block advances the sequence length by one.
 __global__ void __launch_bounds__(D) decode_gqa_merge_kernel(const float* __restrict__ partials,
                                                              __nv_bfloat16* __restrict__ out, int Hq,
                                                              int nsplit, const int* __restrict__ slot_ids,
-                                                             int* seq_len, int max_seqs, int bump, int q_len) {
+                                                             int* seq_len, int max_seqs, int bump, int q_len, int q_total,
+                                                             int u0) {
   const int h = blockIdx.x, i = blockIdx.y, t = threadIdx.x;
+  const long long orow = (long long)(i / q_len) * q_total + u0 + i % q_len;   // token's row of `out`
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const float* p = partials + ((long long)i * Hq + h) * nsplit * PS;
   // launched with programmatic stream serialisation: the grid may start while the split kernel
@@ -416,7 +419,7 @@ __global__ void __launch_bounds__(D) decode_gqa_merge_kernel(const float* __rest
     L += p[s * PS + 1] * f;
     O += p[s * PS + 2 + t] * f;
   }
-  out[((long long)i * Hq + h) * D + t] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
+  out[(orow * Hq + h) * D + t] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
   if (bump && h == 0 && t == 0) {
     const int slot = slot_ids[i / q_len];
     if (slot >= 0 && slot < max_seqs) atomicAdd(&seq_len[slot], 1);
@@ -451,7 +454,7 @@ cudaError_t launch_g(const FastArgs& a, int n_active, __nv_bfloat16* out, int* s
   const float* parts = a.partials;
   const int* slots = a.slot_ids;
   cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_merge_kernel, parts, out, a.Hq, a.nsplit, slots, seq_len,
-                                     a.max_seqs, bump, 1);
+                                     a.max_seqs, bump, 1, 1, 0);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -461,7 +464,8 @@ cudaError_t launch_g(const FastArgs& a, int n_active, __nv_bfloat16* out, int* s
 // The split merge as a programmatic dependent launch (shared with the tensor-core kernel);
 // n_rows = sequences * q_len.
 cudaError_t launch_decode_gqa_merge(const float* partials, void* out, int Hq, int nsplit, const int* slot_ids,
-                                    int n_rows, int q_len, int* seq_len, int max_seqs, int bump, cudaStream_t st) {
+                                    int n_rows, int q_len, int* seq_len, int max_seqs, int bump, cudaStream_t st,
+                                    int q_total, int u0) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -472,7 +476,8 @@ cudaError_t launch_decode_gqa_merge(const float* partials, void* out, int Hq, in
   lc.attrs = attr;
   lc.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&lc, decode_gqa_merge_kernel, partials, static_cast<__nv_bfloat16*>(out), Hq, nsplit,
-                                     slot_ids, seq_len, max_seqs, bump, q_len);
+                                     slot_ids, seq_len, max_seqs, bump, q_len, q_total < q_len ? q_len : q_total,
+                                     q_total < q_len ? 0 : u0);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -50,7 +50,8 @@ struct MmaArgs {
   char* kc; char* vc;
   long long seq_b, head_b;
   int Hq, Hkv, g, Ls, Lr, max_seqs, nsplit;
-  int T;                                        // query tokens per sequence in this step (T * g <= 8)
+  int T;                                        // query tokens per sequence in this launch (T * g <= 8)
+  int QT, u0;                                   // ... which are tokens u0 .. u0 + T - 1 of the QT tokens per sequence in q / k_new / v_new
   float scale_log2;
   const int* seq_len; const int* valid_topk;
   float* partials;                              // [n_active][T][Hq][nsplit][PS]
@@ -141,8 +142,8 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
   char* kc = a.kc + slot * a.seq_b + kvh * a.head_b;
   char* vc = a.vc + slot * a.seq_b + kvh * a.head_b;
   // new rows of this KV head: token u at kn + u * Hkv * D
-  const __nv_bfloat16* kn = a.k_new ? a.k_new + ((long long)i * TQ * a.Hkv + kvh) * D : nullptr;
-  const __nv_bfloat16* vn = a.v_new ? a.v_new + ((long long)i * TQ * a.Hkv + kvh) * D : nullptr;
+  const __nv_bfloat16* kn = a.k_new ? a.k_new + (((long long)i * a.QT + a.u0) * a.Hkv + kvh) * D : nullptr;
+  const __nv_bfloat16* vn = a.v_new ? a.v_new + (((long long)i * a.QT + a.u0) * a.Hkv + kvh) * D : nullptr;
   const long long new_stride = (long long)a.Hkv * D;
 
   // Column n of the MMAs is query token n / g, head n % g of the group (zero beyond T * g).
@@ -151,7 +152,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
   uint32_t qb[KS][2];
   {
     const int tcol = gq / a.g, hcol = gq - tcol * a.g;
-    const __nv_bfloat16* qp = a.q + (((long long)i * TQ + tcol) * a.Hq + (long long)kvh * a.g + hcol) * D + 2 * tq;
+    const __nv_bfloat16* qp = a.q + (((long long)i * a.QT + a.u0 + tcol) * a.Hq + (long long)kvh * a.g + hcol) * D + 2 * tq;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
       qb[ks][0] = gq < ncols ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks) : 0u;
@@ -339,13 +340,16 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
 }
 
 // Merge the splits of one (sequence, query token, query head) for any head size; maxima are in
-// the log2 domain.  Rows of `partials` and `out` are indexed by sequence * q_len + token, and every
-// token's block advances the sequence length by one.
+// the log2 domain.  Rows of `partials` are indexed by sequence * q_len + token; the token is token
+// u0 + (its index) of the q_total per sequence in `out`; every token's block advances the sequence
+// length by one.
 __global__ void __launch_bounds__(128) decode_gqa_mma_merge_kernel(const float* __restrict__ partials,
                                                                    __nv_bfloat16* __restrict__ out, int Hq, int d,
                                                                    int nsplit, const int* __restrict__ slot_ids,
-                                                                   int* seq_len, int max_seqs, int bump, int q_len) {
+                                                                   int* seq_len, int max_seqs, int bump, int q_len, int q_total,
+                                                                   int u0) {
   const int h = blockIdx.x, i = blockIdx.y, ps = d + 2;
+  const long long orow = (long long)(i / q_len) * q_total + u0 + i % q_len;   // token's row of `out`
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const float* p = partials + ((long long)i * Hq + h) * nsplit * ps;
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -363,7 +367,7 @@ __global__ void __launch_bounds__(128) decode_gqa_mma_merge_kernel(const float* 
       const float ms = p[s * ps];
       if (ms != -INFINITY) O += p[s * ps + 2 + t] * exp2f(ms - M);
     }
-    out[((long long)i * Hq + h) * d + t] = __float2bfloat16_rn(O * inv);
+    out[(orow * Hq + h) * d + t] = __float2bfloat16_rn(O * inv);
   }
   if (bump && h == 0 && threadIdx.x == 0) {
     const int slot = slot_ids[i / q_len];
@@ -396,9 +400,11 @@ size_t decode_gqa_mma_partial_floats(const Shape& s, int n_rows, int nsplit) {
 cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_new, const void* v_new,
                                   const int* slot_ids, int n_active, void* k_cache, void* v_cache,
                                   int* seq_len, const int* valid_topk, void* out, float* partials,
-                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len) {
+                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len, int q_total, int u0) {
   if (n_active == 0) return cudaSuccess;
-  if (q_len < 1 || q_len * s.g > GP || (q_len > 1 && (!k_new || q_len > s.Lr))) return cudaErrorInvalidValue;
+  if (q_total < q_len) { q_total = q_len; u0 = 0; }            // the launch's tokens are all the step's tokens
+  if (q_len < 1 || q_len * s.g > GP || (q_len > 1 && (!k_new || q_len > s.Lr)) || u0 < 0 || u0 + q_len > q_total)
+    return cudaErrorInvalidValue;
   umma::EncodeTiledFn enc = umma::encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
   const int D = s.d_qk;
@@ -439,7 +445,7 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   a.kc = static_cast<char*>(k_cache); a.vc = static_cast<char*>(v_cache);
   a.head_b = (long long)s.Sc * D * 2; a.seq_b = a.head_b * s.Hkv;
   a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.Ls = s.Ls; a.Lr = s.Lr; a.max_seqs = s.max_seqs; a.nsplit = nsplit;
-  a.T = q_len;
+  a.T = q_len; a.QT = q_total; a.u0 = u0;
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.seq_len = seq_len; a.valid_topk = valid_topk; a.partials = partials; a.status = status;
   cudaError_t e;
@@ -449,10 +455,10 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   if (e != cudaSuccess) return e;
   if (D == 128)
     return launch_decode_gqa_merge(partials, out, s.Hq, nsplit, slot_ids, n_active * q_len, q_len, seq_len, s.max_seqs,
-                                   k_new != nullptr, st);
+                                   k_new != nullptr, st, q_total, u0);
   e = launch_pdl(decode_gqa_mma_merge_kernel, dim3(s.Hq, n_active * q_len), dim3(128), 0, st,
                  static_cast<const float*>(partials), static_cast<__nv_bfloat16*>(out), s.Hq, D, nsplit, slot_ids, seq_len,
-                 s.max_seqs, (int)(k_new != nullptr), q_len);
+                 s.max_seqs, (int)(k_new != nullptr), q_len, q_total, u0);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }

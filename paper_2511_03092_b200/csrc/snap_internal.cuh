@@ -180,7 +180,8 @@ cudaError_t launch_decode_gqa(const Shape& s, const void* q, const void* k_new, 
                               int nsplit, uint32_t* status, cudaStream_t st);
 
 cudaError_t launch_decode_gqa_merge(const float* partials, void* out, int Hq, int nsplit, const int* slot_ids,
-                                    int n_rows, int q_len, int* seq_len, int max_seqs, int bump, cudaStream_t st);
+                                    int n_rows, int q_len, int* seq_len, int max_seqs, int bump, cudaStream_t st,
+                                    int q_total = 0, int u0 = 0);
 // the same on tensor cores (mma.sync, the group's heads on the N side; head sizes 64, 128, 256): cost independent of the group size
 bool decode_gqa_mma_supported(int dtype, const Shape& s);
 bool decode_use_gqa_mma(int dtype, const Shape& s);     // the choice between the two, shared by all entry points
@@ -189,7 +190,9 @@ size_t decode_gqa_mma_partial_floats(const Shape& s, int n_rows, int nsplit);
 cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_new, const void* v_new,
                                   const int* slot_ids, int n_active, void* k_cache, void* v_cache,
                                   int* seq_len, const int* valid_topk, void* out, float* partials,
-                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len = 1);
+                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len = 1, int q_total = 0, int u0 = 0);
+// (q_len tokens per sequence in one pass, q_len * g <= 8: tokens u0 .. u0 + q_len - 1 of the q_total per sequence that
+// q, k_new, v_new and out hold; q_total = 0: they hold exactly these)
 
 // latent attention (one 576-wide KV row shared by all heads, V = its first 512 dims): mma.sync kernel
 bool decode_mla_supported(int dtype, const Shape& s);
