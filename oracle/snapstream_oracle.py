@@ -405,3 +405,80 @@ def candidate_log2_normalisers(q_obs: np.ndarray, k: np.ndarray, cfg: OracleConf
         m = S.max(axis=1)
         mu[h] = (m + np.log(np.exp(S - m[:, None]).sum(axis=1))) / np.log(2.0)
     return mu
+
+
+# ----------------------------------------------------------------------------
+# Per-step block top-K over the evictable middle of the prompt (the alternative the paper's
+# related-work section leaves to future work: KV blocks with pre-computed statistics, of
+# which the top ones are looked up for every newly decoded token, "in the style of Quest
+# and InfLLM").  The paper fixes nothing beyond that sentence, so everything here is a
+# reading, stated in full:
+#   * the middle of the prompt, positions [Ls, L - Lr), is kept whole and cut into blocks
+#     of `block_tokens` consecutive positions (the last block may be shorter);
+#   * a block's statistics are the element-wise minimum and maximum of its keys per KV
+#     head (the published query-aware page criterion);
+#   * a decode query scores block b of KV head kvh by
+#         U[kvh, b] = sum_{h in group(kvh)} sum_d max(q[h, d] * kmin[kvh, b, d], q[h, d] * kmax[kvh, b, d]),
+#     an upper bound of the group-summed logit q_h . k_j of every key j of the block (the
+#     g query heads of a KV head are summed as in Eq. 1's group reading above);
+#   * the `n_blocks` highest-scoring blocks are attended, ties to the lower block index,
+#     together with the sinks and the rolling window of Eq. 3, which behave as before;
+#     tokens that leave the rolling window during decoding are dropped as in SnapStream.
+# Parity unpinned by the paper: all of the above.  Pinned by the mathematics: the bound
+# property, the one-token-block special case (exact top-k by logit), and equality with
+# attention over everything kept when all blocks are selected.
+# ----------------------------------------------------------------------------
+
+def block_statistics(k: np.ndarray, cfg: OracleConfig, block_tokens: int):
+    """Per-block key minima and maxima over the prompt's middle.  k: [L, Hkv, d_qk].
+    returns (kmin, kmax), each [Hkv, n_blocks, d_qk]; n_blocks = ceil((L - Lsr) / block_tokens)."""
+    k = np.asarray(k, dtype=np.float64)
+    L = k.shape[0]
+    Le = max(L - cfg.l_sr, 0)
+    nb = -(-Le // block_tokens)
+    kmin = np.zeros((cfg.n_kv_heads, nb, cfg.d_qk))
+    kmax = np.zeros((cfg.n_kv_heads, nb, cfg.d_qk))
+    for b in range(nb):
+        lo = cfg.l_sink + b * block_tokens
+        hi = min(lo + block_tokens, cfg.l_sink + Le)
+        kmin[:, b, :] = k[lo:hi].min(axis=0)
+        kmax[:, b, :] = k[lo:hi].max(axis=0)
+    return kmin, kmax
+
+
+def block_upper_bounds(q: np.ndarray, kmin: np.ndarray, kmax: np.ndarray, cfg: OracleConfig) -> np.ndarray:
+    """U[kvh, b] for one decode query q: [Hq, d_qk]. -> [Hkv, n_blocks]."""
+    q = np.asarray(q, dtype=np.float64)
+    nb = kmin.shape[1]
+    U = np.zeros((cfg.n_kv_heads, nb))
+    for kvh in range(cfg.n_kv_heads):
+        for h in range(kvh * cfg.group, (kvh + 1) * cfg.group):
+            U[kvh] += np.maximum(q[h][None, :] * kmin[kvh], q[h][None, :] * kmax[kvh]).sum(axis=1)
+    return U
+
+
+def select_blocks(U_row: np.ndarray, n_blocks: int) -> np.ndarray:
+    """The n_blocks highest-scoring blocks of one KV head, ties to the lower index, ascending."""
+    return select_topk(U_row, n_blocks)
+
+
+def block_positions(blocks: np.ndarray, prompt_len: int, cfg: OracleConfig, block_tokens: int) -> np.ndarray:
+    """Absolute prompt positions covered by the given blocks (ascending)."""
+    end = prompt_len - cfg.l_recent
+    out = []
+    for b in blocks:
+        lo = cfg.l_sink + int(b) * block_tokens
+        out.extend(range(lo, min(lo + block_tokens, end)))
+    return np.asarray(out, dtype=np.int64)
+
+
+def block_decode_step(seq: OracleSequence, prompt_len: int, kmin: np.ndarray, kmax: np.ndarray, n_blocks: int,
+                      block_tokens: int, q: np.ndarray, k_new: np.ndarray, v_new: Optional[np.ndarray]):
+    """One decode step with a per-step block lookup: score the blocks with this token's
+    query, keep the top n_blocks per KV head in place of the prefill top-K set, then
+    append and attend as in `decode_step`.  returns (out [Hq, d_v], blocks per KV head)."""
+    cfg = seq.cfg
+    U = block_upper_bounds(q, kmin, kmax, cfg)
+    chosen = [select_blocks(U[kvh], n_blocks) for kvh in range(cfg.n_kv_heads)]
+    seq.topk_pos = [block_positions(chosen[kvh], prompt_len, cfg, block_tokens) for kvh in range(cfg.n_kv_heads)]
+    return decode_step(seq, q, k_new, v_new), chosen
