@@ -16,8 +16,11 @@
  * and, around it: snap_decode_attn_multi (several new tokens per sequence and step),
  * snap_decode_attn_static (the decode step without a caller-provided scratch buffer),
  * snap_append_kv_concat (the slice-and-concatenate update of Section 3.2.1, as a baseline),
- * and snap_prefill_attn + snap_compress_with_row_stats (the prompt's causal attention emitting
- * the normalisers of Eq. 4, and the compression that consumes them).
+ * snap_prefill_attn + snap_compress_with_row_stats (the prompt's causal attention emitting
+ * the normalisers of Eq. 4, and the compression that consumes them),
+ * and snap_block_stats + snap_block_select + snap_decode_attn_blocks (a per-step block top-K
+ * over the whole middle of the prompt instead of the one-time top-K, the variant the paper's
+ * related-work section leaves to future work).
  *
  * Conventions
  *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are plain
@@ -328,6 +331,57 @@ int snap_append_kv_concat(const snap_config_t* cfg, const snap_layout_t* layout,
                           const void* k_cache_in_dev, const void* v_cache_in_dev,
                           void* k_cache_out_dev, void* v_cache_out_dev,
                           int32_t* seq_len_dev, uint32_t* status_dev, void* cuda_stream);
+
+/*
+ * Per-step block top-K (the paper's related-work section: KV blocks with pre-computed statistics,
+ * of which the top ones are looked up for every newly decoded token, left there to future
+ * work; the criterion is the published query-aware one).  The paper fixes nothing further, so
+ * the definition is this library's:
+ *   - the cache is built by snap_compress with a top-K budget of at least the prompt's middle
+ *     (topk >= L - Ls - Lr): every candidate is then kept, in position order, in the third
+ *     section, valid_topk rows of it;
+ *   - that section is cut into blocks of block_tokens consecutive rows (a multiple of 16, at
+ *     most 1024; the last block may be shorter); a block's statistics are the element-wise
+ *     minimum and maximum of its keys per KV head;
+ *   - a decode query scores block b of KV head kvh by
+ *       U = sum over the query heads h of kvh and the dims d of max(q[h][d] * kmin[b][d], q[h][d] * kmax[b][d]),
+ *     an upper bound of the group-summed logit of every key of the block, and the n_blocks
+ *     highest-scoring blocks are attended, ties to the lower block index, together with the
+ *     sinks and the rolling window, which behave as in snap_decode_attn (Eq. 3 append
+ *     included); rows that leave the window during decoding are dropped as before.
+ * bf16 layers with 64-, 128- or 256-wide heads, a separate V and at most 8 query heads per KV
+ * head; at most 8192 blocks per sequence; SNAP_ERR_UNSUPPORTED otherwise.  The scores are summed
+ * in single precision (the products are exact): two blocks whose scores differ by less than about
+ * 1e-6 relative may come out in either order.
+ *
+ * snap_block_stats    once per prompt, after snap_compress:
+ *   stats_dev  out [max_seqs][Hkv][ceil(topk / block_tokens)][2][d_qk] in the cache's dtype (minimum, then
+ *              maximum), snap_block_stats_bytes(cfg, block_tokens) bytes; the blocks of slot_ids_dev[0 .. n_seqs)
+ *              are written, rows of blocks past a prompt's last one are left alone.
+ * snap_block_select   every step, before the attention:
+ *   q_dev [n_active][Hq][d_qk];  block_idx_dev out [n_active][Hkv][n_blocks] ascending block numbers;
+ *   n_selected_dev out [n_active][Hkv] = min(n_blocks, blocks of that prompt).
+ * snap_decode_attn_blocks   snap_decode_attn that visits only the listed blocks of the third section
+ *   (arguments as there, plus the two arrays snap_block_select wrote, same n_blocks);
+ *   scratch: snap_decode_blocks_workspace_bytes(cfg, n_active, block_tokens, n_blocks).
+ * All three enqueue on cuda_stream and return; device-side conditions go to status_dev.
+ */
+int64_t snap_block_stats_bytes(const snap_config_t* cfg, int32_t block_tokens);
+int snap_block_stats(const snap_config_t* cfg, const snap_layout_t* layout, const int32_t* slot_ids_dev,
+                     int32_t n_seqs, const void* k_cache_dev, const int32_t* valid_topk_dev,
+                     int32_t block_tokens, void* stats_dev, uint32_t* status_dev, void* cuda_stream);
+int snap_block_select(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,
+                      const int32_t* slot_ids_dev, int32_t n_active, const void* stats_dev,
+                      const int32_t* valid_topk_dev, int32_t block_tokens, int32_t n_blocks,
+                      int32_t* block_idx_dev, int32_t* n_selected_dev, uint32_t* status_dev, void* cuda_stream);
+int64_t snap_decode_blocks_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t block_tokens,
+                                           int32_t n_blocks);
+int snap_decode_attn_blocks(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,
+                            const void* k_new_dev, const void* v_new_dev, const int32_t* slot_ids_dev,
+                            int32_t n_active, void* k_cache_dev, void* v_cache_dev, int32_t* seq_len_dev,
+                            const int32_t* valid_topk_dev, int32_t block_tokens, int32_t n_blocks,
+                            const int32_t* block_idx_dev, const int32_t* n_selected_dev, void* out_dev,
+                            void* workspace_dev, size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream);
 
 /*
  * Testing and tuning aids (the paper has no counterpart).  Each option is one non-negative

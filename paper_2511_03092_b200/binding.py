@@ -87,6 +87,16 @@ def lib() -> C.CDLL:
     L.snap_decode_attn_static.argtypes = [pcfg, play, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
     L.snap_debug_set_option.restype = C.c_int
     L.snap_debug_set_option.argtypes = [C.c_int, C.c_int]
+    L.snap_block_stats_bytes.restype = i64
+    L.snap_block_stats_bytes.argtypes = [pcfg, i32]
+    L.snap_block_stats.restype = C.c_int
+    L.snap_block_stats.argtypes = [pcfg, play, vp, i32, vp, vp, i32, vp, vp, vp]
+    L.snap_block_select.restype = C.c_int
+    L.snap_block_select.argtypes = [pcfg, play, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp, vp]
+    L.snap_decode_blocks_workspace_bytes.restype = i64
+    L.snap_decode_blocks_workspace_bytes.argtypes = [pcfg, i32, i32, i32]
+    L.snap_decode_attn_blocks.restype = C.c_int
+    L.snap_decode_attn_blocks.argtypes = [pcfg, play, vp, vp, vp, vp, i32, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp, vp]
     _lib = L
     return L
 
@@ -94,7 +104,9 @@ def lib() -> C.CDLL:
 EXPORTS = ("snap_cache_layout", "snap_compress_workspace_bytes", "snap_decode_workspace_bytes",
            "snap_compress", "snap_append_kv", "snap_append_kv_concat", "snap_decode_attn",
            "snap_decode_multi_workspace_bytes", "snap_decode_attn_multi", "snap_decode_attn_static", "snap_status_string",
-           "snap_kernel_launch_count", "snap_prefill_attn", "snap_compress_with_row_stats", "snap_debug_set_option")
+           "snap_kernel_launch_count", "snap_prefill_attn", "snap_compress_with_row_stats", "snap_debug_set_option",
+           "snap_block_stats_bytes", "snap_block_stats", "snap_block_select", "snap_decode_blocks_workspace_bytes",
+           "snap_decode_attn_blocks")
 
 # testing / tuning options of snap_debug_set_option
 (SNAP_OPT_SCORE_KERNEL, SNAP_OPT_DECODE_GQA_KERNEL, SNAP_OPT_DECODE_LATENT_KERNEL, SNAP_OPT_DECODE_NSPLIT,
@@ -289,3 +301,44 @@ def alloc_cache(cfg: SnapConfig, layout: SnapLayout, device="cuda") -> CacheBuff
     return CacheBuffers(kc, vc, torch.zeros(cfg.max_seqs, dtype=torch.int32, device=device),
                         torch.zeros(cfg.max_seqs, dtype=torch.int32, device=device),
                         torch.zeros(1, dtype=torch.int32, device=device))
+
+
+def snap_block_stats_bytes(cfg: SnapConfig, block_tokens: int) -> int:
+    n = lib().snap_block_stats_bytes(C.byref(cfg), int(block_tokens))
+    if n < 0:
+        raise SnapError(int(n), "snap_block_stats_bytes")
+    return int(n)
+
+
+def snap_block_stats(cfg: SnapConfig, layout: SnapLayout, slot_ids_dev, n_seqs: int, k_cache, valid_topk,
+                     block_tokens: int, stats, status=None, stream=None) -> None:
+    """Per-block key minima and maxima of the third section of the given slots' caches."""
+    _check(lib().snap_block_stats(C.byref(cfg), C.byref(layout), _ptr(slot_ids_dev), int(n_seqs), _ptr(k_cache),
+                                  _ptr(valid_topk), int(block_tokens), _ptr(stats), _ptr(status), _stream(stream)),
+           "snap_block_stats")
+
+
+def snap_block_select(cfg: SnapConfig, layout: SnapLayout, q, slot_ids_dev, n_active: int, stats, valid_topk,
+                      block_tokens: int, n_blocks: int, block_idx, n_selected, status=None, stream=None) -> None:
+    """The n_blocks highest-scoring blocks per (sequence, KV head) for this step's queries."""
+    _check(lib().snap_block_select(C.byref(cfg), C.byref(layout), _ptr(q), _ptr(slot_ids_dev), int(n_active), _ptr(stats),
+                                   _ptr(valid_topk), int(block_tokens), int(n_blocks), _ptr(block_idx), _ptr(n_selected),
+                                   _ptr(status), _stream(stream)), "snap_block_select")
+
+
+def snap_decode_blocks_workspace_bytes(cfg: SnapConfig, n_active: int, block_tokens: int, n_blocks: int) -> int:
+    n = lib().snap_decode_blocks_workspace_bytes(C.byref(cfg), int(n_active), int(block_tokens), int(n_blocks))
+    if n < 0:
+        raise SnapError(int(n), "snap_decode_blocks_workspace_bytes")
+    return int(n)
+
+
+def snap_decode_attn_blocks(cfg: SnapConfig, layout: SnapLayout, q, k_new, v_new, slot_ids_dev, n_active: int, k_cache,
+                            v_cache, seq_len, valid_topk, block_tokens: int, n_blocks: int, block_idx, n_selected, out,
+                            workspace, status=None, stream=None) -> None:
+    """snap_decode_attn over the sinks, the window and the listed blocks of the third section."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().snap_decode_attn_blocks(C.byref(cfg), C.byref(layout), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(slot_ids_dev),
+                                         int(n_active), _ptr(k_cache), _ptr(v_cache), _ptr(seq_len), _ptr(valid_topk),
+                                         int(block_tokens), int(n_blocks), _ptr(block_idx), _ptr(n_selected), _ptr(out),
+                                         _ptr(workspace), ws_bytes, _ptr(status), _stream(stream)), "snap_decode_attn_blocks")

@@ -582,6 +582,107 @@ int64_t snap_decode_multi_workspace_bytes(const snap_config_t* cfg, int32_t n_ac
   return (int64_t)step_stage(cfg, s, n_active).bytes + single;
 }
 
+// ---- per-step block top-K over the third section (block_topk.cu) ----
+
+static int blocks_check(const snap_config_t* cfg, const Shape& s, int block_tokens) {
+  if (block_tokens < 1) return SNAP_ERR_INVALID_ARG;
+  if (!block_topk_supported(cfg->dtype, s, block_tokens) || !decode_use_gqa_mma(cfg->dtype, s)) return SNAP_ERR_UNSUPPORTED;
+  return SNAP_OK;
+}
+// the cache the decode kernel's split rule should assume: the low section plus the visited blocks
+static Shape blocks_shape(Shape s, int block_tokens, int n_blocks) {
+  const long long rows = (long long)n_blocks * block_tokens;
+  s.K = rows < s.K ? (int)rows : s.K;
+  s.Sc = s.Ls + s.Lr + s.K;
+  return s;
+}
+
+int64_t snap_block_stats_bytes(const snap_config_t* cfg, int32_t block_tokens) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  const Shape s = make_shape(cfg);
+  const int bc = blocks_check(cfg, s, block_tokens);
+  if (bc != SNAP_OK) return bc;
+  return (int64_t)s.max_seqs * s.Hkv * block_count_max(s, block_tokens) * 2 * s.d_qk * elt_bytes(cfg->dtype);
+}
+
+int snap_block_stats(const snap_config_t* cfg, const snap_layout_t* layout, const int32_t* slot_ids_dev, int32_t n_seqs,
+                     const void* k_cache_dev, const int32_t* valid_topk_dev, int32_t block_tokens, void* stats_dev,
+                     uint32_t* status_dev, void* cuda_stream) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (!layout) return SNAP_ERR_NULL_POINTER;
+  if (n_seqs < 0) return SNAP_ERR_INVALID_ARG;
+  const Shape s = make_shape(cfg);
+  const int bc = blocks_check(cfg, s, block_tokens);
+  if (bc != SNAP_OK) return bc;
+  if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
+  if (n_seqs == 0) return SNAP_OK;
+  if (!slot_ids_dev || !k_cache_dev || !valid_topk_dev || !stats_dev) return SNAP_ERR_NULL_POINTER;
+  const cudaError_t e = launch_block_stats(s, block_tokens, slot_ids_dev, n_seqs, k_cache_dev, valid_topk_dev, stats_dev,
+                                           status_dev, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+}
+
+int snap_block_select(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev, const int32_t* slot_ids_dev,
+                      int32_t n_active, const void* stats_dev, const int32_t* valid_topk_dev, int32_t block_tokens,
+                      int32_t n_blocks, int32_t* block_idx_dev, int32_t* n_selected_dev, uint32_t* status_dev,
+                      void* cuda_stream) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (!layout) return SNAP_ERR_NULL_POINTER;
+  if (n_active < 0 || n_blocks < 1) return SNAP_ERR_INVALID_ARG;
+  const Shape s = make_shape(cfg);
+  const int bc = blocks_check(cfg, s, block_tokens);
+  if (bc != SNAP_OK) return bc;
+  if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
+  if (n_active == 0) return SNAP_OK;
+  if (!q_dev || !slot_ids_dev || !stats_dev || !valid_topk_dev || !block_idx_dev || !n_selected_dev) return SNAP_ERR_NULL_POINTER;
+  const cudaError_t e = launch_block_select(s, block_tokens, n_blocks, q_dev, slot_ids_dev, n_active, stats_dev, valid_topk_dev,
+                                            block_idx_dev, n_selected_dev, status_dev, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+}
+
+int64_t snap_decode_blocks_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t block_tokens, int32_t n_blocks) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (n_active < 0 || n_blocks < 1) return SNAP_ERR_INVALID_ARG;
+  const Shape s = make_shape(cfg);
+  const int bc = blocks_check(cfg, s, block_tokens);
+  if (bc != SNAP_OK) return bc;
+  const int nsplit = decode_gqa_mma_nsplit(blocks_shape(s, block_tokens, n_blocks), n_active > 0 ? n_active : 1, sm_count());
+  return (int64_t)(decode_gqa_mma_partial_floats(s, n_active, nsplit) * sizeof(float) + 256);
+}
+
+int snap_decode_attn_blocks(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev, const void* k_new_dev,
+                            const void* v_new_dev, const int32_t* slot_ids_dev, int32_t n_active, void* k_cache_dev,
+                            void* v_cache_dev, int32_t* seq_len_dev, const int32_t* valid_topk_dev, int32_t block_tokens,
+                            int32_t n_blocks, const int32_t* block_idx_dev, const int32_t* n_selected_dev, void* out_dev,
+                            void* workspace_dev, size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (!layout) return SNAP_ERR_NULL_POINTER;
+  if (n_active < 0 || n_blocks < 1) return SNAP_ERR_INVALID_ARG;
+  const Shape s = make_shape(cfg);
+  const int bc = blocks_check(cfg, s, block_tokens);
+  if (bc != SNAP_OK) return bc;
+  if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
+  if (n_active == 0) return SNAP_OK;
+  if (!q_dev || !slot_ids_dev || !k_cache_dev || !v_cache_dev || !seq_len_dev || !valid_topk_dev || !block_idx_dev ||
+      !n_selected_dev || !out_dev || !workspace_dev)
+    return SNAP_ERR_NULL_POINTER;
+  if (k_new_dev && !v_new_dev) return SNAP_ERR_NULL_POINTER;
+  const int64_t need = snap_decode_blocks_workspace_bytes(cfg, n_active, block_tokens, n_blocks);
+  if (need < 0) return (int)need;
+  if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
+  const int nsplit = decode_gqa_mma_nsplit(blocks_shape(s, block_tokens, n_blocks), n_active, sm_count());
+  const cudaError_t e = launch_decode_gqa_mma(s, q_dev, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev, v_cache_dev,
+                                              seq_len_dev, valid_topk_dev, out_dev, static_cast<float*>(workspace_dev), nsplit,
+                                              status_dev, static_cast<cudaStream_t>(cuda_stream), 1, 0, 0, block_idx_dev,
+                                              n_selected_dev, n_blocks, block_tokens);
+  return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+}
+
 int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,
                            const void* k_new_dev, const void* v_new_dev, const int32_t* slot_ids_dev,
                            int32_t n_active, int32_t q_len, void* k_cache_dev, void* v_cache_dev,

@@ -56,6 +56,10 @@ struct MmaArgs {
   const int* seq_len; const int* valid_topk;
   float* partials;                              // [n_active][T][Hq][nsplit][PS]
   uint32_t* status;
+  // per-step block lookup (block_topk.cu): NULL, or the blocks of the third section to visit, ascending
+  const int* block_idx;                         // [n_active][Hkv][blocks_cap]
+  const int* n_sel;                             // [n_active][Hkv] entries of block_idx in use
+  int blocks_cap, tpb;                          // tiles per block = block_tokens / 16
 };
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, unsigned parity) {
@@ -118,7 +122,18 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
   } else if (tid == 0 && sp == 0 && kvh == 0 && a.status) {
     atomicOr(a.status, SNAP_DEV_BAD_SLOT);
   }
-  const int nA = (n_low_st + WT - 1) / WT, ntiles = nA + (n_top + WT - 1) / WT;
+  const int* blist = a.block_idx && !bad ? a.block_idx + ((long long)i * a.Hkv + kvh) * a.blocks_cap : nullptr;
+  const int nA = (n_low_st + WT - 1) / WT;
+  const int ntiles = nA + (blist ? a.n_sel[i * a.Hkv + kvh] * a.tpb : (n_top + WT - 1) / WT);
+  // tile j: the low section first, then the third section -- all of it, or the listed blocks only
+  auto rows_of = [&](int j) -> TileRows {
+    if (j < nA || !blist) return tile_rows(j, nA, n_low, Lsr, n_top);
+    const int jj = j - nA, blk = blist[jj / a.tpb];
+    TileRows t;
+    t.row0 = Lsr + (blk * a.tpb + jj % a.tpb) * WT;
+    t.row_end = Lsr + n_top;
+    return t;
+  };
   const int t_begin = (int)((long long)ntiles * sp / a.nsplit);
   const int t_end = (int)((long long)ntiles * (sp + 1) / a.nsplit);
   // this warp's tiles: t_begin + w, t_begin + w + NWARP, ...
@@ -127,7 +142,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
 
   auto issue = [&](int n) {                                     // tile n of this warp -> stage n % NSTAGE
     const int s = n % NSTAGE;
-    const TileRows tr = tile_rows(t_begin + w + n * NWARP, nA, n_low, Lsr, n_top);
+    const TileRows tr = rows_of(t_begin + w + n * NWARP);
     const uint32_t dst = stage0 + s * STAGE_B, bar = bar0 + 8 * s;
     mbar_expect_tx(bar, (unsigned)STAGE_B);
 #pragma unroll
@@ -222,7 +237,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     const bool landed = mbar_wait_bounded(bar0 + 8 * s, parity);
     if (__any_sync(0xffffffffu, !landed)) { timed_out = true; break; }
     const int j = t_begin + w + n * NWARP;
-    const TileRows tr = tile_rows(j, nA, n_low, Lsr, n_top);
+    const TileRows tr = rows_of(j);
     const int nrows = tr.row_end - tr.row0;                    // rows at or past it are masked (may be <= 0)
     const uint32_t sK = stage0 + s * STAGE_B, sV = sK + TENS_B;
     bool ok0 = gq < nrows, ok1 = ok0, ok2 = gq + 8 < nrows, ok3 = ok2;
@@ -400,8 +415,10 @@ size_t decode_gqa_mma_partial_floats(const Shape& s, int n_rows, int nsplit) {
 cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_new, const void* v_new,
                                   const int* slot_ids, int n_active, void* k_cache, void* v_cache,
                                   int* seq_len, const int* valid_topk, void* out, float* partials,
-                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len, int q_total, int u0) {
+                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len, int q_total, int u0,
+                                  const int* block_idx, const int* n_sel, int blocks_cap, int block_tokens) {
   if (n_active == 0) return cudaSuccess;
+  if (block_idx && (!n_sel || blocks_cap < 1 || block_tokens < WT || block_tokens % WT || q_len != 1)) return cudaErrorInvalidValue;
   if (q_total < q_len) { q_total = q_len; u0 = 0; }            // the launch's tokens are all the step's tokens
   if (q_len < 1 || q_len * s.g > GP || (q_len > 1 && (!k_new || q_len > s.Lr)) || u0 < 0 || u0 + q_len > q_total)
     return cudaErrorInvalidValue;
@@ -448,6 +465,7 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   a.T = q_len; a.QT = q_total; a.u0 = u0;
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.seq_len = seq_len; a.valid_topk = valid_topk; a.partials = partials; a.status = status;
+  a.block_idx = block_idx; a.n_sel = n_sel; a.blocks_cap = blocks_cap; a.tpb = block_idx ? block_tokens / WT : 1;
   cudaError_t e;
   if (D == 128) e = launch_d<128, 4>(a, hit->tk, hit->tv, n_active, st);
   else if (D == 64) e = launch_d<64, 4>(a, hit->tk, hit->tv, n_active, st);

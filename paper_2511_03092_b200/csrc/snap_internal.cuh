@@ -190,9 +190,21 @@ size_t decode_gqa_mma_partial_floats(const Shape& s, int n_rows, int nsplit);
 cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_new, const void* v_new,
                                   const int* slot_ids, int n_active, void* k_cache, void* v_cache,
                                   int* seq_len, const int* valid_topk, void* out, float* partials,
-                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len = 1, int q_total = 0, int u0 = 0);
+                                  int nsplit, uint32_t* status, cudaStream_t st, int q_len = 1, int q_total = 0, int u0 = 0,
+                                  const int* block_idx = nullptr, const int* n_sel = nullptr, int blocks_cap = 0,
+                                  int block_tokens = 0);
 // (q_len tokens per sequence in one pass, q_len * g <= 8: tokens u0 .. u0 + q_len - 1 of the q_total per sequence that
 // q, k_new, v_new and out hold; q_total = 0: they hold exactly these)
+
+// (block_idx: per-step block lookup -- only the listed blocks of block_tokens rows of the third section are visited)
+// per-step block top-K: statistics of the third section's blocks, and the per-step selection (block_topk.cu)
+int block_count_max(const Shape& s, int block_tokens);
+bool block_topk_supported(int dtype, const Shape& s, int block_tokens);
+cudaError_t launch_block_stats(const Shape& s, int block_tokens, const int* slot_ids, int n, const void* k_cache,
+                               const int* valid_topk, void* stats, uint32_t* status, cudaStream_t st);
+cudaError_t launch_block_select(const Shape& s, int block_tokens, int n_blocks, const void* q, const int* slot_ids,
+                                int n_active, const void* stats, const int* valid_topk, int* block_idx, int* n_sel,
+                                uint32_t* status, cudaStream_t st);
 
 // latent attention (one 576-wide KV row shared by all heads, V = its first 512 dims): mma.sync kernel
 bool decode_mla_supported(int dtype, const Shape& s);
