@@ -523,6 +523,7 @@ def extras(hp, wl, dev):
     out["prefill_status"] = int(c.status.item())
     hp.compress_prompt(hp.pool[hp.resident[0]], 0)          # restore slot 0
     del p, qf, attn, cws
+    out["block_lookup"] = block_lookup_extra(wl, dev)
     out["concat_update_bytes"] = 2 * wl.batch * wl.n_kv_heads * hp.layout.slots * (wl.d_qk + wl.d_v) * 2
     out["ring_append_bytes"] = 2 * wl.batch * wl.n_kv_heads * (wl.d_qk + wl.d_v) * 2
     torch.cuda.empty_cache()
@@ -530,6 +531,86 @@ def extras(hp, wl, dev):
     out["config1_llama_32k_batch1"] = other_config(synth.CONFIGS[1], dev, n_layers=1)
     out["config3_latent_128k_batch8"] = other_config(synth.CONFIGS[3], dev, n_layers=1)
     out["config4_slice_4_of_32_layers_batch16"] = other_config(synth.CONFIGS[4], dev, n_layers=4)
+    return out
+
+
+def block_lookup_extra(wl, dev, n_seqs=8, L=131072, block_tokens=64, n_blocks=64):
+    """Per-step block top-K (the variant the paper leaves to future work) on the headline layer shape: n_seqs
+    prompts of L tokens kept whole, statistics per 64-token block, and every step the 64 highest-scoring
+    blocks per KV head attended together with sinks and window -- as many rows as the one-time top-K keeps."""
+    from paper_2511_03092_b200 import binding as B
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    cfg = B.make_config(n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, d_qk=wl.d_qk, d_v=wl.d_v, dtype=wl.torch_dtype,
+                        l_sink=wl.l_sink, l_recent=wl.l_recent, topk=L, l_obs=wl.l_obs, pool_kernel=wl.pool_kernel,
+                        softmax_scale=wl.scale, max_seqs=n_seqs)
+    lay = B.snap_cache_layout(cfg)
+    cache = B.alloc_cache(cfg, lay, dev)
+    p = synth.make_prompt(wl, L, SEED + 123, dev)
+    cws = torch.empty(B.snap_compress_workspace_bytes(cfg, [0, L]), dtype=torch.uint8, device=dev)
+    for slot in range(n_seqs):                               # the same prompt in every slot: the kernels do not care
+        B.snap_compress(cfg, lay, p["q_obs"][None], p["k"], p["v"], [0, L], [slot], cache.k_cache, cache.v_cache, cache.seq_len,
+                        cache.valid_topk, None, cws, cache.status)
+    del cws, p
+    slots = torch.arange(n_seqs, dtype=torch.int32, device=dev)
+    stats = torch.empty(B.snap_block_stats_bytes(cfg, block_tokens), dtype=torch.uint8, device=dev)
+    times = []
+    for r in range(4):
+        a, b = ev(), ev()
+        a.record()
+        B.snap_block_stats(cfg, lay, slots, n_seqs, cache.k_cache, cache.valid_topk, block_tokens, stats, cache.status)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    stats_ms = min(times[1:])
+    idx = torch.empty(n_seqs, wl.n_kv_heads, n_blocks, dtype=torch.int32, device=dev)
+    nsel = torch.empty(n_seqs, wl.n_kv_heads, dtype=torch.int32, device=dev)
+    ws = torch.empty(B.snap_decode_blocks_workspace_bytes(cfg, n_seqs, block_tokens, n_blocks), dtype=torch.uint8, device=dev)
+    sws = torch.empty(B.snap_block_select_workspace_bytes(cfg, n_seqs, block_tokens), dtype=torch.uint8, device=dev)
+    ins = [synth.make_decode_inputs(wl, n_seqs, SEED + 7, r, dev) for r in range(4)]
+    outb = torch.empty(n_seqs, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device=dev)
+
+    def select(d):
+        B.snap_block_select(cfg, lay, d["q"], slots, n_seqs, stats, cache.valid_topk, block_tokens, n_blocks, idx, nsel,
+                            sws, cache.status)
+
+    def attend(d):
+        B.snap_decode_attn_blocks(cfg, lay, d["q"], d["k_new"], d["v_new"], slots, n_seqs, cache.k_cache, cache.v_cache,
+                                  cache.seq_len, cache.valid_topk, block_tokens, n_blocks, idx, nsel, outb, ws, cache.status)
+
+    def timed(fn, reps=32):
+        for r in range(4):
+            fn(ins[r % 4])
+        a, b = ev(), ev()
+        a.record()
+        for r in range(reps):
+            fn(ins[r % 4])
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    select_ms = timed(select)
+    attend_ms = timed(attend)
+    step_ms = timed(lambda d: (select(d), attend(d)))
+    n_low = wl.l_sink + wl.l_recent
+    nb = -(-(L - n_low) // block_tokens)
+    row_b = (wl.d_qk + wl.d_v) * 2
+    stats_bytes = n_seqs * wl.n_kv_heads * nb * 2 * wl.d_qk * 2
+    attend_bytes = n_seqs * wl.n_kv_heads * (n_low + n_blocks * block_tokens) * row_b
+    full_bytes = n_seqs * wl.n_kv_heads * L * row_b
+    peak = _peaks()[0]
+    out = {"sequences": n_seqs, "prompt_tokens": L, "block_tokens": block_tokens, "blocks_per_sequence": nb,
+           "blocks_attended_per_kv_head": n_blocks, "statistics_ms_per_batch_once": stats_ms,
+           "statistics_GBps": n_seqs * wl.n_kv_heads * (L - n_low) * wl.d_qk * 2 / (stats_ms * 1e-3) / 1e9,
+           "select_ms": select_ms, "select_bytes": stats_bytes, "select_GBps": stats_bytes / (select_ms * 1e-3) / 1e9,
+           "attend_ms": attend_ms, "attend_bytes": attend_bytes, "attend_GBps": attend_bytes / (attend_ms * 1e-3) / 1e9,
+           "attend_frac_of_measured_hbm": attend_bytes / (attend_ms * 1e-3) / 1e9 / peak,
+           "step_ms_select_plus_attend": step_ms, "tokens_per_s": n_seqs / (step_ms * 1e-3),
+           "step_bytes": stats_bytes + attend_bytes, "step_GBps": (stats_bytes + attend_bytes) / (step_ms * 1e-3) / 1e9,
+           "step_frac_of_measured_hbm": (stats_bytes + attend_bytes) / (step_ms * 1e-3) / 1e9 / peak,
+           "full_kv_bytes_over_step_bytes": full_bytes / (stats_bytes + attend_bytes),
+           "status": int(cache.status.item())}
+    del cache, stats, ws, sws
+    torch.cuda.empty_cache()
     return out
 
 

@@ -351,8 +351,8 @@ int snap_append_kv_concat(const snap_config_t* cfg, const snap_layout_t* layout,
  *     included); rows that leave the window during decoding are dropped as before.
  * bf16 layers with 64-, 128- or 256-wide heads, a separate V and at most 8 query heads per KV
  * head; at most 8192 blocks per sequence; SNAP_ERR_UNSUPPORTED otherwise.  The scores are summed
- * in single precision (the products are exact): two blocks whose scores differ by less than about
- * 1e-6 relative may come out in either order.
+ * in single precision: two blocks whose scores differ by less than about 1e-6 relative may come
+ * out in either order.
  *
  * snap_block_stats    once per prompt, after snap_compress:
  *   stats_dev  out [max_seqs][Hkv][ceil(topk / block_tokens)][2][d_qk] in the cache's dtype (minimum, then
@@ -360,7 +360,8 @@ int snap_append_kv_concat(const snap_config_t* cfg, const snap_layout_t* layout,
  *              are written, rows of blocks past a prompt's last one are left alone.
  * snap_block_select   every step, before the attention:
  *   q_dev [n_active][Hq][d_qk];  block_idx_dev out [n_active][Hkv][n_blocks] ascending block numbers;
- *   n_selected_dev out [n_active][Hkv] = min(n_blocks, blocks of that prompt).
+ *   n_selected_dev out [n_active][Hkv] = min(n_blocks, blocks of that prompt);
+ *   scratch: snap_block_select_workspace_bytes(cfg, n_active, block_tokens) (the scores of every block).
  * snap_decode_attn_blocks   snap_decode_attn that visits only the listed blocks of the third section
  *   (arguments as there, plus the two arrays snap_block_select wrote, same n_blocks);
  *   scratch: snap_decode_blocks_workspace_bytes(cfg, n_active, block_tokens, n_blocks).
@@ -373,7 +374,9 @@ int snap_block_stats(const snap_config_t* cfg, const snap_layout_t* layout, cons
 int snap_block_select(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,
                       const int32_t* slot_ids_dev, int32_t n_active, const void* stats_dev,
                       const int32_t* valid_topk_dev, int32_t block_tokens, int32_t n_blocks,
-                      int32_t* block_idx_dev, int32_t* n_selected_dev, uint32_t* status_dev, void* cuda_stream);
+                      int32_t* block_idx_dev, int32_t* n_selected_dev, void* workspace_dev, size_t workspace_bytes,
+                      uint32_t* status_dev, void* cuda_stream);
+int64_t snap_block_select_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t block_tokens);
 int64_t snap_decode_blocks_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t block_tokens,
                                            int32_t n_blocks);
 int snap_decode_attn_blocks(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev,

@@ -92,7 +92,9 @@ def lib() -> C.CDLL:
     L.snap_block_stats.restype = C.c_int
     L.snap_block_stats.argtypes = [pcfg, play, vp, i32, vp, vp, i32, vp, vp, vp]
     L.snap_block_select.restype = C.c_int
-    L.snap_block_select.argtypes = [pcfg, play, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp, vp]
+    L.snap_block_select.argtypes = [pcfg, play, vp, vp, i32, vp, vp, i32, i32, vp, vp, vp, sz, vp, vp]
+    L.snap_block_select_workspace_bytes.restype = i64
+    L.snap_block_select_workspace_bytes.argtypes = [pcfg, i32, i32]
     L.snap_decode_blocks_workspace_bytes.restype = i64
     L.snap_decode_blocks_workspace_bytes.argtypes = [pcfg, i32, i32, i32]
     L.snap_decode_attn_blocks.restype = C.c_int
@@ -105,7 +107,8 @@ EXPORTS = ("snap_cache_layout", "snap_compress_workspace_bytes", "snap_decode_wo
            "snap_compress", "snap_append_kv", "snap_append_kv_concat", "snap_decode_attn",
            "snap_decode_multi_workspace_bytes", "snap_decode_attn_multi", "snap_decode_attn_static", "snap_status_string",
            "snap_kernel_launch_count", "snap_prefill_attn", "snap_compress_with_row_stats", "snap_debug_set_option",
-           "snap_block_stats_bytes", "snap_block_stats", "snap_block_select", "snap_decode_blocks_workspace_bytes",
+           "snap_block_stats_bytes", "snap_block_stats", "snap_block_select", "snap_block_select_workspace_bytes",
+           "snap_decode_blocks_workspace_bytes",
            "snap_decode_attn_blocks")
 
 # testing / tuning options of snap_debug_set_option
@@ -319,11 +322,19 @@ def snap_block_stats(cfg: SnapConfig, layout: SnapLayout, slot_ids_dev, n_seqs: 
 
 
 def snap_block_select(cfg: SnapConfig, layout: SnapLayout, q, slot_ids_dev, n_active: int, stats, valid_topk,
-                      block_tokens: int, n_blocks: int, block_idx, n_selected, status=None, stream=None) -> None:
+                      block_tokens: int, n_blocks: int, block_idx, n_selected, workspace, status=None, stream=None) -> None:
     """The n_blocks highest-scoring blocks per (sequence, KV head) for this step's queries."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().snap_block_select(C.byref(cfg), C.byref(layout), _ptr(q), _ptr(slot_ids_dev), int(n_active), _ptr(stats),
                                    _ptr(valid_topk), int(block_tokens), int(n_blocks), _ptr(block_idx), _ptr(n_selected),
-                                   _ptr(status), _stream(stream)), "snap_block_select")
+                                   _ptr(workspace), ws_bytes, _ptr(status), _stream(stream)), "snap_block_select")
+
+
+def snap_block_select_workspace_bytes(cfg: SnapConfig, n_active: int, block_tokens: int) -> int:
+    n = lib().snap_block_select_workspace_bytes(C.byref(cfg), int(n_active), int(block_tokens))
+    if n < 0:
+        raise SnapError(int(n), "snap_block_select_workspace_bytes")
+    return int(n)
 
 
 def snap_decode_blocks_workspace_bytes(cfg: SnapConfig, n_active: int, block_tokens: int, n_blocks: int) -> int:

@@ -626,8 +626,8 @@ int snap_block_stats(const snap_config_t* cfg, const snap_layout_t* layout, cons
 
 int snap_block_select(const snap_config_t* cfg, const snap_layout_t* layout, const void* q_dev, const int32_t* slot_ids_dev,
                       int32_t n_active, const void* stats_dev, const int32_t* valid_topk_dev, int32_t block_tokens,
-                      int32_t n_blocks, int32_t* block_idx_dev, int32_t* n_selected_dev, uint32_t* status_dev,
-                      void* cuda_stream) {
+                      int32_t n_blocks, int32_t* block_idx_dev, int32_t* n_selected_dev, void* workspace_dev,
+                      size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream) {
   const int rc = validate(cfg);
   if (rc != SNAP_OK) return rc;
   if (!layout) return SNAP_ERR_NULL_POINTER;
@@ -637,10 +637,23 @@ int snap_block_select(const snap_config_t* cfg, const snap_layout_t* layout, con
   if (bc != SNAP_OK) return bc;
   if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
   if (n_active == 0) return SNAP_OK;
-  if (!q_dev || !slot_ids_dev || !stats_dev || !valid_topk_dev || !block_idx_dev || !n_selected_dev) return SNAP_ERR_NULL_POINTER;
+  if (!q_dev || !slot_ids_dev || !stats_dev || !valid_topk_dev || !block_idx_dev || !n_selected_dev || !workspace_dev)
+    return SNAP_ERR_NULL_POINTER;
+  if (workspace_bytes < block_select_scratch_bytes(s, block_tokens, n_active)) return SNAP_ERR_WORKSPACE_TOO_SMALL;
   const cudaError_t e = launch_block_select(s, block_tokens, n_blocks, q_dev, slot_ids_dev, n_active, stats_dev, valid_topk_dev,
-                                            block_idx_dev, n_selected_dev, status_dev, static_cast<cudaStream_t>(cuda_stream));
+                                            block_idx_dev, n_selected_dev, workspace_dev, status_dev,
+                                            static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
+}
+
+int64_t snap_block_select_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t block_tokens) {
+  const int rc = validate(cfg);
+  if (rc != SNAP_OK) return rc;
+  if (n_active < 0) return SNAP_ERR_INVALID_ARG;
+  const Shape s = make_shape(cfg);
+  const int bc = blocks_check(cfg, s, block_tokens);
+  if (bc != SNAP_OK) return bc;
+  return (int64_t)block_select_scratch_bytes(s, block_tokens, n_active);
 }
 
 int64_t snap_decode_blocks_workspace_bytes(const snap_config_t* cfg, int32_t n_active, int32_t block_tokens, int32_t n_blocks) {

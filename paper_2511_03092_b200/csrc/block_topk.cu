@@ -8,12 +8,16 @@
 //   block_stats_kernel   once per prompt: element-wise minimum and maximum of the keys of every block of
 //                        `block_tokens` consecutive rows of that section (the last block may be
 //                        shorter), per KV head: stats[slot][kvh][block][0 = min, 1 = max][d_qk].
-//   block_select_kernel  every step: block b of KV head kvh scores
+//   block_score_kernel   every step: block b of KV head kvh scores
 //                            U = sum over the group's heads h, dims d of max(q[h][d] * min[d], q[h][d] * max[d]),
-//                        an upper bound of the group-summed logit of every key of the block; the
-//                        n_blocks highest-scoring blocks are listed in ascending order, ties to
-//                        the lower index.  The products of two bf16 values are exact in single
-//                        precision; only the summation order rounds.
+//                        an upper bound of the group-summed logit of every key of the block.  Since
+//                        min <= max, the larger product is q * max for q >= 0 and q * min otherwise, so
+//                        U = max . Q+ + min . Q- with Q+[d] = sum_h max(q[h][d], 0), Q-[d] = sum_h min(q[h][d], 0):
+//                        one pass over the statistics (512 bytes per block at d = 128), a warp-wide
+//                        16-byte load per block, in single precision.
+//   block_select_kernel  the n_blocks highest-scoring blocks of each (sequence, KV head), listed in
+//                        ascending order, ties to the lower index (four 8-bit radix passes over the
+//                        order-preserving integer images of the scores, then an ordered emission).
 // The decode kernel then visits the listed blocks instead of the whole section (decode_gqa_mma.cu).
 #include "snap_internal.cuh"
 
@@ -58,6 +62,7 @@ struct SelectArgs {
   const __nv_bfloat16* q;       // [n_active][Hq][d]
   const __nv_bfloat16* stats;
   const int* slot_ids; const int* valid_topk;
+  unsigned* keys;               // scratch [n_active][Hkv][nb_max]: order-preserving integer images of the scores
   int* block_idx;               // [n_active][Hkv][n_blocks]
   int* n_sel;                   // [n_active][Hkv]
   int Hq, Hkv, g, d, max_seqs, nb_max, bs, n_blocks;
@@ -70,15 +75,96 @@ __device__ __forceinline__ unsigned key_of(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// grid (Hkv, n_active), SEL_NT threads.  Dynamic shared memory: q group as floats [g][d], keys [nb].
+// grid (ceil(nb_max / 64), Hkv, n_active), 256 threads: a warp takes eight blocks, four at a time; a lane owns the same
+// 16-byte chunk (eight dims of the minimum row, or of the maximum row) of every block it visits.
+constexpr int SC_BLOCKS = 64;
+__global__ void __launch_bounds__(256) block_score_kernel(const SelectArgs a) {
+  const int kvh = blockIdx.y, i = blockIdx.z, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int slot = a.slot_ids[i];
+  if (slot < 0 || slot >= a.max_seqs) return;                  // the selection kernel reports it
+  const int nb = min((a.valid_topk[slot] + a.bs - 1) / a.bs, a.nb_max);
+  const int b_first = blockIdx.x * SC_BLOCKS + warp * 8;
+  if (b_first >= nb) return;
+  const int cpr = a.d / 8, cpb = 2 * cpr;                      // 16-byte chunks per row and per block (min row, max row)
+  // this lane's chunks: lane, lane + 32 (d = 256); per chunk eight entries of Q- (minimum row) or Q+ (maximum row)
+  float w[2][8];
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int c = lane + 32 * t;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) w[t][e] = 0.f;
+    if (c < cpb) {
+      const bool is_max = c >= cpr;
+      const int d0 = (is_max ? c - cpr : c) * 8;
+      for (int h = 0; h < a.g; ++h) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(a.q + ((long long)i * a.Hq + (long long)kvh * a.g + h) * a.d + d0);
+        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(p2[e]);
+          w[t][2 * e] += is_max ? fmaxf(f.x, 0.f) : fminf(f.x, 0.f);
+          w[t][2 * e + 1] += is_max ? fmaxf(f.y, 0.f) : fminf(f.y, 0.f);
+        }
+      }
+    }
+  }
+  const uint4* st = reinterpret_cast<const uint4*>(a.stats + (((long long)slot * a.Hkv + kvh) * a.nb_max) * 2 * a.d);
+  unsigned* out = a.keys + ((long long)i * a.Hkv + kvh) * a.nb_max;
+#pragma unroll 1
+  for (int b0 = b_first; b0 < min(b_first + 8, nb); b0 += 4) {
+    uint4 v[4][2];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        const int c = lane + 32 * t;
+        v[k][t] = b0 + k < nb && c < cpb ? st[(long long)(b0 + k) * cpb + c] : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float u = 0.f;
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v[k][t]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(p2[e]);
+          u = fmaf(f.x, w[t][2 * e], u);
+          u = fmaf(f.y, w[t][2 * e + 1], u);
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) u += __shfl_xor_sync(0xffffffffu, u, o);
+      if (lane == 0 && b0 + k < nb) out[b0 + k] = key_of(u);
+    }
+  }
+}
+
+// Block-wide exclusive scan of one int per thread (SEL_NT threads); returns the exclusive prefix and the total.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { const int u = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += u; }
+  __syncthreads();                                             // warp_tot may still be read from the previous scan
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  int before = 0, tot = 0;
+#pragma unroll
+  for (int w2 = 0; w2 < SEL_NT / 32; ++w2) { const int t = warp_tot[w2]; tot += t; if (w2 < warp) before += t; }
+  total = tot;
+  return before + incl - v;
+}
+
+// grid (Hkv, n_active), SEL_NT threads.  Dynamic shared memory: keys [nb].
 __global__ void __launch_bounds__(SEL_NT) block_select_kernel(const SelectArgs a) {
   extern __shared__ unsigned char sel_smem[];
-  float* qs = reinterpret_cast<float*>(sel_smem);                     // [g][d]
-  unsigned* keys = reinterpret_cast<unsigned*>(qs + a.g * a.d);       // [nb]
-  __shared__ int hist[256];
+  unsigned* keys = reinterpret_cast<unsigned*>(sel_smem);             // [nb]
+  __shared__ int hist[256], warp_tot[SEL_NT / 32];
   __shared__ unsigned s_prefix;
-  __shared__ int s_need, s_warp_tot[SEL_NT / 32][2], s_run[2];
-  const int kvh = blockIdx.x, i = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __shared__ int s_need;
+  const int kvh = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int slot = a.slot_ids[i];
   int* out = a.block_idx + ((long long)i * a.Hkv + kvh) * a.n_blocks;
@@ -92,88 +178,59 @@ __global__ void __launch_bounds__(SEL_NT) block_select_kernel(const SelectArgs a
   const int n_top = a.valid_topk[slot];
   const int nb = min((n_top + a.bs - 1) / a.bs, a.nb_max);
   const int want = min(a.n_blocks, nb);
-  for (int e = tid; e < a.g * a.d; e += SEL_NT)
-    qs[e] = __bfloat162float(a.q[((long long)i * a.Hq + (long long)kvh * a.g) * a.d + e]);
-  __syncthreads();
-  // ---- scores: one warp per block, lanes over pairs of dims ----
-  const __nv_bfloat16* st = a.stats + (((long long)slot * a.Hkv + kvh) * a.nb_max) * 2 * a.d;
-  for (int b = warp; b < nb; b += SEL_NT / 32) {
-    const __nv_bfloat16* mn = st + (long long)b * 2 * a.d, *mx = mn + a.d;
-    float u = 0.f;
-    for (int c = 2 * lane; c < a.d; c += 64) {
-      const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(mn + c));
-      const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(mx + c));
-      for (int h = 0; h < a.g; ++h) {
-        const float q0 = qs[h * a.d + c], q1 = qs[h * a.d + c + 1];
-        u += fmaxf(q0 * lo.x, q0 * hi.x) + fmaxf(q1 * lo.y, q1 * hi.y);
-      }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) u += __shfl_xor_sync(0xffffffffu, u, o);
-    if (lane == 0) keys[b] = key_of(u);
-  }
-  __syncthreads();
   if (want == nb) {                                            // every block: no selection needed
     for (int b = tid; b < nb; b += SEL_NT) out[b] = b;
     if (tid == 0) a.n_sel[i * a.Hkv + kvh] = nb;
     return;
   }
+  const unsigned* scored = a.keys + ((long long)i * a.Hkv + kvh) * a.nb_max;
+  for (int b = tid; b < nb; b += SEL_NT) keys[b] = scored[b];
   // ---- the want-th largest key by four 8-bit radix passes ----
-  if (tid == 0) { s_prefix = 0u; s_need = want; }
+  unsigned prefix = 0u;
+  int need = want;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     hist[tid] = 0;                                             // SEL_NT == 256 bins
     __syncthreads();
-    const unsigned prefix = s_prefix, himask = pass == 0 ? 0u : 0xffffffffu << (shift + 8);
+    const unsigned himask = pass == 0 ? 0u : 0xffffffffu << (shift + 8);
     for (int b = tid; b < nb; b += SEL_NT) {
       const unsigned k = keys[b];
       if ((k & himask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
     }
     __syncthreads();
-    if (tid == 0) {
-      int need = s_need, digit = 255;
-      for (; digit > 0; --digit) {                             // from the largest digit down
-        if (hist[digit] >= need) break;
-        need -= hist[digit];
-      }
-      s_prefix = prefix | ((unsigned)digit << shift);
-      s_need = need;                                           // how many of the keys equal so far are still wanted
+    // thread t looks at digit 255 - t: `above` = keys (under the prefix) with a larger digit
+    int total;
+    const int mine = hist[255 - tid];
+    const int above = block_exclusive_scan(mine, warp_tot, total);
+    if (above < need && above + mine >= need) {               // exactly one thread: the digit of the want-th largest key
+      s_prefix = prefix | ((unsigned)(255 - tid) << shift);
+      s_need = need - above;
     }
     __syncthreads();
+    prefix = s_prefix;
+    need = s_need;                                             // how many of the keys equal so far are still wanted
   }
-  const unsigned tau = s_prefix;
-  const int need_eq = s_need;                                  // blocks with key == tau to take, lowest indices first
-  // ---- ordered emission: key > tau, and the first need_eq with key == tau ----
-  if (tid == 0) { s_run[0] = 0; s_run[1] = 0; }                // blocks emitted, equal keys seen
-  __syncthreads();
-  for (int base = 0; base < nb; base += SEL_NT) {
-    const int b = base + tid;
-    const unsigned k = b < nb ? keys[b] : 0u;
-    const int gt = b < nb && k > tau, eq = b < nb && k == tau;
-    // exclusive scans of eq (to rank the equal keys) and of the emitted flags over the chunk
-    int eq_incl = eq;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, eq_incl, o); if (lane >= o) eq_incl += v; }
-    if (lane == 31) s_warp_tot[warp][1] = eq_incl;
-    __syncthreads();
-    int eq_before = s_run[1];
-    for (int w2 = 0; w2 < warp; ++w2) eq_before += s_warp_tot[w2][1];
-    const int take = gt || (eq && eq_before + eq_incl - 1 < need_eq);
-    int tk_incl = take;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, tk_incl, o); if (lane >= o) tk_incl += v; }
-    if (lane == 31) s_warp_tot[warp][0] = tk_incl;
-    __syncthreads();
-    int pos = s_run[0];
-    for (int w2 = 0; w2 < warp; ++w2) pos += s_warp_tot[w2][0];
-    if (take && pos + tk_incl - 1 < want) out[pos + tk_incl - 1] = b;
-    __syncthreads();
-    if (tid == 0) {
-      int t0 = 0, t1 = 0;
-      for (int w2 = 0; w2 < SEL_NT / 32; ++w2) { t0 += s_warp_tot[w2][0]; t1 += s_warp_tot[w2][1]; }
-      s_run[0] += t0; s_run[1] += t1;
-    }
-    __syncthreads();
+  const unsigned tau = prefix;
+  const int need_eq = need;                                    // blocks with key == tau to take, lowest indices first
+  // ---- ordered emission: key > tau, and the first need_eq with key == tau; a thread owns a run of consecutive blocks ----
+  const int run = (nb + SEL_NT - 1) / SEL_NT, b0 = tid * run, b1 = min(b0 + run, nb);
+  int n_eq = 0;
+  for (int b = b0; b < b1; ++b) n_eq += keys[b] == tau;
+  int total;
+  int eq_rank = block_exclusive_scan(n_eq, warp_tot, total);
+  int n_take = 0;
+  for (int b = b0; b < b1; ++b) {
+    const unsigned k = keys[b];
+    n_take += k > tau || (k == tau && eq_rank < need_eq);
+    eq_rank += k == tau;
+  }
+  eq_rank -= n_eq;
+  int pos = block_exclusive_scan(n_take, warp_tot, total);
+  for (int b = b0; b < b1; ++b) {
+    const unsigned k = keys[b];
+    const bool take = k > tau || (k == tau && eq_rank < need_eq);
+    eq_rank += k == tau;
+    if (take && pos < want) out[pos++] = b;
   }
   if (tid == 0) a.n_sel[i * a.Hkv + kvh] = want;
 }
@@ -183,7 +240,7 @@ __global__ void __launch_bounds__(SEL_NT) block_select_kernel(const SelectArgs a
 int block_count_max(const Shape& s, int block_tokens) { return (s.K + block_tokens - 1) / block_tokens; }
 
 bool block_topk_supported(int dtype, const Shape& s, int block_tokens) {
-  return dtype == SNAP_BF16 && !s.v_aliases_k && s.d_qk % 2 == 0 && s.d_qk <= 512 && block_tokens >= 16 && block_tokens % 16 == 0 &&
+  return dtype == SNAP_BF16 && !s.v_aliases_k && s.d_qk % 8 == 0 && s.d_qk <= 256 && block_tokens >= 16 && block_tokens % 16 == 0 &&
          block_tokens <= 1024 && s.K > 0 && block_count_max(s, block_tokens) <= MAX_BLOCKS && s.g <= 8;
 }
 
@@ -201,21 +258,26 @@ cudaError_t launch_block_stats(const Shape& s, int block_tokens, const int* slot
   return cudaGetLastError();
 }
 
+size_t block_select_scratch_bytes(const Shape& s, int block_tokens, int n_active) {
+  return (size_t)n_active * s.Hkv * block_count_max(s, block_tokens) * sizeof(unsigned);
+}
+
 cudaError_t launch_block_select(const Shape& s, int block_tokens, int n_blocks, const void* q, const int* slot_ids,
                                 int n_active, const void* stats, const int* valid_topk, int* block_idx, int* n_sel,
-                                uint32_t* status, cudaStream_t st) {
+                                void* scratch, uint32_t* status, cudaStream_t st) {
   if (n_active == 0) return cudaSuccess;
   SelectArgs a;
   a.q = static_cast<const __nv_bfloat16*>(q);
   a.stats = static_cast<const __nv_bfloat16*>(stats);
   a.slot_ids = slot_ids; a.valid_topk = valid_topk; a.block_idx = block_idx; a.n_sel = n_sel;
+  a.keys = static_cast<unsigned*>(scratch);
   a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.d = s.d_qk; a.max_seqs = s.max_seqs;
   a.nb_max = block_count_max(s, block_tokens); a.bs = block_tokens; a.n_blocks = n_blocks; a.status = status;
-  const size_t smem = (size_t)s.g * s.d_qk * sizeof(float) + (size_t)a.nb_max * sizeof(unsigned);
-  static SmemLimit limit = {};
-  if (smem > 48 * 1024)
-    if (cudaError_t e = ensure_dyn_smem(block_select_kernel, smem, limit)) return e;
-  cudaError_t e = launch_pdl(block_select_kernel, dim3(s.Hkv, n_active), dim3(SEL_NT), smem, st, a);
+  cudaError_t e = launch_pdl(block_score_kernel, dim3((a.nb_max + SC_BLOCKS - 1) / SC_BLOCKS, s.Hkv, n_active), dim3(256), 0, st, a);
+  count_launch();
+  if (e != cudaSuccess) return e;
+  const size_t smem = (size_t)a.nb_max * sizeof(unsigned);
+  e = launch_pdl(block_select_kernel, dim3(s.Hkv, n_active), dim3(SEL_NT), smem, st, a);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -204,7 +204,8 @@ cudaError_t launch_block_stats(const Shape& s, int block_tokens, const int* slot
                                const int* valid_topk, void* stats, uint32_t* status, cudaStream_t st);
 cudaError_t launch_block_select(const Shape& s, int block_tokens, int n_blocks, const void* q, const int* slot_ids,
                                 int n_active, const void* stats, const int* valid_topk, int* block_idx, int* n_sel,
-                                uint32_t* status, cudaStream_t st);
+                                void* scratch, uint32_t* status, cudaStream_t st);
+size_t block_select_scratch_bytes(const Shape& s, int block_tokens, int n_active);
 
 // latent attention (one 576-wide KV row shared by all heads, V = its first 512 dims): mma.sync kernel
 bool decode_mla_supported(int dtype, const Shape& s);

@@ -72,6 +72,7 @@ def _run(wl, lengths, bs, n_blocks, steps, seed):
     block_idx = torch.full((n, wl.n_kv_heads, n_blocks), -9, dtype=torch.int32, device="cuda")
     n_sel = torch.full((n, wl.n_kv_heads), -9, dtype=torch.int32, device="cuda")
     ws = torch.empty(B.snap_decode_blocks_workspace_bytes(layer.cfg, n, bs, n_blocks), dtype=torch.uint8, device="cuda")
+    sws = torch.empty(B.snap_block_select_workspace_bytes(layer.cfg, n, bs), dtype=torch.uint8, device="cuda")
     out = torch.empty(n, wl.n_q_heads, wl.d_v, dtype=torch.bfloat16, device="cuda")
     swaps = 0
     for step in range(steps):
@@ -83,7 +84,7 @@ def _run(wl, lengths, bs, n_blocks, steps, seed):
                     pos = cfg.l_sink + (step * 37 + i * 11) % (L - cfg.l_sr)
                     q[i] = (prompts[i]["k"][pos].float().repeat_interleave(cfg.group, dim=0) * 3.0).to(torch.bfloat16)
         B.snap_block_select(layer.cfg, layer.layout, q.cuda(), slots_dev, n, stats, c.valid_topk, bs, n_blocks, block_idx,
-                            n_sel, c.status)
+                            n_sel, sws, c.status)
         B.snap_decode_attn_blocks(layer.cfg, layer.layout, q.cuda(), d["k_new"].cuda(), d["v_new"].cuda(), slots_dev, n,
                                   c.k_cache, c.v_cache, c.seq_len, c.valid_topk, bs, n_blocks, block_idx, n_sel, out, ws,
                                   c.status)
