@@ -42,7 +42,11 @@ against torch's double-precision causal routine, the running-mean closed form an
 causality; the Eq. 4 normalisers against scipy's logsumexp and by rebuilding Eq. 1.
 Parity unpinned by the paper (fixed only by the readings above): which softmax
 domain, pooling domain, GQA reduction order and ring-fill convention the
-authors' own implementation uses.
+authors' own implementation uses; and the whole per-step block top-K section at
+the end of this file, which the paper only names as future work (its definition
+and its pins -- hand-worked values, the bound property, the one-token-block
+special case, all blocks = everything kept -- are stated there and in
+tests/test_oracle_blocks.py).
 """
 from __future__ import annotations
 
