@@ -800,12 +800,17 @@ def run_case(args):
                (672 MB of cache read per step, ~1.5 GB resident);
     `compress` one prompt of --case-len tokens compressed a few times;
     `prefill`  the same, then the prompt's causal attention (emitting the Eq. 4 normalisers) and the
-               compression that consumes them."""
+               compression that consumes them;
+    `blocks`   the per-step block top-K path over --case-seqs prompts of --case-len tokens kept whole
+               (0.54 GB of cache per 131072-token prompt)."""
     from paper_2511_03092_b200 import binding as B
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     wl = synth.CONFIGS[2]
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if args.case == "blocks":
+        print(json.dumps(dict(case="blocks", **block_lookup_extra(wl, dev, n_seqs=args.case_seqs, L=args.case_len))))
+        return
     if args.case == "decode":
         wl = wl.scaled(prompt_len=(8192, 8192))
         hp = HotPath.__new__(HotPath)
@@ -987,9 +992,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the 128k-compress and full-KV side measurements")
-    ap.add_argument("--case", choices=["decode", "compress", "prefill"], default=None,
+    ap.add_argument("--case", choices=["decode", "compress", "prefill", "blocks"], default=None,
                     help="small single-kernel-family case for profiler captures")
     ap.add_argument("--case-len", type=int, default=131072)
+    ap.add_argument("--case-seqs", type=int, default=8, help="sequences of the `blocks` case")
     ap.add_argument("--workload", type=int, choices=[0, 1, 3, 4], default=None,
                     help="report compress and decode times of another benchmark configuration (context only)")
     args = ap.parse_args()

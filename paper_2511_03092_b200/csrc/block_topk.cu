@@ -75,16 +75,16 @@ __device__ __forceinline__ unsigned key_of(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// grid (ceil(nb_max / 64), Hkv, n_active), 256 threads: a warp takes eight blocks, four at a time; a lane owns the same
+// grid (ceil(nb_max / 256), Hkv, n_active), 256 threads: a warp takes 32 blocks, four at a time; a lane owns the same
 // 16-byte chunk (eight dims of the minimum row, or of the maximum row) of every block it visits.
-constexpr int SC_BLOCKS = 64;
+constexpr int SC_BLOCKS = 256, SC_PER_WARP = SC_BLOCKS / 8;
 __global__ void __launch_bounds__(256) block_score_kernel(const SelectArgs a) {
   const int kvh = blockIdx.y, i = blockIdx.z, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int slot = a.slot_ids[i];
   if (slot < 0 || slot >= a.max_seqs) return;                  // the selection kernel reports it
   const int nb = min((a.valid_topk[slot] + a.bs - 1) / a.bs, a.nb_max);
-  const int b_first = blockIdx.x * SC_BLOCKS + warp * 8;
+  const int b_first = blockIdx.x * SC_BLOCKS + warp * SC_PER_WARP;
   if (b_first >= nb) return;
   const int cpr = a.d / 8, cpb = 2 * cpr;                      // 16-byte chunks per row and per block (min row, max row)
   // this lane's chunks: lane, lane + 32 (d = 256); per chunk eight entries of Q- (minimum row) or Q+ (maximum row)
@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(256) block_score_kernel(const SelectArgs a) {
   const uint4* st = reinterpret_cast<const uint4*>(a.stats + (((long long)slot * a.Hkv + kvh) * a.nb_max) * 2 * a.d);
   unsigned* out = a.keys + ((long long)i * a.Hkv + kvh) * a.nb_max;
 #pragma unroll 1
-  for (int b0 = b_first; b0 < min(b_first + 8, nb); b0 += 4) {
+  for (int b0 = b_first; b0 < min(b_first + SC_PER_WARP, nb); b0 += 4) {
     uint4 v[4][2];
 #pragma unroll
     for (int k = 0; k < 4; ++k)
