@@ -351,8 +351,11 @@ int snap_append_kv_concat(const snap_config_t* cfg, const snap_layout_t* layout,
  *     included); rows that leave the window during decoding are dropped as before.
  * bf16 layers with 64-, 128- or 256-wide heads, a separate V and at most 8 query heads per KV
  * head; at most 8192 blocks per sequence; SNAP_ERR_UNSUPPORTED otherwise.  The scores are summed
- * in single precision: two blocks whose scores differ by less than about 1e-6 relative may come
- * out in either order.
+ * in single precision for every block; the blocks that single precision cannot tell from the
+ * last selected one (a rigorous error bound per block) are scored again in double precision and
+ * ranked by that, so the selection is the one the exact scores give down to relative differences
+ * of about 1e-15.  More than 256 such blocks for one (sequence, KV head): the single-precision
+ * order stands and SNAP_DEV_BAND_OVERFLOW is raised in *status_dev.
  *
  * snap_block_stats    once per prompt, after snap_compress:
  *   stats_dev  out [max_seqs][Hkv][ceil(topk / block_tokens)][2][d_qk] in the cache's dtype (minimum, then
@@ -404,7 +407,8 @@ int snap_decode_attn_blocks(const snap_config_t* cfg, const snap_layout_t* layou
 #define SNAP_OPT_PREFILL_KERNEL 6        /* 1: portable prefill attention kernel    SNAP_PREFILL_PATH=simt   */
 #define SNAP_OPT_PREFILL_SINGLE_HEADS 7  /* 1: one head per CTA in prefill attention  SNAP_PREFILL_HEADS=1   */
 #define SNAP_OPT_REFINE_OFF 8            /* 1: skip the double-precision re-scoring near the top-K
-                                               threshold (single-precision order)  SNAP_REFINE=0            */
+                                               threshold and near the block-selection threshold
+                                               (single-precision order)            SNAP_REFINE=0            */
 #define SNAP_OPT_COUNT 9
 int snap_debug_set_option(int option, int value);
 

@@ -14,10 +14,17 @@
 //                        min <= max, the larger product is q * max for q >= 0 and q * min otherwise, so
 //                        U = max . Q+ + min . Q- with Q+[d] = sum_h max(q[h][d], 0), Q-[d] = sum_h min(q[h][d], 0):
 //                        one pass over the statistics (512 bytes per block at d = 128), a warp-wide
-//                        16-byte load per block, in single precision.
+//                        16-byte load per block, in single precision; next to U the kernel writes
+//                        A = sum of the absolute values of U's terms, which bounds U's rounding error.
 //   block_select_kernel  the n_blocks highest-scoring blocks of each (sequence, KV head), listed in
-//                        ascending order, ties to the lower index (four 8-bit radix passes over the
-//                        order-preserving integer images of the scores, then an ordered emission).
+//                        ascending order, ties to the lower index: four 8-bit radix passes over the
+//                        order-preserving integer images of the scores find the threshold; the blocks
+//                        whose single-precision score cannot be told from the threshold (within
+//                        2e-5 (A + A_threshold)) are scored again in double precision -- a few
+//                        blocks, 256 multiply-adds each -- and ranked by that, so the selection is
+//                        the one the exact scores give (down to 1e-15 relative); then an ordered
+//                        emission.  More than 256 such blocks: the single-precision order stands
+//                        and SNAP_DEV_BAND_OVERFLOW is raised.
 // The decode kernel then visits the listed blocks instead of the whole section (decode_gqa_mma.cu).
 #include "snap_internal.cuh"
 
@@ -62,10 +69,11 @@ struct SelectArgs {
   const __nv_bfloat16* q;       // [n_active][Hq][d]
   const __nv_bfloat16* stats;
   const int* slot_ids; const int* valid_topk;
-  unsigned* keys;               // scratch [n_active][Hkv][nb_max]: order-preserving integer images of the scores
+  uint2* keys;                  // scratch [n_active][Hkv][nb_max]: (order-preserving integer image of U, bits of A)
   int* block_idx;               // [n_active][Hkv][n_blocks]
   int* n_sel;                   // [n_active][Hkv]
   int Hq, Hkv, g, d, max_seqs, nb_max, bs, n_blocks;
+  int no_rescoring;             // testing aid (option SNAP_OPT_REFINE_OFF): keep the single-precision order
   uint32_t* status;
 };
 
@@ -110,7 +118,7 @@ __global__ void __launch_bounds__(256) block_score_kernel(const SelectArgs a) {
     }
   }
   const uint4* st = reinterpret_cast<const uint4*>(a.stats + (((long long)slot * a.Hkv + kvh) * a.nb_max) * 2 * a.d);
-  unsigned* out = a.keys + ((long long)i * a.Hkv + kvh) * a.nb_max;
+  uint2* out = a.keys + ((long long)i * a.Hkv + kvh) * a.nb_max;
 #pragma unroll 1
   for (int b0 = b_first; b0 < min(b_first + SC_PER_WARP, nb); b0 += 4) {
     uint4 v[4][2];
@@ -123,7 +131,7 @@ __global__ void __launch_bounds__(256) block_score_kernel(const SelectArgs a) {
       }
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      float u = 0.f;
+      float u = 0.f, ab = 0.f;
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
         const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v[k][t]);
@@ -132,11 +140,16 @@ __global__ void __launch_bounds__(256) block_score_kernel(const SelectArgs a) {
           const float2 f = __bfloat1622float2(p2[e]);
           u = fmaf(f.x, w[t][2 * e], u);
           u = fmaf(f.y, w[t][2 * e + 1], u);
+          ab = fmaf(fabsf(f.x), fabsf(w[t][2 * e]), ab);
+          ab = fmaf(fabsf(f.y), fabsf(w[t][2 * e + 1]), ab);
         }
       }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) u += __shfl_xor_sync(0xffffffffu, u, o);
-      if (lane == 0 && b0 + k < nb) out[b0 + k] = key_of(u);
+      for (int o = 16; o > 0; o >>= 1) {
+        u += __shfl_xor_sync(0xffffffffu, u, o);
+        ab += __shfl_xor_sync(0xffffffffu, ab, o);
+      }
+      if (lane == 0 && b0 + k < nb) out[b0 + k] = make_uint2(key_of(u), __float_as_uint(ab));
     }
   }
 }
@@ -157,14 +170,24 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int& t
   return before + incl - v;
 }
 
-// grid (Hkv, n_active), SEL_NT threads.  Dynamic shared memory: keys [nb].
+__device__ __forceinline__ float float_of_key(unsigned k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+constexpr int BAND_CAP = 256;
+constexpr float BAND_REL = 2e-5f;      // 256 single-precision multiply-adds: |error| <= 256 * 2^-24 * A = 1.5e-5 A
+
+// grid (Hkv, n_active), SEL_NT threads.  Dynamic shared memory: keys [nb] | take flags [nb].
 __global__ void __launch_bounds__(SEL_NT) block_select_kernel(const SelectArgs a) {
   extern __shared__ unsigned char sel_smem[];
   unsigned* keys = reinterpret_cast<unsigned*>(sel_smem);             // [nb]
+  unsigned char* take = reinterpret_cast<unsigned char*>(keys + a.nb_max);   // [nb]
   __shared__ int hist[256], warp_tot[SEL_NT / 32];
   __shared__ unsigned s_prefix;
-  __shared__ int s_need;
-  const int kvh = blockIdx.x, i = blockIdx.y, tid = threadIdx.x;
+  __shared__ int s_need, s_nband, s_nsure, s_thr_block;
+  __shared__ int band_idx[BAND_CAP];
+  __shared__ double band_u[BAND_CAP];
+  const int kvh = blockIdx.x, i = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int slot = a.slot_ids[i];
   int* out = a.block_idx + ((long long)i * a.Hkv + kvh) * a.n_blocks;
@@ -183,9 +206,10 @@ __global__ void __launch_bounds__(SEL_NT) block_select_kernel(const SelectArgs a
     if (tid == 0) a.n_sel[i * a.Hkv + kvh] = nb;
     return;
   }
-  const unsigned* scored = a.keys + ((long long)i * a.Hkv + kvh) * a.nb_max;
-  for (int b = tid; b < nb; b += SEL_NT) keys[b] = scored[b];
-  // ---- the want-th largest key by four 8-bit radix passes ----
+  const uint2* scored = a.keys + ((long long)i * a.Hkv + kvh) * a.nb_max;
+  for (int b = tid; b < nb; b += SEL_NT) keys[b] = scored[b].x;
+  if (tid == 0) { s_nband = 0; s_nsure = 0; s_thr_block = 0x7fffffff; }
+  // ---- the want-th largest single-precision score by four 8-bit radix passes ----
   unsigned prefix = 0u;
   int need = want;
   for (int pass = 0; pass < 4; ++pass) {
@@ -211,27 +235,105 @@ __global__ void __launch_bounds__(SEL_NT) block_select_kernel(const SelectArgs a
     need = s_need;                                             // how many of the keys equal so far are still wanted
   }
   const unsigned tau = prefix;
-  const int need_eq = need;                                    // blocks with key == tau to take, lowest indices first
-  // ---- ordered emission: key > tau, and the first need_eq with key == tau; a thread owns a run of consecutive blocks ----
+  const int need_eq = need;                                    // single-precision rule: this many of the blocks at the threshold
+  // ---- which blocks can single precision not tell from the threshold? ----
+  for (int b = tid; b < nb; b += SEL_NT)
+    if (keys[b] == tau) atomicMin(&s_thr_block, b);
+  __syncthreads();
+  const float tau_f = float_of_key(tau), a_tau = __uint_as_float(scored[s_thr_block].y);
+  for (int b = tid; b < nb; b += SEL_NT) {
+    const float u = float_of_key(keys[b]);
+    const float band = BAND_REL * (__uint_as_float(scored[b].y) + a_tau);
+    unsigned char t = 0;
+    if (u - tau_f > band) { t = 1; atomicAdd(&s_nsure, 1); }   // above the threshold whatever the rounding
+    else if (tau_f - u <= band) {                              // undecided
+      const int m = atomicAdd(&s_nband, 1);
+      if (m < BAND_CAP) band_idx[m] = b;
+    }
+    take[b] = t;
+  }
+  __syncthreads();
+  const int n_band = s_nband, n_sure = s_nsure;
+  if (n_band <= BAND_CAP && !a.no_rescoring) {
+    // ---- their scores again, in double precision: a warp per block, a lane per 16-byte chunk ----
+    const int cpr = a.d / 8, cpb = 2 * cpr;
+    if (warp < n_band) {
+      double w[2][8];
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        const int c = lane + 32 * t;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) w[t][e] = 0.0;
+        if (c < cpb) {
+          const bool is_max = c >= cpr;
+          const int d0 = (is_max ? c - cpr : c) * 8;
+          for (int h = 0; h < a.g; ++h) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(a.q + ((long long)i * a.Hq + (long long)kvh * a.g + h) * a.d + d0);
+            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 f = __bfloat1622float2(p2[e]);
+              w[t][2 * e] += (double)(is_max ? fmaxf(f.x, 0.f) : fminf(f.x, 0.f));
+              w[t][2 * e + 1] += (double)(is_max ? fmaxf(f.y, 0.f) : fminf(f.y, 0.f));
+            }
+          }
+        }
+      }
+      const uint4* st = reinterpret_cast<const uint4*>(a.stats + (((long long)slot * a.Hkv + kvh) * a.nb_max) * 2 * a.d);
+      for (int m = warp; m < n_band; m += SEL_NT / 32) {
+        double u = 0.0;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          const int c = lane + 32 * t;
+          if (c < cpb) {
+            const uint4 v = st[(long long)band_idx[m] * cpb + c];
+            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 f = __bfloat1622float2(p2[e]);
+              u = fma((double)f.x, w[t][2 * e], u);
+              u = fma((double)f.y, w[t][2 * e + 1], u);
+            }
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) u += __shfl_xor_sync(0xffffffffu, u, o);
+        if (lane == 0) band_u[m] = u;
+      }
+    }
+    __syncthreads();
+    // ---- the best (want - n_sure) of them: larger score first, lower block number on equal scores ----
+    const int room = want - n_sure;
+    for (int m = tid; m < n_band; m += SEL_NT) {
+      const double um = band_u[m];
+      const int bm = band_idx[m];
+      int rank = 0;
+      for (int o = 0; o < n_band; ++o) rank += band_u[o] > um || (band_u[o] == um && band_idx[o] < bm);
+      if (rank < room) take[bm] = 1;
+    }
+  } else {
+    // too many to re-score: the single-precision order stands (blocks at the threshold by block number)
+    if (tid == 0 && a.status && !a.no_rescoring) atomicOr(a.status, SNAP_DEV_BAND_OVERFLOW);
+    const int run0 = (nb + SEL_NT - 1) / SEL_NT, c0 = tid * run0, c1 = min(c0 + run0, nb);
+    int n_eq = 0;
+    for (int b = c0; b < c1; ++b) n_eq += keys[b] == tau;
+    int total;
+    int eq_rank = block_exclusive_scan(n_eq, warp_tot, total);
+    for (int b = c0; b < c1; ++b) {
+      const unsigned k = keys[b];
+      take[b] = k > tau || (k == tau && eq_rank < need_eq);
+      eq_rank += k == tau;
+    }
+  }
+  __syncthreads();
+  // ---- ordered emission: a thread owns a run of consecutive blocks ----
   const int run = (nb + SEL_NT - 1) / SEL_NT, b0 = tid * run, b1 = min(b0 + run, nb);
-  int n_eq = 0;
-  for (int b = b0; b < b1; ++b) n_eq += keys[b] == tau;
-  int total;
-  int eq_rank = block_exclusive_scan(n_eq, warp_tot, total);
   int n_take = 0;
-  for (int b = b0; b < b1; ++b) {
-    const unsigned k = keys[b];
-    n_take += k > tau || (k == tau && eq_rank < need_eq);
-    eq_rank += k == tau;
-  }
-  eq_rank -= n_eq;
+  for (int b = b0; b < b1; ++b) n_take += take[b];
+  int total;
   int pos = block_exclusive_scan(n_take, warp_tot, total);
-  for (int b = b0; b < b1; ++b) {
-    const unsigned k = keys[b];
-    const bool take = k > tau || (k == tau && eq_rank < need_eq);
-    eq_rank += k == tau;
-    if (take && pos < want) out[pos++] = b;
-  }
+  for (int b = b0; b < b1; ++b)
+    if (take[b] && pos < want) out[pos++] = b;
   if (tid == 0) a.n_sel[i * a.Hkv + kvh] = want;
 }
 
@@ -259,7 +361,7 @@ cudaError_t launch_block_stats(const Shape& s, int block_tokens, const int* slot
 }
 
 size_t block_select_scratch_bytes(const Shape& s, int block_tokens, int n_active) {
-  return (size_t)n_active * s.Hkv * block_count_max(s, block_tokens) * sizeof(unsigned);
+  return (size_t)n_active * s.Hkv * block_count_max(s, block_tokens) * sizeof(uint2);
 }
 
 cudaError_t launch_block_select(const Shape& s, int block_tokens, int n_blocks, const void* q, const int* slot_ids,
@@ -270,13 +372,14 @@ cudaError_t launch_block_select(const Shape& s, int block_tokens, int n_blocks, 
   a.q = static_cast<const __nv_bfloat16*>(q);
   a.stats = static_cast<const __nv_bfloat16*>(stats);
   a.slot_ids = slot_ids; a.valid_topk = valid_topk; a.block_idx = block_idx; a.n_sel = n_sel;
-  a.keys = static_cast<unsigned*>(scratch);
+  a.keys = static_cast<uint2*>(scratch);
   a.Hq = s.Hq; a.Hkv = s.Hkv; a.g = s.g; a.d = s.d_qk; a.max_seqs = s.max_seqs;
   a.nb_max = block_count_max(s, block_tokens); a.bs = block_tokens; a.n_blocks = n_blocks; a.status = status;
+  a.no_rescoring = option(SNAP_OPT_REFINE_OFF) != 0;
   cudaError_t e = launch_pdl(block_score_kernel, dim3((a.nb_max + SC_BLOCKS - 1) / SC_BLOCKS, s.Hkv, n_active), dim3(256), 0, st, a);
   count_launch();
   if (e != cudaSuccess) return e;
-  const size_t smem = (size_t)a.nb_max * sizeof(unsigned);
+  const size_t smem = (size_t)a.nb_max * (sizeof(unsigned) + 1) + 16;
   e = launch_pdl(block_select_kernel, dim3(s.Hkv, n_active), dim3(SEL_NT), smem, st, a);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();

@@ -1,6 +1,7 @@
 """Per-step block top-K through the C ABI against the oracle: block statistics byte for byte, the
-per-step selection (exact, up to blocks whose oracle scores lie within 1e-5 relative of the last
-selected one: the kernel sums in single precision), and the attention over sinks, window and the
+per-step selection (exact, up to blocks whose oracle scores lie within 1e-12 relative of the last
+selected one: the kernel re-scores the blocks near its threshold in double precision, the oracle
+sums in double throughout, in another order), and the attention over sinks, window and the
 selected blocks, on ragged batches with prompts that have no middle, a short last block, more
 budget than blocks, and rings that wrap."""
 import numpy as np
@@ -14,7 +15,7 @@ from tests import _harness as H
 
 pytestmark = pytest.mark.gpu
 
-SCORE_REL = 1e-5
+SCORE_REL = 1e-12
 
 
 def _workload(hq, hkv, d, topk, l_recent=48, l_sink=4):
@@ -129,6 +130,89 @@ def test_block_lookup_at_the_benchmark_shape():
     wl = synth.Workload("blocks_128k", 32, 8, 128, 128, "bf16", 4, 1024, 131072, 64, 7, batch=1, prompt_len=(131072, 131072),
                         decode_steps=3, salience="zipf")
     _run(wl, [131072, 40000], 64, 64, steps=3, seed=211)
+
+
+def _near_tie_case(gap_dim_q, seed):
+    """Blocks of identical keys (minimum = maximum, so a block's score is the group-summed logit itself): three strong
+    ones, many weak ones, and a pair of equal strength whose second member is one bf16 step larger in one dim; the query
+    is tiny in that dim, so the pair's scores differ by 1e-9 .. 1e-8 relative -- below what a 256-term single-precision
+    sum resolves, far above what double precision does."""
+    bs, n_blocks, nb = 16, 4, 40
+    wl = _workload(4, 1, 128, topk=nb * bs, l_recent=16, l_sink=0)
+    g = torch.Generator().manual_seed(seed)
+    base = (torch.randn(128, generator=g).abs() + 0.5).to(torch.bfloat16)
+    L = nb * bs + wl.l_recent
+    p = synth.make_prompt(wl, L, seed)
+    k = torch.zeros(L, 1, 128, dtype=torch.bfloat16)
+    strength = torch.ones(nb)
+    strong = [5, 17, 33]
+    pair = (11, 26)
+    strength[strong] = 3.0
+    strength[list(pair)] = 2.0
+    for b in range(nb):
+        k[b * bs:(b + 1) * bs, 0] = (base.float() * strength[b]).to(torch.bfloat16)
+    d_star = 77
+    row = k[pair[1] * bs, 0].clone()
+    step = torch.tensor(row[d_star].view(torch.int16).item() + 1, dtype=torch.int16).view(torch.bfloat16)   # next bf16 up
+    k[pair[1] * bs:(pair[1] + 1) * bs, 0, d_star] = step
+    k[L - wl.l_recent:] = p["k"][L - wl.l_recent:]
+    p["k"] = k
+    q = base.float().repeat(4, 1)
+    q[:, d_star] = gap_dim_q
+    return wl, p, q.to(torch.bfloat16), bs, n_blocks, strong, pair
+
+
+@pytest.mark.parametrize("gap_dim_q,winner", [(2.0 ** -12, 1), (-(2.0 ** -12), 0), (2.0 ** -15, 1), (-(2.0 ** -15), 0)],
+                         ids=["second_larger_q_2^-12", "first_larger_q_2^-12", "second_larger_q_2^-15", "first_larger_q_2^-15"])
+def test_blocks_nearly_tied_at_the_threshold_are_ranked_by_their_exact_scores(snap_option, gap_dim_q, winner):
+    """The last place goes to the member of the pair whose exact score is larger, whichever its block number.  With the
+    re-scoring switched off the single-precision order (a tie, hence the lower block number) must get at least one of
+    the four cases wrong; that run is the evidence that the cases bite."""
+    wl, p, q, bs, n_blocks, strong, pair = _near_tie_case(gap_dim_q, seed=301)
+    cfg = H.oracle_config(wl)
+    kmin, kmax = orc.block_statistics(synth.to_f64(p["k"]), cfg, bs)
+    U = orc.block_upper_bounds(synth.to_f64(q), kmin, kmax, cfg)[0]
+    gap = abs(U[pair[0]] - U[pair[1]]) / abs(U[pair[0]])
+    assert 1e-10 < gap < 1e-7
+    want = sorted(strong + [pair[winner]])
+    assert orc.select_blocks(U, n_blocks).tolist() == want
+    layer = H.GpuLayer(wl, 1)
+    layer.compress([p], [0], want_idx=False)
+    c = layer.cache
+    slots = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stats = torch.zeros(B.snap_block_stats_bytes(layer.cfg, bs), dtype=torch.uint8, device="cuda")
+    B.snap_block_stats(layer.cfg, layer.layout, slots, 1, c.k_cache, c.valid_topk, bs, stats, c.status)
+    idx = torch.zeros(1, 1, n_blocks, dtype=torch.int32, device="cuda")
+    nsel = torch.zeros(1, 1, dtype=torch.int32, device="cuda")
+    sws = torch.empty(B.snap_block_select_workspace_bytes(layer.cfg, 1, bs), dtype=torch.uint8, device="cuda")
+    B.snap_block_select(layer.cfg, layer.layout, q[None].cuda(), slots, 1, stats, c.valid_topk, bs, n_blocks, idx, nsel, sws,
+                        c.status)
+    torch.cuda.synchronize()
+    assert layer.status() == 0
+    assert idx.cpu().numpy()[0, 0].tolist() == want
+
+
+def test_without_rescoring_the_near_ties_are_not_all_resolved(snap_option):
+    snap_option(B.SNAP_OPT_REFINE_OFF, 1)
+    wrong = 0
+    for gap_dim_q, winner in [(2.0 ** -12, 1), (-(2.0 ** -12), 0), (2.0 ** -15, 1), (-(2.0 ** -15), 0)]:
+        wl, p, q, bs, n_blocks, strong, pair = _near_tie_case(gap_dim_q, seed=301)
+        layer = H.GpuLayer(wl, 1)
+        layer.compress([p], [0], want_idx=False)
+        c = layer.cache
+        slots = torch.zeros(1, dtype=torch.int32, device="cuda")
+        stats = torch.zeros(B.snap_block_stats_bytes(layer.cfg, bs), dtype=torch.uint8, device="cuda")
+        B.snap_block_stats(layer.cfg, layer.layout, slots, 1, c.k_cache, c.valid_topk, bs, stats, c.status)
+        idx = torch.zeros(1, 1, n_blocks, dtype=torch.int32, device="cuda")
+        nsel = torch.zeros(1, 1, dtype=torch.int32, device="cuda")
+        sws = torch.empty(B.snap_block_select_workspace_bytes(layer.cfg, 1, bs), dtype=torch.uint8, device="cuda")
+        B.snap_block_select(layer.cfg, layer.layout, q[None].cuda(), slots, 1, stats, c.valid_topk, bs, n_blocks, idx, nsel,
+                            sws, c.status)
+        torch.cuda.synchronize()
+        got = idx.cpu().numpy()[0, 0].tolist()
+        assert sorted(strong) == [b for b in got if b in strong]          # the clear winners are always there
+        wrong += got != sorted(strong + [pair[winner]])
+    assert wrong >= 1
 
 
 def test_block_entry_points_reject_what_they_do_not_serve():
