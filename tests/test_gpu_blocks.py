@@ -119,6 +119,21 @@ def test_block_lookup_steps_match_the_oracle(hq, hkv, d, bs, n_blocks):
     _run(wl, lengths, bs, n_blocks, steps=6, seed=201)
 
 
+@pytest.mark.parametrize("seed", [5, 6])
+def test_random_block_lookup_configurations(seed):
+    """Seeded random layers (group size 1..8, head size 64/128/256, blocks of 16..256 tokens, budgets of 1..40 blocks, sink
+    and window sizes, one to four ragged prompts): statistics, selections, outputs and the final cache image."""
+    rng = np.random.default_rng(seed)
+    for case in range(20):
+        hkv = int(rng.choice([1, 2, 4])); g = int(rng.choice([1, 2, 3, 4, 8])); d = int(rng.choice([64, 128, 256]))
+        bs = int(rng.choice([16, 32, 48, 64, 128, 256])); nblk = int(rng.choice([1, 2, 5, 16, 40]))
+        Ls = int(rng.integers(0, 9)); Lr = int(rng.integers(8, 200)); topk = int(rng.choice([500, 2100, 5000]))
+        lengths = [int(rng.integers(1, Ls + Lr + topk)) for _ in range(int(rng.integers(1, 5)))]
+        wl = synth.Workload("blocks_random", g * hkv, hkv, d, d, "bf16", Ls, Lr, topk, 8, 5, batch=1, prompt_len=(100, 100),
+                            decode_steps=1, salience=str(rng.choice(["zipf", "planted"])), n_planted=8)
+        _run(wl, lengths, bs, nblk, steps=int(rng.integers(1, 6)), seed=1000 * seed + case)
+
+
 def test_more_budget_than_blocks_attends_everything_and_the_ring_wraps():
     wl = _workload(8, 2, 128, topk=600, l_recent=16)
     _run(wl, [300, 616, 90], 64, 12, steps=40, seed=207)       # 12 blocks of budget, at most 10 blocks of middle
