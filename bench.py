@@ -473,25 +473,26 @@ def extras(hp, wl, dev):
         src = dst
     out["concat_update_ms"] = statistics.median(times[2:])
     del bufs
-    # (4) two new tokens per sequence and step (multi-token prediction, Section 5) in one pass over the cache
-    q_len = 2
-    mws = torch.empty(B.snap_decode_multi_workspace_bytes(hp.cfg, wl.batch, q_len), dtype=torch.uint8, device=dev)
-    mout = torch.empty(wl.batch, q_len, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device=dev)
-    stack = lambda key, r: torch.stack([hp.decode_in[(r + u) % DECODE_RING][key] for u in range(q_len)], dim=1).contiguous()
-    ins2 = [(stack("q", r), stack("k_new", r), stack("v_new", r)) for r in range(2)]
-    times = []
-    for r in range(8):
-        q2, k2, v2 = ins2[r % 2]
-        a, b = ev(), ev()
-        a.record()
-        B.snap_decode_attn_multi(hp.cfg, hp.layout, q2, k2, v2, hp.slots_dev, wl.batch, q_len, c.k_cache, c.v_cache,
-                                 c.seq_len, c.valid_topk, mout, mws, c.status)
-        b.record()
-        torch.cuda.synchronize()
-        times.append(a.elapsed_time(b))
-    out["multi_token_q_len"] = q_len
-    out["multi_token_decode_ms"] = statistics.median(times[2:])
-    out["multi_token_tokens_per_s"] = wl.batch * q_len / (out["multi_token_decode_ms"] * 1e-3)
+    # (4) two and four new tokens per sequence and step (multi-token prediction, Section 5) in one pass over the cache
+    for q_len in (2, 4):
+        mws = torch.empty(B.snap_decode_multi_workspace_bytes(hp.cfg, wl.batch, q_len), dtype=torch.uint8, device=dev)
+        mout = torch.empty(wl.batch, q_len, wl.n_q_heads, wl.d_v, dtype=wl.torch_dtype, device=dev)
+        stack = lambda key, r: torch.stack([hp.decode_in[(r + u) % DECODE_RING][key] for u in range(q_len)], dim=1).contiguous()
+        ins2 = [(stack("q", r), stack("k_new", r), stack("v_new", r)) for r in range(2)]
+        times = []
+        for r in range(8):
+            q2, k2, v2 = ins2[r % 2]
+            a, b = ev(), ev()
+            a.record()
+            B.snap_decode_attn_multi(hp.cfg, hp.layout, q2, k2, v2, hp.slots_dev, wl.batch, q_len, c.k_cache, c.v_cache,
+                                     c.seq_len, c.valid_topk, mout, mws, c.status)
+            b.record()
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        tag = "multi_token" if q_len == 2 else f"multi_token_q{q_len}"
+        out[tag + "_q_len"] = q_len
+        out[tag + "_decode_ms"] = statistics.median(times[2:])
+        out[tag + "_tokens_per_s"] = wl.batch * q_len / (out[tag + "_decode_ms"] * 1e-3)
     out["multi_token_status"] = int(c.status.item())
     # (5) the prompt's causal attention emitting the Eq. 4 normalisers, and the compression that takes
     #     them instead of making its own first pass over the keys (one 128k-token prompt, one layer)

@@ -257,8 +257,8 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout,
  *   k_new_dev [n_active][q_len][Hkv][d_qk], v_new_dev [n_active][q_len][Hkv][d_v]   (required)
  *   out_dev   [n_active][q_len][Hq][d_v];  seq_len_dev[slot] += q_len
  * 1 <= q_len <= Lr (SNAP_ERR_INVALID_ARG otherwise).  bf16 layers with 64-, 128- or 256-wide heads
- * and up to 8 query heads per KV head take 8 / (Hq / Hkv) tokens per pass over the cache (all
- * q_len in one pass when q_len * (Hq / Hkv) <= 8, otherwise several passes, each reading its
+ * and up to 8 query heads per KV head take 16 / (Hq / Hkv) tokens per pass over the cache (all
+ * q_len in one pass when q_len * (Hq / Hkv) <= 16, otherwise several passes, each reading its
  * tokens' rows in place); every other layer (fp32, the latent layout -- v_new_dev is then ignored
  * --) is served as the definition reads, q_len single steps: same results, no saving in cache
  * traffic.  The tcgen05 latent kernel reads each token's rows in place; the other single-step

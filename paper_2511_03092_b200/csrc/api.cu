@@ -539,12 +539,12 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout, cons
 static int multi_check(const Shape& s, int q_len) {
   return q_len < 1 || q_len > s.Lr ? SNAP_ERR_INVALID_ARG : SNAP_OK;
 }
-// Tokens per launch of the tensor-core grouped-query kernel: its eight MMA columns hold (token, head)
-// pairs, so 8 / g tokens go in one pass and a longer step takes several passes, each reading its
-// tokens' rows in place.  0: the layout is served by other kernels.
+// Tokens per launch of the tensor-core grouped-query kernel: its MMA columns hold (token, head)
+// pairs, eight or sixteen of them, so 16 / g tokens go in one pass and a longer step takes several
+// passes, each reading its tokens' rows in place.  0: the layout is served by other kernels.
 static int multi_tokens_per_pass(const snap_config_t* cfg, const Shape& s, int q_len) {
   if (!decode_use_gqa_mma(cfg->dtype, s) || s.g > 8) return 0;
-  const int t = 8 / s.g;
+  const int t = 16 / s.g;
   return t < q_len ? t : q_len;
 }
 

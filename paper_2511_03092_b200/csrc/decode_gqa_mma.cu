@@ -18,8 +18,9 @@
 // Fused append (Eq. 3): the warp that stages the new token's slot stores the row to the cache
 // and patches its staged copy.
 //
-// Several new tokens per step (multi-token prediction): the eight columns are then (token,
-// head) pairs, T x g <= 8.  Query t must see the cache as it is after tokens 0..t: the old rows
+// Several new tokens per step (multi-token prediction): the columns are then (token, head)
+// pairs: T x g <= 8 in the usual instantiation, up to 16 in a second one (NG = 2: two groups of
+// eight columns, i.e. two MMAs per fragment of K or V, for steps of three or four tokens at g = 4).  Query t must see the cache as it is after tokens 0..t: the old rows
 // are attended as staged, a window row that token u evicts is masked for the queries from u
 // on, the new rows form one extra tile with a causal mask, and each new row is written to the
 // cache by the warp that has just staged the row it replaces.
@@ -80,9 +81,10 @@ __device__ __forceinline__ TileRows tile_rows(int j, int nA, int n_low, int Lsr,
   return t;
 }
 
-// D: head size (64, 128 or 256); NWARP: warps per CTA (fewer for wide heads, whose stages are larger)
-template <int D, int NWARP>
-__global__ void __launch_bounds__(NWARP * 32, 3)
+// D: head size (64, 128 or 256); NWARP: warps per CTA (fewer for wide heads, whose stages are larger);
+// NG: groups of eight MMA columns (1, or 2 for multi-token steps with 9 to 16 query rows per KV head)
+template <int D, int NWARP, int NG>
+__global__ void __launch_bounds__(NWARP * 32, NG == 1 ? 3 : 2)
 decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
   constexpr int NT = NWARP * 32, NSL = D / 64, CPR = D / 8, KS = D / 16;   // slabs per tensor, 16-byte chunks per row, 16-dim steps
   constexpr int TENS_B = NSL * SLAB_B, STAGE_B = 2 * TENS_B, PS = D + 2;   // stage = K slabs | V slabs
@@ -164,70 +166,101 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
   // Column n of the MMAs is query token n / g, head n % g of the group (zero beyond T * g).
   // B fragments of Q^T for the eight 16-dim steps: column gq, dims 16 ks + 2 tq (+8)
   const int ncols = TQ * a.g;
-  uint32_t qb[KS][2];
-  {
-    const int tcol = gq / a.g, hcol = gq - tcol * a.g;
+  uint32_t qb[NG][KS][2];
+  int tc0[NG], tc1[NG];                          // query tokens of this thread's two columns, per column group
+#pragma unroll
+  for (int gi = 0; gi < NG; ++gi) {
+    const int col = GP * gi + gq;                // this lane's column of the B fragments
+    const int tcol = col / a.g, hcol = col - tcol * a.g;
     const __nv_bfloat16* qp = a.q + (((long long)i * a.QT + a.u0 + tcol) * a.Hq + (long long)kvh * a.g + hcol) * D + 2 * tq;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      qb[ks][0] = gq < ncols ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks) : 0u;
-      qb[ks][1] = gq < ncols ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks + 8) : 0u;
+      qb[gi][ks][0] = col < ncols ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks) : 0u;
+      qb[gi][ks][1] = col < ncols ? *reinterpret_cast<const uint32_t*>(qp + 16 * ks + 8) : 0u;
     }
+    tc0[gi] = (GP * gi + 2 * tq) / a.g;
+    tc1[gi] = (GP * gi + 2 * tq + 1) / a.g;
   }
-  const int tc0 = (2 * tq) / a.g, tc1 = (2 * tq + 1) / a.g;     // query tokens of this thread's two columns
-  float oacc[KS][4];                             // O^T: dims 16 db + gq (+8), columns 2 tq (+1)
+  float oacc[NG][KS][4];                         // O^T: dims 16 db + gq (+8), columns 8 gi + 2 tq (+1)
 #pragma unroll
-  for (int db = 0; db < KS; ++db)
+  for (int gi = 0; gi < NG; ++gi)
 #pragma unroll
-    for (int e = 0; e < 4; ++e) oacc[db][e] = 0.f;
-  float m_ref[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};   // columns 2 tq, 2 tq + 1
+    for (int db = 0; db < KS; ++db)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) oacc[gi][db][e] = 0.f;
+  float m_ref[NG][2], l_part[NG][2];             // columns 8 gi + 2 tq, 8 gi + 2 tq + 1
+#pragma unroll
+  for (int gi = 0; gi < NG; ++gi) { m_ref[gi][0] = m_ref[gi][1] = -INFINITY; l_part[gi][0] = l_part[gi][1] = 0.f; }
   bool timed_out = false;
 
   // ldmatrix lane roles: K (plain): row (lane & 7) + 8 * bit3, chunk + bit4; V (transposed): row (lane & 7) + 8 * bit4, chunk + bit3
   const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_cadd = lane >> 4;
   const int v_row = (lane & 7) + ((lane >> 4) & 1) * 8, v_cadd = (lane >> 3) & 1;
 
-  // One staged tile: okN says whether this thread's value N (rows gq, gq, gq + 8, gq + 8 x columns
-  // 2 tq, 2 tq + 1, 2 tq, 2 tq + 1) takes part.
-  auto process = [&](uint32_t sK, uint32_t sV, bool ok0, bool ok1, bool ok2, bool ok3) {
+  // One staged tile: ok[gi][N] says whether this thread's value N of column group gi (rows gq, gq, gq + 8,
+  // gq + 8 x columns 2 tq, 2 tq + 1, 2 tq, 2 tq + 1) takes part.
+  struct Mask { bool ok[NG][4]; };
+  auto process = [&](uint32_t sK, uint32_t sV, const Mask& mk) {
     // ---- S^T = K tile . Q^T ----
-    float sacc[4] = {0.f, 0.f, 0.f, 0.f};
+    float sacc[NG][4];
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) { sacc[gi][0] = sacc[gi][1] = sacc[gi][2] = sacc[gi][3] = 0.f; }
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
       uint32_t af[4];
       ldsm4(sK + (ks >> 2) * SLAB_B + swz(k_row, (ks & 3) * 2 + k_cadd), af);
-      mma16816(sacc, af, qb[ks][0], qb[ks][1]);
+#pragma unroll
+      for (int gi = 0; gi < NG; ++gi) mma16816(sacc[gi], af, qb[gi][ks][0], qb[gi][ks][1]);
     }
-    const float v0 = ok0 ? sacc[0] * a.scale_log2 : -INFINITY, v1 = ok1 ? sacc[1] * a.scale_log2 : -INFINITY;
-    const float v2 = ok2 ? sacc[2] * a.scale_log2 : -INFINITY, v3 = ok3 ? sacc[3] * a.scale_log2 : -INFINITY;
+    float v[NG][4];
+    bool refresh = false;
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v[gi][e] = mk.ok[gi][e] ? sacc[gi][e] * a.scale_log2 : -INFINITY;
+      refresh = refresh || fmaxf(v[gi][0], v[gi][2]) > m_ref[gi][0] + 8.f || fmaxf(v[gi][1], v[gi][3]) > m_ref[gi][1] + 8.f;
+    }
     // Lazy reference per column: refreshed (accumulators rescaled) only when a warp vote sees a
     // logit 8 above it; the column maxima are then reduced over the lanes that share tq.
-    if (__any_sync(0xffffffffu, fmaxf(v0, v2) > m_ref[0] + 8.f || fmaxf(v1, v3) > m_ref[1] + 8.f)) {
-      float mx0 = fmaxf(v0, v2), mx1 = fmaxf(v1, v3);
+    if (__any_sync(0xffffffffu, refresh)) {
 #pragma unroll
-      for (int o = 4; o <= 16; o <<= 1) {
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+      for (int gi = 0; gi < NG; ++gi) {
+        float mx0 = fmaxf(v[gi][0], v[gi][2]), mx1 = fmaxf(v[gi][1], v[gi][3]);
+#pragma unroll
+        for (int o = 4; o <= 16; o <<= 1) {
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+          mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+        }
+        const float n0 = fmaxf(m_ref[gi][0], mx0), n1 = fmaxf(m_ref[gi][1], mx1);
+        const float a0 = m_ref[gi][0] == -INFINITY ? 0.f : exp2f(m_ref[gi][0] - n0);
+        const float a1 = m_ref[gi][1] == -INFINITY ? 0.f : exp2f(m_ref[gi][1] - n1);
+        m_ref[gi][0] = n0; m_ref[gi][1] = n1;
+        l_part[gi][0] *= a0; l_part[gi][1] *= a1;
+#pragma unroll
+        for (int db = 0; db < KS; ++db) {
+          oacc[gi][db][0] *= a0; oacc[gi][db][1] *= a1; oacc[gi][db][2] *= a0; oacc[gi][db][3] *= a1;
+        }
       }
-      const float n0 = fmaxf(m_ref[0], mx0), n1 = fmaxf(m_ref[1], mx1);
-      const float a0 = m_ref[0] == -INFINITY ? 0.f : exp2f(m_ref[0] - n0), a1 = m_ref[1] == -INFINITY ? 0.f : exp2f(m_ref[1] - n1);
-      m_ref[0] = n0; m_ref[1] = n1;
-      l_part[0] *= a0; l_part[1] *= a1;
-#pragma unroll
-      for (int db = 0; db < KS; ++db) { oacc[db][0] *= a0; oacc[db][1] *= a1; oacc[db][2] *= a0; oacc[db][3] *= a1; }
     }
-    const float r0 = m_ref[0] == -INFINITY ? 0.f : m_ref[0], r1 = m_ref[1] == -INFINITY ? 0.f : m_ref[1];
-    const float p0 = fast_exp2(v0 - r0), p1 = fast_exp2(v1 - r1), p2 = fast_exp2(v2 - r0), p3 = fast_exp2(v3 - r1);
-    l_part[0] += p0 + p2;
-    l_part[1] += p1 + p3;
-    // P^T as the B operand: rows 2 tq (+1) and 2 tq + 8 (+9) of column gq
-    const uint32_t pb0 = movmatrix_t(pack_bf16(p0, p1)), pb1 = movmatrix_t(pack_bf16(p2, p3));
+    uint32_t pb[NG][2];
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+      const float r0 = m_ref[gi][0] == -INFINITY ? 0.f : m_ref[gi][0], r1 = m_ref[gi][1] == -INFINITY ? 0.f : m_ref[gi][1];
+      const float p0 = fast_exp2(v[gi][0] - r0), p1 = fast_exp2(v[gi][1] - r1);
+      const float p2 = fast_exp2(v[gi][2] - r0), p3 = fast_exp2(v[gi][3] - r1);
+      l_part[gi][0] += p0 + p2;
+      l_part[gi][1] += p1 + p3;
+      // P^T as the B operand: rows 2 tq (+1) and 2 tq + 8 (+9) of column gq
+      pb[gi][0] = movmatrix_t(pack_bf16(p0, p1));
+      pb[gi][1] = movmatrix_t(pack_bf16(p2, p3));
+    }
     // ---- O^T += V tile^T . P^T ----
 #pragma unroll
     for (int db = 0; db < KS; ++db) {
       uint32_t af[4];
       ldsm4t(sV + (db >> 2) * SLAB_B + swz(v_row, (db & 3) * 2 + v_cadd), af);
-      mma16816(oacc[db], af, pb0, pb1);
+#pragma unroll
+      for (int gi = 0; gi < NG; ++gi) mma16816(oacc[gi][db], af, pb[gi][0], pb[gi][1]);
     }
   };
 
@@ -240,7 +273,9 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     const TileRows tr = rows_of(j);
     const int nrows = tr.row_end - tr.row0;                    // rows at or past it are masked (may be <= 0)
     const uint32_t sK = stage0 + s * STAGE_B, sV = sK + TENS_B;
-    bool ok0 = gq < nrows, ok1 = ok0, ok2 = gq + 8 < nrows, ok3 = ok2;
+    Mask mk;
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) { mk.ok[gi][0] = mk.ok[gi][1] = gq < nrows; mk.ok[gi][2] = mk.ok[gi][3] = gq + 8 < nrows; }
     if (nrows < WT) {
       // ragged tile: rows past the end may hold anything (memory the caller never wrote), and a
       // zero probability does not silence a NaN in V: clear those V rows
@@ -270,8 +305,11 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
         const int ru = ring_slot(L0 + u, a.Ls, a.Lr);
         if (ru < tr.row0 || ru >= tr.row0 + WT) continue;
         const int r = ru - tr.row0;
-        if (gq == r) { ok0 = ok0 && tc0 < u; ok1 = ok1 && tc1 < u; }
-        if (gq + 8 == r) { ok2 = ok2 && tc0 < u; ok3 = ok3 && tc1 < u; }
+#pragma unroll
+        for (int gi = 0; gi < NG; ++gi) {
+          if (gq == r) { mk.ok[gi][0] = mk.ok[gi][0] && tc0[gi] < u; mk.ok[gi][1] = mk.ok[gi][1] && tc1[gi] < u; }
+          if (gq + 8 == r) { mk.ok[gi][2] = mk.ok[gi][2] && tc0[gi] < u; mk.ok[gi][3] = mk.ok[gi][3] && tc1[gi] < u; }
+        }
         for (int e = lane; e < 2 * CPR; e += 32) {
           const int tens = e / CPR, c = e % CPR;
           reinterpret_cast<uint4*>((tens ? vc : kc) + (long long)ru * (D * 2))[c] =
@@ -279,7 +317,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
         }
       }
     }
-    process(sK, sV, ok0, ok1, ok2, ok3);
+    process(sK, sV, mk);
     __syncwarp();
     if (lane == 0 && n + NSTAGE < T) {
       // the stage was read, and possibly patched, through the generic proxy; the bulk copy that
@@ -302,30 +340,41 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
       *reinterpret_cast<uint4*>(wstages + tens * TENS_B + (c >> 3) * SLAB_B + swz(r, c & 7)) = val;
     }
     __syncwarp();
-    process(stage0, stage0 + TENS_B, gq < TQ && gq <= tc0, gq < TQ && gq <= tc1, false, false);
+    Mask mk;
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+      mk.ok[gi][0] = gq < TQ && gq <= tc0[gi]; mk.ok[gi][1] = gq < TQ && gq <= tc1[gi];
+      mk.ok[gi][2] = gq + 8 < TQ && gq + 8 <= tc0[gi]; mk.ok[gi][3] = gq + 8 < TQ && gq + 8 <= tc1[gi];   // up to 16 tokens
+    }
+    process(stage0, stage0 + TENS_B, mk);
     __syncwarp();
   }
 
   // ---- per-warp result -> this warp's stage memory, then merge the warps ----
-#pragma unroll
-  for (int o = 4; o <= 16; o <<= 1) {
-    l_part[0] += __shfl_xor_sync(0xffffffffu, l_part[0], o);
-    l_part[1] += __shfl_xor_sync(0xffffffffu, l_part[1], o);
-  }
-  float* wm = reinterpret_cast<float*>(wstages);           // [GP] max, [GP] sum, [GP][D] acc
-  float* wl = wm + GP;
-  float* wacc = wl + GP;
+  constexpr int NCOL = NG * GP;
+  float* wm = reinterpret_cast<float*>(wstages);           // [NCOL] max, [NCOL] sum, [NCOL][D] acc
+  float* wl = wm + NCOL;
+  float* wacc = wl + NCOL;
   __syncwarp();
-  if (gq == 0) {
-    wm[2 * tq] = m_ref[0]; wm[2 * tq + 1] = m_ref[1];
-    wl[2 * tq] = l_part[0]; wl[2 * tq + 1] = l_part[1];
-  }
 #pragma unroll
-  for (int db = 0; db < KS; ++db) {
-    wacc[(2 * tq) * D + 16 * db + gq] = oacc[db][0];
-    wacc[(2 * tq + 1) * D + 16 * db + gq] = oacc[db][1];
-    wacc[(2 * tq) * D + 16 * db + gq + 8] = oacc[db][2];
-    wacc[(2 * tq + 1) * D + 16 * db + gq + 8] = oacc[db][3];
+  for (int gi = 0; gi < NG; ++gi) {
+#pragma unroll
+    for (int o = 4; o <= 16; o <<= 1) {
+      l_part[gi][0] += __shfl_xor_sync(0xffffffffu, l_part[gi][0], o);
+      l_part[gi][1] += __shfl_xor_sync(0xffffffffu, l_part[gi][1], o);
+    }
+    const int c0 = GP * gi + 2 * tq;
+    if (gq == 0) {
+      wm[c0] = m_ref[gi][0]; wm[c0 + 1] = m_ref[gi][1];
+      wl[c0] = l_part[gi][0]; wl[c0 + 1] = l_part[gi][1];
+    }
+#pragma unroll
+    for (int db = 0; db < KS; ++db) {
+      wacc[c0 * D + 16 * db + gq] = oacc[gi][db][0];
+      wacc[(c0 + 1) * D + 16 * db + gq] = oacc[gi][db][1];
+      wacc[c0 * D + 16 * db + gq + 8] = oacc[gi][db][2];
+      wacc[(c0 + 1) * D + 16 * db + gq + 8] = oacc[gi][db][3];
+    }
   }
   __syncthreads();
   constexpr int WSTRIDE = NSTAGE * STAGE_B / 4;            // floats between two warps' regions
@@ -339,7 +388,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     for (int ww = 0; ww < NWARP; ++ww) {
       const float mw = base[ww * WSTRIDE + h];
       f[ww] = mw == -INFINITY ? 0.f : exp2f(mw - M);
-      L += base[ww * WSTRIDE + GP + h] * f[ww];
+      L += base[ww * WSTRIDE + NCOL + h] * f[ww];
     }
     const int tcol = h / a.g, hcol = h - tcol * a.g;
     float* ph = a.partials + ((((long long)i * TQ + tcol) * a.Hq + (long long)kvh * a.g + hcol) * a.nsplit + sp) * PS;
@@ -347,7 +396,7 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
     for (int dv = tid; dv < D; dv += NT) {
       float O = 0.f;
 #pragma unroll
-      for (int ww = 0; ww < NWARP; ++ww) O += base[ww * WSTRIDE + 2 * GP + h * D + dv] * f[ww];
+      for (int ww = 0; ww < NWARP; ++ww) O += base[ww * WSTRIDE + 2 * NCOL + h * D + dv] * f[ww];
       ph[2 + dv] = O;
     }
   }
@@ -390,13 +439,14 @@ __global__ void __launch_bounds__(128) decode_gqa_mma_merge_kernel(const float* 
   }
 }
 
-template <int D, int NWARP>
+template <int D, int NWARP, int NG>
 cudaError_t launch_d(const MmaArgs& a, const CUtensorMap& tk, const CUtensorMap& tv, int n_active, cudaStream_t st) {
   constexpr size_t smem = (size_t)NWARP * NSTAGE * (2 * (D / 64) * SLAB_B) + NWARP * NSTAGE * 8 + 1024;
+  static_assert((size_t)NSTAGE * (2 * (D / 64) * SLAB_B) >= (size_t)NG * GP * (D + 2) * sizeof(float), "a warp's result fits its stages");
   static SmemLimit limit = {};
-  if (cudaError_t e = ensure_dyn_smem(decode_gqa_mma_kernel<D, NWARP>, smem, limit)) return e;
-  const cudaError_t e = launch_pdl(decode_gqa_mma_kernel<D, NWARP>, dim3(a.nsplit, a.Hkv, n_active), dim3(NWARP * 32), smem, st,
-                                   a, tk, tv);
+  if (cudaError_t e = ensure_dyn_smem(decode_gqa_mma_kernel<D, NWARP, NG>, smem, limit)) return e;
+  const cudaError_t e = launch_pdl(decode_gqa_mma_kernel<D, NWARP, NG>, dim3(a.nsplit, a.Hkv, n_active), dim3(NWARP * 32), smem,
+                                   st, a, tk, tv);
   count_launch();
   return e;
 }
@@ -420,7 +470,7 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   if (n_active == 0) return cudaSuccess;
   if (block_idx && (!n_sel || blocks_cap < 1 || block_tokens < WT || block_tokens % WT || q_len != 1)) return cudaErrorInvalidValue;
   if (q_total < q_len) { q_total = q_len; u0 = 0; }            // the launch's tokens are all the step's tokens
-  if (q_len < 1 || q_len * s.g > GP || (q_len > 1 && (!k_new || q_len > s.Lr)) || u0 < 0 || u0 + q_len > q_total)
+  if (q_len < 1 || q_len * s.g > 2 * GP || (q_len > 1 && (!k_new || q_len > s.Lr)) || u0 < 0 || u0 + q_len > q_total)
     return cudaErrorInvalidValue;
   umma::EncodeTiledFn enc = umma::encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
@@ -467,9 +517,10 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   a.seq_len = seq_len; a.valid_topk = valid_topk; a.partials = partials; a.status = status;
   a.block_idx = block_idx; a.n_sel = n_sel; a.blocks_cap = blocks_cap; a.tpb = block_idx ? block_tokens / WT : 1;
   cudaError_t e;
-  if (D == 128) e = launch_d<128, 4>(a, hit->tk, hit->tv, n_active, st);
-  else if (D == 64) e = launch_d<64, 4>(a, hit->tk, hit->tv, n_active, st);
-  else e = launch_d<256, 2>(a, hit->tk, hit->tv, n_active, st);
+  const bool wide = q_len * s.g > GP;                          // 9 to 16 (token, head) columns: two column groups
+  if (D == 128) e = wide ? launch_d<128, 4, 2>(a, hit->tk, hit->tv, n_active, st) : launch_d<128, 4, 1>(a, hit->tk, hit->tv, n_active, st);
+  else if (D == 64) e = wide ? launch_d<64, 4, 2>(a, hit->tk, hit->tv, n_active, st) : launch_d<64, 4, 1>(a, hit->tk, hit->tv, n_active, st);
+  else e = wide ? launch_d<256, 2, 2>(a, hit->tk, hit->tv, n_active, st) : launch_d<256, 2, 1>(a, hit->tk, hit->tv, n_active, st);
   if (e != cudaSuccess) return e;
   if (D == 128)
     return launch_decode_gqa_merge(partials, out, s.Hq, nsplit, slot_ids, n_active * q_len, q_len, seq_len, s.max_seqs,

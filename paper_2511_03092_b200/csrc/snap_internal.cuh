@@ -193,7 +193,7 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
                                   int nsplit, uint32_t* status, cudaStream_t st, int q_len = 1, int q_total = 0, int u0 = 0,
                                   const int* block_idx = nullptr, const int* n_sel = nullptr, int blocks_cap = 0,
                                   int block_tokens = 0);
-// (q_len tokens per sequence in one pass, q_len * g <= 8: tokens u0 .. u0 + q_len - 1 of the q_total per sequence that
+// (q_len tokens per sequence in one pass, q_len * g <= 16: tokens u0 .. u0 + q_len - 1 of the q_total per sequence that
 // q, k_new, v_new and out hold; q_total = 0: they hold exactly these)
 
 // (block_idx: per-step block lookup -- only the listed blocks of block_tokens rows of the third section are visited)

@@ -454,9 +454,11 @@ def _run_multi(wl, lengths, q_len, steps, seed):
 
 
 @pytest.mark.parametrize("hq,hkv,q_len", [(16, 4, 2), (8, 4, 4), (8, 4, 3), (4, 4, 8), (32, 4, 1),
-                                          (16, 4, 4), (16, 4, 3), (32, 4, 3), (8, 4, 7), (12, 4, 5)],
+                                          (16, 4, 4), (16, 4, 3), (8, 4, 7), (12, 4, 5), (4, 4, 13),
+                                          (32, 4, 3), (16, 4, 7), (12, 4, 11)],
                          ids=["g4x2", "g2x4", "g2x3", "g1x8", "g8x1",
-                              "g4x4_two_passes", "g4x3_two_passes", "g8x3_three_passes", "g2x7_two_passes", "g3x5_three_passes"])
+                              "g4x4_16_columns", "g4x3_12_columns", "g2x7_14_columns", "g3x5_15_columns", "g1x13_13_columns",
+                              "g8x3_two_passes", "g4x7_two_passes", "g3x11_three_passes"])
 def test_multi_token_decode_steps(hq, hkv, q_len):
     """q_len tokens per step: each query sees the cache as it is after its own token -- window rows
     evicted by later tokens of the step included, those evicted by earlier ones not.  Sequences that
@@ -466,10 +468,10 @@ def test_multi_token_decode_steps(hq, hkv, q_len):
 
 
 @pytest.mark.parametrize("wl,q_len", [(SMALL_BF16, 3), (SMALL_F32, 2), (SMALL_MLA, 3), (LATENT_128, 2)],
-                         ids=["bf16_g4x3_two_passes", "f32_g4x2", "latent_x3", "latent_128_heads_x2"])
+                         ids=["bf16_g4x3", "f32_g4x2", "latent_x3", "latent_128_heads_x2"])
 def test_multi_token_decode_on_shapes_served_step_by_step(wl, q_len):
     """Shapes the tensor-core grouped-query kernel does not take (fp32, the latent layout) go through
-    q_len single steps inside the library, and a step with more than 8 query rows per KV head through
+    q_len single steps inside the library, and a step with more than 16 query rows per KV head through
     several passes of that kernel: same definition, same results."""
     _run_multi(wl, [1, 3, 45, 50, 51, 52, 300, wl.prompt_len[0]], q_len, steps=6, seed=87)
 
