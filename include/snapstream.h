@@ -257,7 +257,7 @@ int snap_decode_attn(const snap_config_t* cfg, const snap_layout_t* layout,
  *   k_new_dev [n_active][q_len][Hkv][d_qk], v_new_dev [n_active][q_len][Hkv][d_v]   (required)
  *   out_dev   [n_active][q_len][Hq][d_v];  seq_len_dev[slot] += q_len
  * 1 <= q_len <= Lr (SNAP_ERR_INVALID_ARG otherwise).  bf16 layers with 64-, 128- or 256-wide heads
- * and up to 8 query heads per KV head take 16 / (Hq / Hkv) tokens per pass over the cache (all
+ * and up to 16 query heads per KV head take 16 / (Hq / Hkv) tokens per pass over the cache (all
  * q_len in one pass when q_len * (Hq / Hkv) <= 16, otherwise several passes, each reading its
  * tokens' rows in place); every other layer (fp32, the latent layout -- v_new_dev is then ignored
  * --) is served as the definition reads, q_len single steps: same results, no saving in cache
@@ -349,7 +349,7 @@ int snap_append_kv_concat(const snap_config_t* cfg, const snap_layout_t* layout,
  *     highest-scoring blocks are attended, ties to the lower block index, together with the
  *     sinks and the rolling window, which behave as in snap_decode_attn (Eq. 3 append
  *     included); rows that leave the window during decoding are dropped as before.
- * bf16 layers with 64-, 128- or 256-wide heads, a separate V and at most 8 query heads per KV
+ * bf16 layers with 64-, 128- or 256-wide heads, a separate V and at most 16 query heads per KV
  * head; at most 8192 blocks per sequence; SNAP_ERR_UNSUPPORTED otherwise.  The scores are summed
  * in single precision for every block; the blocks that single precision cannot tell from the
  * last selected one (a rigorous error bound per block) are scored again in double precision and

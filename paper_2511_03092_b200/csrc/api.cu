@@ -543,7 +543,7 @@ static int multi_check(const Shape& s, int q_len) {
 // pairs, eight or sixteen of them, so 16 / g tokens go in one pass and a longer step takes several
 // passes, each reading its tokens' rows in place.  0: the layout is served by other kernels.
 static int multi_tokens_per_pass(const snap_config_t* cfg, const Shape& s, int q_len) {
-  if (!decode_use_gqa_mma(cfg->dtype, s) || s.g > 8) return 0;
+  if (!decode_use_gqa_mma(cfg->dtype, s) || s.g > 16) return 0;
   const int t = 16 / s.g;
   return t < q_len ? t : q_len;
 }

@@ -343,7 +343,7 @@ int block_count_max(const Shape& s, int block_tokens) { return (s.K + block_toke
 
 bool block_topk_supported(int dtype, const Shape& s, int block_tokens) {
   return dtype == SNAP_BF16 && !s.v_aliases_k && s.d_qk % 8 == 0 && s.d_qk <= 256 && block_tokens >= 16 && block_tokens % 16 == 0 &&
-         block_tokens <= 1024 && s.K > 0 && block_count_max(s, block_tokens) <= MAX_BLOCKS && s.g <= 8;
+         block_tokens <= 1024 && s.K > 0 && block_count_max(s, block_tokens) <= MAX_BLOCKS && s.g <= 16;
 }
 
 cudaError_t launch_block_stats(const Shape& s, int block_tokens, const int* slot_ids, int n, const void* k_cache,

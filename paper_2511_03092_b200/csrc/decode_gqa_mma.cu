@@ -1,5 +1,5 @@
-// Decode attention over the compressed cache (Section 3.3) for bf16 layers with 128-wide heads
-// and 1 to 8 query heads per KV head, on tensor cores -- the HBM-bound kernel of the decode step.
+// Decode attention over the compressed cache (Section 3.3) for bf16 layers with 64-, 128- or 256-wide
+// heads and 1 to 16 query heads per KV head, on tensor cores -- the HBM-bound kernel of the decode step.
 //
 // Split-K flash decoding: grid = splits x KV heads x sequences, warp-private pipelines of 16-row
 // tiles, one partial result per split, a merge kernel.  The arithmetic is mma.sync.m16n8k16
@@ -51,7 +51,7 @@ struct MmaArgs {
   char* kc; char* vc;
   long long seq_b, head_b;
   int Hq, Hkv, g, Ls, Lr, max_seqs, nsplit;
-  int T;                                        // query tokens per sequence in this launch (T * g <= 8)
+  int T;                                        // query tokens per sequence in this launch (T * g <= 16)
   int QT, u0;                                   // ... which are tokens u0 .. u0 + T - 1 of the QT tokens per sequence in q / k_new / v_new
   float scale_log2;
   const int* seq_len; const int* valid_topk;
@@ -455,7 +455,7 @@ cudaError_t launch_d(const MmaArgs& a, const CUtensorMap& tk, const CUtensorMap&
 
 bool decode_gqa_mma_supported(int dtype, const Shape& s) {
   return dtype == SNAP_BF16 && s.d_qk == s.d_v && (s.d_qk == 64 || s.d_qk == 128 || s.d_qk == 256) && !s.v_aliases_k &&
-         s.g >= 1 && s.g <= GP && umma::encode_tiled_fn() != nullptr;
+         s.g >= 1 && s.g <= 2 * GP && umma::encode_tiled_fn() != nullptr;
 }
 
 size_t decode_gqa_mma_partial_floats(const Shape& s, int n_rows, int nsplit) {

@@ -211,10 +211,10 @@ def test_slot_reuse_overwrites_everything():
     H.check_cache_image(layer, H.oracle_compress(wl, p), 0, wl)
 
 
-@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 4), (12, 4), (20, 4), (24, 4), (28, 4), (32, 4)],
-                         ids=["g1", "g2", "g3", "g5", "g6", "g7", "g8"])
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 4), (12, 4), (20, 4), (24, 4), (28, 4), (32, 4), (18, 2), (24, 2), (32, 2)],
+                         ids=["g1", "g2", "g3", "g5", "g6", "g7", "g8", "g9", "g12", "g16"])
 def test_group_sizes(hq, hkv):
-    """Every number of query heads per KV head from 1 to 8 (odd sizes run padded by one head)."""
+    """Numbers of query heads per KV head from 1 to 16 (up to 8 in one group of MMA columns, beyond in two)."""
     wl = SMALL_BF16.scaled(n_q_heads=hq, n_kv_heads=hkv)
     _run_compress_and_decode(wl, [wl.prompt_len[0], 50, 3], seed=13, steps=5)
 
