@@ -146,12 +146,10 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
     auto issue_s = [&](int x, int it, int s) {                // S of head x = Q_x K(it)^T, K in stage s
       const uint32_t sd = tmem_base + COL_S + buf_of(x, it) * BN;
       const uint64_t kd0 = smem_desc(smem_u32(Rs) + s * TILE_B), qdx = qd0 + (uint64_t)((x * TILE_B) >> 4);
+      // one instruction group per 64-dim slab: this warp's instruction chain per MMA is what the tensor pipe waits for
 #pragma unroll
       for (int h = 0; h < 2; ++h)
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          mma_ss_pred(sd, qdx + (uint64_t)((h * SLAB_B) >> 4) + (uint64_t)(ks * 2),
-                      kd0 + (uint64_t)((h * SLAB_B) >> 4) + (uint64_t)(ks * 2), idesc_s, (h | ks) != 0, leader);
+        mma_ss_slab4_pred(sd, qdx + (uint64_t)((h * SLAB_B) >> 4), kd0 + (uint64_t)((h * SLAB_B) >> 4), idesc_s, h != 0, leader);
       commit_pred(sfull_bar(buf_of(x, it)), leader);
     };
     auto issue_pv = [&](int x, int it, int s) -> bool {       // O_x += P_x(it) V(it), V in stage s
@@ -161,10 +159,9 @@ prefill_attn_kernel(const PArgs a, const __grid_constant__ CUtensorMap tmap_q, c
       for (int half = 0; half < 2; ++half) {                  // the first 64 keys go while the rest are exponentiated
         if (!wait_warp(pready_bar(buf_of(x, it), half), phase_of(it), abort_flag)) return false;
         fence_after();
-#pragma unroll
-        for (int ks = 4 * half; ks < 4 * half + 4; ++ks)      // 16 keys per instruction
-          mma_ts_pred(tmem_base + COL_O + x * D, pa + 8 * ks, smem_desc_mn(vst + ks * 16 * 128, SLAB_B), idesc_pv,
-                      (it | ks) != 0, leader);
+        // four instructions of 16 keys each, one group
+        mma_ts_4_pred(tmem_base + COL_O + x * D, pa + 32 * half, smem_desc_mn(vst + half * 64 * 128, SLAB_B), (16 * 128) >> 4,
+                      idesc_pv, (it | half) != 0, leader);
       }
       commit_pred(pvdone_bar(buf_of(x, it)), leader);
       return true;

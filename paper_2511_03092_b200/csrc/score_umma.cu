@@ -194,18 +194,17 @@ score_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_q, 
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t kst = smem_u32(Ks) + s * STAGE_B, qst = smem_u32(Qs);
+        // one instruction group per 64-dim slab (four 16-wide steps)
         if (PASS == 1) {
           for (int mb = 0; mb < MB; ++mb)
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks)
-              mma_bf16(tmem_base + b * 256 + mb * 128,
-                        smem_desc(qst + (ks >> 2) * (R * 128) + mb * HALF_B + (ks & 3) * 32),
-                        smem_desc(kst + (ks >> 2) * HALF_B + (ks & 3) * 32), idesc, ks > 0);
+            for (int h = 0; h < D / 64; ++h)
+              mma_slab4<false>(tmem_base + b * 256 + mb * 128, smem_desc(qst + h * (R * 128) + mb * HALF_B),
+                               smem_desc(kst + h * HALF_B), idesc, h > 0);
         } else {
 #pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks)
-            mma_bf16(tmem_base + b * 256, smem_desc(kst + (ks >> 2) * HALF_B + (ks & 3) * 32),
-                      smem_desc(qst + (ks >> 2) * (R * 128) + (ks & 3) * 32), idesc, ks > 0);
+          for (int h = 0; h < D / 64; ++h)
+            mma_slab4<false>(tmem_base + b * 256, smem_desc(kst + h * HALF_B), smem_desc(qst + h * (R * 128)), idesc, h > 0);
           mma_bf16(tmem_base + b * 256, smem_desc(smem_u32(Kx)), smem_desc(smem_u32(Qx)), idesc, 1);   // - mu_i / scale
         }
         mma_commit(empty_bar(s));        // the stage may be refilled once these MMAs have read it

@@ -294,6 +294,20 @@ __device__ __forceinline__ void mma_ts_2_pred(uint32_t d_tmem, uint32_t a_tmem, 
       "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a1], b1, %4, t;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(b_step), "r"(idesc), "r"(acc_first), "r"(leader) : "memory");
 }
+// four 16-row steps with the A operand in tensor memory (8 columns of bf16 pairs per step), B advancing by b_step
+__device__ __forceinline__ void mma_ts_4_pred(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t b_step, uint32_t idesc,
+                                              uint32_t acc_first, uint32_t leader) {
+  asm volatile(
+      "{\n\t.reg .pred p, t, q;\n\t.reg .b64 b1, b2, b3, st;\n\t.reg .b32 a1, a2, a3;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 t, %4, %4;\n\tsetp.ne.b32 q, %6, 0;\n\t"
+      "cvt.u64.u32 st, %3;\n\tadd.s64 b1, %2, st;\n\tadd.s64 b2, b1, st;\n\tadd.s64 b3, b2, st;\n\t"
+      "add.u32 a1, %1, 8;\n\tadd.u32 a2, %1, 16;\n\tadd.u32 a3, %1, 24;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %4, p;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a1], b1, %4, t;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a2], b2, %4, t;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [a3], b3, %4, t;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(b_step), "r"(idesc), "r"(acc_first), "r"(leader) : "memory");
+}
 // 32 lanes x 16 consecutive columns, registers to tensor memory
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
