@@ -74,9 +74,11 @@ typedef enum snap_status {
 #define SNAP_DEV_BAND_OVERFLOW 4u   /* snap_compress: a KV head had more candidates within the re-scoring
                                        band of its top-K threshold than the band buffer holds (512, or
                                        256 for layers with more than 2^18 query elements per KV head);
-                                       that head keeps its single-precision order.  The results are
-                                       valid; exactly tied scores, which go to the lower position in
-                                       either precision, are the usual cause */
+                                       snap_block_select: more than 256 blocks that single precision
+                                       cannot tell from the threshold.  That head keeps its
+                                       single-precision order.  The results are valid; exactly tied
+                                       scores, which go to the lower position in either precision, are
+                                       the usual cause */
 
 #define SNAP_DEV_INDEX_CHECK 8u     /* only from the checked build of the library (compiled with
                                        -DSNAP_DEBUG_BOUNDS): a data-dependent index -- a selected
