@@ -137,6 +137,33 @@ def test_duplicate_scores_and_exact_ties_at_the_boundary():
         np.testing.assert_array_equal(idx[0][h], seq.topk_pos[h])
 
 
+@pytest.mark.parametrize("copies, take", [(200, 100), (40, 17)])
+def test_many_exact_ties_at_the_threshold_spread_over_the_selection_cluster(copies, take):
+    """One key repeated at scattered positions of a long prompt: its copies score exactly alike, and the
+    budget is set so that the threshold falls among them (`take` of them are kept).  With 200 copies
+    the equal keys outnumber what the selection kernel's CTAs pass around as a list, so every radix
+    digit is resolved by histograms and the copies are shared out among the CTAs by index order; with 40
+    the list short-cut ends the selection.  Either way the lowest positions win, as in the oracle."""
+    base = SMALL_BF16.scaled(n_q_heads=4, n_kv_heads=1, pool_kernel=1)
+    L = 40000
+    p = synth.make_prompt(base, L, seed=5)
+    rng = np.random.default_rng(3)
+    cand = np.arange(base.l_sink, L - base.l_recent)
+    pos = np.sort(rng.choice(cand, size=copies, replace=False))
+    p["k"][pos] = p["k"][pos[0]].clone()
+    scores = H.oracle_compress(base, p).pooled[0]
+    dup = scores[pos[0] - base.l_sink]
+    assert (scores[pos - base.l_sink] == dup).all()
+    above = int((scores > dup).sum())
+    wl = base.scaled(topk=above + take)
+    layer = H.GpuLayer(wl, max_seqs=1)
+    idx = layer.compress([p], [0])
+    seq = H.oracle_compress(wl, p)
+    np.testing.assert_array_equal(idx[0][0], seq.topk_pos[0])
+    kept = np.isin(pos, idx[0][0])
+    assert kept[:take].all() and not kept[take:].any()
+
+
 def test_budget_covers_prompt_equals_dense_attention():
     """K >= number of candidates and no new token: the compressed cache attends like the full one."""
     wl = SMALL_F32.scaled(topk=1024)
