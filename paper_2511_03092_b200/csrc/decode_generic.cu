@@ -35,12 +35,15 @@ struct DecodeArgs {
 
 template <typename T>
 __global__ void __launch_bounds__(NT) decode_split_kernel(const DecodeArgs a) {
+  pdl_wait();                                // the previous step's merge (or whatever came before) has finished
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the merge may take its place and wait
   extern __shared__ float smem[];
   float* qs = smem;                          // [HB][d_qk]
   float* sc = qs + HB * a.d_qk;              // [HB][TR]
   float* m_run = sc + HB * TR;               // [HB]
   float* l_run = m_run + HB;
   float* alpha = l_run + HB;
+  float* sc_x = alpha + HB;                  // [HB][NT / 2] exchange between the CTA's halves (narrow heads)
 
   const int sp = blockIdx.x, i = blockIdx.z;
   const int kvh = blockIdx.y / a.n_hb, hb = blockIdx.y % a.n_hb;
@@ -72,6 +75,10 @@ __global__ void __launch_bounds__(NT) decode_split_kernel(const DecodeArgs a) {
   const int tps = (ntiles + a.nsplit - 1) / a.nsplit;
   const int v0 = min(n_valid, sp * tps * TR), v1 = min(n_valid, (sp + 1) * tps * TR);
 
+  // p.V: a thread owns output dims; with heads of at most NT / 2 dims the CTA's two halves share the rows of a
+  // tile between them (their sums meet in shared memory at the end) instead of leaving one half idle
+  const int nhalf = a.d_v <= NT / 2 ? 2 : 1;
+  const int rhalf = nhalf == 2 ? tid / (NT / 2) : 0, dtid = nhalf == 2 ? tid % (NT / 2) : tid;
   for (int e = tid; e < nh * a.d_qk; e += NT)
     qs[e] = to_f32<T>(static_cast<const T*>(a.q)[((long long)i * a.Hq + h0) * a.d_qk + e]);
   if (tid < HB) { m_run[tid] = -INFINITY; l_run[tid] = 0.f; alpha[tid] = 1.f; }
@@ -85,31 +92,53 @@ __global__ void __launch_bounds__(NT) decode_split_kernel(const DecodeArgs a) {
                 : (a.v_new ? static_cast<const T*>(a.v_new) + ((long long)i * a.Hkv + kvh) * a.d_v : nullptr);
   const int Lsr = a.Ls + a.Lr;
 
+  constexpr int RPW = TR / NWARP;                            // rows per warp and tile
   for (int vb = v0; vb < v1; vb += TR) {
-    // phase 1: logits
-    for (int r = wid; r < TR; r += NWARP) {
-      const int v = vb + r;
-      float s[HB];
+    // phase 1: logits.  A warp takes its RPW rows together, so that the loads of all of them are in flight at
+    // once (row after row, each row's load latency was paid in turn: 37 us per step of a 772-slot fp32 cache).
+    {
+      const T* krow[RPW];
+      bool live[RPW];
 #pragma unroll
-      for (int h = 0; h < HB; ++h) s[h] = 0.f;
-      if (v < v1) {
+      for (int rr = 0; rr < RPW; ++rr) {
+        const int v = vb + wid + rr * NWARP;
+        live[rr] = v < v1;
         const int cs = v < n_low ? v : Lsr + (v - n_low);
-        const T* krow = cs == new_slot ? kn : reinterpret_cast<const T*>(kc + (long long)cs * a.k_row_b);
-        for (int c = lane; c < a.d_qk; c += 32) {
-          const float kv = to_f32<T>(krow[c]);
+        krow[rr] = !live[rr] ? nullptr : cs == new_slot ? kn : reinterpret_cast<const T*>(kc + (long long)cs * a.k_row_b);
+      }
+      float s[RPW][HB];
 #pragma unroll
-          for (int h = 0; h < HB; ++h)
-            if (h < nh) s[h] = fmaf(kv, qs[h * a.d_qk + c], s[h]);
+      for (int rr = 0; rr < RPW; ++rr)
+#pragma unroll
+        for (int h = 0; h < HB; ++h) s[rr][h] = 0.f;
+#pragma unroll 2
+      for (int c = lane; c < a.d_qk; c += 32) {
+        float kv[RPW];
+#pragma unroll
+        for (int rr = 0; rr < RPW; ++rr) kv[rr] = live[rr] ? to_f32<T>(krow[rr][c]) : 0.f;
+#pragma unroll
+        for (int h = 0; h < HB; ++h) {
+          if (h < nh) {
+            const float qv = qs[h * a.d_qk + c];
+#pragma unroll
+            for (int rr = 0; rr < RPW; ++rr) s[rr][h] = fmaf(kv[rr], qv, s[rr][h]);
+          }
         }
       }
 #pragma unroll
-      for (int h = 0; h < HB; ++h) {
+      for (int rr = 0; rr < RPW; ++rr) {
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s[h] += __shfl_xor_sync(0xffffffffu, s[h], o);
-      }
-      if (lane == 0) {
+        for (int h = 0; h < HB; ++h) {
+          if (h < nh) {                                      // nh is uniform over the CTA
 #pragma unroll
-        for (int h = 0; h < HB; ++h) sc[h * TR + r] = v < v1 ? s[h] * a.scale : -INFINITY;
+            for (int o = 16; o > 0; o >>= 1) s[rr][h] += __shfl_xor_sync(0xffffffffu, s[rr][h], o);
+          }
+        }
+        if (lane == 0) {
+          const int r = wid + rr * NWARP;
+#pragma unroll
+          for (int h = 0; h < HB; ++h) sc[h * TR + r] = live[rr] ? s[rr][h] * a.scale : -INFINITY;
+        }
       }
     }
     __syncthreads();
@@ -144,18 +173,26 @@ __global__ void __launch_bounds__(NT) decode_split_kernel(const DecodeArgs a) {
       }
     }
     const int nr = min(TR, v1 - vb);
-    for (int r = 0; r < nr; ++r) {
-      const int v = vb + r;
-      const int cs = v < n_low ? v : Lsr + (v - n_low);
-      const T* vrow = cs == new_slot ? vn : reinterpret_cast<const T*>(vc + (long long)cs * v_row_b);
+    constexpr int VB = 8;                                    // value rows whose loads are in flight together
+    for (int r0 = rhalf * VB; r0 < nr; r0 += VB * nhalf) {   // narrow heads: the two halves of the CTA take alternate groups
 #pragma unroll
       for (int c = 0; c < MAX_DV_PER_THREAD; ++c) {
-        const int dim = tid + c * NT;
+        const int dim = dtid + c * NT;
         if (dim < a.d_v) {
-          const float vv = to_f32<T>(vrow[dim]);
+          float vv[VB];
 #pragma unroll
-          for (int h = 0; h < HB; ++h)
-            if (h < nh) acc[h][c] = fmaf(sc[h * TR + r], vv, acc[h][c]);
+          for (int u = 0; u < VB; ++u) {
+            const int v = vb + r0 + u;
+            const int cs = v < n_low ? v : Lsr + (v - n_low);
+            const T* vrow = cs == new_slot ? vn : reinterpret_cast<const T*>(vc + (long long)cs * v_row_b);
+            vv[u] = r0 + u < nr ? to_f32<T>(vrow[dim]) : 0.f;
+          }
+#pragma unroll
+          for (int u = 0; u < VB; ++u) {
+#pragma unroll
+            for (int h = 0; h < HB; ++h)
+              if (h < nh) acc[h][c] = fmaf(sc[h * TR + r0 + u], vv[u], acc[h][c]);
+          }
         }
       }
     }
@@ -163,6 +200,18 @@ __global__ void __launch_bounds__(NT) decode_split_kernel(const DecodeArgs a) {
   }
 
   // partial results
+  if (nhalf == 2) {
+    float* xs = sc_x;
+    if (rhalf == 1) {
+#pragma unroll
+      for (int h = 0; h < HB; ++h) xs[h * (NT / 2) + dtid] = acc[h][0];
+    }
+    __syncthreads();
+    if (rhalf == 0) {
+#pragma unroll
+      for (int h = 0; h < HB; ++h) acc[h][0] += xs[h * (NT / 2) + dtid];
+    }
+  }
 #pragma unroll
   for (int h = 0; h < HB; ++h) {
     if (h < nh) {
@@ -170,8 +219,8 @@ __global__ void __launch_bounds__(NT) decode_split_kernel(const DecodeArgs a) {
       if (tid == 0) { ph[0] = m_run[h]; ph[1] = l_run[h]; }
 #pragma unroll
       for (int c = 0; c < MAX_DV_PER_THREAD; ++c) {
-        const int dim = tid + c * NT;
-        if (dim < a.d_v) ph[2 + dim] = acc[h][c];
+        const int dim = dtid + c * NT;
+        if (rhalf == 0 && dim < a.d_v) ph[2 + dim] = acc[h][c];
       }
     }
   }
@@ -196,23 +245,37 @@ template <typename T>
 __global__ void decode_merge_kernel(const float* __restrict__ partials, T* __restrict__ out,
                                     int Hq, int d_v, int nsplit, const int* __restrict__ slot_ids,
                                     int* seq_len, int max_seqs, int bump) {
+  pdl_wait();                                // all splits have written their partial results
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next step's kernel waits at its top
   const int h = blockIdx.x, i = blockIdx.y;
   const int ps = d_v + 2;
   const float* p = partials + ((long long)i * Hq + h) * nsplit * ps;
-  float m = -INFINITY;
-  for (int s = 0; s < nsplit; ++s) m = fmaxf(m, p[s * ps]);
-  float l = 0.f;
-  for (int s = 0; s < nsplit; ++s) {
-    const float ms = p[s * ps];
-    if (ms != -INFINITY) l += p[s * ps + 1] * expf(ms - m);
+  // The splits' (m, l) are fetched by one thread each and their weights e^{m_s - m} computed once per block;
+  // the sums over the splits then run with eight loads in flight.  (One load after the other, per thread and
+  // per split, this kernel took 12.5 us for 13 splits of 8 heads.)
+  __shared__ float m_s[64], w_s[64], wl_s[64];               // nsplit <= 64
+  const int tid = threadIdx.x;
+  float l_mine = 0.f;
+  if (tid < nsplit) {
+    m_s[tid] = p[tid * ps];
+    l_mine = p[tid * ps + 1];
   }
+  __syncthreads();
+  float m = -INFINITY;
+  for (int s = 0; s < nsplit; ++s) m = fmaxf(m, m_s[s]);
+  if (tid < nsplit) {
+    const float w = m_s[tid] != -INFINITY ? expf(m_s[tid] - m) : 0.f;
+    w_s[tid] = w;
+    wl_s[tid] = w * l_mine;
+  }
+  __syncthreads();
+  float l = 0.f;
+  for (int s = 0; s < nsplit; ++s) l += wl_s[s];             // same order in every thread
   const float inv = l > 0.f ? 1.f / l : 0.f;
-  for (int dim = threadIdx.x; dim < d_v; dim += blockDim.x) {
+  for (int dim = tid; dim < d_v; dim += blockDim.x) {
     float o = 0.f;
-    for (int s = 0; s < nsplit; ++s) {
-      const float ms = p[s * ps];
-      if (ms != -INFINITY) o += p[s * ps + 2 + dim] * expf(ms - m);
-    }
+#pragma unroll 8
+    for (int s = 0; s < nsplit; ++s) o = fmaf(w_s[s], p[s * ps + 2 + dim], o);
     out[((long long)i * Hq + h) * d_v + dim] = from_f32<T>(o * inv);
   }
   if (bump && h == 0 && threadIdx.x == 0) {
@@ -227,7 +290,7 @@ int decode_generic_nsplit(const Shape& s, int n_active, int sm_count) {
   const int n_hb = (s.g + HB - 1) / HB;
   const long long base = (long long)n_active * s.Hkv * n_hb;
   int nsplit = (int)((4LL * sm_count + base - 1) / base);
-  const int max_split = (s.Sc + 2 * TR - 1) / (2 * TR);
+  const int max_split = (s.Sc + TR - 1) / TR;               // down to one 32-row tile per CTA
   nsplit = nsplit < 1 ? 1 : nsplit;
   nsplit = nsplit > max_split ? max_split : nsplit;
   nsplit = nsplit > 64 ? 64 : nsplit;
@@ -255,24 +318,27 @@ cudaError_t launch_decode_generic(int dtype, const Shape& s, const void* q, cons
   a.max_seqs = s.max_seqs; a.v_aliases_k = s.v_aliases_k; a.n_hb = (s.g + HB - 1) / HB;
   a.nsplit = nsplit; a.scale = s.scale; a.seq_len = seq_len; a.valid_topk = valid_topk;
   a.partials = partials; a.out = out; a.status = status;
-  const size_t smem = (size_t)(HB * s.d_qk + HB * TR + 3 * HB) * sizeof(float);
+  const size_t smem = (size_t)(HB * s.d_qk + HB * TR + 3 * HB + HB * (NT / 2)) * sizeof(float);
   dim3 grid(nsplit, s.Hkv * a.n_hb, n_active);
   dim3 mgrid(s.Hq, n_active);
   const int bump = k_new != nullptr;
+  // both launches are programmatic dependents: each waits at its top for the one before
+  cudaError_t e;
   if (dtype == SNAP_F32) {
-    decode_split_kernel<float><<<grid, NT, smem, st>>>(a);
+    e = launch_pdl(decode_split_kernel<float>, grid, dim3(NT), smem, st, a);
     count_launch();
-    decode_merge_kernel<float><<<mgrid, 128, 0, st>>>(partials, static_cast<float*>(out), s.Hq, s.d_v,
-                                                      nsplit, slot_ids, seq_len, s.max_seqs, bump);
+    if (e == cudaSuccess)
+      e = launch_pdl(decode_merge_kernel<float>, mgrid, dim3(128), 0, st, static_cast<const float*>(partials),
+                     static_cast<float*>(out), s.Hq, s.d_v, nsplit, slot_ids, seq_len, s.max_seqs, bump);
   } else {
-    decode_split_kernel<__nv_bfloat16><<<grid, NT, smem, st>>>(a);
+    e = launch_pdl(decode_split_kernel<__nv_bfloat16>, grid, dim3(NT), smem, st, a);
     count_launch();
-    decode_merge_kernel<__nv_bfloat16><<<mgrid, 128, 0, st>>>(
-        partials, static_cast<__nv_bfloat16*>(out), s.Hq, s.d_v, nsplit, slot_ids, seq_len,
-        s.max_seqs, bump);
+    if (e == cudaSuccess)
+      e = launch_pdl(decode_merge_kernel<__nv_bfloat16>, mgrid, dim3(128), 0, st, static_cast<const float*>(partials),
+                     static_cast<__nv_bfloat16*>(out), s.Hq, s.d_v, nsplit, slot_ids, seq_len, s.max_seqs, bump);
   }
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace snap
