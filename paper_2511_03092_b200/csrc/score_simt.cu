@@ -129,17 +129,25 @@ __global__ void __launch_bounds__(NT) score_stats_kernel(const ScoreArgs a) {
 }
 
 // Merge the per-split statistics: m = max_s m_s, l = sum_s l_s exp(m_s - m), kept as (m, 1/l).
+// One warp per query row, lanes over the splits (a thread per row walking the splits one dependent load and
+// one double-precision exponential at a time took 18 us for 60 splits).
 __global__ void score_combine_kernel(const float2* __restrict__ part, float2* __restrict__ stats,
                                      double* __restrict__ mu64, int nsplit, int R) {
-  const long long z = blockIdx.x;
-  for (int row = threadIdx.x; row < R; row += blockDim.x) {
-    float m = -INFINITY;
-    for (int s = 0; s < nsplit; ++s) m = fmaxf(m, part[(z * nsplit + s) * R + row].x);
-    double l = 0.0;
-    for (int s = 0; s < nsplit; ++s) {
-      const float2 p = part[(z * nsplit + s) * R + row];
-      if (p.y > 0.f) l += (double)p.y * exp((double)p.x - (double)m);
-    }
+  const long long z = blockIdx.y;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= R) return;
+  float m = -INFINITY;
+  for (int s = lane; s < nsplit; s += 32) m = fmaxf(m, part[(z * nsplit + s) * R + row].x);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  double l = 0.0;
+  for (int s = lane; s < nsplit; s += 32) {
+    const float2 p = part[(z * nsplit + s) * R + row];
+    if (p.y > 0.f) l += (double)p.y * exp((double)p.x - (double)m);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+  if (lane == 0) {
     stats[z * R + row] = make_float2(m, (float)(1.0 / l));
     if (mu64) mu64[z * R + row] = ((double)m + log(l)) * 1.4426950408889634074;   // log2 domain, unrounded
   }
@@ -204,7 +212,7 @@ cudaError_t launch_t(const ScoreArgs& a, int max_le, cudaStream_t st) {
     dim3 g1(a.buf.nsplit, (R + BM - 1) / BM, nz);
     score_stats_kernel<T><<<g1, NT, 0, st>>>(a);
     count_launch();
-    score_combine_kernel<<<nz, 256, 0, st>>>(a.buf.part_stats, a.buf.stats, a.buf.ref.mu64, a.buf.nsplit, R);
+    score_combine_kernel<<<dim3((R + 7) / 8, nz), 256, 0, st>>>(a.buf.part_stats, a.buf.stats, a.buf.ref.mu64, a.buf.nsplit, R);
     count_launch();
   }
   dim3 g2((max_le + BN - 1) / BN, 1, nz);
