@@ -410,14 +410,28 @@ __global__ void __launch_bounds__(D) decode_gqa_merge_kernel(const float* __rest
   // launched with programmatic stream serialisation: the grid may start while the split kernel
   // drains; everything the split kernel wrote is visible after this wait
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  float M = -INFINITY;
-  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * PS]);
-  float L = 0.f, O = 0.f;
-  for (int s = 0; s < nsplit; ++s) {
-    const float ms = p[s * PS];
-    const float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
-    L += p[s * PS + 1] * f;
-    O += p[s * PS + 2 + t] * f;
+  float M = -INFINITY, L = 0.f, O = 0.f;
+  if (nsplit <= D) {
+    // The splits' (m, l) are fetched by one thread each; every thread then derives the weights from shared
+    // memory and sums its output dim with eight loads in flight (split after split, each thread paid two
+    // dependent rounds of global loads per split).
+    __shared__ float m_s[D], l_s[D], f_s[D];
+    if (t < nsplit) { m_s[t] = p[t * PS]; l_s[t] = p[t * PS + 1]; }
+    __syncthreads();
+    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, m_s[s]);
+    if (t < nsplit) f_s[t] = m_s[t] == -INFINITY ? 0.f : exp2f(m_s[t] - M);
+    __syncthreads();
+    for (int s = 0; s < nsplit; ++s) L += l_s[s] * f_s[s];
+#pragma unroll 8
+    for (int s = 0; s < nsplit; ++s) O = fmaf(p[s * PS + 2 + t], f_s[s], O);
+  } else {
+    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * PS]);
+    for (int s = 0; s < nsplit; ++s) {
+      const float ms = p[s * PS];
+      const float f = ms == -INFINITY ? 0.f : exp2f(ms - M);
+      L += p[s * PS + 1] * f;
+      O += p[s * PS + 2 + t] * f;
+    }
   }
   out[(orow * Hq + h) * D + t] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
   if (bump && h == 0 && t == 0) {

@@ -417,21 +417,38 @@ __global__ void __launch_bounds__(128) decode_gqa_mma_merge_kernel(const float* 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const float* p = partials + ((long long)i * Hq + h) * nsplit * ps;
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  float M = -INFINITY;
-  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * ps]);
-  float L = 0.f;
-  for (int s = 0; s < nsplit; ++s) {
-    const float ms = p[s * ps];
-    if (ms != -INFINITY) L += p[s * ps + 1] * exp2f(ms - M);
-  }
-  const float inv = L > 0.f ? 1.f / L : 0.f;
-  for (int t = threadIdx.x; t < d; t += blockDim.x) {
-    float O = 0.f;
+  float M = -INFINITY, L = 0.f;
+  if (nsplit <= 128) {                                       // (m, l) fetched by one thread per split, weights in shared memory
+    __shared__ float m_s[128], l_s[128], f_s[128];
+    const int t0 = threadIdx.x;
+    if (t0 < nsplit) { m_s[t0] = p[t0 * ps]; l_s[t0] = p[t0 * ps + 1]; }
+    __syncthreads();
+    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, m_s[s]);
+    if (t0 < nsplit) f_s[t0] = m_s[t0] == -INFINITY ? 0.f : exp2f(m_s[t0] - M);
+    __syncthreads();
+    for (int s = 0; s < nsplit; ++s) L += l_s[s] * f_s[s];
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    for (int t = threadIdx.x; t < d; t += blockDim.x) {
+      float O = 0.f;
+#pragma unroll 8
+      for (int s = 0; s < nsplit; ++s) O = fmaf(p[s * ps + 2 + t], f_s[s], O);
+      out[(orow * Hq + h) * d + t] = __float2bfloat16_rn(O * inv);
+    }
+  } else {
+    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p[s * ps]);
     for (int s = 0; s < nsplit; ++s) {
       const float ms = p[s * ps];
-      if (ms != -INFINITY) O += p[s * ps + 2 + t] * exp2f(ms - M);
+      if (ms != -INFINITY) L += p[s * ps + 1] * exp2f(ms - M);
     }
-    out[(orow * Hq + h) * d + t] = __float2bfloat16_rn(O * inv);
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    for (int t = threadIdx.x; t < d; t += blockDim.x) {
+      float O = 0.f;
+      for (int s = 0; s < nsplit; ++s) {
+        const float ms = p[s * ps];
+        if (ms != -INFINITY) O += p[s * ps + 2 + t] * exp2f(ms - M);
+      }
+      out[(orow * Hq + h) * d + t] = __float2bfloat16_rn(O * inv);
+    }
   }
   if (bump && h == 0 && threadIdx.x == 0) {
     const int slot = slot_ids[i / q_len];
