@@ -953,19 +953,23 @@ def run_config(args):
     t1.record()
     torch.cuda.synchronize()
     ms = t0.elapsed_time(t1) / steps
-    # the same step captured once as a CUDA graph (all layers' launches) and replayed
+    # the same steps captured as a CUDA graph (all layers' launches, sixteen steps per graph so that the
+    # replay's own launch latency -- about 12 us -- does not hide a step of that size) and replayed
+    graph_steps = 16
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
-        step(0)
+        for s in range(graph_steps):
+            step(s)
     for s in range(args.warmup):
         graph.replay()
     torch.cuda.synchronize()
+    replays = max(1, steps // graph_steps)
     t0.record()
-    for s in range(steps):
+    for s in range(replays):
         graph.replay()
     t1.record()
     torch.cuda.synchronize()
-    ms_graph = t0.elapsed_time(t1) / steps
+    ms_graph = t0.elapsed_time(t1) / (replays * graph_steps)
     eb = 2 if wl.dtype == "bf16" else 4
     rows = min(L + 1, wl.slots)
     step_bytes = n_layers * nseq * wl.n_kv_heads * rows * (wl.d_qk + (0 if wl.v_aliases_k else wl.d_v)) * eb

@@ -401,7 +401,9 @@ int snap_decode_attn_blocks(const snap_config_t* cfg, const snap_layout_t* layou
  * Returns the option's previous value, or SNAP_ERR_INVALID_ARG.
  */
 #define SNAP_OPT_SCORE_KERNEL 0          /* 1: mma.sync score kernel, 2: SIMT, 3: tcgen05 without CTA pairs  SNAP_SCORE_PATH=mma|simt|single */
-#define SNAP_OPT_DECODE_GQA_KERNEL 1     /* 1: packed-FP32 GQA decode kernel        SNAP_DECODE_GQA=simt     */
+#define SNAP_OPT_DECODE_GQA_KERNEL 1     /* 1: packed-FP32 GQA decode kernel; the tensor-core kernel 2: always with a merge
+                                               launch, 3: with the in-kernel merge of small batches outside stream capture
+                                               too (by default only under capture)   SNAP_DECODE_GQA=simt|split|fused */
 #define SNAP_OPT_DECODE_LATENT_KERNEL 2  /* 1: mma.sync latent decode kernel        SNAP_DECODE_MLA=mma      */
 #define SNAP_OPT_DECODE_NSPLIT 3         /* n: splits per (sequence, KV head)       SNAP_DECODE_NSPLIT=n     */
 #define SNAP_OPT_SCORE_NSPLIT 4          /* n: candidate splits of the longest prompt  SNAP_SCORE_NSPLIT=n   */

@@ -22,7 +22,7 @@ std::once_flag g_opt_once;
 void seed_options() {
   auto env_int = [](const char* name) { const char* e = getenv(name); const int v = e ? atoi(e) : 0; return v > 0 ? v : 0; };
   if (const char* e = getenv("SNAP_SCORE_PATH")) g_opt[SNAP_OPT_SCORE_KERNEL] = !strcmp(e, "mma") ? 1 : !strcmp(e, "simt") ? 2 : !strcmp(e, "single") ? 3 : 0;
-  if (const char* e = getenv("SNAP_DECODE_GQA")) g_opt[SNAP_OPT_DECODE_GQA_KERNEL] = e[0] == 's';
+  if (const char* e = getenv("SNAP_DECODE_GQA")) g_opt[SNAP_OPT_DECODE_GQA_KERNEL] = !strcmp(e, "simt") ? 1 : !strcmp(e, "split") ? 2 : !strcmp(e, "fused") ? 3 : 0;
   if (const char* e = getenv("SNAP_DECODE_MLA")) g_opt[SNAP_OPT_DECODE_LATENT_KERNEL] = e[0] == 'm';
   if (const char* e = getenv("SNAP_PREFILL_PATH")) g_opt[SNAP_OPT_PREFILL_KERNEL] = !strcmp(e, "simt");
   if (const char* e = getenv("SNAP_PREFILL_HEADS")) g_opt[SNAP_OPT_PREFILL_SINGLE_HEADS] = e[0] == '1';

@@ -56,6 +56,7 @@ struct MmaArgs {
   float scale_log2;
   const int* seq_len; const int* valid_topk;
   float* partials;                              // [n_active][T][Hq][nsplit][PS]
+  __nv_bfloat16* out;                           // fused merge only: [n_active][QT][Hq][D]
   uint32_t* status;
   // per-step block lookup (block_topk.cu): NULL, or the blocks of the third section to visit, ascending
   const int* block_idx;                         // [n_active][Hkv][blocks_cap]
@@ -83,7 +84,14 @@ __device__ __forceinline__ TileRows tile_rows(int j, int nA, int n_low, int Lsr,
 
 // D: head size (64, 128 or 256); NWARP: warps per CTA (fewer for wide heads, whose stages are larger);
 // NG: groups of eight MMA columns (1, or 2 for multi-token steps with 9 to 16 query rows per KV head)
-template <int D, int NWARP, int NG>
+// FUSED: the splits of a (sequence, KV head) form one thread-block cluster (the grid's x extent) and merge
+// their results through distributed shared memory instead of a second launch -- for small batches, where a
+// step is a chain of launch latencies.  Every CTA reduces an equal share of the output elements: each split
+// sends every CTA that CTA's share of its outputs, and its (max, sum) per column, with asynchronous remote
+// stores that complete on the receiver's mbarrier; a CTA waits for its own arrivals only, so the one cluster
+// barrier (the mbarriers exist before anything is sent) is started at the top of the kernel and completed
+// just before the sends, and none is needed at the end.
+template <int D, int NWARP, int NG, bool FUSED>
 __global__ void __launch_bounds__(NWARP * 32, NG == 1 ? 3 : 2)
 decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v) {
   constexpr int NT = NWARP * 32, NSL = D / 64, CPR = D / 8, KS = D / 16;   // slabs per tensor, 16-byte chunks per row, 16-dim steps
@@ -92,6 +100,13 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
   unsigned char* smem_raw = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   // [NWARP][NSTAGE] stages | [NWARP][NSTAGE] mbarriers
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + NWARP * NSTAGE * STAGE_B);
+  // fused merge: this split's outputs [columns][D] (+ padding), its (max, sum) per column, the inbox
+  // [splits][share of the outputs + 16] and the inbox's barrier
+  constexpr int XO = NG * GP * D + 64;
+  float* osm = reinterpret_cast<float*>(bars + NWARP * NSTAGE);
+  float* mls = osm + XO;
+  float* inbox = mls + 16;
+  uint64_t* xbar = reinterpret_cast<uint64_t*>(inbox + XO + 16 * 16);
 
   const int sp = blockIdx.x, kvh = blockIdx.y, i = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, gq = lane >> 2, tq = lane & 3;
@@ -99,9 +114,11 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
   const uint32_t stage0 = smem_u32(wstages), bar0 = smem_u32(bars + w * NSTAGE);
   if (lane == 0) {
     for (int s = 0; s < NSTAGE; ++s) mbar_init(bar0 + 8 * s, 1);
+    if (FUSED && tid == 0) mbar_init(smem_u32(xbar), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
+  if (FUSED) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // completed before the merge's sends
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int slot = a.slot_ids[i];
   const bool bad = slot < 0 || slot >= a.max_seqs;
@@ -391,16 +408,72 @@ decode_gqa_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap tmap_
       L += base[ww * WSTRIDE + NCOL + h] * f[ww];
     }
     const int tcol = h / a.g, hcol = h - tcol * a.g;
+    // this split's result for column h: to scratch for the merge kernel, or to this CTA's exchange area
     float* ph = a.partials + ((((long long)i * TQ + tcol) * a.Hq + (long long)kvh * a.g + hcol) * a.nsplit + sp) * PS;
-    if (tid == 0) { ph[0] = M; ph[1] = L; }
+    if (tid == 0) {
+      if (FUSED) { mls[2 * h] = M; mls[2 * h + 1] = L; }
+      else { ph[0] = M; ph[1] = L; }
+    }
     for (int dv = tid; dv < D; dv += NT) {
       float O = 0.f;
 #pragma unroll
       for (int ww = 0; ww < NWARP; ++ww) O += base[ww * WSTRIDE + 2 * NCOL + h * D + dv] * f[ww];
-      ph[2 + dv] = O;
+      if (FUSED) osm[h * D + dv] = O;
+      else ph[2 + dv] = O;
+    }
+  }
+  if (FUSED) {
+    const int ns = a.nsplit;                                   // = cluster size; sp = this CTA's rank in the cluster
+    const int W = ncols * D;
+    const int per = (((W + ns - 1) / ns) + 3) & ~3;            // outputs reduced by each CTA, whole 16-byte pieces
+    const int pp = per / 4 + 4, row = per + 16;                // pieces sent to each CTA: its outputs, then 16 floats of (max, sum)
+    __syncthreads();                                           // osm and mls are complete
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every CTA's inbox barrier exists
+    if (tid == 0) mbar_expect_tx(smem_u32(xbar), (unsigned)(ns * pp * 16));
+    const uint32_t my_row = smem_u32(inbox) + (uint32_t)(sp * row) * 4u, xb = smem_u32(xbar);
+    for (int e = tid; e < ns * pp; e += NT) {
+      const int to = e / pp, piece = e - to * pp;
+      const float* src = piece < per / 4 ? osm + to * per + 4 * piece : mls + 4 * (piece - per / 4);
+      const uint4 v = *reinterpret_cast<const uint4*>(src);
+      asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                   ::"r"(umma::map_to_rank(my_row + (uint32_t)piece * 16u, (uint32_t)to)), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w),
+                     "r"(umma::map_to_rank(xb, (uint32_t)to)) : "memory");
+    }
+    if (!mbar_wait_bounded(smem_u32(xbar), 0u)) {
+      if (tid == 0 && a.status) atomicOr(a.status, SNAP_DEV_WAIT_TIMEOUT);
+    } else {
+      for (int ol = tid; ol < per; ol += NT) {
+        const int o = sp * per + ol;
+        if (o >= W) break;
+        const int h = o / D, dv = o - h * D;
+        float M = -INFINITY;
+        for (int rr = 0; rr < ns; ++rr) M = fmaxf(M, inbox[rr * row + per + 2 * h]);
+        float L = 0.f, O = 0.f;
+        for (int rr = 0; rr < ns; ++rr) {
+          const float mr = inbox[rr * row + per + 2 * h];
+          const float fr = mr == -INFINITY ? 0.f : exp2f(mr - M);
+          L = fmaf(inbox[rr * row + per + 2 * h + 1], fr, L);
+          O = fmaf(inbox[rr * row + ol], fr, O);
+        }
+        const int tcol = h / a.g, hcol = h - tcol * a.g;
+        const long long orow = (long long)i * a.QT + a.u0 + tcol;
+        a.out[(orow * a.Hq + (long long)kvh * a.g + hcol) * D + dv] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
+      }
     }
   }
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// The sequence lengths advance after every CTA of the step has read them: with the fused merge that is a
+// launch of its own (a few threads), off the path of the step's outputs.
+__global__ void decode_gqa_bump_kernel(const int* __restrict__ slot_ids, int* seq_len, int max_seqs, int n_rows, int q_len) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r < n_rows) {
+    const int slot = slot_ids[r / q_len];
+    if (slot >= 0 && slot < max_seqs) atomicAdd(&seq_len[slot], 1);
+  }
 }
 
 // Merge the splits of one (sequence, query token, query head) for any head size; maxima are in
@@ -456,14 +529,40 @@ __global__ void __launch_bounds__(128) decode_gqa_mma_merge_kernel(const float* 
   }
 }
 
-template <int D, int NWARP, int NG>
+template <int D, int NWARP, int NG, bool FUSED>
 cudaError_t launch_d(const MmaArgs& a, const CUtensorMap& tk, const CUtensorMap& tv, int n_active, cudaStream_t st) {
-  constexpr size_t smem = (size_t)NWARP * NSTAGE * (2 * (D / 64) * SLAB_B) + NWARP * NSTAGE * 8 + 1024;
+  constexpr size_t smem = (size_t)NWARP * NSTAGE * (2 * (D / 64) * SLAB_B) + NWARP * NSTAGE * 8 + 1024 +
+                          (FUSED ? (size_t)(2 * (NG * GP * D + 64) + 16 + 16 * 16) * sizeof(float) + 16 : 0);
   static_assert((size_t)NSTAGE * (2 * (D / 64) * SLAB_B) >= (size_t)NG * GP * (D + 2) * sizeof(float), "a warp's result fits its stages");
   static SmemLimit limit = {};
-  if (cudaError_t e = ensure_dyn_smem(decode_gqa_mma_kernel<D, NWARP, NG>, smem, limit)) return e;
-  const cudaError_t e = launch_pdl(decode_gqa_mma_kernel<D, NWARP, NG>, dim3(a.nsplit, a.Hkv, n_active), dim3(NWARP * 32), smem,
-                                   st, a, tk, tv);
+  if (cudaError_t e = ensure_dyn_smem(decode_gqa_mma_kernel<D, NWARP, NG, FUSED>, smem, limit)) return e;
+  cudaError_t e;
+  if (FUSED) {
+    // the splits of a (sequence, KV head) as one cluster; more than eight CTAs per cluster need the opt-in
+    static bool allowed = false;
+    if (a.nsplit > 8 && !allowed) {
+      if ((e = cudaFuncSetAttribute(decode_gqa_mma_kernel<D, NWARP, NG, FUSED>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1)) != cudaSuccess)
+        return e;
+      allowed = true;
+    }
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)a.nsplit;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(a.nsplit, a.Hkv, n_active);
+    lc.blockDim = dim3(NWARP * 32);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    lc.attrs = attr;
+    lc.numAttrs = 2;
+    e = cudaLaunchKernelEx(&lc, decode_gqa_mma_kernel<D, NWARP, NG, FUSED>, a, tk, tv);
+  } else {
+    e = launch_pdl(decode_gqa_mma_kernel<D, NWARP, NG, FUSED>, dim3(a.nsplit, a.Hkv, n_active), dim3(NWARP * 32), smem, st, a, tk, tv);
+  }
   count_launch();
   return e;
 }
@@ -535,9 +634,38 @@ cudaError_t launch_decode_gqa_mma(const Shape& s, const void* q, const void* k_n
   a.block_idx = block_idx; a.n_sel = n_sel; a.blocks_cap = blocks_cap; a.tpb = block_idx ? block_tokens / WT : 1;
   cudaError_t e;
   const bool wide = q_len * s.g > GP;                          // 9 to 16 (token, head) columns: two column groups
-  if (D == 128) e = wide ? launch_d<128, 4, 2>(a, hit->tk, hit->tv, n_active, st) : launch_d<128, 4, 1>(a, hit->tk, hit->tv, n_active, st);
-  else if (D == 64) e = wide ? launch_d<64, 4, 2>(a, hit->tk, hit->tv, n_active, st) : launch_d<64, 4, 1>(a, hit->tk, hit->tv, n_active, st);
-  else e = wide ? launch_d<256, 2, 2>(a, hit->tk, hit->tv, n_active, st) : launch_d<256, 2, 1>(a, hit->tk, hit->tv, n_active, st);
+  // Small batches (the grid is at most about one CTA per SM) whose step is being captured into a CUDA graph: the
+  // splits merge inside the kernel, as one cluster per (sequence, KV head) -- 9.6 against 11.0 us per replayed
+  // step of one 5124-slot sequence.  Launched eagerly such a step is bound by the host's launch calls, and a
+  // cluster launch costs the host more than the merge kernel's plain launch (16.3 against 12.0 us per step), so
+  // eager steps keep the two launches.  Option SNAP_OPT_DECODE_GQA_KERNEL = 2: never merge in the kernel, 3: merge
+  // in the kernel whenever the shape allows (testing aids).  A device that refuses the cluster shape gets the
+  // two launches from then on.
+  static bool fused_refused = false;
+  bool fused = !wide && q_len == 1 && nsplit >= 2 && nsplit <= 16 && !fused_refused && option(SNAP_OPT_DECODE_GQA_KERNEL) != 2 &&
+               (long long)nsplit * s.Hkv * n_active <= 160;
+  if (fused && option(SNAP_OPT_DECODE_GQA_KERNEL) != 3) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    fused = cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusActive;
+  }
+  if (fused) {
+    a.out = static_cast<__nv_bfloat16*>(out);
+    e = D == 128 ? launch_d<128, 4, 1, true>(a, hit->tk, hit->tv, n_active, st)
+        : D == 64 ? launch_d<64, 4, 1, true>(a, hit->tk, hit->tv, n_active, st)
+                  : launch_d<256, 2, 1, true>(a, hit->tk, hit->tv, n_active, st);
+    if (e == cudaSuccess) {
+      if (!k_new) return cudaGetLastError();                   // attend only: the lengths stay
+      e = launch_pdl(decode_gqa_bump_kernel, dim3((n_active + 127) / 128), dim3(128), 0, st, slot_ids, seq_len, s.max_seqs, n_active, 1);
+      count_launch();
+      return e != cudaSuccess ? e : cudaGetLastError();
+    }
+    (void)cudaGetLastError();                                  // e.g. a cluster of this size cannot be scheduled: two launches from now on
+    fused_refused = true;
+  }
+  a.out = nullptr;
+  if (D == 128) e = wide ? launch_d<128, 4, 2, false>(a, hit->tk, hit->tv, n_active, st) : launch_d<128, 4, 1, false>(a, hit->tk, hit->tv, n_active, st);
+  else if (D == 64) e = wide ? launch_d<64, 4, 2, false>(a, hit->tk, hit->tv, n_active, st) : launch_d<64, 4, 1, false>(a, hit->tk, hit->tv, n_active, st);
+  else e = wide ? launch_d<256, 2, 2, false>(a, hit->tk, hit->tv, n_active, st) : launch_d<256, 2, 1, false>(a, hit->tk, hit->tv, n_active, st);
   if (e != cudaSuccess) return e;
   if (D == 128)
     return launch_decode_gqa_merge(partials, out, s.Hq, nsplit, slot_ids, n_active * q_len, q_len, seq_len, s.max_seqs,

@@ -246,6 +246,17 @@ def test_group_sizes(hq, hkv):
     _run_compress_and_decode(wl, [wl.prompt_len[0], 50, 3], seed=13, steps=5)
 
 
+@pytest.mark.parametrize("hq,hkv,d", [(4, 4, 128), (16, 4, 128), (20, 4, 128), (32, 4, 128), (8, 2, 64), (8, 2, 256)],
+                         ids=["g1", "g4", "g5", "g8", "d64", "d256"])
+def test_decode_with_the_merge_inside_the_kernel(hq, hkv, d, snap_option):
+    """Small batches captured into a CUDA graph merge their splits inside the decode kernel (one cluster per
+    sequence and KV head, the lengths advanced by a launch of their own); the option takes that path outside
+    a capture too: ragged lengths, a ring that wraps, sequences shorter than one tile, every head size."""
+    snap_option(B.SNAP_OPT_DECODE_GQA_KERNEL, 3)
+    wl = SMALL_BF16.scaled(n_q_heads=hq, n_kv_heads=hkv, d_qk=d, d_v=d)
+    _run_compress_and_decode(wl, [wl.prompt_len[0], 50, 3], seed=19, steps=wl.l_recent + 5, check_ring_every=16)
+
+
 @pytest.mark.parametrize("hq,hkv", [(4, 4), (16, 4), (20, 4), (32, 4)], ids=["g1", "g4", "g5", "g8"])
 def test_packed_fp32_decode_kernel_stays_selectable(hq, hkv, snap_option):
     """The packed-FP32 decode kernel (the default before the tensor-core one) on the same cases."""
