@@ -559,7 +559,18 @@ cudaError_t launch_d(const MmaArgs& a, const CUtensorMap& tk, const CUtensorMap&
     lc.stream = st;
     lc.attrs = attr;
     lc.numAttrs = 2;
+    // can the device hold a cluster of this size at all?  Asked once per size, before the launch: a launch that
+    // fails inside a stream capture would invalidate the caller's capture.
+    static int fits[17] = {};
+    if (fits[a.nsplit] == 0) {
+      int n_clusters = 0;
+      fits[a.nsplit] = cudaOccupancyMaxActiveClusters(&n_clusters, decode_gqa_mma_kernel<D, NWARP, NG, FUSED>, &lc) == cudaSuccess &&
+                               n_clusters >= 1 ? 1 : -1;
+      if (fits[a.nsplit] < 0) (void)cudaGetLastError();
+    }
+    if (fits[a.nsplit] < 0) return cudaErrorInvalidClusterSize;
     e = cudaLaunchKernelEx(&lc, decode_gqa_mma_kernel<D, NWARP, NG, FUSED>, a, tk, tv);
+    if (e != cudaSuccess) return e;
   } else {
     e = launch_pdl(decode_gqa_mma_kernel<D, NWARP, NG, FUSED>, dim3(a.nsplit, a.Hkv, n_active), dim3(NWARP * 32), smem, st, a, tk, tv);
   }
