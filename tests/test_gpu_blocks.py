@@ -134,6 +134,14 @@ def test_random_block_lookup_configurations(seed):
         _run(wl, lengths, bs, nblk, steps=int(rng.integers(1, 6)), seed=1000 * seed + case)
 
 
+def test_block_lookup_with_the_merge_inside_the_decode_kernel(snap_option):
+    """The block list and the in-kernel merge of small batches (taken under stream capture; the option takes it here)
+    together: ragged prompts, several steps."""
+    snap_option(B.SNAP_OPT_DECODE_GQA_KERNEL, 3)
+    wl = _workload(8, 2, 128, topk=2100)
+    _run(wl, [30, 52 + 64, 700, 2052], 64, 6, steps=6, seed=231)
+
+
 def test_more_budget_than_blocks_attends_everything_and_the_ring_wraps():
     wl = _workload(8, 2, 128, topk=600, l_recent=16)
     _run(wl, [300, 616, 90], 64, 12, steps=40, seed=207)       # 12 blocks of budget, at most 10 blocks of middle
