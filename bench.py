@@ -679,6 +679,24 @@ def other_config(wl, dev, n_layers):
         torch.cuda.synchronize()
         groups.append(a.elapsed_time(b) / 16)
     ms = statistics.mean(groups)
+    # small batches are bound by the host's launch calls when launched one by one: the same sixteen steps as one
+    # CUDA graph, replayed (the GPU's own time per step)
+    ms_graph = None
+    if nseq * n_layers <= 8:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for s in range(16):
+                step(s)
+        for r in range(3):
+            graph.replay()
+        a, b = ev(), ev()
+        a.record()
+        for r in range(8):
+            graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        ms_graph = a.elapsed_time(b) / (8 * 16)
+        del graph
     eb = 2 if wl.dtype == "bf16" else 4
     rows = min(L + 1, wl.slots)
     step_bytes = n_layers * nseq * wl.n_kv_heads * rows * (wl.d_qk + (0 if wl.v_aliases_k else wl.d_v)) * eb
@@ -690,6 +708,7 @@ def other_config(wl, dev, n_layers):
            "compress_us_note": "median of single calls, each followed by a synchronise",
            "compress_us_per_prompt_layer_back_to_back": comp_b2b_us,
            "decode_ms_per_step": ms, "decode_ms_per_layer_step": ms / n_layers,
+           "decode_ms_per_step_replayed_from_a_cuda_graph_of_16_steps": ms_graph,
            "decode_tokens_per_s_this_slice": nseq / (ms * 1e-3),
            "decode_bytes_per_step": step_bytes, "decode_GBps": step_bytes / (ms * 1e-3) / 1e9,
            "decode_frac_of_measured_hbm": step_bytes / (ms * 1e-3) / 1e9 / peak,
