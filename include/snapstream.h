@@ -24,7 +24,8 @@
  *
  * Conventions
  *   - "dev" pointers are CUDA device pointers on the current device, "host" pointers are plain
- *     host memory.  Every device buffer must be 16-byte aligned.
+ *     host memory.  Every device buffer must be 16-byte aligned (the tensors, caches, outputs and
+ *     workspaces are checked: SNAP_ERR_INVALID_ARG, nothing launched).
  *   - The caller owns every buffer.  The library allocates no device memory; all work is
  *     enqueued on the CUDA stream given and the calls return without synchronising.
  *   - What the library keeps between calls, all of it on the host: per device, the SM count and

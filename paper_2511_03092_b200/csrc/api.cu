@@ -91,6 +91,11 @@ Shape make_shape(const snap_config_t* c) {
 }
 
 size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+// Every device buffer must start on a 16-byte boundary (the kernels use 16-byte accesses and bulk copies); a
+// pointer that does not is refused here rather than left to fault on the device.  NULL passes: optional
+// arguments are checked for presence separately.
+template <typename... P>
+bool misaligned(const P*... p) { return (((reinterpret_cast<uintptr_t>(p) & 15u) != 0) || ...); }
 
 // Option SNAP_OPT_SCORE_KERNEL = 1 (mma.sync) or 2 (SIMT) forces a slower score kernel, 3 keeps the
 // tcgen05 kernels but without CTA pairs (testing aids); default: the best one.
@@ -247,6 +252,7 @@ int decode_step_with_scratch(const snap_config_t* cfg, const snap_layout_t* layo
     return SNAP_ERR_NULL_POINTER;
   if (!cfg->v_aliases_k && !v_cache_dev) return SNAP_ERR_NULL_POINTER;
   if (k_new_dev && !cfg->v_aliases_k && !v_new_dev) return SNAP_ERR_NULL_POINTER;
+  if (misaligned(q_dev, k_new_dev, v_new_dev, k_cache_dev, v_cache_dev, out_dev) || misaligned(scratch)) return SNAP_ERR_INVALID_ARG;
   const Shape s = make_shape(cfg);
   if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
   const DecodePlan p = plan_decode(cfg->dtype, s, n_active);
@@ -370,6 +376,7 @@ int snap_prefill_attn(const snap_config_t* cfg, const void* q_dev,
   const Shape s = make_shape(cfg);
   if (n_seq == 0 || cu_seqlens_host[n_seq] == cu_seqlens_host[0]) return SNAP_OK;
   if (!q_dev || !k_dev || !out_dev || (!cfg->v_aliases_k && !v_dev)) return SNAP_ERR_NULL_POINTER;
+  if (misaligned(q_dev, k_dev, v_dev, out_dev)) return SNAP_ERR_INVALID_ARG;
   const int eb = elt_bytes(cfg->dtype);
   if ((k_token_stride * eb) % 16 || (k_head_stride * eb) % 16 || k_token_stride < s.d_qk) return SNAP_ERR_INVALID_ARG;
   if (!cfg->v_aliases_k && ((v_token_stride * eb) % 16 || (v_head_stride * eb) % 16 || v_token_stride < s.d_v))
@@ -413,6 +420,7 @@ int snap_compress_with_row_stats(const snap_config_t* cfg, const snap_layout_t* 
   if (n_seq == 0) return SNAP_OK;
   if (!k_dev || !k_cache_dev || !seq_len_dev || !valid_topk_dev) return SNAP_ERR_NULL_POINTER;
   if (!cfg->v_aliases_k && (!v_dev || !v_cache_dev)) return SNAP_ERR_NULL_POINTER;
+  if (misaligned(q_obs_dev, k_dev, v_dev, k_cache_dev, v_cache_dev, workspace_dev)) return SNAP_ERR_INVALID_ARG;
   const Shape s = make_shape(cfg);
   if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
   const int eb = elt_bytes(cfg->dtype);
@@ -513,6 +521,7 @@ int snap_append_kv(const snap_config_t* cfg, const snap_layout_t* layout, const 
   if (n_active == 0) return SNAP_OK;
   if (!k_new_dev || !slot_ids_dev || !k_cache_dev || !seq_len_dev) return SNAP_ERR_NULL_POINTER;
   if (!cfg->v_aliases_k && (!v_new_dev || !v_cache_dev)) return SNAP_ERR_NULL_POINTER;
+  if (misaligned(k_new_dev, v_new_dev, k_cache_dev, v_cache_dev)) return SNAP_ERR_INVALID_ARG;
   const Shape s = make_shape(cfg);
   if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
   if (launch_append(cfg->dtype, s, k_new_dev, v_new_dev, slot_ids_dev, n_active, k_cache_dev,
@@ -619,6 +628,7 @@ int snap_block_stats(const snap_config_t* cfg, const snap_layout_t* layout, cons
   if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
   if (n_seqs == 0) return SNAP_OK;
   if (!slot_ids_dev || !k_cache_dev || !valid_topk_dev || !stats_dev) return SNAP_ERR_NULL_POINTER;
+  if (misaligned(k_cache_dev, stats_dev)) return SNAP_ERR_INVALID_ARG;
   const cudaError_t e = launch_block_stats(s, block_tokens, slot_ids_dev, n_seqs, k_cache_dev, valid_topk_dev, stats_dev,
                                            status_dev, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SNAP_OK : SNAP_ERR_CUDA;
@@ -639,6 +649,7 @@ int snap_block_select(const snap_config_t* cfg, const snap_layout_t* layout, con
   if (n_active == 0) return SNAP_OK;
   if (!q_dev || !slot_ids_dev || !stats_dev || !valid_topk_dev || !block_idx_dev || !n_selected_dev || !workspace_dev)
     return SNAP_ERR_NULL_POINTER;
+  if (misaligned(q_dev, stats_dev, workspace_dev)) return SNAP_ERR_INVALID_ARG;
   if (workspace_bytes < block_select_scratch_bytes(s, block_tokens, n_active)) return SNAP_ERR_WORKSPACE_TOO_SMALL;
   const cudaError_t e = launch_block_select(s, block_tokens, n_blocks, q_dev, slot_ids_dev, n_active, stats_dev, valid_topk_dev,
                                             block_idx_dev, n_selected_dev, workspace_dev, status_dev,
@@ -685,6 +696,7 @@ int snap_decode_attn_blocks(const snap_config_t* cfg, const snap_layout_t* layou
       !n_selected_dev || !out_dev || !workspace_dev)
     return SNAP_ERR_NULL_POINTER;
   if (k_new_dev && !v_new_dev) return SNAP_ERR_NULL_POINTER;
+  if (misaligned(q_dev, k_new_dev, v_new_dev, k_cache_dev, v_cache_dev, out_dev, workspace_dev)) return SNAP_ERR_INVALID_ARG;
   const int64_t need = snap_decode_blocks_workspace_bytes(cfg, n_active, block_tokens, n_blocks);
   if (need < 0) return (int)need;
   if (workspace_bytes < (size_t)need) return SNAP_ERR_WORKSPACE_TOO_SMALL;
@@ -713,6 +725,7 @@ int snap_decode_attn_multi(const snap_config_t* cfg, const snap_layout_t* layout
       !workspace_dev)
     return SNAP_ERR_NULL_POINTER;
   if (!s.v_aliases_k && (!v_new_dev || !v_cache_dev)) return SNAP_ERR_NULL_POINTER;
+  if (misaligned(q_dev, k_new_dev, v_new_dev, k_cache_dev, v_cache_dev, out_dev, workspace_dev)) return SNAP_ERR_INVALID_ARG;
   if (layout->slots != s.Sc) return SNAP_ERR_INVALID_ARG;
   const int64_t need = snap_decode_multi_workspace_bytes(cfg, n_active, q_len);
   if (need < 0) return (int)need;

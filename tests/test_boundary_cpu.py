@@ -96,6 +96,17 @@ def test_workspace_queries_and_argument_errors_without_gpu():
     assert lib.snap_append_kv(C.byref(cfg), C.byref(lay), one, one, one, -1, one, one, one, None, None) == -1
     assert lib.snap_decode_attn(C.byref(cfg), C.byref(lay), one, None, None, one, 0, one, one, one, one, one,
                                 one, 0, None, None) == 0                     # nothing to do
+    # device buffers that do not start on a 16-byte boundary are refused before anything is launched
+    odd = C.c_void_p(264)
+    assert lib.snap_compress(C.byref(cfg), C.byref(lay), one, odd, 1024, 128, one, 1024, 128, cu, ok_slot, 1,
+                             one, one, one, one, None, one, 1 << 40, None, None) == -1
+    assert lib.snap_compress(C.byref(cfg), C.byref(lay), one, one, 1024, 128, one, 1024, 128, cu, ok_slot, 1,
+                             one, one, one, one, None, odd, 1 << 40, None, None) == -1
+    assert lib.snap_decode_attn(C.byref(cfg), C.byref(lay), odd, None, None, one, 4, one, one, one, one, one,
+                                one, 1 << 40, None, None) == -1
+    assert lib.snap_decode_attn(C.byref(cfg), C.byref(lay), one, None, None, one, 4, one, one, one, one, one,
+                                odd, 1 << 40, None, None) == -1
+    assert lib.snap_append_kv(C.byref(cfg), C.byref(lay), one, one, one, 2, odd, one, one, None, None) == -1
     two = C.c_void_p(512)
     cc = lambda *a: lib.snap_append_kv_concat(C.byref(cfg), C.byref(lay), *a)
     assert cc(one, one, one, 2, one, one, one, one, one, None, None) == -1   # in place: output must differ from input
